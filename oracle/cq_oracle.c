@@ -1,0 +1,294 @@
+/*
+ * CPU oracle for Coupled Quantization (CQ) of LLM KV caches -- TEST INFRASTRUCTURE.
+ *
+ * Plain, slow, fp64.  It exists to check the CUDA library and to be timed as a
+ * CPU baseline; it shares no code with the CUDA path and the product never
+ * calls it.  Every function states the passage of the paper it follows.
+ *
+ * Conventions
+ *   D  head_dim, c channels per group, G = D / c groups, b bits per code,
+ *   K = 2^b centroids per group.
+ *   x          fp16 bit patterns, row-major [n_vec][n_heads][D]
+ *   codebooks  fp32, row-major [n_heads][G][K][c]
+ *   codes      int32, row-major [n_vec][n_heads][G]       (encode)
+ *              int32, row-major [n_seq][max_tokens][n_kv_heads][G] (attention)
+ * fp16 and fp32 inputs are widened exactly to fp64; all arithmetic is fp64.
+ * OpenMP parallelises only over independent items (vectors, or (sequence,
+ * query head) pairs); there is no blocking, fusion or reordering inside an item.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* IEEE binary16 bit pattern -> double, exact. */
+static double half_to_double(uint16_t h)
+{
+    int sign = (h >> 15) & 1;
+    int expo = (h >> 10) & 0x1f;
+    int mant = h & 0x3ff;
+    double v;
+    if (expo == 0)
+        v = ldexp((double)mant, -24);               /* subnormal or zero */
+    else if (expo == 31)
+        v = mant ? NAN : INFINITY;
+    else
+        v = ldexp((double)(mant | 0x400), expo - 25);
+    return sign ? -v : v;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/*
+ * CQ encode (Section 3.2: the channels of a key/value vector are split into
+ * equal, non-overlapping groups of c contiguous channels and every group is
+ * replaced by the index of its nearest centroid in L2 distance; this is the
+ * map CQ(.) inside Eq. 5).
+ *
+ * d_j = sum_{i<c} (x[g c + i] - C[h][g][j][i])^2, code = argmin_j d_j, lowest
+ * index on exact ties.  d_best / d_second (may be NULL) receive the smallest
+ * and second smallest distance of each (vector, head, group), which the
+ * near-tie acceptance rule of the tests needs (d_second = +inf when K == 1).
+ */
+void oracle_encode(const uint16_t *x, const float *codebooks, int64_t n_vec,
+                   int n_heads, int D, int c, int b, int32_t *codes,
+                   double *d_best, double *d_second)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+#pragma omp parallel for schedule(static)
+    for (int64_t v = 0; v < n_vec; ++v) {
+        for (int h = 0; h < n_heads; ++h) {
+            const uint16_t *xv = x + (v * n_heads + h) * (int64_t)D;
+            for (int g = 0; g < G; ++g) {
+                const float *cb = codebooks + ((int64_t)h * G + g) * K * c;
+                double best = INFINITY, second = INFINITY;
+                int32_t arg = 0;
+                for (int j = 0; j < K; ++j) {
+                    double d = 0.0;
+                    for (int i = 0; i < c; ++i) {
+                        double diff = half_to_double(xv[g * c + i]) - (double)cb[j * c + i];
+                        d += diff * diff;
+                    }
+                    if (d < best) {
+                        second = best;
+                        best = d;
+                        arg = j;
+                    } else if (d < second) {
+                        second = d;
+                    }
+                }
+                int64_t o = (v * n_heads + h) * G + g;
+                codes[o] = arg;
+                if (d_best) d_best[o] = best;
+                if (d_second) d_second[o] = second;
+            }
+        }
+    }
+}
+
+/*
+ * Squared L2 distance between each group of x and the centroid named by an
+ * arbitrary code (same definition of distance as oracle_encode, Section 3.2).
+ * Used to judge a code that differs from the oracle's.
+ */
+void oracle_code_distance(const uint16_t *x, const float *codebooks, const int32_t *codes,
+                          int64_t n_vec, int n_heads, int D, int c, int b, double *dist)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+#pragma omp parallel for schedule(static)
+    for (int64_t v = 0; v < n_vec; ++v)
+        for (int h = 0; h < n_heads; ++h)
+            for (int g = 0; g < G; ++g) {
+                int64_t o = (v * n_heads + h) * G + g;
+                const float *cj = codebooks + (((int64_t)h * G + g) * K + codes[o]) * c;
+                double d = 0.0;
+                for (int i = 0; i < c; ++i) {
+                    double diff = half_to_double(x[(v * n_heads + h) * (int64_t)D + g * c + i]) - (double)cj[i];
+                    d += diff * diff;
+                }
+                dist[o] = d;
+            }
+}
+
+/*
+ * Dequantisation CQ(A) (Section 3.2.1: the reconstruction whose error
+ * ||A - CQ(A)||_F^2 the centroid objectives measure): channel g c + i of the
+ * reconstruction is component i of centroid codes[g] of group g.
+ */
+void oracle_dequant(const int32_t *codes, const float *codebooks, int64_t n_vec,
+                    int n_heads, int D, int c, int b, double *xhat)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+    for (int64_t v = 0; v < n_vec; ++v)
+        for (int h = 0; h < n_heads; ++h)
+            for (int g = 0; g < G; ++g) {
+                int32_t j = codes[(v * n_heads + h) * G + g];
+                const float *cj = codebooks + (((int64_t)h * G + g) * K + j) * c;
+                for (int i = 0; i < c; ++i)
+                    xhat[(v * n_heads + h) * (int64_t)D + g * c + i] = (double)cj[i];
+            }
+}
+
+/*
+ * Decode attention over a CQ-coded cache, dense form (Eq. 1 with the cached
+ * keys and values replaced by their CQ reconstructions, Section 3.2):
+ *   Khat_t = dequant(k_codes[t]), Vhat_t = dequant(v_codes[t])
+ *   s_t = scale * <q, Khat_t>,  p = softmax(s_0 .. s_{n-1}),  out = sum_t p_t Vhat_t
+ * for the first n = seq_lens[s] cached tokens of sequence s.  Query head hq
+ * reads KV head hq / (n_q_heads / n_kv_heads).  n == 0 gives a zero row.
+ *
+ *   q    fp16 bits [n_seq][n_q_heads][D]
+ *   out  fp64      [n_seq][n_q_heads][D]
+ */
+void oracle_decode_dense(const uint16_t *q, const int32_t *k_codes, const int32_t *v_codes,
+                         const float *k_cb, const float *v_cb, const int32_t *seq_lens,
+                         double scale, int n_seq, int n_q_heads, int n_kv_heads, int D,
+                         int c, int b, int64_t max_tokens, double *out)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+    const int R = n_q_heads / n_kv_heads;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int s = 0; s < n_seq; ++s) {
+        for (int hq = 0; hq < n_q_heads; ++hq) {
+            const int hkv = hq / R;
+            const int64_t n = seq_lens[s];
+            double *o = out + ((int64_t)s * n_q_heads + hq) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            if (n <= 0) continue;
+            double *qd = (double *)malloc(sizeof(double) * D);
+            double *score = (double *)malloc(sizeof(double) * n);
+            for (int d = 0; d < D; ++d)
+                qd[d] = half_to_double(q[((int64_t)s * n_q_heads + hq) * D + d]);
+            double smax = -INFINITY;
+            for (int64_t t = 0; t < n; ++t) {
+                const int32_t *kc = k_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                double dot = 0.0;
+                for (int g = 0; g < G; ++g) {
+                    const float *cj = k_cb + (((int64_t)hkv * G + g) * K + kc[g]) * c;
+                    for (int i = 0; i < c; ++i) dot += qd[g * c + i] * (double)cj[i];
+                }
+                score[t] = scale * dot;
+                if (score[t] > smax) smax = score[t];
+            }
+            double denom = 0.0;
+            for (int64_t t = 0; t < n; ++t) {
+                score[t] = exp(score[t] - smax);
+                denom += score[t];
+            }
+            for (int64_t t = 0; t < n; ++t) {
+                const int32_t *vc = v_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                double p = score[t] / denom;
+                for (int g = 0; g < G; ++g) {
+                    const float *cj = v_cb + (((int64_t)hkv * G + g) * K + vc[g]) * c;
+                    for (int i = 0; i < c; ++i) o[g * c + i] += p * (double)cj[i];
+                }
+            }
+            free(qd);
+            free(score);
+        }
+    }
+}
+
+/*
+ * The same attention in the lookup-table form the CUDA library is asked to
+ * use: a per-query table LUT[g][j] = scale * <q_g, Ck[g][j]>, scores as sums
+ * of table entries, softmax online over n_chunks contiguous context chunks,
+ * softmax weights binned per V code, bins multiplied by the V centroids, and
+ * chunk partials (m, l, acc) merged with the log-sum-exp rule.  It is an exact
+ * re-association of Eq. 1 and serves only to cross-check oracle_decode_dense.
+ */
+void oracle_decode_lut(const uint16_t *q, const int32_t *k_codes, const int32_t *v_codes,
+                       const float *k_cb, const float *v_cb, const int32_t *seq_lens,
+                       double scale, int n_seq, int n_q_heads, int n_kv_heads, int D,
+                       int c, int b, int64_t max_tokens, int n_chunks, double *out)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+    const int R = n_q_heads / n_kv_heads;
+    if (n_chunks < 1) n_chunks = 1;
+    for (int s = 0; s < n_seq; ++s) {
+        for (int hq = 0; hq < n_q_heads; ++hq) {
+            const int hkv = hq / R;
+            const int64_t n = seq_lens[s];
+            double *o = out + ((int64_t)s * n_q_heads + hq) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            if (n <= 0) continue;
+            double *lut = (double *)malloc(sizeof(double) * G * K);
+            double *bins = (double *)malloc(sizeof(double) * G * K);
+            double *acc = (double *)malloc(sizeof(double) * D);
+            double *tot = (double *)calloc(D, sizeof(double));
+            for (int g = 0; g < G; ++g)
+                for (int j = 0; j < K; ++j) {
+                    const float *cj = k_cb + (((int64_t)hkv * G + g) * K + j) * c;
+                    double dot = 0.0;
+                    for (int i = 0; i < c; ++i)
+                        dot += half_to_double(q[((int64_t)s * n_q_heads + hq) * D + g * c + i]) * (double)cj[i];
+                    lut[g * K + j] = scale * dot;
+                }
+            double M = -INFINITY, L = 0.0;   /* running max and normaliser of merged chunks */
+            for (int ch = 0; ch < n_chunks; ++ch) {
+                int64_t t0 = n * ch / n_chunks, t1 = n * (ch + 1) / n_chunks;
+                if (t1 <= t0) continue;
+                double m = -INFINITY, l = 0.0;
+                for (int64_t t = t0; t < t1; ++t) {
+                    const int32_t *kc = k_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                    double sc = 0.0;
+                    for (int g = 0; g < G; ++g) sc += lut[g * K + kc[g]];
+                    if (sc > m) m = sc;
+                }
+                memset(bins, 0, sizeof(double) * G * K);
+                for (int64_t t = t0; t < t1; ++t) {
+                    const int32_t *kc = k_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                    const int32_t *vc = v_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                    double sc = 0.0;
+                    for (int g = 0; g < G; ++g) sc += lut[g * K + kc[g]];
+                    double p = exp(sc - m);
+                    l += p;
+                    for (int g = 0; g < G; ++g) bins[g * K + vc[g]] += p;
+                }
+                for (int g = 0; g < G; ++g)
+                    for (int i = 0; i < c; ++i) {
+                        double a = 0.0;
+                        for (int j = 0; j < K; ++j)
+                            a += bins[g * K + j] * (double)v_cb[(((int64_t)hkv * G + g) * K + j) * c + i];
+                        acc[g * c + i] = a;
+                    }
+                /* merge partial (m, l, acc) into (M, L, tot) */
+                double Mn = m > M ? m : M;
+                double wo = (M == -INFINITY) ? 0.0 : exp(M - Mn);
+                double wn = exp(m - Mn);
+                for (int d = 0; d < D; ++d) tot[d] = tot[d] * wo + acc[d] * wn;
+                L = L * wo + l * wn;
+                M = Mn;
+            }
+            for (int d = 0; d < D; ++d) o[d] = tot[d] / L;
+            free(lut);
+            free(bins);
+            free(acc);
+            free(tot);
+        }
+    }
+}

@@ -1,0 +1,278 @@
+"""Pins of the fp64 CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each pin is chosen so that a
+plausible slip in the oracle (wrong group or head index, transposed codebook,
+dropped scale, wrong GQA mapping, missing normalisation) breaks it.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+rng = np.random.default_rng(20240503)
+
+
+def rand_case(n_vec, n_heads, D, c, b, scale_x=1.0):
+    x = (scale_x * rng.standard_normal((n_vec, n_heads, D))).astype(np.float16)
+    cb = rng.standard_normal((n_heads, D // c, 1 << b, c)).astype(np.float32)
+    return x, cb
+
+
+# ----------------------------------------------------------------------------- encode
+
+def test_fp16_widening_is_exact():
+    # K = 1 centroid at 0, c = 1: distance is x^2, so every finite fp16 bit pattern
+    # must come back as numpy's own widening squared.
+    bits = np.arange(65536, dtype=np.uint16)
+    vals = bits.view(np.float16).astype(np.float64)
+    keep = np.isfinite(vals)
+    x = bits[keep].reshape(-1, 1, 1)
+    cb = np.zeros((1, 1, 1, 1), dtype=np.float32)
+    codes, d1, _ = oracle.encode(x, cb, 1, 0)
+    assert (codes == 0).all()
+    assert np.array_equal(d1.ravel(), vals[keep] ** 2)
+
+
+def test_hand_worked_scalar_and_pair_cases():
+    # c = 1, centroids {0, 10}: 4 -> 0, 6 -> 1, 5 is an exact tie -> lowest index.
+    x = np.array([4.0, 6.0, 5.0, -3.0, 11.0], dtype=np.float16).reshape(5, 1, 1)
+    cb = np.array([0.0, 10.0], dtype=np.float32).reshape(1, 1, 2, 1)
+    codes, d1, d2 = oracle.encode(x, cb, 1, 1)
+    assert codes.ravel().tolist() == [0, 1, 0, 0, 1]
+    assert d1.ravel().tolist() == [16.0, 16.0, 25.0, 9.0, 1.0]
+    assert d2.ravel().tolist() == [36.0, 36.0, 25.0, 169.0, 121.0]
+    # c = 2, b = 2, one vector of two groups with different codebooks per group.
+    # group 0 = (1, 1): centroids (0,0) d=2, (2,2) d=2, (1,2) d=1, (3,1) d=4 -> 2
+    # group 1 = (-2, 0): centroids (0,0) d=4, (-2,1) d=1, (-3,0) d=1, (5,5) -> tie 1/2 -> 1
+    x = np.array([1, 1, -2, 0], dtype=np.float16).reshape(1, 1, 4)
+    cb = np.array([[[0, 0], [2, 2], [1, 2], [3, 1]],
+                   [[0, 0], [-2, 1], [-3, 0], [5, 5]]], dtype=np.float32).reshape(1, 2, 4, 2)
+    codes, d1, d2 = oracle.encode(x, cb, 2, 2)
+    assert codes.ravel().tolist() == [2, 1]
+    assert d1.ravel().tolist() == [1.0, 1.0]
+    assert d2.ravel().tolist() == [2.0, 1.0]
+
+
+@pytest.mark.parametrize("c,b", [(1, 1), (2, 2), (4, 3), (8, 2), (2, 3)])
+def test_brute_force_python_loops(c, b):
+    # Integer-valued tiny inputs, distances by pure-Python integer arithmetic.
+    D, n_vec, n_heads = 8, 6, 2
+    x = rng.integers(-4, 5, size=(n_vec, n_heads, D)).astype(np.float16)
+    cb = rng.integers(-4, 5, size=(n_heads, D // c, 1 << b, c)).astype(np.float32)
+    codes, d1, d2 = oracle.encode(x, cb, c, b)
+    for v, h, g in itertools.product(range(n_vec), range(n_heads), range(D // c)):
+        ds = []
+        for j in range(1 << b):
+            ds.append(sum((int(x[v, h, g * c + i]) - int(cb[h, g, j, i])) ** 2 for i in range(c)))
+        best = min(ds)
+        assert codes[v, h, g] == ds.index(best)          # first occurrence
+        assert d1[v, h, g] == best
+        assert d2[v, h, g] == sorted(ds)[1]
+
+
+@pytest.mark.parametrize("c,b", [(2, 8), (4, 8), (8, 8), (8, 5)])
+def test_codebook_contains_inputs_gives_zero_error(c, b):
+    # Every input group is one of its group's centroids: distance exactly 0,
+    # code = lowest index holding that centroid, reconstruction = input.
+    D, n_heads, K = 32, 3, 1 << b
+    cb = rng.standard_normal((n_heads, D // c, K, c)).astype(np.float16).astype(np.float32)
+    cb[:, :, K - 1, :] = cb[:, :, 3, :]                   # duplicate: index 3 must win over K-1
+    pick = rng.integers(0, K, size=(50, n_heads, D // c))
+    x = np.empty((50, n_heads, D), dtype=np.float16)
+    for v, h, g in itertools.product(range(50), range(n_heads), range(D // c)):
+        x[v, h, g * c:(g + 1) * c] = cb[h, g, pick[v, h, g]]
+    codes, d1, _ = oracle.encode(x, cb, c, b)
+    want = np.where(pick == K - 1, 3, pick)
+    assert np.array_equal(codes, want)
+    assert (d1 == 0).all()
+    assert np.array_equal(oracle.dequant(codes, cb, c, b), x.astype(np.float64))
+
+
+def test_c1_reduces_to_scalar_bucketing():
+    # With one channel per group CQ is channel-wise non-uniform quantisation
+    # (Section 2.3): nearest scalar centroid = bucket between sorted midpoints.
+    D, b = 16, 4
+    x = rng.standard_normal((200, 1, D)).astype(np.float16)
+    cb = rng.standard_normal((1, D, 1 << b, 1)).astype(np.float32)
+    codes, _, _ = oracle.encode(x, cb, 1, b)
+    for ch in range(D):
+        cent = cb[0, ch, :, 0].astype(np.float64)
+        order = np.argsort(cent, kind="stable")
+        mids = (cent[order][1:] + cent[order][:-1]) / 2
+        want = order[np.searchsorted(mids, x[:, 0, ch].astype(np.float64), side="left")]
+        assert np.array_equal(codes[:, 0, ch], want)
+
+
+@pytest.mark.parametrize("c,b", [(2, 8), (4, 6), (8, 8)])
+def test_matches_torch_cdist_argmin(c, b):
+    D, n_heads = 64, 3
+    x, cb = rand_case(40, n_heads, D, c, b)
+    codes, d1, d2 = oracle.encode(x, cb, c, b)
+    xt = torch.from_numpy(x.astype(np.float64))
+    for h in range(n_heads):
+        for g in range(D // c):
+            dist = torch.cdist(xt[:, h, g * c:(g + 1) * c], torch.from_numpy(cb[h, g].astype(np.float64))) ** 2
+            assert np.array_equal(codes[:, h, g], dist.argmin(dim=1).numpy())
+            top2 = dist.topk(2, dim=1, largest=False).values.numpy()
+            np.testing.assert_allclose(d1[:, h, g], top2[:, 0], rtol=1e-9)   # cdist takes a sqrt
+            np.testing.assert_allclose(d2[:, h, g], top2[:, 1], rtol=1e-9)
+
+
+def test_single_code_change_never_lowers_error():
+    # Objective of CQ(.) in Eq. 5: nearest-centroid assignment minimises ||A - CQ(A)||_F^2.
+    D, c, b = 32, 4, 6
+    x, cb = rand_case(30, 2, D, c, b)
+    codes, _, _ = oracle.encode(x, cb, c, b)
+    base = ((oracle.dequant(codes, cb, c, b) - x.astype(np.float64)) ** 2).sum()
+    for _ in range(200):
+        alt = codes.copy()
+        v, h, g = rng.integers(30), rng.integers(2), rng.integers(D // c)
+        alt[v, h, g] = rng.integers(1 << b)
+        err = ((oracle.dequant(alt, cb, c, b) - x.astype(np.float64)) ** 2).sum()
+        assert err >= base - 1e-9
+    dist = oracle.code_distance(x, cb, codes, c, b)
+    np.testing.assert_allclose(dist.sum(), base, rtol=1e-12)
+
+
+def test_sizes_match_paper_tables():
+    for line in open(os.path.join(GOLDEN, "table4_centroid_params.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        _, layers, heads, hd, bits, printed = line.split()
+        n = int(layers) * 2 * int(heads) * int(hd) * (1 << int(bits))
+        assert round(n / 1e6, 2) == float(printed)
+        for c in (2, 4, 8):   # the count does not depend on the coupling c
+            cb_shape = (int(heads), int(hd) // c, 1 << int(bits), c)
+            assert int(layers) * 2 * int(np.prod(cb_shape)) == n
+    for line in open(os.path.join(GOLDEN, "table1_bits_per_fpn.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        _, c, b, printed = line.split()
+        assert int(b) / int(c) == float(printed)
+
+
+# ----------------------------------------------------------------------------- attention
+
+def attn_case(n_seq, Hq, Hkv, D, c, b, max_tokens, lens=None):
+    q = rng.standard_normal((n_seq, Hq, D)).astype(np.float16)
+    kc = rng.integers(0, 1 << b, size=(n_seq, max_tokens, Hkv, D // c)).astype(np.int32)
+    vc = rng.integers(0, 1 << b, size=(n_seq, max_tokens, Hkv, D // c)).astype(np.int32)
+    kcb = rng.standard_normal((Hkv, D // c, 1 << b, c)).astype(np.float32)
+    vcb = rng.standard_normal((Hkv, D // c, 1 << b, c)).astype(np.float32)
+    sl = np.full(n_seq, max_tokens, dtype=np.int32) if lens is None else np.asarray(lens, dtype=np.int32)
+    return q, kc, vc, kcb, vcb, sl
+
+
+def torch_dense(q, kc, vc, kcb, vcb, sl, scale, c, b):
+    """Eq. 1 with library routines: gather, matmul, torch.softmax, all fp64."""
+    n_seq, Hq, D = q.shape
+    Hkv = kc.shape[2]
+    G = D // c
+    R = Hq // Hkv
+    out = np.zeros((n_seq, Hq, D))
+    for s in range(n_seq):
+        n = int(sl[s])
+        if n == 0:
+            continue
+        for hq in range(Hq):
+            h = hq // R
+            gi = torch.arange(G)
+            K = torch.from_numpy(kcb[h].astype(np.float64))[gi[None, :], torch.from_numpy(kc[s, :n, h].astype(np.int64))].reshape(n, D)
+            V = torch.from_numpy(vcb[h].astype(np.float64))[gi[None, :], torch.from_numpy(vc[s, :n, h].astype(np.int64))].reshape(n, D)
+            p = torch.softmax(scale * (K @ torch.from_numpy(q[s, hq].astype(np.float64))), dim=0)
+            out[s, hq] = (p[None, :] @ V).numpy()[0]
+    return out
+
+
+@pytest.mark.parametrize("c,b,Hq,Hkv", [(8, 8, 4, 2), (4, 8, 2, 2), (2, 5, 6, 2)])
+def test_dense_matches_torch_softmax(c, b, Hq, Hkv):
+    D = 32
+    args = attn_case(3, Hq, Hkv, D, c, b, 37, lens=[37, 5, 0])
+    got = oracle.decode_dense(*args, 0.31, c, b)
+    want = torch_dense(*args, 0.31, c, b)
+    np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-13)
+    assert (got[2] == 0).all()                     # empty context -> zero row
+
+
+@pytest.mark.parametrize("n_chunks", [1, 2, 7, 53])
+def test_lut_form_equals_dense_form_for_any_chunking(n_chunks):
+    args = attn_case(2, 4, 2, 64, 8, 8, 53, lens=[53, 20])
+    dense = oracle.decode_dense(*args, 1 / np.sqrt(64), 8, 8)
+    lut = oracle.decode_lut(*args, 1 / np.sqrt(64), 8, 8, n_chunks=n_chunks)
+    np.testing.assert_allclose(lut, dense, rtol=1e-12, atol=1e-14)
+
+
+def test_lut_sum_equals_scaled_dot_with_reconstruction():
+    # sum_g LUT_g[code_g] = scale <q, Khat>, checked through a context of two tokens:
+    # out = sigma(s0 - s1) V0 + (1 - sigma) V1 with s from an independent numpy dot.
+    D, c, b = 16, 4, 3
+    q, kc, vc, kcb, vcb, sl = attn_case(1, 1, 1, D, c, b, 2)
+    scale = 0.7
+    khat = oracle.dequant(kc[0], kcb, c, b)[:, 0]     # (2, D)
+    vhat = oracle.dequant(vc[0], vcb, c, b)[:, 0]
+    s = scale * khat @ q[0, 0].astype(np.float64)
+    w0 = 1 / (1 + np.exp(s[1] - s[0]))
+    want = w0 * vhat[0] + (1 - w0) * vhat[1]
+    for fn in (lambda: oracle.decode_dense(q, kc, vc, kcb, vcb, sl, scale, c, b),
+               lambda: oracle.decode_lut(q, kc, vc, kcb, vcb, sl, scale, c, b, n_chunks=2)):
+        np.testing.assert_allclose(fn()[0, 0], want, rtol=1e-12, atol=1e-14)
+
+
+def test_one_token_context_returns_its_value_reconstruction():
+    D, c, b = 128, 8, 8
+    q, kc, vc, kcb, vcb, _ = attn_case(3, 4, 2, D, c, b, 5)
+    sl = np.ones(3, dtype=np.int32)
+    out = oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 0.088, c, b)
+    for s in range(3):
+        vhat = oracle.dequant(vc[s, :1], vcb, c, b)[0]          # (Hkv, D)
+        for hq in range(4):
+            assert np.array_equal(out[s, hq], vhat[hq // 2])
+
+
+def test_zero_query_gives_mean_and_score_shift_is_invisible():
+    D, c, b = 32, 4, 4
+    q, kc, vc, kcb, vcb, sl = attn_case(1, 2, 1, D, c, b, 19)
+    kcb = np.round(kcb * 64) / 64                       # so that the shift below is exact in fp32
+    out0 = oracle.decode_dense(np.zeros_like(q), kc, vc, kcb, vcb, sl, 0.5, c, b)
+    vhat = oracle.dequant(vc[0, :, :, :], vcb, c, b)[:, 0]
+    np.testing.assert_allclose(out0[0, 0], vhat.mean(axis=0), rtol=1e-12, atol=1e-14)
+    base = oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 0.5, c, b)
+    shifted = kcb.copy()
+    shifted[0, 3] += np.array([0.5, -1.25, 2.0, 0.75], dtype=np.float32)   # same shift for every centroid of group 3
+    np.testing.assert_allclose(oracle.decode_dense(q, kc, vc, shifted, vcb, sl, 0.5, c, b), base,
+                               rtol=1e-9, atol=1e-12)
+
+
+def test_token_permutation_and_gqa_replication():
+    D, c, b = 32, 8, 6
+    q, kc, vc, kcb, vcb, sl = attn_case(2, 4, 2, D, c, b, 23, lens=[23, 11])
+    base = oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 0.2, c, b)
+    kp, vp = kc.copy(), vc.copy()
+    for s in range(2):
+        perm = rng.permutation(int(sl[s]))
+        kp[s, :sl[s]] = kc[s, perm]
+        vp[s, :sl[s]] = vc[s, perm]
+    np.testing.assert_allclose(oracle.decode_dense(q, kp, vp, kcb, vcb, sl, 0.2, c, b), base,
+                               rtol=1e-11, atol=1e-13)
+    # GQA with R = 2 equals MHA with every KV head (codes and codebooks) repeated twice.
+    rep = lambda a, ax: np.repeat(a, 2, axis=ax)
+    mha = oracle.decode_dense(q, rep(kc, 2), rep(vc, 2), rep(kcb, 0), rep(vcb, 0), sl, 0.2, c, b)
+    assert np.array_equal(mha, base)
+    # tokens past seq_len are never read
+    kc2 = kc.copy()
+    kc2[1, 11:] = (kc2[1, 11:] + 1) % (1 << b)
+    assert np.array_equal(oracle.decode_dense(q, kc2, vc, kcb, vcb, sl, 0.2, c, b), base)
+
+
+def test_scale_is_applied_to_scores_only():
+    D, c, b = 16, 2, 3
+    q, kc, vc, kcb, vcb, sl = attn_case(1, 1, 1, D, c, b, 9)
+    a = oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 0.25, c, b)
+    b2 = oracle.decode_dense(q, kc, vc, (0.25 * kcb.astype(np.float64)).astype(np.float32), vcb, sl, 1.0, c, b)
+    np.testing.assert_allclose(a, b2, rtol=1e-6)      # 0.25 is a power of two: kcb scaling is exact
+    assert np.abs(a - oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 1.0, c, b)).max() > 1e-3
