@@ -1,0 +1,186 @@
+/*
+ * cq.h -- C ABI of the Coupled Quantization (CQ) KV-cache library for NVIDIA B200 (sm_100a).
+ *
+ * CQ (arXiv 2405.03917, Section 3.2) splits the head_dim channels of every key
+ * or value vector into G = head_dim / c groups of c contiguous channels and
+ * stores, per group, the b-bit index of the nearest of 2^b group-specific
+ * centroids ("CQ-<c>c<b>b").  This library holds the two data-parallel steps
+ * that touch every cached token:
+ *
+ *   cq_encode       vectors -> codes           (Section 3.2; the map CQ(.) of Eq. 5)
+ *   cq_decode_attn  single-query attention that reads only the codes
+ *                   (Eq. 1 with K and V replaced by their CQ reconstructions)
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The
+ *     caller owns all buffers, including the workspace; the library allocates
+ *     nothing and keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     enqueue work and return; they never synchronise, except cq_decode_step_host.
+ *   - Every function that returns int returns a cq_status: arguments are checked
+ *     on the host before anything is launched, a failed check launches nothing,
+ *     and a CUDA launch error is reported as CQ_ERR_CUDA.  Nothing aborts or traps.
+ *   - Supported shapes: c divides head_dim, head_dim <= 256, 1 <= b <= 8 (codes
+ *     are one uint8 each), n_q_heads a multiple of n_kv_heads.  Tuned kernels
+ *     exist for head_dim 128 with CQ-2c8b, CQ-4c8b and CQ-8c8b; every other
+ *     supported shape runs on generic sm_100a kernels (never on the CPU).
+ *   - Inputs must be finite.
+ *
+ * Code layout (version cq_layout_version() == 1).  Codes of one (sequence, head)
+ * are stored in blocks of CQ_TOKEN_BLOCK = 16 tokens, group-major inside a block:
+ *
+ *   byte offset of (seq s, head h, token t, group g) =
+ *       (((s * n_heads + h) * NB + t / 16) * G + g) * 16 + t % 16,   NB = ceil(max_tokens / 16)
+ *
+ * so the 16 codes of one group for 16 consecutive tokens are one aligned 16-byte
+ * word.  cq_codes_to_rowmajor / cq_codes_from_rowmajor convert to and from the
+ * plain [n_seq][max_tokens][n_heads][G] order.
+ */
+#ifndef CQ_H_
+#define CQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CQ_TOKEN_BLOCK 16
+
+typedef enum {
+    CQ_OK = 0,
+    CQ_ERR_NULL = -1,        /* a required pointer is NULL                                  */
+    CQ_ERR_SHAPE = -2,       /* zero / negative dims, c does not divide head_dim, Hq % Hkv, */
+                             /* token range outside [0, max_tokens]                         */
+    CQ_ERR_UNSUPPORTED = -3, /* b outside [1, 8], head_dim > 256                            */
+    CQ_ERR_ALIGN = -4,       /* a pointer is not aligned as documented                      */
+    CQ_ERR_WORKSPACE = -5,   /* workspace smaller than the matching *_workspace_bytes()     */
+    CQ_ERR_CUDA = -6         /* a CUDA runtime call or launch failed                        */
+} cq_status;
+
+/* Version of the code layout described above. */
+int cq_layout_version(void);
+
+/* Static, human-readable name of a cq_status value. */
+const char *cq_status_string(int status);
+
+/*
+ * Bytes of one code buffer (K or V) for n_seq sequences of capacity max_tokens:
+ * n_seq * n_heads * ceil(max_tokens / 16) * G * 16 (the paper's "bits per FPN"
+ * b / c of Section 4, with b rounded up to one byte and the capacity rounded up
+ * to a token block).  Returns 0 for invalid arguments.
+ */
+size_t cq_codes_bytes(int64_t n_seq, int64_t max_tokens, int n_heads, int head_dim, int c, int b);
+
+/*
+ * CQ encode (Section 3.2): for every vector and every group g, the index
+ *   argmin_j  sum_{i<c} (x[g*c+i] - codebooks[h][g][j][i])^2 ,  lowest j on exact ties,
+ * evaluated in fp32 (distances that differ by less than about 1e-6 relative may
+ * resolve either way).
+ *
+ *   x_fp16       [n_seq][n_tokens][n_heads][head_dim] fp16, 16-byte aligned
+ *   codebooks    [n_heads][G][2^b][c] fp32, 16-byte aligned
+ *   seq_offsets  NULL, or [n_seq] int32: per-sequence first cache position
+ *   codes_out    code buffer of cq_codes_bytes(n_seq, max_tokens, ...) bytes, 16-byte
+ *                aligned; token i of sequence s is written at cache position
+ *                token_offset + (seq_offsets ? seq_offsets[s] : 0) + i.  Positions
+ *                outside [0, max_tokens) are skipped.  Other positions are untouched
+ *                (appending one token rewrites G single bytes per head).
+ * Requires 0 <= token_offset and, without seq_offsets, token_offset + n_tokens <= max_tokens.
+ */
+int cq_encode(const void *x_fp16, const float *codebooks, const int32_t *seq_offsets,
+              int64_t n_seq, int64_t n_tokens, int64_t token_offset, int64_t max_tokens,
+              int n_heads, int head_dim, int c, int b, void *codes_out, void *stream);
+
+/*
+ * Layout converters.  rowmajor is uint8 [n_seq][max_tokens][n_heads][G].
+ * to_rowmajor reads every position < max_tokens of the library layout;
+ * from_rowmajor writes every position < max_tokens (block padding is zeroed).
+ */
+int cq_codes_to_rowmajor(const void *codes, int64_t n_seq, int64_t max_tokens, int n_heads,
+                         int head_dim, int c, int b, void *rowmajor_out, void *stream);
+int cq_codes_from_rowmajor(const void *rowmajor, int64_t n_seq, int64_t max_tokens, int n_heads,
+                           int head_dim, int c, int b, void *codes_out, void *stream);
+
+/*
+ * Workspace of cq_decode_attn: split-K partials (running max, normaliser and
+ * head_dim accumulators per (sequence, query head, context split)).
+ * Returns 0 for invalid arguments.
+ */
+size_t cq_decode_attn_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim,
+                                      int c, int b, int64_t max_tokens);
+
+/*
+ * Single-query decode attention over a CQ-coded cache.  For sequence s and query
+ * head hq (which reads KV head hq / (n_q_heads / n_kv_heads)), over the first
+ * n = seq_lens[s] cached tokens:
+ *
+ *   s_t = scale * <q, Khat_t>,  p = softmax(s_0..s_{n-1}),  out = sum_t p_t Vhat_t     (Eq. 1)
+ *
+ * where Khat_t / Vhat_t are the CQ reconstructions of token t (Section 3.2).  The
+ * kernels never form Khat or Vhat: scores are sums over groups of a per-query table
+ * LUT[g][j] = scale * <q_g, k_cb[g][j]>, softmax is online over context splits,
+ * softmax weights are accumulated in bins per V code and the bins are multiplied
+ * by the V centroids -- an exact re-association of Eq. 1, evaluated in fp32.
+ *
+ *   q_fp16     [n_seq][n_q_heads][head_dim] fp16
+ *   k_codes, v_codes   code buffers in the library layout, capacity max_tokens,
+ *                      n_kv_heads heads, 16-byte aligned
+ *   k_cb, v_cb [n_kv_heads][G][2^b][c] fp32
+ *   seq_lens   [n_seq] int32, each in [0, max_tokens]; values outside are clamped;
+ *              seq_lens[s] == 0 gives a zero output row
+ *   out        [n_seq][n_q_heads][head_dim] fp32
+ *   workspace  at least cq_decode_attn_workspace_bytes(...) bytes, 16-byte aligned;
+ *              contents on entry are ignored
+ */
+int cq_decode_attn(const void *q_fp16, const void *k_codes, const void *v_codes,
+                   const float *k_cb, const float *v_cb, const int32_t *seq_lens, float scale,
+                   int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                   int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
+                   void *stream);
+
+/*
+ * Same operation with an explicit kernel choice, for tests and benchmarks:
+ * variant 0 = automatic (what cq_decode_attn uses), 1 = generic kernel,
+ * 2 = tuned kernel (CQ_ERR_UNSUPPORTED when the shape has none).
+ */
+int cq_decode_attn_variant(const void *q_fp16, const void *k_codes, const void *v_codes,
+                           const float *k_cb, const float *v_cb, const int32_t *seq_lens, float scale,
+                           int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                           int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
+                           int variant, void *stream);
+
+/* cq_encode with an explicit kernel choice (same variant numbers). */
+int cq_encode_variant(const void *x_fp16, const float *codebooks, const int32_t *seq_offsets,
+                      int64_t n_seq, int64_t n_tokens, int64_t token_offset, int64_t max_tokens,
+                      int n_heads, int head_dim, int c, int b, void *codes_out, int variant,
+                      void *stream);
+
+/*
+ * One decode step of one layer driven from HOST buffers (the end-to-end path):
+ * copies the step's query and the new token's key and value vectors to the
+ * device, appends the new token's codes at position seq_lens_host[s] of every
+ * sequence (cq_encode), attends over seq_lens_host[s] + 1 tokens (cq_decode_attn)
+ * and copies the result back.  Synchronises `stream` before returning.
+ *
+ *   q_host       [n_seq][n_q_heads][head_dim] fp16   (pinned memory recommended)
+ *   k_new_host, v_new_host   [n_seq][n_kv_heads][head_dim] fp16
+ *   seq_lens_host [n_seq] int32: tokens already cached, each < max_tokens
+ *   k_codes, v_codes, k_cb, v_cb   device, as in cq_decode_attn (codes are updated)
+ *   out_host     [n_seq][n_q_heads][head_dim] fp32
+ *   workspace    device, at least cq_decode_step_host_workspace_bytes(...) bytes
+ */
+size_t cq_decode_step_host_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim,
+                                           int c, int b, int64_t max_tokens);
+int cq_decode_step_host(const void *q_host, const void *k_new_host, const void *v_new_host,
+                        const int32_t *seq_lens_host, void *k_codes, void *v_codes,
+                        const float *k_cb, const float *v_cb, float scale,
+                        int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                        int64_t max_tokens, float *out_host, void *workspace, size_t workspace_bytes,
+                        void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CQ_H_ */

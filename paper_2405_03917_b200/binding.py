@@ -1,0 +1,209 @@
+"""ctypes binding of `libcq.so`: argument marshalling only, same names as the C ABI.
+
+Every function takes torch tensors (device tensors for device pointers, CPU tensors for
+the `_host` arguments), checks dtype / contiguity / device, and forwards raw pointers and
+sizes.  A non-zero cq_status raises CQError.  Work is enqueued on torch's current stream.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libcq.so")
+
+# Every symbol include/cq.h declares.
+EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant",
+           "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
+           "cq_decode_attn_variant", "cq_decode_step_host_workspace_bytes", "cq_decode_step_host"]
+
+
+class CQError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {cq_status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2405_03917_b200.build` "
+                              "(needs nvcc); this package has no CPU or PyTorch fallback")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i64, i32, f32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.cq_layout_version.restype = i32
+        L.cq_status_string.restype = ctypes.c_char_p
+        L.cq_status_string.argtypes = [i32]
+        L.cq_codes_bytes.restype = sz
+        L.cq_codes_bytes.argtypes = [i64, i64, i32, i32, i32, i32]
+        L.cq_encode.restype = i32
+        L.cq_encode.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, i32, i32, i32, vp, vp]
+        L.cq_encode_variant.restype = i32
+        L.cq_encode_variant.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, i32, i32, i32, vp, i32, vp]
+        for f in (L.cq_codes_to_rowmajor, L.cq_codes_from_rowmajor):
+            f.restype = i32
+            f.argtypes = [vp, i64, i64, i32, i32, i32, i32, vp, vp]
+        L.cq_decode_attn_workspace_bytes.restype = sz
+        L.cq_decode_attn_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
+        L.cq_decode_attn.restype = i32
+        L.cq_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp, sz, vp]
+        L.cq_decode_attn_variant.restype = i32
+        L.cq_decode_attn_variant.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp,
+                                             sz, i32, vp]
+        L.cq_decode_step_host_workspace_bytes.restype = sz
+        L.cq_decode_step_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
+        L.cq_decode_step_host.restype = i32
+        L.cq_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64,
+                                          vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name}: CUDA tensor expected")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: contiguous {dtype} tensor expected, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _host(t: torch.Tensor, dtype, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError(f"{name}: CPU tensor expected")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: contiguous {dtype} tensor expected, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise CQError(status, where)
+
+
+def cq_layout_version() -> int:
+    return int(lib().cq_layout_version())
+
+
+def cq_status_string(status: int) -> str:
+    return lib().cq_status_string(int(status)).decode()
+
+
+def cq_codes_bytes(n_seq: int, max_tokens: int, n_heads: int, head_dim: int, c: int, b: int) -> int:
+    return int(lib().cq_codes_bytes(n_seq, max_tokens, n_heads, head_dim, c, b))
+
+
+def cq_encode(x: torch.Tensor, codebooks: torch.Tensor, c: int, b: int, codes_out: torch.Tensor, max_tokens: int,
+              token_offset: int = 0, seq_offsets: Optional[torch.Tensor] = None, variant: int = 0) -> torch.Tensor:
+    """x fp16 (n_seq, n_tokens, n_heads, head_dim); codebooks fp32 (n_heads, G, 2^b, c);
+    codes_out uint8 buffer of cq_codes_bytes(...) bytes, updated in place and returned."""
+    n_seq, n_tokens, n_heads, head_dim = x.shape
+    if tuple(codebooks.shape) != (n_heads, head_dim // max(c, 1), 1 << b, c):
+        raise ValueError(f"codebooks shape {tuple(codebooks.shape)} does not match heads/groups/centroids")
+    need = cq_codes_bytes(n_seq, max_tokens, n_heads, head_dim, c, b)
+    if need and codes_out.numel() < need:
+        raise ValueError(f"codes_out holds {codes_out.numel()} bytes, {need} needed")
+    so = None if seq_offsets is None else _dev(seq_offsets, torch.int32, "seq_offsets")
+    if seq_offsets is not None and seq_offsets.numel() != n_seq:
+        raise ValueError("seq_offsets must have n_seq entries")
+    st = lib().cq_encode_variant(_dev(x, torch.float16, "x"), _dev(codebooks, torch.float32, "codebooks"), so,
+                                 n_seq, n_tokens, token_offset, max_tokens, n_heads, head_dim, c, b,
+                                 _dev(codes_out, torch.uint8, "codes_out"), variant, _stream())
+    _check(st, "cq_encode")
+    return codes_out
+
+
+def cq_codes_to_rowmajor(codes: torch.Tensor, n_seq: int, max_tokens: int, n_heads: int, head_dim: int, c: int,
+                         b: int) -> torch.Tensor:
+    out = torch.empty(n_seq, max_tokens, n_heads, head_dim // c, dtype=torch.uint8, device=codes.device)
+    st = lib().cq_codes_to_rowmajor(_dev(codes, torch.uint8, "codes"), n_seq, max_tokens, n_heads, head_dim, c, b,
+                                    out.data_ptr(), _stream())
+    _check(st, "cq_codes_to_rowmajor")
+    return out
+
+
+def cq_codes_from_rowmajor(rowmajor: torch.Tensor, head_dim: int, c: int, b: int) -> torch.Tensor:
+    n_seq, max_tokens, n_heads, G = rowmajor.shape
+    if G * c != head_dim:
+        raise ValueError("last dimension must be head_dim / c")
+    out = torch.empty(cq_codes_bytes(n_seq, max_tokens, n_heads, head_dim, c, b), dtype=torch.uint8,
+                      device=rowmajor.device)
+    st = lib().cq_codes_from_rowmajor(_dev(rowmajor, torch.uint8, "rowmajor"), n_seq, max_tokens, n_heads, head_dim,
+                                      c, b, out.data_ptr(), _stream())
+    _check(st, "cq_codes_from_rowmajor")
+    return out
+
+
+def cq_decode_attn_workspace_bytes(n_seq: int, n_q_heads: int, n_kv_heads: int, head_dim: int, c: int, b: int,
+                                   max_tokens: int) -> int:
+    return int(lib().cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens))
+
+
+def cq_decode_attn(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor,
+                   v_cb: torch.Tensor, seq_lens: torch.Tensor, scale: float, c: int, b: int, max_tokens: int,
+                   out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   variant: int = 0) -> torch.Tensor:
+    """q fp16 (n_seq, Hq, head_dim); codes in the library layout; codebooks fp32
+    (Hkv, G, 2^b, c); seq_lens int32 (n_seq,).  Returns out fp32 (n_seq, Hq, head_dim)."""
+    n_seq, n_q_heads, head_dim = q.shape
+    n_kv_heads = k_cb.shape[0]
+    for nm, cb in (("k_cb", k_cb), ("v_cb", v_cb)):
+        if tuple(cb.shape) != (n_kv_heads, head_dim // max(c, 1), 1 << b, c):
+            raise ValueError(f"{nm} shape {tuple(cb.shape)} does not match heads/groups/centroids")
+    need_codes = cq_codes_bytes(n_seq, max_tokens, n_kv_heads, head_dim, c, b)
+    if need_codes and (k_codes.numel() < need_codes or v_codes.numel() < need_codes):
+        raise ValueError(f"code buffers must hold {need_codes} bytes")
+    if seq_lens.numel() != n_seq:
+        raise ValueError("seq_lens must have n_seq entries")
+    if out is None:
+        out = torch.empty(n_seq, n_q_heads, head_dim, dtype=torch.float32, device=q.device)
+    if workspace is None:
+        nbytes = cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens)
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    st = lib().cq_decode_attn_variant(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+                                      _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
+                                      _dev(v_cb, torch.float32, "v_cb"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                      float(scale), n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
+                                      _dev(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
+                                      workspace.numel(), variant, _stream())
+    _check(st, "cq_decode_attn")
+    return out
+
+
+def cq_decode_step_host_workspace_bytes(n_seq: int, n_q_heads: int, n_kv_heads: int, head_dim: int, c: int, b: int,
+                                        max_tokens: int) -> int:
+    return int(lib().cq_decode_step_host_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens))
+
+
+def cq_decode_step_host(q_host: torch.Tensor, k_new_host: torch.Tensor, v_new_host: torch.Tensor,
+                        seq_lens_host: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor,
+                        k_cb: torch.Tensor, v_cb: torch.Tensor, scale: float, c: int, b: int, max_tokens: int,
+                        out_host: torch.Tensor, workspace: torch.Tensor) -> torch.Tensor:
+    """One decode step from host buffers: H2D copies, append-encode, attention, D2H copy, stream sync."""
+    n_seq, n_q_heads, head_dim = q_host.shape
+    n_kv_heads = k_cb.shape[0]
+    st = lib().cq_decode_step_host(_host(q_host, torch.float16, "q_host"), _host(k_new_host, torch.float16, "k_new_host"),
+                                   _host(v_new_host, torch.float16, "v_new_host"),
+                                   _host(seq_lens_host, torch.int32, "seq_lens_host"),
+                                   _dev(k_codes, torch.uint8, "k_codes"), _dev(v_codes, torch.uint8, "v_codes"),
+                                   _dev(k_cb, torch.float32, "k_cb"), _dev(v_cb, torch.float32, "v_cb"), float(scale),
+                                   n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
+                                   _host(out_host, torch.float32, "out_host"),
+                                   _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream())
+    _check(st, "cq_decode_step_host")
+    return out_host

@@ -1,0 +1,250 @@
+// extern "C" entry points of the CQ library: host-side validation and dispatch only.
+#include "cq_common.cuh"
+
+using namespace cq;
+
+namespace {
+
+constexpr int kMaxHeadDim = 256;
+constexpr int64_t kGenericMaxTableEntries = 24576;   // (G * 2^b) floats x 2 tables must fit shared memory
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates the quantiser shape and fills `sh`; n_q_heads == n_kv_heads for encode-side calls.
+int make_shape(int64_t n_seq, int64_t max_tokens, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+               Shape* sh)
+{
+    if (n_seq <= 0 || max_tokens <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0 || c <= 0)
+        return CQ_ERR_SHAPE;
+    if (head_dim % c != 0 || n_q_heads % n_kv_heads != 0) return CQ_ERR_SHAPE;
+    if (b < 1 || b > 8 || head_dim > kMaxHeadDim) return CQ_ERR_UNSUPPORTED;
+    if (n_seq * (int64_t)n_q_heads > (int64_t)1 << 24) return CQ_ERR_UNSUPPORTED;
+    sh->n_seq = n_seq;
+    sh->max_tokens = max_tokens;
+    sh->n_blocks = (max_tokens + kTokenBlock - 1) / kTokenBlock;
+    sh->n_q_heads = n_q_heads;
+    sh->n_kv_heads = n_kv_heads;
+    sh->head_dim = head_dim;
+    sh->c = c;
+    sh->b = b;
+    sh->G = head_dim / c;
+    sh->K = 1 << b;
+    sh->R = n_q_heads / n_kv_heads;
+    return CQ_OK;
+}
+
+// Partial slots per (sequence, query head) that the workspace must hold for any variant.
+int max_parts(const Shape& sh)
+{
+    int p = decode_generic_splits(sh);
+    if (decode_tuned_supported(sh)) {
+        const int t = decode_tuned_parts(sh);
+        if (t > p) p = t;
+    }
+    return p;
+}
+
+size_t partial_bytes(const Shape& sh)
+{
+    return (size_t)sh.n_seq * sh.n_q_heads * max_parts(sh) * partial_stride(sh.head_dim) * sizeof(float);
+}
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+int cq_layout_version(void) { return 1; }
+
+const char* cq_status_string(int status)
+{
+    switch (status) {
+        case CQ_OK: return "CQ_OK";
+        case CQ_ERR_NULL: return "CQ_ERR_NULL: a required pointer is NULL";
+        case CQ_ERR_SHAPE: return "CQ_ERR_SHAPE: invalid dimensions or token range";
+        case CQ_ERR_UNSUPPORTED: return "CQ_ERR_UNSUPPORTED: shape outside what the library was built for";
+        case CQ_ERR_ALIGN: return "CQ_ERR_ALIGN: pointer not 16-byte aligned";
+        case CQ_ERR_WORKSPACE: return "CQ_ERR_WORKSPACE: workspace too small";
+        case CQ_ERR_CUDA: return "CQ_ERR_CUDA: CUDA runtime error";
+        default: return "unknown cq_status";
+    }
+}
+
+size_t cq_codes_bytes(int64_t n_seq, int64_t max_tokens, int n_heads, int head_dim, int c, int b)
+{
+    Shape sh;
+    if (make_shape(n_seq, max_tokens, n_heads, n_heads, head_dim, c, b, &sh) != CQ_OK) return 0;
+    return (size_t)sh.n_seq * n_heads * sh.n_blocks * sh.G * kTokenBlock;
+}
+
+int cq_encode_variant(const void* x_fp16, const float* codebooks, const int32_t* seq_offsets, int64_t n_seq,
+                      int64_t n_tokens, int64_t token_offset, int64_t max_tokens, int n_heads, int head_dim, int c,
+                      int b, void* codes_out, int variant, void* stream)
+{
+    if (!x_fp16 || !codebooks || !codes_out) return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_heads, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (n_tokens < 0 || token_offset < 0) return CQ_ERR_SHAPE;
+    if (!seq_offsets && token_offset + n_tokens > max_tokens) return CQ_ERR_SHAPE;
+    if (!aligned16(x_fp16) || !aligned16(codebooks) || !aligned16(codes_out)) return CQ_ERR_ALIGN;
+    if (variant < 0 || variant > 2) return CQ_ERR_SHAPE;
+    if (n_tokens == 0) return CQ_OK;
+    const bool tuned_ok = encode_tuned_supported(sh);
+    if (variant == 2 && !tuned_ok) return CQ_ERR_UNSUPPORTED;
+    const bool use_tuned = variant == 2 || (variant == 0 && tuned_ok);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    cudaError_t e = use_tuned
+                        ? launch_encode_tuned(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh, n_tokens,
+                                              token_offset, static_cast<uint8_t*>(codes_out), cs)
+                        : launch_encode_generic(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh,
+                                                n_tokens, token_offset, static_cast<uint8_t*>(codes_out), cs);
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_encode(const void* x_fp16, const float* codebooks, const int32_t* seq_offsets, int64_t n_seq, int64_t n_tokens,
+              int64_t token_offset, int64_t max_tokens, int n_heads, int head_dim, int c, int b, void* codes_out,
+              void* stream)
+{
+    return cq_encode_variant(x_fp16, codebooks, seq_offsets, n_seq, n_tokens, token_offset, max_tokens, n_heads,
+                             head_dim, c, b, codes_out, 0, stream);
+}
+
+int cq_codes_to_rowmajor(const void* codes, int64_t n_seq, int64_t max_tokens, int n_heads, int head_dim, int c,
+                         int b, void* rowmajor_out, void* stream)
+{
+    if (!codes || !rowmajor_out) return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_heads, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (!aligned16(codes)) return CQ_ERR_ALIGN;
+    cudaError_t e = launch_to_rowmajor(static_cast<const uint8_t*>(codes), sh, static_cast<uint8_t*>(rowmajor_out),
+                                       static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_codes_from_rowmajor(const void* rowmajor, int64_t n_seq, int64_t max_tokens, int n_heads, int head_dim, int c,
+                           int b, void* codes_out, void* stream)
+{
+    if (!rowmajor || !codes_out) return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_heads, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (!aligned16(codes_out)) return CQ_ERR_ALIGN;
+    cudaError_t e = launch_from_rowmajor(static_cast<const uint8_t*>(rowmajor), sh, static_cast<uint8_t*>(codes_out),
+                                         static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+size_t cq_decode_attn_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                                      int64_t max_tokens)
+{
+    Shape sh;
+    if (make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh) != CQ_OK) return 0;
+    return round_up(partial_bytes(sh), 256);
+}
+
+int cq_decode_attn_variant(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
+                           const float* v_cb, const int32_t* seq_lens, float scale, int n_seq, int n_q_heads,
+                           int n_kv_heads, int head_dim, int c, int b, int64_t max_tokens, float* out, void* workspace,
+                           size_t workspace_bytes, int variant, void* stream)
+{
+    if (!q_fp16 || !k_codes || !v_codes || !k_cb || !v_cb || !seq_lens || !out || !workspace) return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (variant < 0 || variant > 2) return CQ_ERR_SHAPE;
+    if (!aligned16(k_codes) || !aligned16(v_codes) || !aligned16(workspace) || !aligned16(k_cb) || !aligned16(v_cb) ||
+        (reinterpret_cast<uintptr_t>(q_fp16) & 1u) || (reinterpret_cast<uintptr_t>(out) & 3u))
+        return CQ_ERR_ALIGN;
+    if (workspace_bytes < round_up(partial_bytes(sh), 256)) return CQ_ERR_WORKSPACE;
+    const bool tuned_ok = decode_tuned_supported(sh);
+    if (variant == 2 && !tuned_ok) return CQ_ERR_UNSUPPORTED;
+    const bool use_tuned = variant == 2 || (variant == 0 && tuned_ok);
+    if (!use_tuned && (int64_t)sh.G * sh.K > kGenericMaxTableEntries) return CQ_ERR_UNSUPPORTED;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const __half* q = static_cast<const __half*>(q_fp16);
+    const uint8_t* kc = static_cast<const uint8_t*>(k_codes);
+    const uint8_t* vc = static_cast<const uint8_t*>(v_codes);
+    float* partials = static_cast<float*>(workspace);
+    cudaError_t e = use_tuned ? launch_decode_tuned(q, kc, vc, k_cb, v_cb, seq_lens, scale, sh, out, partials, cs)
+                              : launch_decode_generic(q, kc, vc, k_cb, v_cb, seq_lens, scale, sh, out, partials, cs);
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_decode_attn(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb, const float* v_cb,
+                   const int32_t* seq_lens, float scale, int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c,
+                   int b, int64_t max_tokens, float* out, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return cq_decode_attn_variant(q_fp16, k_codes, v_codes, k_cb, v_cb, seq_lens, scale, n_seq, n_q_heads, n_kv_heads,
+                                  head_dim, c, b, max_tokens, out, workspace, workspace_bytes, 0, stream);
+}
+
+// Staging area of cq_decode_step_host inside the caller's workspace (all 256-byte aligned):
+//   [q fp16][k_new fp16][v_new fp16][seq_lens int32][seq_lens+1 int32][out fp32][attention workspace]
+size_t cq_decode_step_host_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                                           int64_t max_tokens)
+{
+    const size_t attn = cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens);
+    if (attn == 0) return 0;
+    const size_t q = round_up((size_t)n_seq * n_q_heads * head_dim * 2, 256);
+    const size_t kv = round_up((size_t)n_seq * n_kv_heads * head_dim * 2, 256);
+    const size_t sl = round_up((size_t)n_seq * 4, 256);
+    const size_t o = round_up((size_t)n_seq * n_q_heads * head_dim * 4, 256);
+    return q + 2 * kv + 2 * sl + o + attn;
+}
+
+int cq_decode_step_host(const void* q_host, const void* k_new_host, const void* v_new_host,
+                        const int32_t* seq_lens_host, void* k_codes, void* v_codes, const float* k_cb,
+                        const float* v_cb, float scale, int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c,
+                        int b, int64_t max_tokens, float* out_host, void* workspace, size_t workspace_bytes,
+                        void* stream)
+{
+    if (!q_host || !k_new_host || !v_new_host || !seq_lens_host || !k_codes || !v_codes || !k_cb || !v_cb ||
+        !out_host || !workspace)
+        return CQ_ERR_NULL;
+    const size_t need = cq_decode_step_host_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens);
+    if (need == 0) {
+        Shape sh;
+        return make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
+    }
+    if (workspace_bytes < need) return CQ_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return CQ_ERR_ALIGN;
+    for (int s = 0; s < n_seq; ++s)
+        if (seq_lens_host[s] < 0 || seq_lens_host[s] >= max_tokens) return CQ_ERR_SHAPE;
+
+    const size_t qb = (size_t)n_seq * n_q_heads * head_dim * 2;
+    const size_t kvb = (size_t)n_seq * n_kv_heads * head_dim * 2;
+    const size_t slb = (size_t)n_seq * 4;
+    const size_t ob = (size_t)n_seq * n_q_heads * head_dim * 4;
+    char* w = static_cast<char*>(workspace);
+    char* d_q = w;                 w += round_up(qb, 256);
+    char* d_k = w;                 w += round_up(kvb, 256);
+    char* d_v = w;                 w += round_up(kvb, 256);
+    int32_t* d_sl = reinterpret_cast<int32_t*>(w);   w += round_up(slb, 256);
+    int32_t* d_sl1 = reinterpret_cast<int32_t*>(w);  w += round_up(slb, 256);
+    float* d_out = reinterpret_cast<float*>(w);      w += round_up(ob, 256);
+    void* attn_ws = w;
+    const size_t attn_bytes = workspace_bytes - (size_t)(w - static_cast<char*>(workspace));
+
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    // The new token is appended at position seq_lens[s]; the attention then reads seq_lens[s] + 1 tokens.
+    if (cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    if (cudaMemcpyAsync(d_k, k_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    if (cudaMemcpyAsync(d_v, v_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    if (cudaMemcpyAsync(d_sl, seq_lens_host, slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    int st = cq_encode(d_k, k_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, k_codes, stream);
+    if (st != CQ_OK) return st;
+    st = cq_encode(d_v, v_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, v_codes, stream);
+    if (st != CQ_OK) return st;
+    if (launch_add_one(d_sl, d_sl1, n_seq, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    st = cq_decode_attn(d_q, k_codes, v_codes, k_cb, v_cb, d_sl1, scale, n_seq, n_q_heads, n_kv_heads, head_dim, c, b,
+                        max_tokens, d_out, attn_ws, attn_bytes, stream);
+    if (st != CQ_OK) return st;
+    if (cudaMemcpyAsync(out_host, d_out, ob, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return CQ_ERR_CUDA;
+    return CQ_OK;
+}
+
+}  // extern "C"

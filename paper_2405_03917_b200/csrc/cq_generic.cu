@@ -1,0 +1,309 @@
+// Generic sm_100a kernels of the CQ library: they accept every supported (head_dim, c, b)
+// and favour plainness over speed.  The tuned kernels live in cq_encode.cu / cq_decode.cu.
+#include "cq_common.cuh"
+
+namespace cq {
+
+// ------------------------------------------------------------------------------------------
+// Encode (Section 3.2 of the paper): nearest centroid in L2 per group of c contiguous channels.
+// One thread per (sequence, head, group, token); the token index is the fastest-varying one
+// so that a warp reads one codebook (broadcast) and writes consecutive bytes of a code word.
+// ------------------------------------------------------------------------------------------
+__global__ void encode_generic_kernel(const __half* __restrict__ x, const float* __restrict__ cb,
+                                      const int32_t* __restrict__ seq_offsets, Shape sh, int64_t n_tokens,
+                                      int64_t token_offset, uint8_t* __restrict__ codes)
+{
+    const int n_heads = sh.n_kv_heads;
+    const int64_t total = sh.n_seq * n_heads * sh.G * n_tokens;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = idx % n_tokens;
+        int64_t rest = idx / n_tokens;
+        const int g = (int)(rest % sh.G);
+        rest /= sh.G;
+        const int h = (int)(rest % n_heads);
+        const int64_t s = rest / n_heads;
+        const int64_t pos = token_offset + (seq_offsets ? seq_offsets[s] : 0) + i;
+        if (pos < 0 || pos >= sh.max_tokens) continue;
+        const __half* xv = x + ((s * n_tokens + i) * n_heads + h) * (int64_t)sh.head_dim + g * sh.c;
+        const float* cg = cb + ((int64_t)h * sh.G + g) * sh.K * sh.c;
+        float best = INFINITY;
+        int arg = 0;
+        for (int j = 0; j < sh.K; ++j) {
+            float d = 0.f;
+            for (int k = 0; k < sh.c; ++k) {
+                const float diff = __half2float(xv[k]) - cg[j * sh.c + k];
+                d = fmaf(diff, diff, d);
+            }
+            if (d < best) {   // strict: lowest index wins exact ties
+                best = d;
+                arg = j;
+            }
+        }
+        codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + pos % kTokenBlock] = (uint8_t)arg;
+    }
+}
+
+cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
+                                  int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st)
+{
+    const int64_t total = sh.n_seq * sh.n_kv_heads * sh.G * n_tokens;
+    if (total == 0) return cudaSuccess;
+    const int threads = 256;
+    const int64_t blocks = (total + threads - 1) / threads;
+    const int grid = (int)(blocks < 148 * 64 ? blocks : 148 * 64);
+    encode_generic_kernel<<<grid, threads, 0, st>>>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Layout converters between the library layout and [n_seq][max_tokens][n_heads][G].
+// One thread per code word (16 tokens of one group).
+// ------------------------------------------------------------------------------------------
+__global__ void to_rowmajor_kernel(const uint8_t* __restrict__ codes, Shape sh, uint8_t* __restrict__ rm)
+{
+    const int n_heads = sh.n_kv_heads;
+    const int64_t words = sh.n_seq * n_heads * sh.n_blocks * sh.G;
+    for (int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; w < words; w += (int64_t)gridDim.x * blockDim.x) {
+        const int g = (int)(w % sh.G);
+        int64_t rest = w / sh.G;
+        const int64_t blk = rest % sh.n_blocks;
+        rest /= sh.n_blocks;
+        const int h = (int)(rest % n_heads);
+        const int64_t s = rest / n_heads;
+        const uint8_t* src = codes + w * kTokenBlock;
+        for (int k = 0; k < kTokenBlock; ++k) {
+            const int64_t t = blk * kTokenBlock + k;
+            if (t < sh.max_tokens) rm[((s * sh.max_tokens + t) * n_heads + h) * sh.G + g] = src[k];
+        }
+    }
+}
+
+__global__ void from_rowmajor_kernel(const uint8_t* __restrict__ rm, Shape sh, uint8_t* __restrict__ codes)
+{
+    const int n_heads = sh.n_kv_heads;
+    const int64_t words = sh.n_seq * n_heads * sh.n_blocks * sh.G;
+    for (int64_t w = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; w < words; w += (int64_t)gridDim.x * blockDim.x) {
+        const int g = (int)(w % sh.G);
+        int64_t rest = w / sh.G;
+        const int64_t blk = rest % sh.n_blocks;
+        rest /= sh.n_blocks;
+        const int h = (int)(rest % n_heads);
+        const int64_t s = rest / n_heads;
+        uint8_t* dst = codes + w * kTokenBlock;
+        for (int k = 0; k < kTokenBlock; ++k) {
+            const int64_t t = blk * kTokenBlock + k;
+            dst[k] = t < sh.max_tokens ? rm[((s * sh.max_tokens + t) * n_heads + h) * sh.G + g] : (uint8_t)0;
+        }
+    }
+}
+
+__global__ void add_one_kernel(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int n)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = src[i] + 1;
+}
+
+cudaError_t launch_add_one(const int32_t* src, int32_t* dst, int n, cudaStream_t st)
+{
+    add_one_kernel<<<(n + 255) / 256, 256, 0, st>>>(src, dst, n);
+    return cudaGetLastError();
+}
+
+static int words_grid(const Shape& sh)
+{
+    const int64_t words = sh.n_seq * sh.n_kv_heads * sh.n_blocks * sh.G;
+    const int64_t blocks = (words + 255) / 256;
+    return (int)(blocks < 148 * 32 ? (blocks > 0 ? blocks : 1) : 148 * 32);
+}
+
+cudaError_t launch_to_rowmajor(const uint8_t* codes, const Shape& sh, uint8_t* rowmajor, cudaStream_t st)
+{
+    to_rowmajor_kernel<<<words_grid(sh), 256, 0, st>>>(codes, sh, rowmajor);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_from_rowmajor(const uint8_t* rowmajor, const Shape& sh, uint8_t* codes, cudaStream_t st)
+{
+    from_rowmajor_kernel<<<words_grid(sh), 256, 0, st>>>(rowmajor, sh, codes);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Decode attention, generic form.  One CTA per (context split, query head, sequence):
+//   LUT[g][j] = scale*log2(e) * <q_g, Ck[g][j]>            (scores live in the log2 domain)
+//   per tile of blockDim tokens: s_t = sum_g LUT[g][kcode], online max, p_t = 2^(s_t - m),
+//   bins[g][vcode] += p_t (shared-memory float atomics)
+//   acc[g*c+i] = sum_j bins[g][j] * Cv[g][j][i];  partial = (m, l, acc)
+// The partials of all splits are merged by merge_kernel.
+// ------------------------------------------------------------------------------------------
+constexpr int kGenericThreads = 256;
+
+__device__ inline float block_reduce_max(float v, float* red)
+{
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = red[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = fmaxf(r, red[w]);
+    __syncthreads();
+    return r;
+}
+
+__device__ inline float block_reduce_sum(float v, float* red)
+{
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) r += red[w];
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(kGenericThreads)
+decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
+                      const float* __restrict__ kcb, const float* __restrict__ vcb,
+                      const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int n_splits,
+                      float* __restrict__ partials)
+{
+    extern __shared__ __align__(16) float smem_f[];
+    float* lut = smem_f;                       // [G][K]
+    float* bins = lut + sh.G * sh.K;           // [G][K]
+    __shared__ float red[kGenericThreads / 32];
+
+    const int split = blockIdx.x % n_splits;
+    const int hq = (blockIdx.x / n_splits) % sh.n_q_heads;
+    const int64_t s = blockIdx.x / (n_splits * sh.n_q_heads);
+    const int hkv = hq / sh.R;
+    const int GK = sh.G * sh.K;
+
+    int64_t n = seq_lens[s];
+    n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
+    const int64_t nblk = (n + kTokenBlock - 1) / kTokenBlock;
+    const int64_t t_begin = nblk * split / n_splits * kTokenBlock;
+    int64_t t_end = nblk * (split + 1) / n_splits * kTokenBlock;
+    if (t_end > n) t_end = n;
+
+    float* part = partials + ((s * sh.n_q_heads + hq) * n_splits + split) * (int64_t)partial_stride(sh.head_dim);
+    if (t_end <= t_begin) {          // empty split: neutral element of the merge
+        if (threadIdx.x == 0) { part[0] = -INFINITY; part[1] = 0.f; }
+        for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) part[2 + d] = 0.f;
+        return;
+    }
+
+    const __half* qv = q + (s * sh.n_q_heads + hq) * (int64_t)sh.head_dim;
+    for (int e = threadIdx.x; e < GK; e += blockDim.x) {
+        const int g = e / sh.K;
+        const float* cj = kcb + ((int64_t)hkv * GK + e) * sh.c;
+        float dot = 0.f;
+        for (int k = 0; k < sh.c; ++k) dot = fmaf(__half2float(qv[g * sh.c + k]), cj[k], dot);
+        lut[e] = dot * scale_log2e;
+        bins[e] = 0.f;
+    }
+    __syncthreads();
+
+    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    float m_run = -INFINITY;
+    float l_thr = 0.f;
+    for (int64_t t0 = t_begin; t0 < t_end; t0 += blockDim.x) {
+        const int64_t t = t0 + threadIdx.x;
+        const bool valid = t < t_end;
+        const int64_t word0 = (t / kTokenBlock) * sh.G * kTokenBlock + t % kTokenBlock;
+        float sc = -INFINITY;
+        if (valid) {
+            sc = 0.f;
+            for (int g = 0; g < sh.G; ++g) sc += lut[g * sh.K + kbase[word0 + g * kTokenBlock]];
+        }
+        const float m_tile = block_reduce_max(sc, red);
+        if (m_tile > m_run) {
+            const float f = exp2f(m_run - m_tile);      // 0 when m_run is -inf
+            for (int e = threadIdx.x; e < GK; e += blockDim.x) bins[e] *= f;
+            l_thr *= f;
+            m_run = m_tile;
+            __syncthreads();
+        }
+        if (valid) {
+            const float p = exp2f(sc - m_run);
+            l_thr += p;
+            for (int g = 0; g < sh.G; ++g) atomicAdd(&bins[g * sh.K + vbase[word0 + g * kTokenBlock]], p);
+        }
+        __syncthreads();
+    }
+    const float l = block_reduce_sum(l_thr, red);
+    if (threadIdx.x == 0) { part[0] = m_run; part[1] = l; }
+    for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) {
+        const int g = d / sh.c, k = d % sh.c;
+        const float* cv = vcb + ((int64_t)hkv * GK + g * sh.K) * sh.c + k;
+        float a = 0.f;
+        for (int j = 0; j < sh.K; ++j) a = fmaf(bins[g * sh.K + j], cv[j * sh.c], a);
+        part[2 + d] = a;
+    }
+}
+
+int decode_generic_splits(const Shape& sh)
+{
+    // enough CTAs for a few waves of 148 SMs, at least 256 tokens per split
+    const int64_t items = sh.n_seq * sh.n_q_heads;
+    int64_t want = (148 * 8 + items - 1) / (items > 0 ? items : 1);
+    const int64_t cap = (sh.max_tokens + 255) / 256;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    return (int)want;
+}
+
+// out[d] = sum_p 2^(m_p - M) acc_p[d] / sum_p 2^(m_p - M) l_p,  M = max_p m_p  (log-sum-exp merge)
+__global__ void merge_kernel(const float* __restrict__ partials, int n_parts, Shape sh, float* __restrict__ out)
+{
+    const int hq = blockIdx.x % sh.n_q_heads;
+    const int64_t s = blockIdx.x / sh.n_q_heads;
+    const int stride = partial_stride(sh.head_dim);
+    const float* base = partials + (s * sh.n_q_heads + hq) * (int64_t)n_parts * stride;
+    float M = -INFINITY;
+    for (int p = 0; p < n_parts; ++p) M = fmaxf(M, base[p * stride]);
+    float* o = out + (s * sh.n_q_heads + hq) * (int64_t)sh.head_dim;
+    if (M == -INFINITY) {           // empty context
+        for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) o[d] = 0.f;
+        return;
+    }
+    float L = 0.f;
+    for (int p = 0; p < n_parts; ++p) {
+        const float m = base[p * stride];
+        if (m != -INFINITY) L += exp2f(m - M) * base[p * stride + 1];
+    }
+    for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) {
+        float a = 0.f;
+        for (int p = 0; p < n_parts; ++p) {
+            const float m = base[p * stride];
+            if (m != -INFINITY) a = fmaf(exp2f(m - M), base[p * stride + 2 + d], a);
+        }
+        o[d] = a / L;
+    }
+}
+
+cudaError_t launch_merge(const float* partials, int n_parts, const Shape& sh, float* out, cudaStream_t st)
+{
+    const unsigned grid = (unsigned)(sh.n_q_heads * sh.n_seq);
+    merge_kernel<<<grid, 128, 0, st>>>(partials, n_parts, sh, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
+                                  const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
+                                  float* out, float* partials, cudaStream_t st)
+{
+    const int n_splits = decode_generic_splits(sh);
+    const size_t smem = (size_t)2 * sh.G * sh.K * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(decode_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)(n_splits * sh.n_q_heads * sh.n_seq);
+    decode_generic_kernel<<<grid, kGenericThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
+                                                               n_splits, partials);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_merge(partials, n_splits, sh, out, st);
+}
+
+}  // namespace cq

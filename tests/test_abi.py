@@ -1,0 +1,96 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every
+symbol the header declares, sizes follow the documented layout, and invalid
+arguments are rejected before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2405_03917_b200 as cq
+from paper_2405_03917_b200 import build as cq_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    cq_build.build()
+    return cq.lib()
+
+
+def header_functions():
+    text = open(os.path.join(ROOT, "include", "cq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cq_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = header_functions()
+    assert len(names) >= 10
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in include/cq.h but not exported"
+    assert sorted(cq.EXPORTS) == names
+
+
+def test_layout_version_and_status_strings(L):
+    assert cq.cq_layout_version() == 1
+    assert cq.cq_status_string(0) == "CQ_OK"
+    for st in range(-6, 0):
+        assert cq.cq_status_string(st).startswith("CQ_ERR_")
+    assert "unknown" in cq.cq_status_string(17)
+
+
+def test_code_buffer_sizes():
+    # one byte per (token, head, group), capacity rounded up to 16-token blocks
+    assert cq.cq_codes_bytes(1, 1024, 1, 128, 8, 8) == 1024 * 16
+    assert cq.cq_codes_bytes(16, 4096, 32, 128, 4, 8) == 16 * 4096 * 32 * 32          # 64 MiB (config 1)
+    assert cq.cq_codes_bytes(64, 16384, 8, 128, 8, 8) == 64 * 16384 * 8 * 16          # 128 MiB (config 2)
+    assert cq.cq_codes_bytes(8, 8192, 32, 128, 2, 8) == 8 * 8192 * 32 * 64            # 128 MiB (config 3)
+    assert cq.cq_codes_bytes(2, 17, 3, 64, 4, 5) == 2 * 3 * 2 * 16 * 16               # 17 tokens -> 2 blocks
+    # invalid shapes give 0
+    assert cq.cq_codes_bytes(1, 16, 1, 128, 3, 8) == 0      # c does not divide head_dim
+    assert cq.cq_codes_bytes(1, 16, 1, 128, 8, 9) == 0      # b > 8
+    assert cq.cq_codes_bytes(0, 16, 1, 128, 8, 8) == 0
+    assert cq.cq_codes_bytes(1, 16, 1, 512, 8, 8) == 0      # head_dim > 256
+
+
+def test_workspace_sizes_are_positive_and_reject_bad_shapes():
+    assert cq.cq_decode_attn_workspace_bytes(64, 32, 8, 128, 8, 8, 16384) > 0
+    assert cq.cq_decode_attn_workspace_bytes(64, 32, 5, 128, 8, 8, 16384) == 0   # Hq % Hkv
+    assert cq.cq_decode_step_host_workspace_bytes(4, 8, 2, 128, 8, 8, 100) > \
+        cq.cq_decode_attn_workspace_bytes(4, 8, 2, 128, 8, 8, 100)
+
+
+def test_argument_validation_happens_on_the_host(L):
+    # Fake, suitably aligned non-NULL addresses: every call below must fail validation
+    # before touching them (nothing is launched, so no GPU is needed).
+    p = 0x10000
+    enc = lambda **kw: L.cq_encode(*[kw.get(k, d) for k, d in [
+        ("x", p), ("cb", p), ("so", None), ("n_seq", 1), ("n_tok", 4), ("off", 0), ("cap", 16),
+        ("heads", 1), ("D", 128), ("c", 8), ("b", 8), ("out", p), ("stream", None)]])
+    assert enc(x=None) == -1
+    assert enc(out=None) == -1
+    assert enc(c=3) == -2
+    assert enc(n_seq=0) == -2
+    assert enc(n_tok=17) == -2                 # past capacity
+    assert enc(off=-1) == -2
+    assert enc(b=0) == -3
+    assert enc(b=9) == -3
+    assert enc(D=512, c=8) == -3
+    assert enc(x=p + 2) == -4
+    assert enc(n_tok=0) == 0                   # nothing to do, nothing launched
+
+    dec = lambda **kw: L.cq_decode_attn(*[kw.get(k, d) for k, d in [
+        ("q", p), ("kc", p), ("vc", p), ("kcb", p), ("vcb", p), ("sl", p), ("scale", ctypes.c_float(0.1)),
+        ("n_seq", 2), ("hq", 4), ("hkv", 2), ("D", 128), ("c", 8), ("b", 8), ("cap", 64), ("out", p),
+        ("ws", p), ("ws_bytes", 1 << 30), ("stream", None)]])
+    assert dec(q=None) == -1
+    assert dec(ws=None) == -1
+    assert dec(hkv=3) == -2
+    assert dec(c=5) == -2
+    assert dec(b=12) == -3
+    assert dec(kc=p + 8) == -4
+    assert dec(ws_bytes=16) == -5
+    conv = L.cq_codes_to_rowmajor(None, 1, 16, 1, 128, 8, 8, p, None)
+    assert conv == -1

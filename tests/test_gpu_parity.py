@@ -1,0 +1,262 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the fp64 CPU oracle,
+element by element, on the same seeded inputs.  Sizes here are ones the oracle finishes
+in seconds; the BASELINE-sized workloads are in test_gpu_full_size.py."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2405_03917_b200 as cq
+from paper_2405_03917_b200 import synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def encode_both(x, cb, c, b, max_tokens, variant=0, token_offset=0):
+    """x (n_seq, n_tokens, n_heads, D) fp16 CPU, cb fp32 CPU -> (gpu rowmajor codes np, oracle triple)."""
+    n_seq, n_tokens, n_heads, D = x.shape
+    buf = torch.zeros(cq.cq_codes_bytes(n_seq, max_tokens, n_heads, D, c, b), dtype=torch.uint8, device=DEV)
+    cq.cq_encode(x.to(DEV), cb.to(DEV), c, b, buf, max_tokens, token_offset=token_offset, variant=variant)
+    rm = cq.cq_codes_to_rowmajor(buf, n_seq, max_tokens, n_heads, D, c, b).cpu().numpy()
+    return buf, rm
+
+
+# ------------------------------------------------------------------------------- encode
+
+@pytest.mark.parametrize("variant", [1, 0])
+def test_config0_encode_bit_exact(variant):
+    w = synth.WORKLOADS[0]
+    ties = 0
+    for is_v in (False, True):
+        x = synth.layer_activations(w, 0, is_v, w.n_seq, w.n_tokens)
+        cb = synth.layer_codebooks(w, 0, is_v)
+        _, rm = encode_both(x, cb, w.c, w.b, w.n_tokens, variant)
+        n, total = H.check_codes(x.numpy().reshape(-1, 1, 128), cb.numpy(), rm.reshape(-1, 1, w.G), w.c, w.b)
+        ties += n
+    assert ties <= 2 * 1024 * 16 // 1000          # near-ties are rare
+
+
+@pytest.mark.parametrize("c,b,head_dim,n_heads,n_tokens", [
+    (2, 8, 128, 3, 100), (4, 8, 128, 2, 77), (8, 8, 128, 2, 130), (1, 4, 64, 2, 33), (16, 8, 128, 1, 50),
+    (8, 5, 64, 3, 47), (4, 1, 32, 2, 19), (8, 8, 256, 1, 40), (2, 3, 16, 5, 16),
+])
+def test_encode_shapes_and_ragged_tails(c, b, head_dim, n_heads, n_tokens):
+    xk, xv, kcb, vcb, _ = H.generic_case(11 * c + b, 2, n_tokens, n_heads, n_heads, head_dim, c, b)
+    for x, cb in ((xk, kcb), (xv, vcb)):
+        for variant in (1, 0):
+            _, rm = encode_both(x, cb, c, b, n_tokens, variant)
+            H.check_codes(x.numpy().reshape(-1, n_heads, head_dim), cb.numpy(),
+                          rm.reshape(-1, n_heads, head_dim // c), c, b)
+
+
+def test_encode_codebook_contains_inputs_and_exact_ties():
+    # inputs equal to centroids -> that centroid's lowest index; duplicated centroids -> lowest index
+    c, b, D, H_ = 8, 8, 128, 2
+    g = torch.Generator().manual_seed(5)
+    cb = torch.randn(H_, D // c, 256, c, generator=g).to(torch.float16).to(torch.float32)
+    cb[:, :, 200] = cb[:, :, 7]
+    pick = torch.randint(0, 256, (1, 64, H_, D // c), generator=g)
+    hh = torch.arange(H_)[None, :, None]
+    gg = torch.arange(D // c)[None, None, :]
+    x = cb[hh, gg, pick[0]].reshape(1, 64, H_, D)        # group g of token t = centroid pick[t, h, g]
+    for variant in (1, 0):
+        _, rm = encode_both(x.to(torch.float16), cb, c, b, 64, variant)
+        want = torch.where(pick == 200, torch.tensor(7), pick).numpy()
+        assert np.array_equal(rm.astype(np.int64), want)
+
+
+def test_append_positions_and_untouched_bytes():
+    c, b, D, nh, cap = 8, 8, 128, 2, 70
+    xk, _, kcb, _, _ = H.generic_case(3, 3, cap, nh, nh, D, c, b)
+    full, rm_full = encode_both(xk, kcb, c, b, cap)
+    # prefill 40 tokens, then append tokens 40..69 one call of 30 tokens at offset 40
+    buf = torch.full((cq.cq_codes_bytes(3, cap, nh, D, c, b),), 0, dtype=torch.uint8, device=DEV)
+    cq.cq_encode(xk[:, :40].contiguous().to(DEV), kcb.to(DEV), c, b, buf, cap)
+    cq.cq_encode(xk[:, 40:].contiguous().to(DEV), kcb.to(DEV), c, b, buf, cap, token_offset=40)
+    assert torch.equal(buf, full)
+    # per-sequence offsets: single-token append at positions (5, 69, 0); everything else untouched
+    buf2 = full.clone()
+    offs = torch.tensor([5, 69, 0], dtype=torch.int32, device=DEV)
+    newtok = xk[:, 10:11].contiguous()
+    cq.cq_encode(newtok.to(DEV), kcb.to(DEV), c, b, buf2, cap, seq_offsets=offs)
+    rm2 = cq.cq_codes_to_rowmajor(buf2, 3, cap, nh, D, c, b).cpu().numpy()
+    want = rm_full.copy()
+    for s, p in enumerate([5, 69, 0]):
+        want[s, p] = rm_full[s, 10]
+    assert np.array_equal(rm2, want)
+    # offsets past the capacity are skipped, not written out of bounds
+    offs_bad = torch.tensor([cap, cap + 5, 3], dtype=torch.int32, device=DEV)
+    buf3 = full.clone()
+    cq.cq_encode(newtok.to(DEV), kcb.to(DEV), c, b, buf3, cap, seq_offsets=offs_bad)
+    rm3 = cq.cq_codes_to_rowmajor(buf3, 3, cap, nh, D, c, b).cpu().numpy()
+    want3 = rm_full.copy()
+    want3[2, 3] = rm_full[2, 10]
+    assert np.array_equal(rm3, want3)
+
+
+def test_layout_roundtrip_matches_documented_offsets():
+    n_seq, cap, nh, D, c, b = 2, 37, 3, 64, 4, 8
+    G = D // c
+    rm = torch.randint(0, 256, (n_seq, cap, nh, G), dtype=torch.uint8)
+    buf = cq.cq_codes_from_rowmajor(rm.to(DEV), D, c, b)
+    assert buf.numel() == cq.cq_codes_bytes(n_seq, cap, nh, D, c, b)
+    back = cq.cq_codes_to_rowmajor(buf, n_seq, cap, nh, D, c, b).cpu()
+    assert torch.equal(back, rm)
+    host = buf.cpu().numpy()
+    NB = (cap + 15) // 16
+    for (s, t, h, g) in [(0, 0, 0, 0), (1, 36, 2, 15), (0, 17, 1, 3), (1, 16, 0, 9)]:
+        off = (((s * nh + h) * NB + t // 16) * G + g) * 16 + t % 16
+        assert host[off] == rm[s, t, h, g]
+
+
+# ------------------------------------------------------------------------------- attention
+
+def attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, scale, c, b, variant):
+    """Codes are the ORACLE's (row-major int32 numpy); both sides read the same codes."""
+    n_seq, cap, n_kv, G = kc_rm.shape
+    D = G * c
+    kb = cq.cq_codes_from_rowmajor(torch.from_numpy(kc_rm.astype(np.uint8)).to(DEV), D, c, b)
+    vb = cq.cq_codes_from_rowmajor(torch.from_numpy(vc_rm.astype(np.uint8)).to(DEV), D, c, b)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    out = cq.cq_decode_attn(q.to(DEV), kb, vb, kcb.to(DEV), vcb.to(DEV), sl, scale, c, b, cap, variant=variant)
+    ref = oracle.decode_dense(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32),
+                              scale, c, b)
+    return out.cpu().numpy(), ref
+
+
+@pytest.mark.parametrize("variant", [1, 0])
+def test_config0_end_to_end(variant):
+    # encode K and V on the GPU, check codes; then attention on the oracle's codes
+    w = synth.WORKLOADS[0]
+    xk = synth.layer_activations(w, 0, False, 1, w.n_tokens)
+    xv = synth.layer_activations(w, 0, True, 1, w.n_tokens)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    q = synth.queries(0, 0, 1, 1)
+    kc_rm, kres = H.oracle_encode_rowmajor(xk, kcb, w.c, w.b)
+    vc_rm, vres = H.oracle_encode_rowmajor(xv, vcb, w.c, w.b)
+    _, gk = encode_both(xk, kcb, w.c, w.b, w.n_tokens, variant)
+    _, gv = encode_both(xv, vcb, w.c, w.b, w.n_tokens, variant)
+    H.check_codes(xk.numpy().reshape(-1, 1, 128), kcb.numpy(), gk.reshape(-1, 1, w.G), w.c, w.b, kres)
+    H.check_codes(xv.numpy().reshape(-1, 1, 128), vcb.numpy(), gv.reshape(-1, 1, w.G), w.c, w.b, vres)
+    out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [w.n_tokens], 128 ** -0.5, w.c, w.b, variant)
+    H.check_attn(out, ref, "config 0")
+
+
+@pytest.mark.parametrize("c,n_q,n_kv,lens", [
+    (8, 4, 1, [1, 15, 16, 17, 0, 333]),          # GQA R=4, one-token, block edges, empty
+    (8, 2, 2, [2049, 700]),                      # MHA, spans several splits
+    (4, 2, 2, [257, 31]),
+    (4, 4, 2, [1000, 1]),
+    (2, 2, 2, [129, 64]),
+    (2, 2, 1, [300]),
+    (8, 8, 1, [90, 200]),                        # R = 8
+    (8, 3, 3, [50]),
+])
+def test_attention_small_cases(c, n_q, n_kv, lens):
+    b, D = 8, 128
+    cap = max(max(lens), 1) + 5
+    w = H.small_workload("t", 90 + c, c, b, len(lens), n_q, n_kv, cap)
+    xk = synth.layer_activations(w, 0, False, len(lens), cap)
+    xv = synth.layer_activations(w, 0, True, len(lens), cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    q = synth.queries(w.config, 0, len(lens), n_q)
+    kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+    for variant in (1, 0):
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, D ** -0.5, c, b, variant)
+        H.check_attn(out, ref, f"c={c} lens={lens} variant={variant}")
+        for s, n in enumerate(lens):
+            if n == 0:
+                assert (out[s] == 0).all()
+            if n == 1:      # a context of one token returns that token's V reconstruction
+                vhat = oracle.dequant(vc_rm[s, :1].reshape(1, n_kv, -1), vcb.numpy(), c, b)[0]
+                for hq in range(n_q):
+                    np.testing.assert_allclose(out[s, hq], vhat[hq // (n_q // n_kv)], rtol=1e-6, atol=1e-6)
+
+
+@pytest.mark.parametrize("c,b,head_dim,n_q,n_kv", [(1, 4, 64, 2, 2), (16, 8, 128, 2, 1), (8, 5, 64, 4, 2),
+                                                   (4, 1, 32, 2, 2), (8, 8, 256, 2, 1), (2, 3, 16, 3, 3)])
+def test_attention_generic_shapes(c, b, head_dim, n_q, n_kv):
+    lens = [61, 7]
+    cap = 64
+    xk, xv, kcb, vcb, q = H.generic_case(100 + c * b, 2, cap, n_q, n_kv, head_dim, c, b)
+    kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+    out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, head_dim ** -0.5, c, b, 0)
+    H.check_attn(out, ref, f"generic c={c} b={b} D={head_dim}")
+
+
+def test_attention_peaked_and_flat_softmax():
+    # a query aligned with one key (peaked weights) and a zero query (uniform weights)
+    c, b, D, cap = 8, 8, 128, 1500
+    w = H.small_workload("t", 77, c, b, 2, 1, 1, cap)
+    xk = synth.layer_activations(w, 0, False, 2, cap)
+    xv = synth.layer_activations(w, 0, True, 2, cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+    q = torch.zeros(2, 1, D, dtype=torch.float16)
+    q[0, 0] = (4.0 * xk[0, 321, 0].float()).clamp(-60000, 60000).to(torch.float16)
+    for variant in (1, 0):
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [cap, cap], 1.0, c, b, variant)
+        H.check_attn(out, ref, f"peaked/flat variant={variant}")
+
+
+def test_token_permutation_and_seq_len_padding_invariance():
+    c, b, D, cap, n = 8, 8, 128, 640, 600
+    w = H.small_workload("t", 55, c, b, 1, 4, 1, cap)
+    xk = synth.layer_activations(w, 0, False, 1, cap)
+    xv = synth.layer_activations(w, 0, True, 1, cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    q = synth.queries(55, 0, 1, 4)
+    kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+    base, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [n], D ** -0.5, c, b, 0)
+    H.check_attn(base, ref)
+    perm = np.random.default_rng(1).permutation(n)
+    kp, vp = kc_rm.copy(), vc_rm.copy()
+    kp[0, :n], vp[0, :n] = kc_rm[0, perm], vc_rm[0, perm]
+    kp[0, n:] = 255 - kp[0, n:]                       # garbage past seq_len must not matter
+    out, _ = attn_both(q, kp, vp, kcb, vcb, [n], D ** -0.5, c, b, 0)
+    np.testing.assert_allclose(out, base, rtol=0, atol=2e-5)
+
+
+def test_decode_step_from_host_buffers():
+    c, b, D, cap, n_seq, n_q, n_kv = 8, 8, 128, 200, 3, 4, 2
+    w = H.small_workload("t", 66, c, b, n_seq, n_q, n_kv, cap)
+    xk = synth.layer_activations(w, 0, False, n_seq, cap)
+    xv = synth.layer_activations(w, 0, True, n_seq, cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    q = synth.queries(66, 0, n_seq, n_q)
+    lens = [150, 0, 199]                       # tokens already cached; the step appends one more
+    kbuf, _ = encode_both(xk, kcb, c, b, cap)
+    vbuf, _ = encode_both(xv, vcb, c, b, cap)
+    k_new = torch.stack([xk[s, 7] for s in range(n_seq)]).contiguous()      # (n_seq, n_kv, D)
+    v_new = torch.stack([xv[s, 9] for s in range(n_seq)]).contiguous()
+    ws = torch.empty(cq.cq_decode_step_host_workspace_bytes(n_seq, n_q, n_kv, D, c, b, cap), dtype=torch.uint8,
+                     device=DEV)
+    out_host = torch.empty(n_seq, n_q, D, dtype=torch.float32).pin_memory()
+    cq.cq_decode_step_host(q.pin_memory(), k_new.pin_memory(), v_new.pin_memory(),
+                           torch.tensor(lens, dtype=torch.int32), kbuf, vbuf, kcb.to(DEV), vcb.to(DEV),
+                           D ** -0.5, c, b, cap, out_host, ws)
+    # oracle: same cache with the new token written at position lens[s], context lens[s] + 1
+    xk2, xv2 = xk.clone(), xv.clone()
+    for s, n in enumerate(lens):
+        xk2[s, n], xv2[s, n] = k_new[s], v_new[s]
+    kc_rm, _ = H.oracle_encode_rowmajor(xk2, kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv2, vcb, c, b)
+    ref = oracle.decode_dense(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(),
+                              np.asarray([n + 1 for n in lens], np.int32), D ** -0.5, c, b)
+    H.check_attn(out_host.numpy(), ref, "host step")
+    got_k = cq.cq_codes_to_rowmajor(kbuf, n_seq, cap, n_kv, D, c, b).cpu().numpy()
+    for s, n in enumerate(lens):
+        H.check_codes(k_new[s:s + 1].numpy(), kcb.numpy(), got_k[s, n][None], c, b)
+
+
+def test_library_is_loaded_from_the_tree():
+    import os
+    assert os.path.samefile(os.path.dirname(cq.library_path()), os.path.dirname(cq.__file__))
+    maps = open("/proc/self/maps").read()
+    assert "libcq.so" in maps
