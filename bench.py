@@ -1,0 +1,453 @@
+#!/usr/bin/env python
+"""Benchmark of the CQ hot path on B200.
+
+One "step" is one decode step of one layer on the headline workload (config 2 of
+the benchmark spec: CQ-8c8b, Mistral-7B-shaped GQA, batch 64, context 16384): the new token's
+key and value vectors are CQ-encoded and appended (cq_encode, K and V), then every query
+head attends over the coded cache (cq_decode_attn).  Inputs are seeded and synthetic.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg2|cfg1|cfg4|cfg0] [--extras none|default|all]
+
+Prints ONE JSON line (rank 0).  `value` is KV tokens/s with everything resident in HBM;
+`e2e` is the same metric through cq_decode_step_host with host buffers; `roofline` is the
+decode-attention call against the measured HBM copy bandwidth; `cpu_baseline` is the fp64
+CPU oracle on a bounded sample.  With --impl reference the oracle itself is the timed arm.
+Under torchrun every rank runs its own replica of the batch (weak scaling, no collective
+on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2405_03917_b200 import synth  # noqa: E402
+
+HBM_FALLBACK_GBS = 6650.0
+METRIC = "cq_decode_attn_kv_tokens_per_s"
+UNIT = "KV tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if backend == "nccl":
+            torch.cuda.set_device(local)
+        dist.init_process_group(backend=backend)
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# --------------------------------------------------------------------------------- setup
+
+class DecodeState:
+    """Device-resident coded cache of one layer of a workload, built with the CUDA encode."""
+
+    def __init__(self, w: synth.Workload, layer: int, dev, cq, lens=None):
+        self.w, self.dev = w, dev
+        D, c, b = w.head_dim, w.c, w.b
+        self.lens_cpu = w.lengths() if lens is None else lens
+        self.cap = w.n_tokens
+        nbytes = cq.cq_codes_bytes(w.n_seq, self.cap, w.n_kv_heads, D, c, b)
+        self.k_codes = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+        self.v_codes = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+        self.k_cb = synth.layer_codebooks(w, layer, False).to(dev)
+        self.v_cb = synth.layer_codebooks(w, layer, True).to(dev)
+        # encode head by head so that at most one head's activations are alive
+        for is_v, codes, cb in ((False, self.k_codes, self.k_cb), (True, self.v_codes, self.v_cb)):
+            x = synth.layer_activations(w, layer, is_v, w.n_seq, self.cap, device=dev)
+            cq.cq_encode(x, cb, c, b, codes, self.cap)
+            # the step's new token: a fresh draw per (sequence, head)
+            new = torch.stack([synth.head_source(w.config, layer, h, is_v).activations(w.n_seq, dev, stream=2)
+                               for h in range(w.n_kv_heads)], dim=1).contiguous()
+            if is_v:
+                self.v_new = new
+            else:
+                self.k_new = new
+            del x
+        self.q = synth.queries(w.config, layer, w.n_seq, w.n_q_heads, device=dev)
+        self.seq_lens = self.lens_cpu.to(dev)
+        self.append_pos = (self.lens_cpu - 1).to(dev)
+        self.out = torch.empty(w.n_seq, w.n_q_heads, D, dtype=torch.float32, device=dev)
+        self.ws = torch.empty(max(256, cq.cq_decode_attn_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, c, b,
+                                                                        self.cap)), dtype=torch.uint8, device=dev)
+        self.scale = D ** -0.5
+
+    def kv_tokens(self) -> int:
+        return int(self.lens_cpu.sum().item())
+
+    def algorithmic_bytes(self) -> int:
+        """Bytes decode attention must read per call: one byte per (token, KV head, group) for K
+        and for V, both codebooks once per KV head, queries; plus the output it writes."""
+        w = self.w
+        codes = 2 * self.kv_tokens() * w.n_kv_heads * w.G
+        books = 2 * w.n_kv_heads * w.G * (1 << w.b) * w.c * 4
+        qo = w.n_seq * w.n_q_heads * w.head_dim * (2 + 4)
+        return codes + books + qo
+
+    def step(self, cq, ev=None):
+        """Append-encode the new token (K, V) at the last position, then attend."""
+        w = self.w
+        cq.cq_encode(self.k_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim), self.k_cb, w.c, w.b, self.k_codes,
+                     self.cap, seq_offsets=self.append_pos)
+        cq.cq_encode(self.v_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim), self.v_cb, w.c, w.b, self.v_codes,
+                     self.cap, seq_offsets=self.append_pos)
+        if ev is not None:
+            ev[0].record()
+        cq.cq_decode_attn(self.q, self.k_codes, self.v_codes, self.k_cb, self.v_cb, self.seq_lens, self.scale,
+                          w.c, w.b, self.cap, out=self.out, workspace=self.ws)
+        if ev is not None:
+            ev[1].record()
+
+
+def time_steps(fn, steps, warmup, world, dev):
+    for _ in range(warmup):
+        fn(None)
+    torch.cuda.synchronize()
+    barrier(world)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    inner = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    e0.record()
+    for i in range(steps):
+        fn(inner[i])
+    e1.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    total_ms = e0.elapsed_time(e1)
+    inner_ms = [a.elapsed_time(b) for a, b in inner]
+    return max_over_ranks(total_ms, world, dev), inner_ms
+
+
+# ----------------------------------------------------------------------------- CPU oracle
+
+def oracle_sample_state(w: synth.Workload, n_sample_seq: int = 1):
+    """Oracle-side copy of the first sequences of the workload: the cache is encoded by the
+    oracle itself (untimed set-up), never read from the CUDA path."""
+    import oracle
+    layer = 0
+    lens = w.lengths()[:n_sample_seq].numpy().astype(np.int32)
+    cap = int(lens.max())
+    st = {"lens": lens, "cap": cap}
+    # CPU and CUDA generators give different draws of the same distribution, so the sample is
+    # drawn directly at its own size.
+    for is_v, key in ((False, "k"), (True, "v")):
+        cb = synth.layer_codebooks(w, layer, is_v).numpy()
+        x = synth.layer_activations(w, layer, is_v, n_sample_seq, cap)
+        xn = x.numpy().reshape(n_sample_seq * cap, w.n_kv_heads, w.head_dim)
+        codes, _, _ = oracle.encode(xn, cb, w.c, w.b)
+        st[key + "_cb"] = cb
+        st[key + "_codes"] = codes.reshape(n_sample_seq, cap, w.n_kv_heads, w.G)
+        new = torch.stack([synth.head_source(w.config, layer, h, is_v).activations(w.n_seq, "cpu", stream=2)
+                           for h in range(w.n_kv_heads)], dim=1)[:n_sample_seq]
+        st[key + "_new"] = new.numpy().reshape(n_sample_seq, w.n_kv_heads, w.head_dim)
+    st["q"] = synth.queries(w.config, layer, w.n_seq, w.n_q_heads)[:n_sample_seq].numpy()
+    return st
+
+
+def oracle_step(w, st):
+    """The same step on the CPU oracle: encode the new token (K, V), write its codes at the
+    last position, dense attention over the reconstructed cache."""
+    import oracle
+    for key in ("k", "v"):
+        codes, _, _ = oracle.encode(st[key + "_new"], st[key + "_cb"], w.c, w.b)
+        for s, n in enumerate(st["lens"]):
+            st[key + "_codes"][s, n - 1] = codes[s]
+    return oracle.decode_dense(st["q"], st["k_codes"], st["v_codes"], st["k_cb"], st["v_cb"], st["lens"],
+                               w.head_dim ** -0.5, w.c, w.b)
+
+
+def time_oracle(w, steps, warmup):
+    import oracle
+    st = oracle_sample_state(w, 1)
+    for _ in range(warmup):
+        oracle_step(w, st)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(w, st)
+    dt = (time.perf_counter() - t0) / steps
+    toks = int(st["lens"].sum())
+    return {"value": toks / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"sequence 0 of the batch ({toks} tokens, all {w.n_kv_heads} KV heads / {w.n_q_heads} query "
+                      f"heads): append-encode + dense attention, mean of {steps} steps; cache encoded by the "
+                      f"oracle beforehand (untimed)",
+            "ms_per_step": dt * 1e3}
+
+
+# ------------------------------------------------------------------------------- extras
+
+def extra_encode_cfg3(cq, dev, reps=5):
+    """Prefill encode throughput on config 3 (CQ-2c8b, 8 x 8192 tokens x 32 heads, K and V)."""
+    w = synth.WORKLOADS[3]
+    D = w.head_dim
+    res = {}
+    xs, cbs, bufs = [], [], []
+    for is_v in (False, True):
+        xs.append(synth.layer_activations(w, 0, is_v, w.n_seq, w.n_tokens, device=dev))
+        cbs.append(synth.layer_codebooks(w, 0, is_v).to(dev))
+        bufs.append(torch.zeros(cq.cq_codes_bytes(w.n_seq, w.n_tokens, w.n_kv_heads, D, w.c, w.b), dtype=torch.uint8,
+                                device=dev))
+    def run():
+        for x, cb, buf in zip(xs, cbs, bufs):
+            cq.cq_encode(x, cb, w.c, w.b, buf, w.n_tokens)
+    for _ in range(2):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    tokens = w.n_seq * w.n_tokens
+    vectors = 2 * tokens * w.n_kv_heads
+    res = {"workload": w.name, "ms": ms, "tokens_per_s": tokens / (ms * 1e-3), "vectors_per_s": vectors / (ms * 1e-3),
+           "useful_tflops": vectors * 2 * D * (1 << w.b) / (ms * 1e-3) / 1e12,
+           "gbs": (vectors * (D * 2 + w.G) + 2 * w.n_kv_heads * D * (1 << w.b) * 4) / (ms * 1e-3) / 1e9}
+    return res
+
+
+def extra_decode(cq, dev, w, reps=20):
+    st = DecodeState(w, 0, dev, cq)
+    for _ in range(3):
+        st.step(cq)
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for e in evs:
+        st.step(cq, e)
+    torch.cuda.synchronize()
+    ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
+    hbm, _ = measured_peaks()
+    gbs = st.algorithmic_bytes() / (ms * 1e-3) / 1e9
+    return {"workload": w.name, "decode_ms": ms, "kv_tokens_per_s": st.kv_tokens() / (ms * 1e-3),
+            "query_heads_per_s": w.n_seq * w.n_q_heads / (ms * 1e-3), "gbs": gbs, "frac_of_measured_hbm": gbs / hbm}
+
+
+# --------------------------------------------------------------------------------- main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg4"])
+    ap.add_argument("--extras", default="default", choices=["none", "default", "all"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    w = synth.WORKLOADS[int(args.workload[3])]
+    config = {"workload": w.name, "c": w.c, "b": w.b, "n_seq": w.n_seq, "n_q_heads": w.n_q_heads,
+              "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "context": w.n_tokens, "layers_per_step": 1,
+              "step": "append-encode new token (K,V) + decode attention",
+              "l2": "inputs exceed L2 (code buffers > 126 MB)" if w.name.startswith(("cfg2", "cfg4")) else
+                    "inputs fit L2 (small case)"}
+
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        if rank != 0:
+            return 0
+        steps = max(1, min(args.steps, 20))
+        r = time_oracle(w, steps, max(1, min(args.warmup, 2)))
+        line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+                "steps": steps, "warmup": max(1, min(args.warmup, 2)), "ms_per_step": r["ms_per_step"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": config,
+                "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+                "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --impl ours needs a CUDA device: the library has no CPU fallback")
+    import paper_2405_03917_b200 as cq
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+
+    st = DecodeState(w, 0, dev, cq)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    total_ms, inner_ms = time_steps(lambda ev: st.step(cq, ev), args.steps, args.warmup, world, dev)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = total_ms / args.steps
+    kv_tokens = st.kv_tokens() * world
+    value = kv_tokens / (ms_per_step * 1e-3)
+
+    # end to end: host buffers in, host result out, through cq_decode_step_host
+    D = w.head_dim
+    ws_h = torch.empty(cq.cq_decode_step_host_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, w.c, w.b, st.cap),
+                       dtype=torch.uint8, device=dev)
+    q_h, k_h, v_h = st.q.cpu().pin_memory(), st.k_new.cpu().pin_memory(), st.v_new.cpu().pin_memory()
+    lens_h = (st.lens_cpu - 1).contiguous()
+    out_h = torch.empty(w.n_seq, w.n_q_heads, D, dtype=torch.float32).pin_memory()
+    def e2e_step():
+        cq.cq_decode_step_host(q_h, k_h, v_h, lens_h, st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.scale, w.c, w.b,
+                               st.cap, out_h, ws_h)
+    for _ in range(3):
+        e2e_step()
+    torch.cuda.synchronize()
+    barrier(world)
+    t0 = time.perf_counter()
+    n_e2e = max(5, args.steps // 2)
+    for _ in range(n_e2e):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, world, dev)
+    h2d = q_h.numel() * 2 + k_h.numel() * 2 + v_h.numel() * 2 + lens_h.numel() * 4
+    d2h = out_h.numel() * 4
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return 0
+
+    hbm, which = measured_peaks()
+    dec_ms = statistics.mean(inner_ms)
+    achieved = st.algorithmic_bytes() / (dec_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "cq_decode_attn (main kernel + split merge)", "achieved": achieved,
+                "peak": hbm, "peak_source": which, "unit": "GB/s", "frac": achieved / hbm,
+                "frac_of_8tbs_nominal": achieved / 8000.0, "traffic": None,
+                "algorithmic_bytes_per_launch": st.algorithmic_bytes(), "launch_ms": dec_ms}
+    tr = os.path.join(ROOT, "profiles", "decode_traffic.json")
+    if os.path.exists(tr):
+        try:
+            t = json.load(open(tr)).get(w.name)
+            if t:
+                roofline["traffic"] = t["dram_bytes_per_launch"]
+                roofline["traffic_source"] = t.get("source")
+        except Exception:
+            pass
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "query_heads_per_s": w.n_seq * w.n_q_heads * world / (ms_per_step * 1e-3),
+            "clocks": clocks,
+            "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": args.steps * 4,
+            "roofline": roofline}
+
+    if args.extras != "none" and world == 1:
+        extras = {}
+        try:
+            extras["encode"] = extra_encode_cfg3(cq, dev)
+            if args.extras == "all":
+                extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
+        except Exception as e:      # extras never hide the headline number
+            extras["error"] = repr(e)
+        line["extras"] = extras
+    if not args.no_cpu_baseline and world == 1:
+        del st
+        torch.cuda.empty_cache()
+        r = time_oracle(w, 10, 1)
+        line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
