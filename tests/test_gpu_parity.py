@@ -204,6 +204,44 @@ def test_attention_peaked_and_flat_softmax():
         H.check_attn(out, ref, f"peaked/flat variant={variant}")
 
 
+def test_weight_unit_is_coarsened_on_flat_and_on_rising_scores():
+    # (a) zero query over a long context: every weight equals the maximum, so integer bins
+    #     must coarsen their unit instead of overflowing; (b) tokens sorted by rising score,
+    #     with a large scale: the running maximum grows in every round.
+    c, b, D, cap = 8, 8, 128, 20000
+    w = H.small_workload("t", 78, c, b, 2, 1, 1, cap)
+    xk = synth.layer_activations(w, 0, False, 2, cap)
+    xv = synth.layer_activations(w, 0, True, 2, cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+    q = synth.queries(78, 0, 2, 1)
+    q[0] = 0
+    scale = 0.7
+    khat = oracle.dequant(kc_rm[1].reshape(cap, 1, -1), kcb.numpy(), c, b)[:, 0]        # (cap, D)
+    order = np.argsort(khat @ q[1, 0].double().numpy(), kind="stable")
+    kc_rm[1], vc_rm[1] = kc_rm[1][order], vc_rm[1][order]
+    for variant in (1, 0):
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [cap, cap - 3], scale, c, b, variant)
+        H.check_attn(out, ref, f"flat/rising variant={variant}")
+
+
+def test_attention_multi_chunk_gqa_and_mha_long():
+    # contexts long enough for several chunks per (sequence, KV head) and ragged ends
+    for c, n_q, n_kv, lens in ((8, 4, 1, [9000, 4097]), (4, 1, 1, [5000]), (8, 2, 1, [6001]), (4, 2, 1, [4500])):
+        b, D = 8, 128
+        cap = max(lens) + 11
+        w = H.small_workload("t", 120 + c + n_q, c, b, len(lens), n_q, n_kv, cap)
+        xk = synth.layer_activations(w, 0, False, len(lens), cap)
+        xv = synth.layer_activations(w, 0, True, len(lens), cap)
+        kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+        q = synth.queries(w.config, 0, len(lens), n_q)
+        kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
+        vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, D ** -0.5, c, b, 0)
+        H.check_attn(out, ref, f"long c={c} Hq={n_q} Hkv={n_kv}")
+
+
 def test_token_permutation_and_seq_len_padding_invariance():
     c, b, D, cap, n = 8, 8, 128, 640, 600
     w = H.small_workload("t", 55, c, b, 1, 4, 1, cap)
