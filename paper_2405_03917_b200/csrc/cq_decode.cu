@@ -52,9 +52,17 @@ struct Cfg {
     static constexpr int kPlanes = kLaneHeads;                           // 32-word planes per table row
     static constexpr int kSlots = G / 4;                                 // code words (16 tokens each) per lane
     static constexpr int kBlocksPerIter = (G == 16 && R >= 2) ? 4 : 8;   // 16-token blocks per warp iteration
+#ifdef CQ_TUNE_WARPS1
+    static constexpr int kWarps = (kPlanes == 1) ? CQ_TUNE_WARPS1 : 16;
+#else
     static constexpr int kWarps = (kPlanes == 1) ? 8 : 16;
+#endif
     static constexpr int kThreads = kWarps * 32;
-    static constexpr int kMinBlocks = (kPlanes == 1) ? (G == 16 ? 3 : 2) : 1;
+#ifdef CQ_TUNE_MINBLK
+    static constexpr int kMinBlocks = (kPlanes == 1) ? CQ_TUNE_MINBLK : 1;
+#else
+    static constexpr int kMinBlocks = (kPlanes == 1) ? 2 : 1;     // 128 registers per thread in every configuration
+#endif
     static constexpr int kRoundTokens = kWarps * kBlocksPerIter * 16;    // tokens a CTA handles per iteration
     static_assert(kPlanes == 1 || kPlanes == 2, "table rows hold one or two planes");
     // One plane: K and V planes share a row (K at +0, V at +128).  Two planes: separate tables.
@@ -68,14 +76,12 @@ struct Cfg {
     {
         return kHalfRows ? 16 * (r >> 2) + 4 * ((r + m) & 3) + p : 4 * ((r + m) & 7) + p;
     }
-    // group / query head (relative to the KV head's first query head) of a table word
+    // group of a table word, and the (plane, word) that holds (group g, query head h of the KV head)
     __device__ static __forceinline__ int group_of(int w) { return kHalfRows ? (w & 15) : w; }
-    __device__ static __forceinline__ int head_of(int plane, int w)
-    {
-        if (!kHalfRows) return plane;
-        if (R == 1) return 0;
-        return 2 * plane + (w >> 4);
-    }
+    __device__ static __forceinline__ int plane_of(int h) { return kHalfRows ? (R <= 2 ? 0 : h >> 1) : h; }
+    __device__ static __forceinline__ int word_of(int g, int h) { return kHalfRows ? (R == 1 ? 0 : (h & 1) * 16) + g : g; }
+    static constexpr int kGroupsPerWarp = G / kWarps;
+    static_assert(G % kWarps == 0 && kSlots % 4 == 0, "ownership of groups by warps; four code words per MMA");
 };
 
 struct Ctl {
@@ -98,6 +104,14 @@ __device__ __forceinline__ uint4 ldg_codes(const uint4* p)
     return v;
 }
 
+// shared-memory load that keeps its place among the other volatile statements
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
@@ -109,9 +123,76 @@ __device__ __forceinline__ float ex2(float x)
 __device__ __forceinline__ void mma_rowsum(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
 {
     const uint32_t ones = 0x3c003c00u;   // half2(1, 1)
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(ones), "r"(ones));
+}
+
+template <int kC>
+__device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC])
+{
+    static_assert(kC == 4 || kC == 8, "centroids of 4 or 8 channels");
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
+    if (kC == 8) {
+        const float4 b = *reinterpret_cast<const float4*>(p + 4);
+        cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
+    }
+}
+
+// half2 (hi, lo) with hi + lo ~= v to about 22 bits: hi in the low half, lo in the high half
+__device__ __forceinline__ uint32_t pack_hi_lo(float v)
+{
+    const __half hi = __float2half_rn(v);
+    const __half lo = __float2half_rn(v - __half2float(hi));
+    return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+}
+
+// Sum of a[0..kC) over the 32 lanes of a warp, with the channels folded while they are exchanged:
+// the step with lane mask 16 keeps half of the channels in each half warp, and so on, so that
+// after log2(kC) steps every lane holds one channel; the remaining steps finish that channel.
+// The result of lane L is the total of channel fold_channel_of<kC>(L).
+template <int kC>
+__device__ __forceinline__ int fold_channel_of(int lane)
+{
+    return kC == 8 ? ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)
+                   : ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+}
+template <int kC>
+__device__ __forceinline__ float fold_channels(const float (&a)[kC], int lane)
+{
+    float h4[kC / 2];
+    {
+        const bool up = lane & 16;
+#pragma unroll
+        for (int i = 0; i < kC / 2; ++i) {
+            const float keep = up ? a[i + kC / 2] : a[i];
+            const float send = up ? a[i] : a[i + kC / 2];
+            h4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+    }
+    float h2[kC / 4];
+    {
+        const bool up = lane & 8;
+#pragma unroll
+        for (int i = 0; i < kC / 4; ++i) {
+            const float keep = up ? h4[i + kC / 4] : h4[i];
+            const float send = up ? h4[i] : h4[i + kC / 4];
+            h2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+    }
+    float v;
+    if (kC == 8) {
+        const bool up = lane & 4;
+        const float keep = up ? h2[1 % (kC / 4)] : h2[0];
+        const float send = up ? h2[0] : h2[1 % (kC / 4)];
+        v = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    } else {
+        v = h2[0] + __shfl_xor_sync(0xffffffffu, h2[0], 4);
+    }
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
 }
 
 // byte `k` (0..15) of a 16-byte code word
@@ -167,38 +248,46 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     if (threadIdx.x == 3) ctl->lut_absmax = 0.f;
     for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
         qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)hkv * R) * 128 + i]) * scale_log2e;
+    // bins start at zero (16-byte stores over the V planes)
+    for (int i = threadIdx.x; i < kRows * 8 * C::kPlanes; i += C::kThreads)
+        *reinterpret_cast<uint4*>(smem + C::kVOffset + (i / (8 * C::kPlanes)) * kRowBytes + (i % (8 * C::kPlanes)) * 16) =
+            make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
 
-    // lane `lane` fills word `lane` of every plane, for the code values j = warp, warp + kWarps, ...
-    {
+    // Table build.  A warp owns whole groups and its lanes walk the code values j, so the
+    // codebook is read in contiguous runs.  A column of the table (fixed word, 32 consecutive
+    // rows) would fall into one bank, so the build writes row j rotated by j words and a second
+    // pass un-rotates every row.  Entries are half2 (hi, lo) of LUT * 2^-kexp; kexp = 0 unless an
+    // entry reaches 2^15 (then the build is repeated once with the exponent that fits).
+    float lut_scale = 1.f;           // scores in table units * lut_scale = log2-domain scores
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        const float inv = 1.f / lut_scale;
         float absmax = 0.f;
-        const int g = C::group_of(lane);
-        float qreg[C::kPlanes][kC];
+#pragma unroll 1
+        for (int gi = 0; gi < C::kGroupsPerWarp; ++gi) {
+            const int g = warp * C::kGroupsPerWarp + gi;
+            float qreg[R][kC];
 #pragma unroll
-        for (int pl = 0; pl < C::kPlanes; ++pl)
+            for (int h = 0; h < R; ++h)
 #pragma unroll
-            for (int i = 0; i < kC; ++i) qreg[pl][i] = qs[C::head_of(pl, lane) * 128 + g * kC + i];
-        const float* cg = kcb + ((int64_t)hkv * G + g) * kRows * kC;
-#pragma unroll 4
-        for (int j = warp; j < kRows; j += C::kWarps) {
-            float cv[kC];
-            if (kC == 8) {
-                const float4 a = *reinterpret_cast<const float4*>(cg + j * 8);
-                const float4 b = *reinterpret_cast<const float4*>(cg + j * 8 + 4);
-                cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
-                cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
-            } else {
-                const float4 a = *reinterpret_cast<const float4*>(cg + j * 4);
-                cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
-            }
+                for (int i = 0; i < kC; ++i) qreg[h][i] = qs[h * 128 + g * kC + i] * inv;
+            const float* cg = kcb + ((int64_t)hkv * G + g) * kRows * kC;
 #pragma unroll
-            for (int pl = 0; pl < C::kPlanes; ++pl) {
-                float dot = 0.f;
+            for (int jb = 0; jb < kRows / 32; ++jb) {
+                const int j = jb * 32 + lane;
+                float cv[kC];
+                load_centroid<kC>(cg + j * kC, cv);
 #pragma unroll
-                for (int i = 0; i < kC; ++i) dot = fmaf(qreg[pl][i], cv[i], dot);
-                absmax = fmaxf(absmax, fabsf(dot));
-                *reinterpret_cast<float*>(smem + j * kRowBytes + pl * 128 + lane * 4) = dot;
-                *reinterpret_cast<uint32_t*>(smem + C::kVOffset + j * kRowBytes + pl * 128 + lane * 4) = 0u;
+                for (int h = 0; h < R; ++h) {
+                    float dot = 0.f;
+#pragma unroll
+                    for (int i = 0; i < kC; ++i) dot = fmaf(qreg[h][i], cv[i], dot);
+                    absmax = fmaxf(absmax, fabsf(dot));
+                    const uint32_t e = pack_hi_lo(dot);
+                    uint8_t* row = smem + j * kRowBytes + C::plane_of(h) * 128;
+                    *reinterpret_cast<uint32_t*>(row + ((C::word_of(g, h) + j) & 31) * 4) = e;
+                    if (C::kReplica) *reinterpret_cast<uint32_t*>(row + ((16 + g + j) & 31) * 4) = e;
+                }
             }
         }
         absmax = fmaxf(absmax, __shfl_xor_sync(0xffffffffu, absmax, 16));
@@ -207,29 +296,24 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         absmax = fmaxf(absmax, __shfl_xor_sync(0xffffffffu, absmax, 2));
         absmax = fmaxf(absmax, __shfl_xor_sync(0xffffffffu, absmax, 1));
         if (lane == 0) atomicMax(reinterpret_cast<int*>(&ctl->lut_absmax), __float_as_int(absmax));
-    }
-    __syncthreads();
-    // Entries become half2 (hi, lo) of LUT * 2^-kexp, with kexp chosen so that |hi| < 2^15.
-    int kexp = 0;
-    {
+        __syncthreads();
+        const float amax = ctl->lut_absmax;
+        if (attempt == 1 || amax < 32768.f) break;       // same decision in every thread
         int ex;
-        frexpf(ctl->lut_absmax, &ex);            // absmax < 2^ex
-        kexp = ex > 15 ? ex - 15 : 0;
+        frexpf(amax, &ex);                                // amax < 2^ex
+        lut_scale = exp2f((float)(ex - 15));
+        __syncthreads();
+        if (threadIdx.x == 0) ctl->lut_absmax = 0.f;
+        __syncthreads();
     }
-    const float lut_scale = exp2f((float)kexp);     // scores in table units * lut_scale = log2-domain scores
-    {
-        const float inv = exp2f(-(float)kexp);
-#pragma unroll 4
-        for (int j = warp; j < kRows; j += C::kWarps)
+    for (int j = warp; j < kRows; j += C::kWarps)
 #pragma unroll
-            for (int pl = 0; pl < C::kPlanes; ++pl) {
-                uint32_t* e = reinterpret_cast<uint32_t*>(smem + j * kRowBytes + pl * 128 + lane * 4);
-                const float v = __uint_as_float(*e) * inv;
-                const __half hi = __float2half_rn(v);
-                const __half lo = __float2half_rn(v - __half2float(hi));
-                *e = (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
-            }
-    }
+        for (int pl = 0; pl < C::kPlanes; ++pl) {
+            uint8_t* row = smem + j * kRowBytes + pl * 128;
+            const uint32_t e = *reinterpret_cast<const uint32_t*>(row + ((lane + j) & 31) * 4);
+            __syncwarp();
+            *reinterpret_cast<uint32_t*>(row + lane * 4) = e;
+        }
     __syncthreads();
 
     // ---------------------------------------------------------------- main loop over the chunk
@@ -237,23 +321,27 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     const int64_t blk_lim = (t_end + kTokenBlock - 1) / kTokenBlock;       // blocks holding a valid token
     const int n_iters = (int)((t_end - t_begin + C::kRoundTokens - 1) / C::kRoundTokens);
     const int qb = (C::kBlocksPerIter == 8) ? r : (r & 3);                 // block of this quad inside the warp's iteration
-    const uint4* kbase = reinterpret_cast<const uint4*>(kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0));
-    const uint4* vbase = reinterpret_cast<const uint4*>(vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0));
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+#ifdef CQ_TUNE_KBATCH
+    constexpr int kBatch = CQ_TUNE_KBATCH;
+#else
+    constexpr int kBatch = C::kSlots >= 8 ? 2 : 4;                         // tokens whose lookups are in flight together
+#endif
 
     uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a plane, per code word
-    int slot_group[C::kSlots];
 #pragma unroll
-    for (int m = 0; m < C::kSlots; ++m) {
-        const int w = C::word(r, p, m);
-        lane_off[m] = 4u * w;
-        slot_group[m] = C::group_of(w);
-    }
+    for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m);
+    // code words of this lane: word (block, group) sits at (block * G + group) * 16 bytes
+    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
 
     uint4 kw[C::kSlots], vw[C::kSlots];
-    auto load_words = [&](uint4 (&dst)[C::kSlots], const uint4* base, int64_t blk) {
+    auto load_words = [&](uint4 (&dst)[C::kSlots], const uint8_t* base, int64_t blk) {
         if (blk < blk_lim) {
+            const uint8_t* bp = base + blk * (G * kTokenBlock);
 #pragma unroll
-            for (int m = 0; m < C::kSlots; ++m) dst[m] = ldg_codes(base + blk * G + slot_group[m]);
+            for (int m = 0; m < C::kSlots; ++m)
+                dst[m] = ldg_codes(reinterpret_cast<const uint4*>(bp + C::group_of(lane_off[m] >> 2) * kTokenBlock));
         } else {
 #pragma unroll
             for (int m = 0; m < C::kSlots; ++m) dst[m] = make_uint4(0u, 0u, 0u, 0u);
@@ -265,40 +353,53 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     load_words(kw, kbase, blk0 + (int64_t)warp * C::kBlocksPerIter + qb);
 
     for (int it = 0; it < n_iters; ++it) {
-        const int64_t blk = blk0 + ((int64_t)it * C::kWarps + warp) * C::kBlocksPerIter + qb;
+        const int64_t blk_warp = blk0 + ((int64_t)it * C::kWarps + warp) * C::kBlocksPerIter;
+        const int64_t blk = blk_warp + qb;
         load_words(vw, vbase, blk);
 
-        // K side: scores of this quad's 16 tokens, for the query heads this lane serves
+        // K side: scores of this quad's 16 tokens for the query heads this lane serves.  One MMA
+        // per (token, head) and per 4 code words: fragment rows r and r + 8 carry two halves of
+        // the same token's lookups, so the token's score is the sum of both row sums.
         float sc[C::kLaneHeads][16];
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj)
+        for (int k0 = 0; k0 < 16; k0 += kBatch)
 #pragma unroll
             for (int u = 0; u < C::kLaneHeads; ++u) {
-                float d[4] = {0.f, 0.f, 0.f, 0.f};
+                // all lookups of a batch of tokens are issued before the first MMA needs one
+                uint32_t a[kBatch][C::kSlots];
 #pragma unroll
-                for (int m = 0; m < C::kSlots; m += 2) {
-                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(smem + u * 128 + row_index(kw[m], jj, lane_off[m]));
-                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(smem + u * 128 + row_index(kw[m], jj + 8, lane_off[m]));
-                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(smem + u * 128 + row_index(kw[m + 1], jj, lane_off[m + 1]));
-                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(smem + u * 128 + row_index(kw[m + 1], jj + 8, lane_off[m + 1]));
-                    mma_rowsum(d, a0, a1, a2, a3);
+                for (int kk = 0; kk < kBatch; ++kk)
+#pragma unroll
+                    for (int m = 0; m < C::kSlots; ++m)
+                        a[kk][m] = lds_u32(smem_base + u * 128 + row_index(kw[m], k0 + kk, lane_off[m]));
+#pragma unroll
+                for (int kk = 0; kk < kBatch; ++kk) {
+                    float tot = 0.f;
+#pragma unroll
+                    for (int m = 0; m < C::kSlots; m += 4) {
+                        float d[4] = {0.f, 0.f, 0.f, 0.f};
+                        mma_rowsum(d, a[kk][m], a[kk][m + 1], a[kk][m + 2], a[kk][m + 3]);
+                        tot += d[0] + d[2];
+                    }
+                    sc[u][k0 + kk] = tot;
                 }
-                sc[u][jj] = d[0];
-                sc[u][jj + 8] = d[2];
             }
 
-        // mask tokens past the end of the context, take the maximum
-        const int64_t tok0 = blk * kTokenBlock;
+        // tokens past the end of the context get -inf (only the warp that holds the ragged end pays)
+        if ((blk_warp + C::kBlocksPerIter) * kTokenBlock > t_end) {
+            const int64_t tok0 = blk * kTokenBlock;
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+#pragma unroll
+                for (int u = 0; u < C::kLaneHeads; ++u)
+                    if (tok0 + k >= t_end) sc[u][k] = -INFINITY;
+        }
         float mx = -INFINITY;
 #pragma unroll
         for (int k = 0; k < 16; ++k)
 #pragma unroll
-            for (int u = 0; u < C::kLaneHeads; ++u) {
-                const float v = (tok0 + k < t_end) ? sc[u][k] * lut_scale : -INFINITY;
-                sc[u][k] = v;
-                mx = fmaxf(mx, v);
-            }
-        const int wmax = __reduce_max_sync(0xffffffffu, enc_float(mx));
+            for (int u = 0; u < C::kLaneHeads; ++u) mx = fmaxf(mx, sc[u][k]);
+        const int wmax = __reduce_max_sync(0xffffffffu, enc_float(mx * lut_scale));
         if (lane == 0) atomicMax(&ctl->rmax[it % 3], wmax);
         __syncthreads();
         const float round_max = dec_float(ctl->rmax[it % 3]);
@@ -308,40 +409,51 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         load_words(kw, kbase, blk + (int64_t)C::kWarps * C::kBlocksPerIter);
 
         if (round_max > -INFINITY) {
-            // unit exponent for this round (every thread computes the same values)
+            // Unit exponent for this round; every thread computes the same values.  Common case:
+            // the maximum fits the current unit and no bin can overflow.
             const float cm = ceilf(round_max);
-            float e_new = e_unit;
-            if (!(cm - e_unit <= (float)kMaxWeightBits)) e_new = cm - (float)kUnitBits;
-            unsigned long long bound;
-            for (;;) {
-                const float shf = e_new - e_unit;                                     // >= 0, +inf on first use
-                bound = (shf >= 64.f) ? 0ull : (bin_bound >> (int)shf);
-                const float dexp = cm - e_new;                                        // <= kMaxWeightBits
-                const unsigned long long wtop = dexp <= 0.f ? 1ull : (1ull << (int)dexp);
-                bound += 1ull + (unsigned long long)C::kRoundTokens * (wtop + (wtop >> 20) + 1ull);
-                if (bound < (1ull << 32)) break;
-                e_new += 2.f;
+            const float dexp0 = cm - e_unit;                                    // +inf before the first round
+            bool keep = dexp0 <= (float)kMaxWeightBits;
+            if (keep) {
+                const unsigned long long wtop = dexp0 <= 0.f ? 1ull : (1ull << (int)dexp0);
+                const unsigned long long b2 = bin_bound + (unsigned long long)C::kRoundTokens * (wtop + (wtop >> 20) + 1ull);
+                keep = b2 < (1ull << 32);
+                if (keep) bin_bound = b2;
             }
-            if (e_new > e_unit && e_unit > -INFINITY) {
-                const float shf = e_new - e_unit;
-                const int k = shf >= 32.f ? 32 : (int)shf;
-                for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
-                    uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes +
-                                                               (i % (32 * C::kPlanes)) * 4);
-                    const uint32_t v = *bp;
-                    *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
+            if (!keep) {
+                float e_new = e_unit;
+                if (!(dexp0 <= (float)kMaxWeightBits)) e_new = cm - (float)kUnitBits;
+                unsigned long long bound;
+                for (;;) {
+                    const float shf = e_new - e_unit;                                 // >= 0, +inf on first use
+                    bound = (shf >= 64.f) ? 0ull : (bin_bound >> (int)shf);
+                    const float dexp = cm - e_new;                                    // <= kMaxWeightBits
+                    const unsigned long long wtop = dexp <= 0.f ? 1ull : (1ull << (int)dexp);
+                    bound += 1ull + (unsigned long long)C::kRoundTokens * (wtop + (wtop >> 20) + 1ull);
+                    if (bound < (1ull << 32)) break;
+                    e_new += 2.f;
                 }
-                __syncthreads();
+                if (e_new > e_unit && e_unit > -INFINITY) {
+                    const float shf = e_new - e_unit;
+                    const int k = shf >= 32.f ? 32 : (int)shf;
+                    for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
+                        uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes +
+                                                                   (i % (32 * C::kPlanes)) * 4);
+                        const uint32_t v = *bp;
+                        *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
+                    }
+                    __syncthreads();
+                }
+                e_unit = e_new;
+                bin_bound = bound;
             }
-            e_unit = e_new;
-            bin_bound = bound;
 
             // V side: integer weights into the bins of this lane's groups
 #pragma unroll
             for (int k = 0; k < 16; ++k)
 #pragma unroll
                 for (int u = 0; u < C::kLaneHeads; ++u) {
-                    const uint32_t w = __float2uint_rn(ex2(sc[u][k] - e_unit));
+                    const uint32_t w = __float2uint_rn(ex2(fmaf(sc[u][k], lut_scale, -e_unit)));
 #pragma unroll
                     for (int m = 0; m < C::kSlots; ++m)
                         atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 +
@@ -352,80 +464,66 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     __syncthreads();
 
     // ---------------------------------------------------------------- epilogue: bins x V centroids
-    // lane `lane` owns word `lane` of every plane and sums over the code values of its warp.
-    {
-        const int g = C::group_of(lane);
+    // Same ownership as the table build: a warp owns whole groups, lanes walk the code values.
+    // Rows are first rotated by their index so that a column read is bank-conflict free.
+    for (int j = warp; j < kRows; j += C::kWarps)
+#pragma unroll
+        for (int pl = 0; pl < C::kPlanes; ++pl) {
+            uint8_t* row = smem + C::kVOffset + j * kRowBytes + pl * 128;
+            const uint32_t v = *reinterpret_cast<const uint32_t*>(row + lane * 4);
+            __syncwarp();
+            *reinterpret_cast<uint32_t*>(row + ((lane + j) & 31) * 4) = v;
+        }
+    __syncthreads();
+#pragma unroll 1
+    for (int gi = 0; gi < C::kGroupsPerWarp; ++gi) {
+        const int g = warp * C::kGroupsPerWarp + gi;
         const float* cg = vcb + ((int64_t)hkv * G + g) * kRows * kC;
-        float acc[C::kPlanes][kC];
-        float lsum[C::kPlanes];
+        float acc[R][kC];
+        float lsum[R];                        // sum of the group's bins (the normaliser)
 #pragma unroll
-        for (int pl = 0; pl < C::kPlanes; ++pl) {
-            lsum[pl] = 0.f;
+        for (int h = 0; h < R; ++h) {
+            lsum[h] = 0.f;
 #pragma unroll
-            for (int i = 0; i < kC; ++i) acc[pl][i] = 0.f;
+            for (int i = 0; i < kC; ++i) acc[h][i] = 0.f;
         }
-#pragma unroll 4
-        for (int j = warp; j < kRows; j += C::kWarps) {
+#pragma unroll
+        for (int jb = 0; jb < kRows / 32; ++jb) {
+            const int j = jb * 32 + lane;
             float cv[kC];
-            if (kC == 8) {
-                const float4 a = *reinterpret_cast<const float4*>(cg + j * 8);
-                const float4 b = *reinterpret_cast<const float4*>(cg + j * 8 + 4);
-                cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
-                cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
-            } else {
-                const float4 a = *reinterpret_cast<const float4*>(cg + j * 4);
-                cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
-            }
+            load_centroid<kC>(cg + j * kC, cv);
 #pragma unroll
-            for (int pl = 0; pl < C::kPlanes; ++pl) {
-                const float bv = (float)*reinterpret_cast<const uint32_t*>(smem + C::kVOffset + j * kRowBytes + pl * 128 + lane * 4);
-                lsum[pl] += bv;
+            for (int h = 0; h < R; ++h) {
+                const uint8_t* row = smem + C::kVOffset + j * kRowBytes + C::plane_of(h) * 128;
+                uint32_t bi = *reinterpret_cast<const uint32_t*>(row + ((C::word_of(g, h) + j) & 31) * 4);
+                if (C::kReplica) bi += *reinterpret_cast<const uint32_t*>(row + ((16 + g + j) & 31) * 4);
+                const float bv = (float)bi;
+                if (gi == 0) lsum[h] += bv;
 #pragma unroll
-                for (int i = 0; i < kC; ++i) acc[pl][i] = fmaf(bv, cv[i], acc[pl][i]);
+                for (int i = 0; i < kC; ++i) acc[h][i] = fmaf(bv, cv[i], acc[h][i]);
             }
         }
-        if (C::kReplica) {       // the two halves of the plane are partial sums of the same bins
+        // Sum over the 32 lanes.  The kC channel sums are folded while they are exchanged: after
+        // the steps with lane masks 16, 8 (and 4 for kC = 8) a lane holds one channel, the
+        // remaining steps finish that channel.
 #pragma unroll
-            for (int i = 0; i < kC; ++i) acc[0][i] += __shfl_xor_sync(0xffffffffu, acc[0][i], 16);
-            lsum[0] += __shfl_xor_sync(0xffffffffu, lsum[0], 16);
+        for (int h = 0; h < R; ++h) {
+            float v = fold_channels<kC>(acc[h], lane);
+            // lane holds channel fold_channel_of<kC>(lane) summed over the lanes that share it
+            const int ch = fold_channel_of<kC>(lane);
+            if ((lane & (kC == 8 ? 3 : 7)) == 0) part_base[(int64_t)h * n_parts * stride + 2 + g * kC + ch] = v;
         }
-        __syncthreads();         // every warp is done reading the K table region reused below
-        // scratch (over the K table rows, which are no longer needed): [warp][plane][lane][kC + 1]
-        float* scratch = reinterpret_cast<float*>(smem);
-        static_assert(C::kWarps * C::kPlanes * 32 * (kC + 1) * 4 <= C::kTableBytes, "scratch must fit the tables");
-        // The scratch overwrites table rows (with one plane, bins included): the barrier above
-        // guarantees that every bin has been read.
+        if (g == 0) {
 #pragma unroll
-        for (int pl = 0; pl < C::kPlanes; ++pl) {
-            float* dst = scratch + ((warp * C::kPlanes + pl) * 32 + lane) * (kC + 1);
+            for (int h = 0; h < R; ++h) {
+                float l = lsum[h];
 #pragma unroll
-            for (int i = 0; i < kC; ++i) dst[i] = acc[pl][i];
-            dst[kC] = lsum[pl];
-        }
-        __syncthreads();
-        // one thread per (query head, channel): sum the warps' partial sums, write the partial
-        for (int o = threadIdx.x; o < R * 130; o += C::kThreads) {
-            const int h = o / 130, d = o % 130;
-            float* dstp = part_base + (int64_t)h * n_parts * stride;
-            if (d == 0) {
-                dstp[0] = e_unit;                 // reference exponent of this partial (log2 domain)
-                continue;
+                for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+                if (lane == 0) {
+                    part_base[(int64_t)h * n_parts * stride + 0] = e_unit;       // reference exponent (log2 domain)
+                    part_base[(int64_t)h * n_parts * stride + 1] = l;            // normaliser, in the same unit
+                }
             }
-            // word / plane that holds (head h, group gg)
-            const int gg = d == 1 ? 0 : (d - 2) / kC;
-            const int ch = d == 1 ? kC : (d - 2) % kC;
-            int pl, w;
-            if (C::kHalfRows) {
-                pl = (R <= 2) ? 0 : h / 2;
-                w = (R == 1 ? 0 : (h & 1) * 16) + gg;
-            } else {
-                pl = h;
-                w = gg;
-            }
-            float sum = 0.f;
-#pragma unroll
-            for (int wp = 0; wp < C::kWarps; ++wp) sum += scratch[((wp * C::kPlanes + pl) * 32 + w) * (kC + 1) + ch];
-            dstp[d] = sum;
         }
     }
 }
@@ -445,8 +543,9 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
     return cudaGetLastError();
 }
 
-// Context chunk per CTA: a multiple of the CTA's round, at least 2048 tokens, small enough for
-// about eight CTA waves on 148 SMs when the batch allows it.
+// Context chunk per CTA.  The table build and the bins x centroids product are paid once per
+// chunk, so chunks are long (up to 16384 tokens); they are halved only while the grid would not
+// give every CTA slot of the 148 SMs two CTAs, and never below 2048 tokens.
 template <int G, int R>
 int chunk_for(const Shape& sh)
 {
@@ -454,12 +553,13 @@ int chunk_for(const Shape& sh)
 #ifdef CQ_TUNE_CHUNK_TOKENS
     return CQ_TUNE_CHUNK_TOKENS;
 #endif
+    const int64_t round = C::kRoundTokens;
     const int64_t items = sh.n_seq * sh.n_kv_heads;
     const int64_t slots = 148 * C::kMinBlocks;
-    int64_t splits = (slots * 8 + items - 1) / items;
-    int64_t chunk = (sh.max_tokens + splits - 1) / splits;
-    if (chunk < 2048) chunk = 2048;
-    chunk = (chunk + C::kRoundTokens - 1) / C::kRoundTokens * C::kRoundTokens;
+    int64_t chunk = (sh.max_tokens + round - 1) / round * round;
+    if (chunk > 16384) chunk = 16384;
+    while (chunk > 2048 && items * ((sh.max_tokens + chunk - 1) / chunk) < 2 * slots)
+        chunk = (chunk / 2 + round - 1) / round * round;
     return (int)chunk;
 }
 
