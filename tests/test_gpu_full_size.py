@@ -1,0 +1,147 @@
+"""Parity at the full workload sizes, in the launch configuration bench.py times.
+
+The caches are built exactly as the benchmark builds them (CUDA encode of seeded synthetic
+activations, `bench.DecodeState`).  The oracle cannot recompute a whole workload, so a seeded
+sample of (sequence, KV head) items is checked one by one:
+
+* codes: the item's activations are drawn again with the same seeded generator, the oracle
+  encodes them on the CPU, and the CUDA codes of the item must match under the near-tie rule;
+* attention: the item's slice of the code buffers is overwritten with the ORACLE's codes (so no
+  oracle input comes from the CUDA path), the full-size attention call runs, and the item's
+  query heads must match the oracle's dense attention within the tolerance.
+
+Items are independent, so the other items of the batch (still CUDA-encoded) cannot influence
+the checked outputs.
+"""
+import numpy as np
+import pytest
+import torch
+
+import bench
+import oracle
+import paper_2405_03917_b200 as cq
+from paper_2405_03917_b200 import synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def item_activations(w, layer, is_v, head, s, cap):
+    """fp16 activations (cap, 128) of sequence s, head `head`, drawn as DecodeState draws them."""
+    src = synth.head_source(w.config, layer, head, is_v)
+    x = src.activations(w.n_seq * cap, DEV).view(w.n_seq, cap, w.head_dim)[s]
+    return x.cpu()
+
+
+def item_slice(w, cap, s, h):
+    nb = (cap + 15) // 16
+    size = nb * w.G * 16
+    start = (s * w.n_kv_heads + h) * size
+    return slice(start, start + size)
+
+
+def check_items(w, layer, st, items):
+    """items: list of (sequence, KV head).  Returns (near_ties, codes_checked, worst max-abs, worst rel-L2)."""
+    cap, D, c, b = st.cap, w.head_dim, w.c, w.b
+    R = w.n_q_heads // w.n_kv_heads
+    ties = total = 0
+    oracle_codes = {}
+    for (s, h) in items:
+        n = int(st.lens_cpu[s])
+        assert n >= 1
+        for is_v, buf, cb in ((False, st.k_codes, st.k_cb), (True, st.v_codes, st.v_cb)):
+            x = item_activations(w, layer, is_v, h, s, cap)                      # (cap, 128) fp16
+            cbh = cb[h:h + 1].cpu().numpy()
+            res = oracle.encode(x.numpy().reshape(cap, 1, D), cbh, c, b)
+            got = cq.cq_codes_to_rowmajor(buf[item_slice(w, cap, s, h)].clone(), 1, cap, 1, D, c, b).cpu().numpy()
+            t, tot = H.check_codes(x.numpy().reshape(cap, 1, D), cbh, got.reshape(cap, 1, w.G), c, b, res)
+            ties += t
+            total += tot
+            oracle_codes[(s, h, is_v)] = res[0].reshape(1, cap, 1, w.G)
+            # the attention below reads the oracle's codes for this item
+            patched = cq.cq_codes_from_rowmajor(
+                torch.from_numpy(res[0].astype(np.uint8).reshape(1, cap, 1, w.G)).to(DEV), D, c, b)
+            buf[item_slice(w, cap, s, h)] = patched
+    out = cq.cq_decode_attn(st.q, st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.seq_lens, st.scale, c, b, cap,
+                            out=st.out, workspace=st.ws)
+    torch.cuda.synchronize()
+    out = out.cpu().numpy()
+    worst_abs = worst_rel = 0.0
+    for (s, h) in items:
+        n = int(st.lens_cpu[s])
+        q = st.q[s, h * R:(h + 1) * R].cpu().numpy().reshape(1, R, D)
+        ref = oracle.decode_dense(q, oracle_codes[(s, h, False)], oracle_codes[(s, h, True)],
+                                  st.k_cb[h:h + 1].cpu().numpy(), st.v_cb[h:h + 1].cpu().numpy(),
+                                  np.array([n], np.int32), st.scale, c, b)
+        a, r = H.check_attn(out[s, h * R:(h + 1) * R], ref[0], f"{w.name} item (seq {s}, kv head {h})")
+        worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
+    return ties, total, worst_abs, worst_rel
+
+
+def seeded_items(w, n_items, seed, must=()):
+    rng = np.random.default_rng(seed)
+    items = list(must)
+    while len(items) < n_items:
+        it = (int(rng.integers(w.n_seq)), int(rng.integers(w.n_kv_heads)))
+        if it not in items:
+            items.append(it)
+    return items
+
+
+def test_config1_llama2_7b_4c8b_decode_full_size():
+    w = synth.WORKLOADS[1]
+    st = bench.DecodeState(w, 0, torch.device(DEV), cq)
+    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 16, 101))       # 16 items = 16 query heads x 4096 tokens
+    assert ties <= total // 500
+    print(f"config 1: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
+
+
+def test_config2_mistral_gqa_8c8b_decode_full_size():
+    w = synth.WORKLOADS[2]
+    st = bench.DecodeState(w, 0, torch.device(DEV), cq)
+    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 6, 202))        # 6 KV heads = 24 query heads x 16384 tokens
+    assert ties <= total // 500
+    print(f"config 2: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
+
+
+def test_config3_2c8b_prefill_encode_full_size():
+    w = synth.WORKLOADS[3]
+    D, c, b = w.head_dim, w.c, w.b
+    rng = np.random.default_rng(303)
+    for is_v in (False, True):
+        x = synth.layer_activations(w, 0, is_v, w.n_seq, w.n_tokens, device=DEV)
+        cb = synth.layer_codebooks(w, 0, is_v).to(DEV)
+        buf = torch.zeros(cq.cq_codes_bytes(w.n_seq, w.n_tokens, w.n_kv_heads, D, c, b), dtype=torch.uint8, device=DEV)
+        cq.cq_encode(x, cb, c, b, buf, w.n_tokens)
+        torch.cuda.synchronize()
+        ties = total = 0
+        for _ in range(8):                                                    # 8 x 8192 = 65536 vectors per tensor
+            s, h = int(rng.integers(w.n_seq)), int(rng.integers(w.n_kv_heads))
+            xs = x[s, :, h].cpu().numpy().reshape(w.n_tokens, 1, D)
+            got = cq.cq_codes_to_rowmajor(buf[item_slice(w, w.n_tokens, s, h)].clone(), 1, w.n_tokens, 1, D, c, b)
+            t, tot = H.check_codes(xs, cb[h:h + 1].cpu().numpy(), got.cpu().numpy().reshape(w.n_tokens, 1, w.G), c, b)
+            ties += t
+            total += tot
+        assert ties <= total // 500
+        print(f"config 3 {'V' if is_v else 'K'}: {total} codes checked, {ties} near-ties")
+        del x, buf
+
+
+def test_config4_llama2_13b_8c8b_layers_full_size():
+    # 8 of the 40 layers, each at the full per-layer shape (32 sequences x 40 heads, seeded lengths in
+    # [8192, 32768]); two items per layer, the shortest or the longest sequence among them
+    w = synth.WORKLOADS[4]
+    lens = w.lengths()
+    s_short, s_long = int(lens.argmin()), int(lens.argmax())
+    worst = (0.0, 0.0)
+    for k, layer in enumerate((0, 5, 11, 17, 23, 29, 34, 39)):
+        st = bench.DecodeState(w, layer, torch.device(DEV), cq)
+        rng = np.random.default_rng(400 + layer)
+        must = [((s_short if k % 2 == 0 else s_long), int(rng.integers(w.n_kv_heads)))]
+        ties, total, a, r = check_items(w, layer, st, seeded_items(w, 2, 404 + layer, must))
+        assert ties <= total // 500
+        worst = (max(worst[0], a), max(worst[1], r))
+        del st
+        torch.cuda.empty_cache()
+    print(f"config 4: worst attention max-abs {worst[0]:.2e} rel-L2 {worst[1]:.2e}")
