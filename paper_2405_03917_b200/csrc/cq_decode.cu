@@ -41,6 +41,7 @@ constexpr int kRows = 256;            // code values
 constexpr int kRowBytes = 256;        // bytes per table row
 constexpr int kUnitBits = 27;         // weight of the running-maximum token: (2^26, 2^27]
 constexpr int kMaxWeightBits = 30;    // a score may exceed the unit exponent by at most this
+constexpr float kBinLimit = 4.2e9f;   // bins stay below 2^32 with room for the rounding of the float bounds
 
 template <int G, int R>
 struct Cfg {
@@ -68,7 +69,7 @@ struct Cfg {
     // One plane: K and V planes share a row (K at +0, V at +128).  Two planes: separate tables.
     static constexpr int kVOffset = (kPlanes == 1) ? 128 : kRows * kRowBytes;
     static constexpr int kTableBytes = (kPlanes == 1) ? kRows * kRowBytes : 2 * kRows * kRowBytes;
-    static constexpr int kCtlBytes = 64 + R * 128 * 4;                   // control words + scaled query
+    static constexpr int kCtlBytes = 128 + R * 128 * 4;                  // control words + scaled query
     static constexpr int kSmemBytes = kTableBytes + kCtlBytes;
 
     // word inside a plane that lane (r, p) uses for its m-th code word
@@ -80,14 +81,32 @@ struct Cfg {
     __device__ static __forceinline__ int group_of(int w) { return kHalfRows ? (w & 15) : w; }
     __device__ static __forceinline__ int plane_of(int h) { return kHalfRows ? (R <= 2 ? 0 : h >> 1) : h; }
     __device__ static __forceinline__ int word_of(int g, int h) { return kHalfRows ? (R == 1 ? 0 : (h & 1) * 16) + g : g; }
+    // query head (of the KV head) that lane row r serves as its u-th head, and the head a table word belongs to
+    __device__ static __forceinline__ int lane_head(int u, int r) { return kHalfRows ? (R == 1 ? 0 : 2 * u + (r >> 2)) : u; }
+    __device__ static __forceinline__ int head_of_word(int word_in_row)
+    {
+        const int plane = word_in_row >> 5, w = word_in_row & 31;
+        return kHalfRows ? (R == 1 ? 0 : 2 * plane + (w >> 4)) : plane;
+    }
+    // v[lane_head(u, r)] without indexing a register array by a run-time value
+    template <int N>
+    __device__ static __forceinline__ float pick(const float (&v)[N], int u, int r)
+    {
+        float out = v[0];
+#pragma unroll
+        for (int h = 1; h < N; ++h) out = lane_head(u, r) == h ? v[h] : out;
+        return out;
+    }
     static constexpr int kGroupsPerWarp = G / kWarps;
     static_assert(G % kWarps == 0 && kSlots % 4 == 0, "ownership of groups by warps; four code words per MMA");
 };
 
 struct Ctl {
-    int rmax[3];        // per-iteration maximum score of the CTA (order-preserving int encoding)
-    float lut_absmax;   // largest |LUT| entry, as float bits (non-negative, so int order works)
+    int rmax[3][4];            // per round and query head: ceil of the largest score (order-preserving int encoding)
+    unsigned int rsum[3][4];   // per round and query head: sum of the round's weights, rounded up, in units of 256
+    float lut_absmax;          // largest |LUT| entry, as float bits (non-negative, so int order works)
 };
+static_assert(sizeof(Ctl) <= 128, "control block");
 
 __device__ __forceinline__ int enc_float(float f)
 {
@@ -217,7 +236,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     constexpr int kC = C::kC;
     extern __shared__ __align__(1024) uint8_t smem[];
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + C::kTableBytes);
-    float* qs = reinterpret_cast<float*>(smem + C::kTableBytes + 64);      // [R][128], scaled by scale*log2(e)
+    float* qs = reinterpret_cast<float*>(smem + C::kTableBytes + 128);     // [R][128], scaled by scale*log2(e)
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int r = lane >> 2, p = lane & 3;
@@ -244,8 +263,11 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     }
 
     // ---------------------------------------------------------------- set-up: query, LUT, bins
-    if (threadIdx.x < 3) ctl->rmax[threadIdx.x] = INT_MIN;
-    if (threadIdx.x == 3) ctl->lut_absmax = 0.f;
+    if (threadIdx.x < 12) {
+        ctl->rmax[threadIdx.x >> 2][threadIdx.x & 3] = INT_MIN;
+        ctl->rsum[threadIdx.x >> 2][threadIdx.x & 3] = 0u;
+    }
+    if (threadIdx.x == 12) ctl->lut_absmax = 0.f;
     for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
         qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)hkv * R) * 128 + i]) * scale_log2e;
     // bins start at zero (16-byte stores over the V planes)
@@ -348,8 +370,15 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         }
     };
 
-    float e_unit = -INFINITY;              // log2 of the weight unit; integer-valued once set
-    unsigned long long bin_bound = 0;      // upper bound on every bin
+    // Per query head of this KV head, identical in every thread: log2 of the weight unit (integer
+    // valued once set) and an upper bound on the sum of all weights added since the bins were
+    // last coarsened (hence on every bin).
+    float e_unit[R], total[R];
+#pragma unroll
+    for (int h = 0; h < R; ++h) { e_unit[h] = -INFINITY; total[h] = 0.f; }
+    constexpr bool kSplit = C::kHalfRows && R >= 2;      // the two half warps serve different query heads
+    const unsigned grp_mask = kSplit ? (lane < 16 ? 0x0000ffffu : 0xffff0000u) : 0xffffffffu;
+    const bool grp_leader = kSplit ? (lane & 15) == 0 : lane == 0;
     load_words(kw, kbase, blk0 + (int64_t)warp * C::kBlocksPerIter + qb);
 
     for (int it = 0; it < n_iters; ++it) {
@@ -394,71 +423,131 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 for (int u = 0; u < C::kLaneHeads; ++u)
                     if (tok0 + k >= t_end) sc[u][k] = -INFINITY;
         }
-        float mx = -INFINITY;
+        // Per head: reference exponent ref = ceil(largest score of this (half) warp), the weights
+        // 2^(score - ref) <= 1 kept as floats in place of the scores, and their sum.
+        const int slot = it % 3;
+        float ref[C::kLaneHeads], zsum[C::kLaneHeads];
 #pragma unroll
-        for (int k = 0; k < 16; ++k)
+        for (int u = 0; u < C::kLaneHeads; ++u) {
+            float mx = -INFINITY;
 #pragma unroll
-            for (int u = 0; u < C::kLaneHeads; ++u) mx = fmaxf(mx, sc[u][k]);
-        const int wmax = __reduce_max_sync(0xffffffffu, enc_float(mx * lut_scale));
-        if (lane == 0) atomicMax(&ctl->rmax[it % 3], wmax);
+            for (int k = 0; k < 16; ++k) mx = fmaxf(mx, sc[u][k]);
+            const float gm = dec_float(__reduce_max_sync(grp_mask, enc_float(mx * lut_scale)));
+            const bool any = gm > -INFINITY;
+            ref[u] = any ? ceilf(gm) : 0.f;
+            if (grp_leader) atomicMax(&ctl->rmax[slot][C::lane_head(u, r)], enc_float(any ? ref[u] : -INFINITY));
+            float z = 0.f;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const float wf = ex2(fmaf(sc[u][k], lut_scale, -ref[u]));
+                sc[u][k] = wf;
+                z += wf;
+            }
+            z = p == 0 ? z : 0.f;                        // the four lanes of a quad hold the same tokens
+#pragma unroll
+            for (int o = kSplit ? 8 : 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+            zsum[u] = z;
+        }
+        if (it == 0) {
+            // first round: the unit is set from the round's maximum before the sums are formed
+            __syncthreads();
+#pragma unroll
+            for (int h = 0; h < R; ++h) e_unit[h] = dec_float(ctl->rmax[slot][h]) - (float)kUnitBits;
+        }
+#pragma unroll
+        for (int u = 0; u < C::kLaneHeads; ++u) {
+            const float eu = C::template pick<R>(e_unit, u, r);
+            // the round's weights of this (half) warp in the current unit, rounded up, in units of 256
+            // (a u32 shared-memory add is fast, the 64-bit form is not)
+            const float cw = (zsum[u] * ex2(ref[u] - eu) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
+            const unsigned int ci = cw < 6.7e7f ? (unsigned int)cw : (1u << 26);     // saturates; 32 of these still fit
+            if (grp_leader) atomicAdd(&ctl->rsum[slot][C::lane_head(u, r)], ci);
+        }
         __syncthreads();
-        const float round_max = dec_float(ctl->rmax[it % 3]);
-        if (threadIdx.x == 0) ctl->rmax[(it + 2) % 3] = INT_MIN;
+        float cm[R], rs[R];
+        bool all_keep = true;
+#pragma unroll
+        for (int h = 0; h < R; ++h) {
+            cm[h] = dec_float(ctl->rmax[slot][h]);
+            const unsigned int sraw = ctl->rsum[slot][h];
+            rs[h] = sraw >= (1u << 26) ? INFINITY : (float)sraw * 256.f;
+            const bool keep = !(cm[h] > -INFINITY) ||
+                              (cm[h] - e_unit[h] <= (float)kMaxWeightBits && total[h] + rs[h] < kBinLimit);
+            all_keep = all_keep && keep;
+        }
+        if (threadIdx.x < 4) {
+            ctl->rmax[(it + 2) % 3][threadIdx.x] = INT_MIN;
+            ctl->rsum[(it + 2) % 3][threadIdx.x] = 0u;
+        }
 
         // the next iteration's K words travel while the V side runs
         load_words(kw, kbase, blk + (int64_t)C::kWarps * C::kBlocksPerIter);
 
-        if (round_max > -INFINITY) {
-            // Unit exponent for this round; every thread computes the same values.  Common case:
-            // the maximum fits the current unit and no bin can overflow.
-            const float cm = ceilf(round_max);
-            const float dexp0 = cm - e_unit;                                    // +inf before the first round
-            bool keep = dexp0 <= (float)kMaxWeightBits;
-            if (keep) {
-                const unsigned long long wtop = dexp0 <= 0.f ? 1ull : (1ull << (int)dexp0);
-                const unsigned long long b2 = bin_bound + (unsigned long long)C::kRoundTokens * (wtop + (wtop >> 20) + 1ull);
-                keep = b2 < (1ull << 32);
-                if (keep) bin_bound = b2;
-            }
-            if (!keep) {
-                float e_new = e_unit;
-                if (!(dexp0 <= (float)kMaxWeightBits)) e_new = cm - (float)kUnitBits;
-                unsigned long long bound;
-                for (;;) {
-                    const float shf = e_new - e_unit;                                 // >= 0, +inf on first use
-                    bound = (shf >= 64.f) ? 0ull : (bin_bound >> (int)shf);
-                    const float dexp = cm - e_new;                                    // <= kMaxWeightBits
-                    const unsigned long long wtop = dexp <= 0.f ? 1ull : (1ull << (int)dexp);
-                    bound += 1ull + (unsigned long long)C::kRoundTokens * (wtop + (wtop >> 20) + 1ull);
-                    if (bound < (1ull << 32)) break;
-                    e_new += 2.f;
+        if (all_keep) {
+#pragma unroll
+            for (int h = 0; h < R; ++h)
+                if (cm[h] > -INFINITY) total[h] = (total[h] + rs[h]) * 1.000001f;
+        } else {
+            // Some head needs a coarser unit: its top score left the range, or a bin could pass 2^32.
+            float shift[R];
+#pragma unroll
+            for (int h = 0; h < R; ++h) {
+                shift[h] = 0.f;
+                if (!(cm[h] > -INFINITY)) continue;
+                const bool range_ok = cm[h] - e_unit[h] <= (float)kMaxWeightBits;
+                if (range_ok && total[h] + rs[h] < kBinLimit) {
+                    total[h] = (total[h] + rs[h]) * 1.000001f;
+                    continue;
                 }
-                if (e_new > e_unit && e_unit > -INFINITY) {
-                    const float shf = e_new - e_unit;
-                    const int k = shf >= 32.f ? 32 : (int)shf;
-                    for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
-                        uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes +
-                                                                   (i % (32 * C::kPlanes)) * 4);
-                        const uint32_t v = *bp;
-                        *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
-                    }
-                    __syncthreads();
+                float e_new = range_ok ? e_unit[h] + 2.f : cm[h] - (float)kUnitBits;
+                const bool measured = range_ok && rs[h] < INFINITY;      // else: worst case of the round
+                float est = 0.f;
+                bool fits = false;
+                for (int tries = 0; tries < 48 && !fits; ++tries) {      // 2 bits per try: 96 bits always suffice
+                    const float down = ex2(e_unit[h] - e_new);            // 2^-shift, 0 when the shift is huge
+                    const float rnew = (measured ? rs[h] * down
+                                                 : (float)C::kRoundTokens * ex2(fmaxf(cm[h] - e_new, 0.f)) * 1.0001f) +
+                                       (float)C::kRoundTokens;
+                    est = (total[h] * down + 1.f + rnew) * 1.000001f;
+                    fits = est < kBinLimit;
+                    if (!fits) e_new += 2.f;
                 }
-                e_unit = e_new;
-                bin_bound = bound;
+                if (!fits) {                                              // not reachable with finite inputs
+                    e_new = fmaxf(cm[h] + 1.f, e_unit[h] + 40.f);
+                    est = 2.f * (float)C::kRoundTokens + 2.f;
+                }
+                shift[h] = e_new - e_unit[h];
+                e_unit[h] = e_new;
+                total[h] = est;
             }
+            for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
+                const int word = i % (32 * C::kPlanes);
+                const int hw = C::head_of_word(word);
+                float sf = shift[0];
+#pragma unroll
+                for (int h = 1; h < R; ++h) sf = hw == h ? shift[h] : sf;
+                if (sf > 0.f) {
+                    const int k = sf >= 32.f ? 32 : (int)sf;
+                    uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes + word * 4);
+                    const uint32_t v = *bp;
+                    *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
+                }
+            }
+            __syncthreads();
+        }
 
-            // V side: integer weights into the bins of this lane's groups
+        // V side: integer weights into the bins of this lane's groups
 #pragma unroll
-            for (int k = 0; k < 16; ++k)
+        for (int u = 0; u < C::kLaneHeads; ++u) {
+            const float f = ex2(ref[u] - C::template pick<R>(e_unit, u, r));      // power of two <= 2^kMaxWeightBits
 #pragma unroll
-                for (int u = 0; u < C::kLaneHeads; ++u) {
-                    const uint32_t w = __float2uint_rn(ex2(fmaf(sc[u][k], lut_scale, -e_unit)));
+            for (int k = 0; k < 16; ++k) {
+                const uint32_t w = __float2uint_rn(sc[u][k] * f);
 #pragma unroll
-                    for (int m = 0; m < C::kSlots; ++m)
-                        atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 +
-                                                                  row_index(vw[m], k, lane_off[m])), w);
-                }
+                for (int m = 0; m < C::kSlots; ++m)
+                    atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 +
+                                                              row_index(vw[m], k, lane_off[m])), w);
+            }
         }
     }
     __syncthreads();
@@ -520,7 +609,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
                 if (lane == 0) {
-                    part_base[(int64_t)h * n_parts * stride + 0] = e_unit;       // reference exponent (log2 domain)
+                    part_base[(int64_t)h * n_parts * stride + 0] = e_unit[h];    // reference exponent (log2 domain)
                     part_base[(int64_t)h * n_parts * stride + 1] = l;            // normaliser, in the same unit
                 }
             }
