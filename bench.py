@@ -1,8 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the CQ hot path on B200.
 
-One "step" is one decode step of one layer on the headline workload (config 2 of
-the benchmark spec: CQ-8c8b, Mistral-7B-shaped GQA, batch 64, context 16384): the new token's
+One "step" is one decode step over every layer of the workload (default: CQ-8c8b on a
+Mistral-7B-shaped GQA layer, batch 64, context 16384, one layer): per layer the new token's
 key and value vectors are CQ-encoded and appended (cq_encode, K and V), then every query
 head attends over the coded cache (cq_decode_attn).  Inputs are seeded and synthetic.
 
@@ -11,8 +11,9 @@ head attends over the coded cache (cq_decode_attn).  Inputs are seeded and synth
 
 Prints ONE JSON line (rank 0).  `value` is KV tokens/s with everything resident in HBM;
 `e2e` is the same metric through cq_decode_step_host with host buffers; `roofline` is the
-decode-attention call against the measured HBM copy bandwidth; `cpu_baseline` is the fp64
-CPU oracle on a bounded sample.  With --impl reference the oracle itself is the timed arm.
+decode-attention kernel against the measured HBM copy bandwidth (`shared_memory` beside it
+gives the same launch against the SM's shared-memory pipe, the unit that actually limits
+it); `cpu_baseline` is the fp64 CPU oracle on a bounded sample.  With --impl reference the oracle itself is the timed arm.
 Under torchrun every rank runs its own replica of the batch (weak scaling, no collective
 on the data path).
 """
@@ -336,7 +337,7 @@ def main():
 
     w = synth.WORKLOADS[int(args.workload[3])]
     config = {"workload": w.name, "c": w.c, "b": w.b, "n_seq": w.n_seq, "n_q_heads": w.n_q_heads,
-              "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "context": w.n_tokens, "layers_per_step": 1,
+              "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "context": w.n_tokens, "layers_per_step": w.n_layers,
               "step": "append-encode new token (K,V) + decode attention",
               "l2": "inputs exceed L2 (code buffers > 126 MB)" if w.name.startswith(("cfg2", "cfg4")) else
                     "inputs fit L2 (small case)"}
@@ -364,27 +365,36 @@ def main():
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
 
-    st = DecodeState(w, 0, dev, cq)
+    states = [DecodeState(w, layer, dev, cq) for layer in range(w.n_layers)]
+    st = states[0]
     torch.cuda.synchronize()
+
+    def step(ev):
+        # the events bracket the decode-attention call of the last layer
+        for i, sti in enumerate(states):
+            sti.step(cq, ev if (ev is not None and i == len(states) - 1) else None)
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    total_ms, inner_ms = time_steps(lambda ev: st.step(cq, ev), args.steps, args.warmup, world, dev)
+    total_ms, inner_ms = time_steps(step, args.steps, args.warmup, world, dev)
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step = total_ms / args.steps
-    kv_tokens = st.kv_tokens() * world
+    kv_tokens = sum(x.kv_tokens() for x in states) * world
     value = kv_tokens / (ms_per_step * 1e-3)
 
     # end to end: host buffers in, host result out, through cq_decode_step_host
     D = w.head_dim
     ws_h = torch.empty(cq.cq_decode_step_host_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, w.c, w.b, st.cap),
                        dtype=torch.uint8, device=dev)
-    q_h, k_h, v_h = st.q.cpu().pin_memory(), st.k_new.cpu().pin_memory(), st.v_new.cpu().pin_memory()
+    host = [(x.q.cpu().pin_memory(), x.k_new.cpu().pin_memory(), x.v_new.cpu().pin_memory()) for x in states]
     lens_h = (st.lens_cpu - 1).contiguous()
     out_h = torch.empty(w.n_seq, w.n_q_heads, D, dtype=torch.float32).pin_memory()
+
     def e2e_step():
-        cq.cq_decode_step_host(q_h, k_h, v_h, lens_h, st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.scale, w.c, w.b,
-                               st.cap, out_h, ws_h)
+        for x, (q_h, k_h, v_h) in zip(states, host):
+            cq.cq_decode_step_host(q_h, k_h, v_h, lens_h, x.k_codes, x.v_codes, x.k_cb, x.v_cb, x.scale, w.c, w.b,
+                                   x.cap, out_h, ws_h)
     for _ in range(3):
         e2e_step()
     torch.cuda.synchronize()
@@ -395,8 +405,9 @@ def main():
         e2e_step()
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / n_e2e, world, dev)
-    h2d = q_h.numel() * 2 + k_h.numel() * 2 + v_h.numel() * 2 + lens_h.numel() * 4
-    d2h = out_h.numel() * 4
+    q_h, k_h, v_h = host[0]
+    h2d = len(states) * (q_h.numel() * 2 + k_h.numel() * 2 + v_h.numel() * 2 + lens_h.numel() * 4)
+    d2h = len(states) * out_h.numel() * 4
 
     if rank != 0:
         if world > 1:
@@ -405,12 +416,13 @@ def main():
         return 0
 
     hbm, which = measured_peaks()
+    last = states[-1]
     dec_ms = statistics.mean(inner_ms)
-    achieved = st.algorithmic_bytes() / (dec_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "cq_decode_attn (main kernel + split merge)", "achieved": achieved,
-                "peak": hbm, "peak_source": which, "unit": "GB/s", "frac": achieved / hbm,
-                "frac_of_8tbs_nominal": achieved / 8000.0, "traffic": None,
-                "algorithmic_bytes_per_launch": st.algorithmic_bytes(), "launch_ms": dec_ms}
+    achieved = last.algorithmic_bytes() / (dec_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_tuned_kernel + merge_kernel (one cq_decode_attn call, one layer)",
+                "achieved": achieved, "peak": hbm, "peak_source": which + " copy bandwidth", "unit": "GB/s",
+                "frac": achieved / hbm, "frac_of_8tbs_nominal": achieved / 8000.0, "traffic": None,
+                "algorithmic_bytes_per_launch": last.algorithmic_bytes(), "launch_ms": dec_ms}
     tr = os.path.join(ROOT, "profiles", "decode_traffic.json")
     if os.path.exists(tr):
         try:
@@ -420,16 +432,24 @@ def main():
                 roofline["traffic_source"] = t.get("source")
         except Exception:
             pass
+    # The unit that limits the kernel: one 4-byte shared-memory lookup and one 4-byte shared-memory
+    # add per (token, KV head, group, query head of the KV head), 32 lanes per clock and SM.
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    lane_ops = 2.0 * last.kv_tokens() * w.n_kv_heads * w.G * (w.n_q_heads // w.n_kv_heads)
+    smem_peak = 148 * 32 * sm_mhz * 1e6
+    shared = {"bound": "shared-memory pipe (32 lanes/clk/SM x 148 SMs x sampled SM clock)",
+              "achieved": lane_ops / (dec_ms * 1e-3), "peak": smem_peak, "unit": "lane-ops/s",
+              "frac": lane_ops / (dec_ms * 1e-3) / smem_peak}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
-            "query_heads_per_s": w.n_seq * w.n_q_heads * world / (ms_per_step * 1e-3),
+            "query_heads_per_s": w.n_seq * w.n_q_heads * len(states) * world / (ms_per_step * 1e-3),
             "clocks": clocks,
             "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": args.steps * 4,
-            "roofline": roofline}
+            "gpu_launches": args.steps * 4 * len(states),
+            "roofline": roofline, "shared_memory": shared}
 
     if args.extras != "none" and world == 1:
         extras = {}
@@ -437,11 +457,12 @@ def main():
             extras["encode"] = extra_encode_cfg3(cq, dev)
             if args.extras == "all":
                 extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
+                extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
         except Exception as e:      # extras never hide the headline number
             extras["error"] = repr(e)
         line["extras"] = extras
     if not args.no_cpu_baseline and world == 1:
-        del st
+        del st, states, last
         torch.cuda.empty_cache()
         r = time_oracle(w, 10, 1)
         line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}

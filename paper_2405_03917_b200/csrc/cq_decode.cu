@@ -123,14 +123,6 @@ __device__ __forceinline__ uint4 ldg_codes(const uint4* p)
     return v;
 }
 
-// shared-memory load that keeps its place among the other volatile statements
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
-{
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
@@ -343,11 +335,10 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     const int64_t blk_lim = (t_end + kTokenBlock - 1) / kTokenBlock;       // blocks holding a valid token
     const int n_iters = (int)((t_end - t_begin + C::kRoundTokens - 1) / C::kRoundTokens);
     const int qb = (C::kBlocksPerIter == 8) ? r : (r & 3);                 // block of this quad inside the warp's iteration
-    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
 #ifdef CQ_TUNE_KBATCH
     constexpr int kBatch = CQ_TUNE_KBATCH;
 #else
-    constexpr int kBatch = C::kSlots >= 8 ? 2 : 4;                         // tokens whose lookups are in flight together
+    constexpr int kBatch = (C::kSlots * C::kLaneHeads >= 8) ? 2 : 4;       // tokens whose lookups are in flight together
 #endif
 
     uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a plane, per code word
@@ -391,28 +382,33 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         // the same token's lookups, so the token's score is the sum of both row sums.
         float sc[C::kLaneHeads][16];
 #pragma unroll
-        for (int k0 = 0; k0 < 16; k0 += kBatch)
+        for (int k0 = 0; k0 < 16; k0 += kBatch) {
+            // All lookups of a batch of tokens are issued before the first MMA needs one.  The row
+            // index of a code is formed once and serves every head (the planes are 128 bytes apart).
+            uint32_t a[kBatch][C::kLaneHeads][C::kSlots];
 #pragma unroll
-            for (int u = 0; u < C::kLaneHeads; ++u) {
-                // all lookups of a batch of tokens are issued before the first MMA needs one
-                uint32_t a[kBatch][C::kSlots];
+            for (int kk = 0; kk < kBatch; ++kk)
 #pragma unroll
-                for (int kk = 0; kk < kBatch; ++kk)
+                for (int m = 0; m < C::kSlots; ++m) {
+                    const uint32_t idx = row_index(kw[m], k0 + kk, lane_off[m]);
 #pragma unroll
-                    for (int m = 0; m < C::kSlots; ++m)
-                        a[kk][m] = lds_u32(smem_base + u * 128 + row_index(kw[m], k0 + kk, lane_off[m]));
+                    for (int u = 0; u < C::kLaneHeads; ++u)
+                        a[kk][u][m] = *reinterpret_cast<const volatile uint32_t*>(smem + u * 128 + idx);
+                }
 #pragma unroll
-                for (int kk = 0; kk < kBatch; ++kk) {
+            for (int kk = 0; kk < kBatch; ++kk)
+#pragma unroll
+                for (int u = 0; u < C::kLaneHeads; ++u) {
                     float tot = 0.f;
 #pragma unroll
                     for (int m = 0; m < C::kSlots; m += 4) {
                         float d[4] = {0.f, 0.f, 0.f, 0.f};
-                        mma_rowsum(d, a[kk][m], a[kk][m + 1], a[kk][m + 2], a[kk][m + 3]);
+                        mma_rowsum(d, a[kk][u][m], a[kk][u][m + 1], a[kk][u][m + 2], a[kk][u][m + 3]);
                         tot += d[0] + d[2];
                     }
                     sc[u][k0 + kk] = tot;
                 }
-            }
+        }
 
         // tokens past the end of the context get -inf (only the warp that holds the ragged end pays)
         if ((blk_warp + C::kBlocksPerIter) * kTokenBlock > t_end) {
@@ -541,14 +537,17 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         for (int u = 0; u < C::kLaneHeads; ++u) {
             const float f = ex2(ref[u] - C::template pick<R>(e_unit, u, r));      // power of two <= 2^kMaxWeightBits
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const uint32_t w = __float2uint_rn(sc[u][k] * f);
-#pragma unroll
-                for (int m = 0; m < C::kSlots; ++m)
-                    atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 +
-                                                              row_index(vw[m], k, lane_off[m])), w);
-            }
+            for (int k = 0; k < 16; ++k) sc[u][k] = __uint_as_float(__float2uint_rn(sc[u][k] * f));
         }
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+#pragma unroll
+            for (int m = 0; m < C::kSlots; ++m) {
+                const uint32_t idx = row_index(vw[m], k, lane_off[m]);
+#pragma unroll
+                for (int u = 0; u < C::kLaneHeads; ++u)
+                    atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 + idx), __float_as_uint(sc[u][k]));
+            }
     }
     __syncthreads();
 
@@ -634,7 +633,7 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
 
 // Context chunk per CTA.  The table build and the bins x centroids product are paid once per
 // chunk, so chunks are long (up to 16384 tokens); they are halved only while the grid would not
-// give every CTA slot of the 148 SMs two CTAs, and never below 2048 tokens.
+// give the CTA slots of the 148 SMs one and a half CTAs each, and never below 2048 tokens.
 template <int G, int R>
 int chunk_for(const Shape& sh)
 {
@@ -647,7 +646,7 @@ int chunk_for(const Shape& sh)
     const int64_t slots = 148 * C::kMinBlocks;
     int64_t chunk = (sh.max_tokens + round - 1) / round * round;
     if (chunk > 16384) chunk = 16384;
-    while (chunk > 2048 && items * ((sh.max_tokens + chunk - 1) / chunk) < 2 * slots)
+    while (chunk > 2048 && 2 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
         chunk = (chunk / 2 + round - 1) / round * round;
     return (int)chunk;
 }

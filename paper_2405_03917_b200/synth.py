@@ -106,7 +106,7 @@ def seq_lens_uniform(config: int, n_seq: int, lo: int, hi: int) -> torch.Tensor:
 
 @dataclasses.dataclass
 class Workload:
-    """Shapes of one BASELINE configuration."""
+    """Shapes of one benchmark configuration."""
     name: str
     config: int
     c: int

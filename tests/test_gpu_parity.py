@@ -1,6 +1,6 @@
 """GPU parity tests: the CUDA library (through its C ABI) against the fp64 CPU oracle,
 element by element, on the same seeded inputs.  Sizes here are ones the oracle finishes
-in seconds; the BASELINE-sized workloads are in test_gpu_full_size.py."""
+in seconds; the full-size workloads are in test_gpu_full_size.py."""
 import numpy as np
 import pytest
 import torch
