@@ -141,6 +141,37 @@ int cq_decode_attn(const void *q_fp16, const void *k_codes, const void *v_codes,
                    void *stream);
 
 /*
+ * cq_decode_attn for callers that have no device memory to give as a workspace and cannot
+ * obtain any.  (The paper has no counterpart to this entry point; it exists for the way the
+ * library gets embedded.)  Typical cases: a serving process that handed every free byte of
+ * HBM to its KV-cache pool at start-up, so a later cudaMalloc fails or stalls the device; or
+ * a plug-in that is called with nothing but the raw input and output pointers and has no
+ * route to its host's allocator.
+ *
+ * The split-K partials live in a fixed array of CQ_STATIC_WORKSPACE_BYTES bytes that is part
+ * of the library image: every GPU that loads the library holds these bytes until the process
+ * exits.  The function allocates and frees nothing, on the host or on the device.
+ *
+ *   - Arguments, layouts and result are those of cq_decode_attn, minus the workspace.
+ *   - Shapes whose partials need more than CQ_STATIC_WORKSPACE_BYTES
+ *     (cq_decode_attn_workspace_bytes(...) tells) are rejected with CQ_ERR_WORKSPACE and
+ *     nothing is launched; use cq_decode_attn with your own workspace for those.
+ *   - The first call on each device looks up the device address of the array (the device
+ *     must be current, as for every call); make that first call before any stream capture
+ *     begins.  A failure of the look-up is reported as CQ_ERR_CUDA.
+ *   - All calls on a device share the one array.  It keeps what the last call left in it;
+ *     that is harmless, because every call overwrites each partial it later reads and
+ *     nothing has to start at zero.  Two calls that overlap on the GPU (different streams,
+ *     or different host threads without ordering) race on the array and give wrong results:
+ *     order them on one stream or with events.
+ */
+#define CQ_STATIC_WORKSPACE_BYTES (4u << 20)
+int cq_decode_attn_static(const void *q_fp16, const void *k_codes, const void *v_codes,
+                          const float *k_cb, const float *v_cb, const int32_t *seq_lens, float scale,
+                          int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                          int64_t max_tokens, float *out, void *stream);
+
+/*
  * Same operation with an explicit kernel choice, for tests and benchmarks:
  * variant 0 = automatic (what cq_decode_attn uses), 1 = generic kernel,
  * 2 = tuned kernel (CQ_ERR_UNSUPPORTED when the shape has none).

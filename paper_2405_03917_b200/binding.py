@@ -18,7 +18,8 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 # Every symbol include/cq.h declares.
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
-           "cq_decode_attn_variant", "cq_decode_step_host_workspace_bytes", "cq_decode_step_host"]
+           "cq_decode_attn_variant", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
+           "cq_decode_step_host"]
 
 
 class CQError(RuntimeError):
@@ -62,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.cq_decode_attn_variant.restype = i32
         L.cq_decode_attn_variant.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp,
                                              sz, i32, vp]
+        L.cq_decode_attn_static.restype = i32
+        L.cq_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp]
         L.cq_decode_step_host_workspace_bytes.restype = sz
         L.cq_decode_step_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
         L.cq_decode_step_host.restype = i32
@@ -182,6 +185,27 @@ def cq_decode_attn(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor
                                       _dev(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
                                       workspace.numel(), variant, _stream())
     _check(st, "cq_decode_attn")
+    return out
+
+
+STATIC_WORKSPACE_BYTES = 4 << 20      # CQ_STATIC_WORKSPACE_BYTES of include/cq.h
+
+
+def cq_decode_attn_static(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor,
+                          v_cb: torch.Tensor, seq_lens: torch.Tensor, scale: float, c: int, b: int, max_tokens: int,
+                          out: torch.Tensor) -> torch.Tensor:
+    """cq_decode_attn without a workspace: the partials go to the array built into the library
+    (shapes that need more than STATIC_WORKSPACE_BYTES raise CQError with CQ_ERR_WORKSPACE).
+    This wrapper allocates nothing either: `out` is the caller's.  Calls that overlap on the
+    GPU share the array and must be ordered by the caller."""
+    n_seq, n_q_heads, head_dim = q.shape
+    n_kv_heads = k_cb.shape[0]
+    st = lib().cq_decode_attn_static(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+                                     _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
+                                     _dev(v_cb, torch.float32, "v_cb"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                     float(scale), n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
+                                     _dev(out, torch.float32, "out"), _stream())
+    _check(st, "cq_decode_attn_static")
     return out
 
 

@@ -1,4 +1,6 @@
 // extern "C" entry points of the CQ library: host-side validation and dispatch only.
+#include <mutex>
+
 #include "cq_common.cuh"
 
 using namespace cq;
@@ -179,6 +181,55 @@ int cq_decode_attn(const void* q_fp16, const void* k_codes, const void* v_codes,
 {
     return cq_decode_attn_variant(q_fp16, k_codes, v_codes, k_cb, v_cb, seq_lens, scale, n_seq, n_q_heads, n_kv_heads,
                                   head_dim, c, b, max_tokens, out, workspace, workspace_bytes, 0, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// cq_decode_attn_static: the split-K partials live in this array instead of a caller workspace.
+// In host code the name `g_static_workspace` is only a handle for the runtime, not a device
+// address; the address a kernel can use comes from cudaGetSymbolAddress, looked up once per
+// device and remembered here.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_workspace[CQ_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};          // device address of g_static_workspace, per device ordinal
+
+// Device address of the array on the current device; nullptr (and *err set) when the look-up fails.
+void* static_workspace(cudaError_t* err)
+{
+    int dev = -1;
+    *err = cudaGetDevice(&dev);
+    if (*err != cudaSuccess) return nullptr;
+    if (dev < 0 || dev >= kMaxDevices) { *err = cudaErrorInvalidDevice; return nullptr; }
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        *err = cudaGetSymbolAddress(&p, g_static_workspace);
+        if (*err != cudaSuccess) return nullptr;
+        g_static_ptr[dev] = p;
+    }
+    return g_static_ptr[dev];
+}
+}  // namespace
+
+int cq_decode_attn_static(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
+                          const float* v_cb, const int32_t* seq_lens, float scale, int n_seq, int n_q_heads,
+                          int n_kv_heads, int head_dim, int c, int b, int64_t max_tokens, float* out, void* stream)
+{
+    if (!q_fp16 || !k_codes || !v_codes || !k_cb || !v_cb || !seq_lens || !out) return CQ_ERR_NULL;
+    const size_t need = cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens);
+    if (need == 0) {
+        Shape sh;
+        return make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
+    }
+    if (need > (size_t)CQ_STATIC_WORKSPACE_BYTES) return CQ_ERR_WORKSPACE;     // too large for the built-in array
+    cudaError_t err = cudaSuccess;
+    void* ws = static_workspace(&err);
+    if (!ws) return CQ_ERR_CUDA;
+    return cq_decode_attn(q_fp16, k_codes, v_codes, k_cb, v_cb, seq_lens, scale, n_seq, n_q_heads, n_kv_heads,
+                          head_dim, c, b, max_tokens, out, ws, (size_t)CQ_STATIC_WORKSPACE_BYTES, stream);
 }
 
 // Staging area of cq_decode_step_host inside the caller's workspace (all 256-byte aligned):
