@@ -41,7 +41,8 @@ constexpr int kRows = 256;            // code values
 constexpr int kRowBytes = 256;        // bytes per table row
 constexpr int kUnitBits = 27;         // weight of the running-maximum token: (2^26, 2^27]
 constexpr int kMaxWeightBits = 30;    // a score may exceed the unit exponent by at most this
-constexpr float kBinLimit = 4.2e9f;   // bins stay below 2^32 with room for the rounding of the float bounds
+constexpr unsigned int kBinLimit256 = 16000000u;   // bins stay below 2^32: bound on their sum, in units of 256
+constexpr int kUnset = INT_MIN;                    // no score seen yet
 
 template <int G, int R>
 struct Cfg {
@@ -90,9 +91,9 @@ struct Cfg {
     }
     // v[lane_head(u, r)] without indexing a register array by a run-time value
     template <int N>
-    __device__ static __forceinline__ float pick(const float (&v)[N], int u, int r)
+    __device__ static __forceinline__ int pick(const int (&v)[N], int u, int r)
     {
-        float out = v[0];
+        int out = v[0];
 #pragma unroll
         for (int h = 1; h < N; ++h) out = lane_head(u, r) == h ? v[h] : out;
         return out;
@@ -102,7 +103,7 @@ struct Cfg {
 };
 
 struct Ctl {
-    int rmax[3][4];            // per round and query head: ceil of the largest score (order-preserving int encoding)
+    int rmax[3][4];            // per round and query head: ceil of the largest score (kUnset: no token)
     unsigned int rsum[3][4];   // per round and query head: sum of the round's weights, rounded up, in units of 256
     float lut_absmax;          // largest |LUT| entry, as float bits (non-negative, so int order works)
 };
@@ -121,6 +122,13 @@ __device__ __forceinline__ uint4 ldg_codes(const uint4* p)
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
+}
+
+// 2^d for an integer d; 0 below the normal range, saturates at 2^127
+__device__ __forceinline__ float pow2i(int d)
+{
+    d = d > 127 ? 127 : d;
+    return d < -126 ? 0.f : __int_as_float((127 + d) << 23);
 }
 
 __device__ __forceinline__ float ex2(float x)
@@ -256,7 +264,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 
     // ---------------------------------------------------------------- set-up: query, LUT, bins
     if (threadIdx.x < 12) {
-        ctl->rmax[threadIdx.x >> 2][threadIdx.x & 3] = INT_MIN;
+        ctl->rmax[threadIdx.x >> 2][threadIdx.x & 3] = kUnset;
         ctl->rsum[threadIdx.x >> 2][threadIdx.x & 3] = 0u;
     }
     if (threadIdx.x == 12) ctl->lut_absmax = 0.f;
@@ -361,12 +369,13 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         }
     };
 
-    // Per query head of this KV head, identical in every thread: log2 of the weight unit (integer
-    // valued once set) and an upper bound on the sum of all weights added since the bins were
-    // last coarsened (hence on every bin).
-    float e_unit[R], total[R];
+    // Per query head of this KV head, identical in every thread: log2 of the weight unit (unset
+    // before the first round) and an upper bound, in units of 256, on the sum of all weights added
+    // since the bins were last coarsened (hence on every bin).
+    int e_unit[R];
+    unsigned int total[R];
 #pragma unroll
-    for (int h = 0; h < R; ++h) { e_unit[h] = -INFINITY; total[h] = 0.f; }
+    for (int h = 0; h < R; ++h) { e_unit[h] = kUnset; total[h] = 0u; }
     constexpr bool kSplit = C::kHalfRows && R >= 2;      // the two half warps serve different query heads
     const unsigned grp_mask = kSplit ? (lane < 16 ? 0x0000ffffu : 0xffff0000u) : 0xffffffffu;
     const bool grp_leader = kSplit ? (lane & 15) == 0 : lane == 0;
@@ -419,10 +428,13 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 for (int u = 0; u < C::kLaneHeads; ++u)
                     if (tok0 + k >= t_end) sc[u][k] = -INFINITY;
         }
-        // Per head: reference exponent ref = ceil(largest score of this (half) warp), the weights
-        // 2^(score - ref) <= 1 kept as floats in place of the scores, and their sum.
+        // Per head: reference exponent ref = ceil(largest score of this (half) warp).  The four lanes
+        // of a quad hold the same 16 scores; lane p turns tokens p, p+4, p+8, p+12 into weights
+        // 2^(score - ref) <= 1 (exponentials are the scarce resource here), and the integer weights
+        // are handed round the quad by shuffles just before the bins are updated.
         const int slot = it % 3;
-        float ref[C::kLaneHeads], zsum[C::kLaneHeads];
+        int ref[C::kLaneHeads];
+        float wown[C::kLaneHeads][4], zsum[C::kLaneHeads];
 #pragma unroll
         for (int u = 0; u < C::kLaneHeads; ++u) {
             float mx = -INFINITY;
@@ -430,16 +442,18 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             for (int k = 0; k < 16; ++k) mx = fmaxf(mx, sc[u][k]);
             const float gm = dec_float(__reduce_max_sync(grp_mask, enc_float(mx * lut_scale)));
             const bool any = gm > -INFINITY;
-            ref[u] = any ? ceilf(gm) : 0.f;
-            if (grp_leader) atomicMax(&ctl->rmax[slot][C::lane_head(u, r)], enc_float(any ? ref[u] : -INFINITY));
+            ref[u] = any ? (int)fminf(fmaxf(ceilf(gm), -1.0e9f), 1.0e9f) : 0;
+            if (grp_leader && any) atomicMax(&ctl->rmax[slot][C::lane_head(u, r)], ref[u]);
+            const float fref = (float)ref[u];
             float z = 0.f;
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const float wf = ex2(fmaf(sc[u][k], lut_scale, -ref[u]));
-                sc[u][k] = wf;
-                z += wf;
+            for (int j = 0; j < 4; ++j) {
+                const float s01 = (p & 1) ? sc[u][4 * j + 1] : sc[u][4 * j];
+                const float s23 = (p & 1) ? sc[u][4 * j + 3] : sc[u][4 * j + 2];
+                const float own = (p & 2) ? s23 : s01;                    // score of token 4 j + p
+                wown[u][j] = ex2(fmaf(own, lut_scale, -fref));
+                z += wown[u][j];
             }
-            z = p == 0 ? z : 0.f;                        // the four lanes of a quad hold the same tokens
 #pragma unroll
             for (int o = kSplit ? 8 : 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
             zsum[u] = z;
@@ -448,31 +462,30 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             // first round: the unit is set from the round's maximum before the sums are formed
             __syncthreads();
 #pragma unroll
-            for (int h = 0; h < R; ++h) e_unit[h] = dec_float(ctl->rmax[slot][h]) - (float)kUnitBits;
+            for (int h = 0; h < R; ++h) e_unit[h] = ctl->rmax[slot][h] - kUnitBits;
         }
 #pragma unroll
         for (int u = 0; u < C::kLaneHeads; ++u) {
-            const float eu = C::template pick<R>(e_unit, u, r);
+            const int eu = C::template pick<R>(e_unit, u, r);
             // the round's weights of this (half) warp in the current unit, rounded up, in units of 256
             // (a u32 shared-memory add is fast, the 64-bit form is not)
-            const float cw = (zsum[u] * ex2(ref[u] - eu) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
+            const float cw = (zsum[u] * pow2i(ref[u] - eu) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
             const unsigned int ci = cw < 6.7e7f ? (unsigned int)cw : (1u << 26);     // saturates; 32 of these still fit
             if (grp_leader) atomicAdd(&ctl->rsum[slot][C::lane_head(u, r)], ci);
         }
         __syncthreads();
-        float cm[R], rs[R];
+        int cm[R];
+        unsigned int rs[R];
         bool all_keep = true;
 #pragma unroll
         for (int h = 0; h < R; ++h) {
-            cm[h] = dec_float(ctl->rmax[slot][h]);
-            const unsigned int sraw = ctl->rsum[slot][h];
-            rs[h] = sraw >= (1u << 26) ? INFINITY : (float)sraw * 256.f;
-            const bool keep = !(cm[h] > -INFINITY) ||
-                              (cm[h] - e_unit[h] <= (float)kMaxWeightBits && total[h] + rs[h] < kBinLimit);
+            cm[h] = ctl->rmax[slot][h];
+            rs[h] = ctl->rsum[slot][h];
+            const bool keep = cm[h] == kUnset || (cm[h] - e_unit[h] <= kMaxWeightBits && total[h] + rs[h] < kBinLimit256);
             all_keep = all_keep && keep;
         }
         if (threadIdx.x < 4) {
-            ctl->rmax[(it + 2) % 3][threadIdx.x] = INT_MIN;
+            ctl->rmax[(it + 2) % 3][threadIdx.x] = kUnset;
             ctl->rsum[(it + 2) % 3][threadIdx.x] = 0u;
         }
 
@@ -481,49 +494,47 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 
         if (all_keep) {
 #pragma unroll
-            for (int h = 0; h < R; ++h)
-                if (cm[h] > -INFINITY) total[h] = (total[h] + rs[h]) * 1.000001f;
+            for (int h = 0; h < R; ++h) total[h] += rs[h];                 // rs is 0 for a head without tokens
         } else {
             // Some head needs a coarser unit: its top score left the range, or a bin could pass 2^32.
-            float shift[R];
+            int shift[R];
 #pragma unroll
             for (int h = 0; h < R; ++h) {
-                shift[h] = 0.f;
-                if (!(cm[h] > -INFINITY)) continue;
-                const bool range_ok = cm[h] - e_unit[h] <= (float)kMaxWeightBits;
-                if (range_ok && total[h] + rs[h] < kBinLimit) {
-                    total[h] = (total[h] + rs[h]) * 1.000001f;
+                shift[h] = 0;
+                if (cm[h] == kUnset) continue;
+                const bool range_ok = cm[h] - e_unit[h] <= kMaxWeightBits;
+                if (range_ok && total[h] + rs[h] < kBinLimit256) {
+                    total[h] += rs[h];
                     continue;
                 }
-                float e_new = range_ok ? e_unit[h] + 2.f : cm[h] - (float)kUnitBits;
-                const bool measured = range_ok && rs[h] < INFINITY;      // else: worst case of the round
+                const bool measured = range_ok && rs[h] < (1u << 26);    // else: worst case of the round
+                int e_new = range_ok ? e_unit[h] + 2 : cm[h] - kUnitBits;
                 float est = 0.f;
                 bool fits = false;
                 for (int tries = 0; tries < 48 && !fits; ++tries) {      // 2 bits per try: 96 bits always suffice
-                    const float down = ex2(e_unit[h] - e_new);            // 2^-shift, 0 when the shift is huge
-                    const float rnew = (measured ? rs[h] * down
-                                                 : (float)C::kRoundTokens * ex2(fmaxf(cm[h] - e_new, 0.f)) * 1.0001f) +
+                    const float down = pow2i(e_unit[h] - e_new);          // 2^-shift, 0 when the shift is huge
+                    const float rnew = (measured ? (float)rs[h] * 256.f * down
+                                                 : (float)C::kRoundTokens * pow2i(cm[h] > e_new ? cm[h] - e_new : 0) * 1.0001f) +
                                        (float)C::kRoundTokens;
-                    est = (total[h] * down + 1.f + rnew) * 1.000001f;
-                    fits = est < kBinLimit;
-                    if (!fits) e_new += 2.f;
+                    est = ((float)total[h] * 256.f * down + 1.f + rnew) * 1.000001f;
+                    fits = est < 256.f * (float)kBinLimit256;
+                    if (!fits) e_new += 2;
                 }
                 if (!fits) {                                              // not reachable with finite inputs
-                    e_new = fmaxf(cm[h] + 1.f, e_unit[h] + 40.f);
+                    e_new = (cm[h] + 1 > e_unit[h] + 40) ? cm[h] + 1 : e_unit[h] + 40;
                     est = 2.f * (float)C::kRoundTokens + 2.f;
                 }
                 shift[h] = e_new - e_unit[h];
                 e_unit[h] = e_new;
-                total[h] = est;
+                total[h] = (unsigned int)(est * (1.f / 256.f)) + 1u;
             }
             for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
                 const int word = i % (32 * C::kPlanes);
                 const int hw = C::head_of_word(word);
-                float sf = shift[0];
+                int k = shift[0];
 #pragma unroll
-                for (int h = 1; h < R; ++h) sf = hw == h ? shift[h] : sf;
-                if (sf > 0.f) {
-                    const int k = sf >= 32.f ? 32 : (int)sf;
+                for (int h = 1; h < R; ++h) k = hw == h ? shift[h] : k;
+                if (k > 0) {
                     uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes + word * 4);
                     const uint32_t v = *bp;
                     *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
@@ -532,22 +543,27 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             __syncthreads();
         }
 
-        // V side: integer weights into the bins of this lane's groups
+        // V side: integer weights (own tokens), handed round the quad, into the bins of this lane's groups
+        uint32_t wint[C::kLaneHeads][4];
 #pragma unroll
         for (int u = 0; u < C::kLaneHeads; ++u) {
-            const float f = ex2(ref[u] - C::template pick<R>(e_unit, u, r));      // power of two <= 2^kMaxWeightBits
+            const float f = pow2i(ref[u] - C::template pick<R>(e_unit, u, r));     // power of two <= 2^kMaxWeightBits
 #pragma unroll
-            for (int k = 0; k < 16; ++k) sc[u][k] = __uint_as_float(__float2uint_rn(sc[u][k] * f));
+            for (int j = 0; j < 4; ++j) wint[u][j] = __float2uint_rn(wown[u][j] * f);
         }
 #pragma unroll
-        for (int k = 0; k < 16; ++k)
+        for (int k = 0; k < 16; ++k) {
+            uint32_t wk[C::kLaneHeads];
+#pragma unroll
+            for (int u = 0; u < C::kLaneHeads; ++u) wk[u] = __shfl_sync(0xffffffffu, wint[u][k >> 2], (lane & ~3) | (k & 3));
 #pragma unroll
             for (int m = 0; m < C::kSlots; ++m) {
                 const uint32_t idx = row_index(vw[m], k, lane_off[m]);
 #pragma unroll
                 for (int u = 0; u < C::kLaneHeads; ++u)
-                    atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 + idx), __float_as_uint(sc[u][k]));
+                    atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 + idx), wk[u]);
             }
+        }
     }
     __syncthreads();
 
@@ -608,7 +624,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
                 if (lane == 0) {
-                    part_base[(int64_t)h * n_parts * stride + 0] = e_unit[h];    // reference exponent (log2 domain)
+                    part_base[(int64_t)h * n_parts * stride + 0] = (float)e_unit[h];   // reference exponent (log2 domain)
                     part_base[(int64_t)h * n_parts * stride + 1] = l;            // normaliser, in the same unit
                 }
             }
