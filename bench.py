@@ -53,6 +53,15 @@ def measured_peaks():
     return HBM_FALLBACK_GBS, "fallback"
 
 
+def kernel_source_hash():
+    """sha256 over the decode kernel's source files (the kernel the roofline object describes)."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("cq_decode.cu", "cq_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2405_03917_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -69,7 +78,7 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=f,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -254,21 +263,28 @@ def oracle_step(w, st):
                                w.head_dim ** -0.5, w.c, w.b)
 
 
-def time_oracle(w, steps, warmup):
+def time_oracle(w, steps, warmup, target_s=None):
+    """Times oracle_step on sequence 0 of the batch.  With target_s the step count is chosen so
+    that the timed region is about that many seconds of CPU work."""
     import oracle
     st = oracle_sample_state(w, 1)
     for _ in range(warmup):
         oracle_step(w, st)
+    if target_s is not None:
+        t0 = time.perf_counter()
+        oracle_step(w, st)
+        one = max(time.perf_counter() - t0, 1e-6)
+        steps = int(min(max(target_s / one, 3), 5000))
     t0 = time.perf_counter()
     for _ in range(steps):
         oracle_step(w, st)
     dt = (time.perf_counter() - t0) / steps
     toks = int(st["lens"].sum())
     return {"value": toks / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"sequence 0 of the batch ({toks} tokens, all {w.n_kv_heads} KV heads / {w.n_q_heads} query "
-                      f"heads): append-encode + dense attention, mean of {steps} steps; cache encoded by the "
-                      f"oracle beforehand (untimed)",
-            "ms_per_step": dt * 1e3}
+            "sample": f"sequence 0 of the batch, layer 0 ({toks} tokens, all {w.n_kv_heads} KV heads / {w.n_q_heads} query "
+                      f"heads): append-encode + dense attention, mean of {steps} steps ({dt * steps:.1f} s); cache encoded "
+                      f"by the oracle beforehand (untimed)",
+            "ms_per_step": dt * 1e3, "steps": steps}
 
 
 # ------------------------------------------------------------------------------- extras
@@ -326,8 +342,8 @@ def extra_decode(cq, dev, w, reps=20):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg4"])
     ap.add_argument("--extras", default="default", choices=["none", "default", "all"])
@@ -427,7 +443,8 @@ def main():
     if os.path.exists(tr):
         try:
             t = json.load(open(tr)).get(w.name)
-            if t:
+            # the counters describe one build of the kernel: any later edit of its source voids them
+            if t and t.get("kernel_source_sha256") == kernel_source_hash():
                 roofline["traffic"] = t["dram_bytes_per_launch"]
                 roofline["traffic_source"] = t.get("source")
         except Exception:
@@ -464,7 +481,7 @@ def main():
     if not args.no_cpu_baseline and world == 1:
         del st, states, last
         torch.cuda.empty_cache()
-        r = time_oracle(w, 10, 1)
+        r = time_oracle(w, 10, 1, target_s=12.0)
         line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
     print(json.dumps(line))
     return 0
