@@ -98,13 +98,17 @@ struct Cfg {
         for (int h = 1; h < N; ++h) out = lane_head(u, r) == h ? v[h] : out;
         return out;
     }
+    static constexpr int kLog2Groups = kWarps == 16 ? 4 : 3;             // log2 of the warps that add to a head's bins per round
     static constexpr int kGroupsPerWarp = G / kWarps;
     static_assert(G % kWarps == 0 && kSlots % 4 == 0, "ownership of groups by warps; four code words per MMA");
 };
 
 struct Ctl {
-    int rmax[3][4];            // per round and query head: ceil of the largest score (kUnset: no token)
-    unsigned int rsum[3][4];   // per round and query head: sum of the round's weights, rounded up, in units of 256
+    int e_cur[4];              // per query head: log2 of the weight unit of its bins (kUnset before the first tokens)
+    unsigned int total[4];     // per query head: bound, in units of 256, on the sum of the weights added since the last coarsening
+    int req_ref[4];            // coarsening request: largest score exponent the requesters need to represent
+    int req_need[4];           // coarsening request: log2 bound of the largest round sum of one (half) warp
+    int want;                  // non-zero: a warp asks every warp to stop adding and coarsen
     float lut_absmax;          // largest |LUT| entry, as float bits (non-negative, so int order works)
 };
 static_assert(sizeof(Ctl) <= 128, "control block");
@@ -122,6 +126,13 @@ __device__ __forceinline__ uint4 ldg_codes(const uint4* p)
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
+}
+
+// Barrier 1 of the CTA, for the coarsening events: warps reach it from different places of the
+// code (bar.sync counts arrivals per barrier, whatever instruction they come from).
+__device__ __forceinline__ void event_barrier(int n_threads)
+{
+    asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory");
 }
 
 // 2^d for an integer d; 0 below the normal range, saturates at 2^127
@@ -263,11 +274,13 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     }
 
     // ---------------------------------------------------------------- set-up: query, LUT, bins
-    if (threadIdx.x < 12) {
-        ctl->rmax[threadIdx.x >> 2][threadIdx.x & 3] = kUnset;
-        ctl->rsum[threadIdx.x >> 2][threadIdx.x & 3] = 0u;
+    if (threadIdx.x < 4) {
+        ctl->e_cur[threadIdx.x] = kUnset;
+        ctl->total[threadIdx.x] = 0u;
+        ctl->req_ref[threadIdx.x] = kUnset;
+        ctl->req_need[threadIdx.x] = kUnset;
     }
-    if (threadIdx.x == 12) ctl->lut_absmax = 0.f;
+    if (threadIdx.x == 4) { ctl->want = 0; ctl->lut_absmax = 0.f; }
     for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
         qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)hkv * R) * 128 + i]) * scale_log2e;
     // bins start at zero (16-byte stores over the V planes)
@@ -369,13 +382,69 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         }
     };
 
-    // Per query head of this KV head, identical in every thread: log2 of the weight unit (unset
-    // before the first round) and an upper bound, in units of 256, on the sum of all weights added
-    // since the bins were last coarsened (hence on every bin).
-    int e_unit[R];
-    unsigned int total[R];
+    // Weight units.  Each query head's bins count in units of 2^e_cur[h].  A warp adds its tokens'
+    // weights without waiting for the others as long as (a) its largest score fits the unit
+    // (weight <= 2^kMaxWeightBits) and (b) its reservation keeps the head's running total - a bound
+    // on every bin - below 2^32.  Otherwise it raises `want`; every warp joins the coarsening
+    // event at its next check (or at the end of its loop): barrier, bins shifted right, new unit,
+    // barrier.  No warp is inside its V side during an event, so bins and unit stay consistent.
+    auto coarsen = [&]() {                       // entered by every thread, right after the event's first barrier
+        int shift[R], e_next[R];
+        unsigned int t_next[R];
+        bool any_shift = false;
 #pragma unroll
-    for (int h = 0; h < R; ++h) { e_unit[h] = kUnset; total[h] = 0u; }
+        for (int h = 0; h < R; ++h) {
+            const int e = ctl->e_cur[h], cmr = ctl->req_ref[h], need = ctl->req_need[h];
+            const unsigned int tot = ctl->total[h];
+            int e_new = e;
+            shift[h] = 0;
+            t_next[h] = tot;
+            if (cmr != kUnset) {
+                // range: the largest score must fit; room: one round of every warp takes at most half of 2^32
+                if (e == kUnset || cmr - e > kMaxWeightBits) e_new = cmr - kUnitBits;
+                const int room = need + C::kLog2Groups - 31;
+                if (need != kUnset && room > e_new) e_new = room;
+            }
+            if (e != kUnset) {
+                // the weights already in the bins keep a sixteenth of the range at most after an event
+                for (int tries = 0; tries < 24; ++tries) {              // 2 bits per try: bounded
+                    const int k = e_new - e;
+                    if ((k >= 32 ? 0u : tot >> k) < kBinLimit256 / 16u) break;
+                    e_new += 2;
+                }
+                shift[h] = e_new - e;
+                t_next[h] = (shift[h] >= 32 ? 0u : tot >> shift[h]) + 1u;
+                any_shift = any_shift || shift[h] > 0;
+            }
+            e_next[h] = e_new;
+        }
+        if (any_shift) {
+            for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
+                const int word = i % (32 * C::kPlanes);
+                const int hw = C::head_of_word(word);
+                int k = shift[0];
+#pragma unroll
+                for (int h = 1; h < R; ++h) k = hw == h ? shift[h] : k;
+                if (k > 0) {
+                    uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes + word * 4);
+                    const uint32_t v = *bp;
+                    *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
+                }
+            }
+        }
+        event_barrier(C::kThreads);                         // every thread has read the request and rescaled its bins
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int h = 0; h < R; ++h) {
+                ctl->e_cur[h] = e_next[h];
+                ctl->total[h] = t_next[h];
+                ctl->req_ref[h] = kUnset;
+                ctl->req_need[h] = kUnset;
+            }
+            ctl->want = 0;
+        }
+        event_barrier(C::kThreads);                         // the new state is visible
+    };
     constexpr bool kSplit = C::kHalfRows && R >= 2;      // the two half warps serve different query heads
     const unsigned grp_mask = kSplit ? (lane < 16 ? 0x0000ffffu : 0xffff0000u) : 0xffffffffu;
     const bool grp_leader = kSplit ? (lane & 15) == 0 : lane == 0;
@@ -432,9 +501,9 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         // of a quad hold the same 16 scores; lane p turns tokens p, p+4, p+8, p+12 into weights
         // 2^(score - ref) <= 1 (exponentials are the scarce resource here), and the integer weights
         // are handed round the quad by shuffles just before the bins are updated.
-        const int slot = it % 3;
         int ref[C::kLaneHeads];
         float wown[C::kLaneHeads][4], zsum[C::kLaneHeads];
+        bool any_tokens = false;
 #pragma unroll
         for (int u = 0; u < C::kLaneHeads; ++u) {
             float mx = -INFINITY;
@@ -442,9 +511,9 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             for (int k = 0; k < 16; ++k) mx = fmaxf(mx, sc[u][k]);
             const float gm = dec_float(__reduce_max_sync(grp_mask, enc_float(mx * lut_scale)));
             const bool any = gm > -INFINITY;
-            ref[u] = any ? (int)fminf(fmaxf(ceilf(gm), -1.0e9f), 1.0e9f) : 0;
-            if (grp_leader && any) atomicMax(&ctl->rmax[slot][C::lane_head(u, r)], ref[u]);
-            const float fref = (float)ref[u];
+            any_tokens = any_tokens || any;
+            ref[u] = any ? (int)fminf(fmaxf(ceilf(gm), -1.0e9f), 1.0e9f) : kUnset;
+            const float fref = any ? (float)ref[u] : 0.f;
             float z = 0.f;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -458,96 +527,73 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             for (int o = kSplit ? 8 : 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
             zsum[u] = z;
         }
-        if (it == 0) {
-            // first round: the unit is set from the round's maximum before the sums are formed
-            __syncthreads();
+        any_tokens = __any_sync(0xffffffffu, any_tokens);
+
+        // Reserve room for this warp's weights, or ask for a coarser unit.  Bounded: every event
+        // coarsens the refused head by at least two bits.
+        int eu[C::kLaneHeads];
+        for (int attempt = 0; attempt < 64; ++attempt) {
+            if (*reinterpret_cast<volatile int*>(&ctl->want) != 0) {
+                // someone needs a coarser unit: tell the event what this warp will need, then join it
+                if (grp_leader)
 #pragma unroll
-            for (int h = 0; h < R; ++h) e_unit[h] = ctl->rmax[slot][h] - kUnitBits;
-        }
+                    for (int u = 0; u < C::kLaneHeads; ++u)
+                        if (ref[u] != kUnset) {
+                            atomicMax(&ctl->req_ref[C::lane_head(u, r)], ref[u]);
+                            atomicMax(&ctl->req_need[C::lane_head(u, r)], ref[u] + ilogbf(fmaxf(zsum[u], 1e-30f)) + 1);
+                        }
+                event_barrier(C::kThreads);
+                coarsen();
+                continue;
+            }
+            if (!any_tokens) break;
+            bool ok = true;
+            unsigned int mine[C::kLaneHeads];
 #pragma unroll
-        for (int u = 0; u < C::kLaneHeads; ++u) {
-            const int eu = C::template pick<R>(e_unit, u, r);
-            // the round's weights of this (half) warp in the current unit, rounded up, in units of 256
-            // (a u32 shared-memory add is fast, the 64-bit form is not)
-            const float cw = (zsum[u] * pow2i(ref[u] - eu) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
-            const unsigned int ci = cw < 6.7e7f ? (unsigned int)cw : (1u << 26);     // saturates; 32 of these still fit
-            if (grp_leader) atomicAdd(&ctl->rsum[slot][C::lane_head(u, r)], ci);
-        }
-        __syncthreads();
-        int cm[R];
-        unsigned int rs[R];
-        bool all_keep = true;
+            for (int u = 0; u < C::kLaneHeads; ++u) {
+                const int h = C::lane_head(u, r);
+                eu[u] = *reinterpret_cast<volatile int*>(&ctl->e_cur[h]);
+                mine[u] = 0u;
+                if (ref[u] == kUnset) continue;
+                if (eu[u] == kUnset || ref[u] - eu[u] > kMaxWeightBits) { ok = false; continue; }
+                // this (half) warp's weights in the current unit, rounded up, in units of 256
+                const float cw = (zsum[u] * pow2i(ref[u] - eu[u]) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
+                const unsigned int ci = (unsigned int)fminf(cw, 6.7e7f);
+                unsigned int old = 0u;
+                if (grp_leader) old = atomicAdd(&ctl->total[h], ci);
+                old = __shfl_sync(0xffffffffu, old, kSplit ? (lane & 16) : 0);
+                mine[u] = ci;
+                if (old + ci >= kBinLimit256) ok = false;
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) break;
+            // give the reservations back, publish what is needed, raise the request, join the event
+            if (grp_leader) {
 #pragma unroll
-        for (int h = 0; h < R; ++h) {
-            cm[h] = ctl->rmax[slot][h];
-            rs[h] = ctl->rsum[slot][h];
-            const bool keep = cm[h] == kUnset || (cm[h] - e_unit[h] <= kMaxWeightBits && total[h] + rs[h] < kBinLimit256);
-            all_keep = all_keep && keep;
-        }
-        if (threadIdx.x < 4) {
-            ctl->rmax[(it + 2) % 3][threadIdx.x] = kUnset;
-            ctl->rsum[(it + 2) % 3][threadIdx.x] = 0u;
+                for (int u = 0; u < C::kLaneHeads; ++u) {
+                    const int h = C::lane_head(u, r);
+                    if (mine[u]) atomicSub(&ctl->total[h], mine[u]);
+                    if (ref[u] != kUnset) {
+                        atomicMax(&ctl->req_ref[h], ref[u]);
+                        atomicMax(&ctl->req_need[h], ref[u] + ilogbf(fmaxf(zsum[u], 1e-30f)) + 1);
+                    }
+                }
+                atomicExch(&ctl->want, 1);
+            }
+            event_barrier(C::kThreads);
+            coarsen();
         }
 
         // the next iteration's K words travel while the V side runs
         load_words(kw, kbase, blk + (int64_t)C::kWarps * C::kBlocksPerIter);
 
-        if (all_keep) {
-#pragma unroll
-            for (int h = 0; h < R; ++h) total[h] += rs[h];                 // rs is 0 for a head without tokens
-        } else {
-            // Some head needs a coarser unit: its top score left the range, or a bin could pass 2^32.
-            int shift[R];
-#pragma unroll
-            for (int h = 0; h < R; ++h) {
-                shift[h] = 0;
-                if (cm[h] == kUnset) continue;
-                const bool range_ok = cm[h] - e_unit[h] <= kMaxWeightBits;
-                if (range_ok && total[h] + rs[h] < kBinLimit256) {
-                    total[h] += rs[h];
-                    continue;
-                }
-                const bool measured = range_ok && rs[h] < (1u << 26);    // else: worst case of the round
-                int e_new = range_ok ? e_unit[h] + 2 : cm[h] - kUnitBits;
-                float est = 0.f;
-                bool fits = false;
-                for (int tries = 0; tries < 48 && !fits; ++tries) {      // 2 bits per try: 96 bits always suffice
-                    const float down = pow2i(e_unit[h] - e_new);          // 2^-shift, 0 when the shift is huge
-                    const float rnew = (measured ? (float)rs[h] * 256.f * down
-                                                 : (float)C::kRoundTokens * pow2i(cm[h] > e_new ? cm[h] - e_new : 0) * 1.0001f) +
-                                       (float)C::kRoundTokens;
-                    est = ((float)total[h] * 256.f * down + 1.f + rnew) * 1.000001f;
-                    fits = est < 256.f * (float)kBinLimit256;
-                    if (!fits) e_new += 2;
-                }
-                if (!fits) {                                              // not reachable with finite inputs
-                    e_new = (cm[h] + 1 > e_unit[h] + 40) ? cm[h] + 1 : e_unit[h] + 40;
-                    est = 2.f * (float)C::kRoundTokens + 2.f;
-                }
-                shift[h] = e_new - e_unit[h];
-                e_unit[h] = e_new;
-                total[h] = (unsigned int)(est * (1.f / 256.f)) + 1u;
-            }
-            for (int i = threadIdx.x; i < kRows * 32 * C::kPlanes; i += C::kThreads) {
-                const int word = i % (32 * C::kPlanes);
-                const int hw = C::head_of_word(word);
-                int k = shift[0];
-#pragma unroll
-                for (int h = 1; h < R; ++h) k = hw == h ? shift[h] : k;
-                if (k > 0) {
-                    uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset + (i / (32 * C::kPlanes)) * kRowBytes + word * 4);
-                    const uint32_t v = *bp;
-                    *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
-                }
-            }
-            __syncthreads();
-        }
+        if (!any_tokens) continue;
 
         // V side: integer weights (own tokens), handed round the quad, into the bins of this lane's groups
         uint32_t wint[C::kLaneHeads][4];
 #pragma unroll
         for (int u = 0; u < C::kLaneHeads; ++u) {
-            const float f = pow2i(ref[u] - C::template pick<R>(e_unit, u, r));     // power of two <= 2^kMaxWeightBits
+            const float f = ref[u] == kUnset ? 0.f : pow2i(ref[u] - eu[u]);      // power of two <= 2^kMaxWeightBits
 #pragma unroll
             for (int j = 0; j < 4; ++j) wint[u][j] = __float2uint_rn(wown[u][j] * f);
         }
@@ -564,6 +610,12 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + u * 128 + idx), wk[u]);
             }
         }
+    }
+    // Warps that are done keep joining coarsening events until every warp is done.
+    for (int guard = 0; guard < 4096; ++guard) {
+        event_barrier(C::kThreads);
+        if (*reinterpret_cast<volatile int*>(&ctl->want) == 0) break;
+        coarsen();
     }
     __syncthreads();
 
@@ -624,7 +676,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
                 if (lane == 0) {
-                    part_base[(int64_t)h * n_parts * stride + 0] = (float)e_unit[h];   // reference exponent (log2 domain)
+                    part_base[(int64_t)h * n_parts * stride + 0] = (float)ctl->e_cur[h];   // reference exponent (log2 domain)
                     part_base[(int64_t)h * n_parts * stride + 1] = l;            // normaliser, in the same unit
                 }
             }
