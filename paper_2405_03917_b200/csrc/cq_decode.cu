@@ -11,11 +11,12 @@
 //
 // Why integers: on sm_100a a shared-memory `red.add.u32` retires a warp's 32 bank-distinct
 // updates in about one cycle, while the f32 / f16x2 / u64 forms run several times slower.
-// Integer adds are also associative, so the result does not depend on the order in which
-// warps reach a bin.  The unit exponent e is kept at least 26 bits below the running maximum
-// score and is coarsened (bins shifted right, with rounding) whenever a score would need more
-// than 30 bits or a bin could overflow 32 bits; both events are rare and cost one pass over
-// the bins.
+// Integer adds are also associative, so a bin does not depend on the order in which warps
+// reach it.  Every query head has its own unit exponent e: it starts 27 bits below the first
+// scores' maximum, and it is coarsened (bins shifted right, with rounding) only when a score
+// would need more than 30 bits or the running total of the weights - a bound on every bin -
+// would pass 2^32.  Warps reserve their weights on that total with one atomic add and do not
+// wait for each other; a coarsening is a rare event that every warp joins (see `coarsen`).
 //
 // Shared-memory traffic, not HBM, is what limits this kernel once the code stream is
 // coalesced: each (token, group, query head) costs one 4-byte table lookup and one 4-byte
@@ -561,7 +562,8 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 const unsigned int ci = (unsigned int)fminf(cw, 6.7e7f);
                 unsigned int old = 0u;
                 if (grp_leader) old = atomicAdd(&ctl->total[h], ci);
-                old = __shfl_sync(0xffffffffu, old, kSplit ? (lane & 16) : 0);
+                // (group mask: with two heads per warp the other half warp may have left this iteration)
+                old = __shfl_sync(grp_mask, old, kSplit ? (lane & 16) : 0);
                 mine[u] = ci;
                 if (old + ci >= kBinLimit256) ok = false;
             }

@@ -204,26 +204,33 @@ def test_attention_peaked_and_flat_softmax():
         H.check_attn(out, ref, f"peaked/flat variant={variant}")
 
 
-def test_weight_unit_is_coarsened_on_flat_and_on_rising_scores():
-    # (a) zero query over a long context: every weight equals the maximum, so integer bins
-    #     must coarsen their unit instead of overflowing; (b) tokens sorted by rising score,
-    #     with a large scale: the running maximum grows in every round.
-    c, b, D, cap = 8, 8, 128, 20000
-    w = H.small_workload("t", 78, c, b, 2, 1, 1, cap)
-    xk = synth.layer_activations(w, 0, False, 2, cap)
-    xv = synth.layer_activations(w, 0, True, 2, cap)
+@pytest.mark.parametrize("c,n_q,n_kv", [(8, 1, 1), (8, 4, 1), (8, 2, 1), (4, 1, 1), (4, 2, 1)])
+def test_weight_unit_is_coarsened_on_flat_and_on_rising_scores(c, n_q, n_kv):
+    # Stress of the integer weight unit, for every tuned kernel shape.  Sequence 0: zero queries over
+    # a long context (every weight equals the maximum, so the bins must coarsen their unit instead of
+    # overflowing).  Sequence 1: tokens sorted by rising score of query head 0 with a large scale (the
+    # running maximum keeps growing, and the other heads of a GQA group see different maxima).
+    # Sequence 2: the same tokens in falling order (the first tokens dominate, the tail is tiny).
+    b, D, cap = 8, 128, 20000
+    w = H.small_workload("t", 78 + c + n_q, c, b, 3, n_q, n_kv, cap)
+    xk = synth.layer_activations(w, 0, False, 3, cap)
+    xv = synth.layer_activations(w, 0, True, 3, cap)
     kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
     kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, c, b)
     vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
-    q = synth.queries(78, 0, 2, 1)
+    q = synth.queries(w.config, 0, 3, n_q)
     q[0] = 0
+    q[2] = q[1]
     scale = 0.7
-    khat = oracle.dequant(kc_rm[1].reshape(cap, 1, -1), kcb.numpy(), c, b)[:, 0]        # (cap, D)
+    khat = oracle.dequant(kc_rm[1].reshape(cap, n_kv, -1), kcb.numpy(), c, b)[:, 0]     # (cap, D)
     order = np.argsort(khat @ q[1, 0].double().numpy(), kind="stable")
+    kc_rm[2], vc_rm[2] = kc_rm[1][order[::-1]], vc_rm[1][order[::-1]]
     kc_rm[1], vc_rm[1] = kc_rm[1][order], vc_rm[1][order]
     for variant in (1, 0):
-        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [cap, cap - 3], scale, c, b, variant)
-        H.check_attn(out, ref, f"flat/rising variant={variant}")
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [cap, cap - 3, cap - 17], scale, c, b, variant)
+        H.check_attn(out, ref, f"flat/rising/falling c={c} Hq={n_q} variant={variant}")
+        for s_ in range(3):                      # per sequence too: a large row must not hide a small one
+            H.check_attn(out[s_], ref[s_], f"flat/rising/falling seq {s_} c={c} Hq={n_q} variant={variant}")
 
 
 def test_attention_multi_chunk_gqa_and_mha_long():
