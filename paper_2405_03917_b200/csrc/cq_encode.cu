@@ -13,15 +13,17 @@
 //     A: x words | x words | x words | (1, 1)        | (X_hi, X_lo) | (1, 0)
 //     B: -2C_hi  | -2C_lo  | -2C_lo2 | (N_hi, N_lo)  | (1, 1)       | (N_lo2, 0)
 // (N = ||C_j||^2, X = ||x_g||^2; c = 8 needs two MMAs per tile, c = 4 drops N_lo2).
-// The accumulator lanes then run a streaming (best, second-best) selection over the 256
-// centroids with the centroid index packed into the low mantissa byte, four lanes of a quad
-// are merged with shuffles, and the winner is accepted only if the second-best score is
-// farther away than a bound on the evaluation error.  Otherwise (near-ties, exact ties,
-// out-of-range codebooks) the warp recomputes that (vector, group) exactly: direct form
-// sum (x - C)^2 in fp32, lowest index on ties -- the arithmetic of the generic kernel.
+// The accumulator lanes then keep, per vector, the smallest score of four subsets of their
+// columns, with the centroid index packed into the low mantissa byte (one 3-input min per two
+// scores).  The smallest of a quad's 16 subset minima names the winner's subset, whose 16
+// centroids are evaluated exactly (direct form sum (x - C)^2 in fp32); the second smallest subset
+// minimum bounds every other centroid from below, and the exact winner is accepted only if that
+// bound is farther away than a bound on the evaluation error.  Otherwise (near-ties, exact ties
+// across subsets, out-of-range codebooks) the warp recomputes that (vector, group) over all 256
+// centroids exactly, lowest index on ties -- the arithmetic of the generic kernel.
 //
-// The selection, not the tensor pipe, is what bounds this kernel: about 3.5 ALU-pipe
-// operations per (vector, centroid) pair.
+// The selection, not the tensor pipe, is what bounds this kernel: the ALU pipe (min / logic,
+// 64 lanes per clock and SM) is about 77 % busy, the tensor pipe about 14 %.
 #include "cq_common.cuh"
 
 namespace cq {
@@ -70,16 +72,6 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], u
     asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// Streaming selection of the smallest and second smallest of the values seen so far.
-// Values are floats whose low mantissa byte carries the centroid index.
-__device__ __forceinline__ void select2(float& best, float& second, float v0, float v1)
-{
-    const float lo = fminf(v0, v1), hi = fmaxf(v0, v1);
-    const float t = fmaxf(best, lo);
-    best = fminf(best, lo);
-    second = min3f(second, hi, t);
 }
 
 // Prepares the B operand of group g of head h: thread t handles centroid t.
@@ -270,6 +262,7 @@ encode_tuned_kernel(const __half* __restrict__ x, const float* __restrict__ cb, 
 
         // A operands of this warp's m-tiles
         uint32_t a[kMT][C::kSteps][4];
+        uint32_t xwreg[kMT][2];            // the x word this lane loaded, per row
         float Xrow[kMT][2];
 #pragma unroll
         for (int mt = 0; mt < kMT; ++mt) {
@@ -293,45 +286,66 @@ encode_tuned_kernel(const __half* __restrict__ x, const float* __restrict__ cb, 
                     }
                 }
                 Xrow[mt][hf] = X[hf];
+                xwreg[mt][hf] = xw[hf];
             }
             build_a<kC>(xw, X, p, a[mt]);
         }
 
-        float best[kMT][2], second[kMT][2];
+        // Selection.  Every lane keeps, per row, the smallest score of four subsets of its columns
+        // (n-tile index mod 4), index packed into the low mantissa byte: one 3-input min per two
+        // scores.  The smallest of the quad's 16 subset minima names the winner's subset; its 16
+        // centroids are then evaluated exactly, and the second smallest subset minimum bounds every
+        // other centroid from below.
+        float sb[kMT][2][4];
 #pragma unroll
         for (int mt = 0; mt < kMT; ++mt)
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) { best[mt][hf] = kInfBits; second[mt][hf] = kInfBits; }
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) sb[mt][hf][q] = kInfBits;
 
         const uint32_t keep = 0xffffff00u;
         const uint2* bsrc = reinterpret_cast<const uint2*>(bbuf[cur]) + lane;
-#pragma unroll 8
-        for (int nt = 0; nt < 32; ++nt) {
-            uint2 b[C::kSteps];
+#pragma unroll 2
+        for (int nt0 = 0; nt0 < 32; nt0 += 4) {
 #pragma unroll
-            for (int st = 0; st < C::kSteps; ++st) b[st] = bsrc[st * 1024 + nt * 32];
-            const uint32_t i0 = nt * 8, i1 = nt * 8 + 1;      // centroid index without the lane's 2p
+            for (int q = 0; q < 4; ++q) {
+                const int nt = nt0 + q;
+                uint2 b[C::kSteps];
 #pragma unroll
-            for (int mt = 0; mt < kMT; ++mt) {
-                float d[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int st = 0; st < C::kSteps; ++st) b[st] = bsrc[st * 1024 + nt * 32];
+                const uint32_t i0 = nt * 8, i1 = nt * 8 + 1;      // centroid index without the lane's 2p
 #pragma unroll
-                for (int st = 0; st < C::kSteps; ++st) mma_f16(d, a[mt][st], b[st].x, b[st].y);
-                const float v0p = __uint_as_float((__float_as_uint(d[0]) & keep) | i0);
-                const float v1p = __uint_as_float((__float_as_uint(d[1]) & keep) | i1);
-                const float v2p = __uint_as_float((__float_as_uint(d[2]) & keep) | i0);
-                const float v3p = __uint_as_float((__float_as_uint(d[3]) & keep) | i1);
-                select2(best[mt][0], second[mt][0], v0p, v1p);
-                select2(best[mt][1], second[mt][1], v2p, v3p);
+                for (int mt = 0; mt < kMT; ++mt) {
+                    float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int st = 0; st < C::kSteps; ++st) mma_f16(d, a[mt][st], b[st].x, b[st].y);
+                    const float v0p = __uint_as_float((__float_as_uint(d[0]) & keep) | i0);
+                    const float v1p = __uint_as_float((__float_as_uint(d[1]) & keep) | i1);
+                    const float v2p = __uint_as_float((__float_as_uint(d[2]) & keep) | i0);
+                    const float v3p = __uint_as_float((__float_as_uint(d[3]) & keep) | i1);
+                    sb[mt][0][q] = min3f(sb[mt][0][q], v0p, v1p);
+                    sb[mt][1][q] = min3f(sb[mt][1][q], v2p, v3p);
+                }
             }
         }
 
-        // merge the quad, certify, store
+        // merge the quad, evaluate the winner's subset exactly, certify, store
 #pragma unroll
         for (int mt = 0; mt < kMT; ++mt)
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-                float b = __uint_as_float(__float_as_uint(best[mt][hf]) | (2u * p));
-                float s2 = __uint_as_float(__float_as_uint(second[mt][hf]) | (2u * p));
+                float b, s2;
+                {
+                    const uint32_t pb = 2u * p;
+                    const float t0 = __uint_as_float(__float_as_uint(sb[mt][hf][0]) | pb);
+                    const float t1 = __uint_as_float(__float_as_uint(sb[mt][hf][1]) | pb);
+                    const float t2 = __uint_as_float(__float_as_uint(sb[mt][hf][2]) | pb);
+                    const float t3 = __uint_as_float(__float_as_uint(sb[mt][hf][3]) | pb);
+                    const float lo01 = fminf(t0, t1), hi01 = fmaxf(t0, t1), lo23 = fminf(t2, t3), hi23 = fmaxf(t2, t3);
+                    b = fminf(lo01, lo23);
+                    s2 = min3f(fmaxf(lo01, lo23), hi01, hi23);
+                }
 #pragma unroll
                 for (int o = 1; o <= 2; o <<= 1) {
                     const float ob = __shfl_xor_sync(0xffffffffu, b, o);
@@ -340,14 +354,51 @@ encode_tuned_kernel(const __half* __restrict__ x, const float* __restrict__ cb, 
                     b = fminf(b, ob);
                     s2 = min3f(s2, os, t);
                 }
+                // the winner's subset: lane pw of the quad, n-tiles qw, qw + 4, ..., qw + 28
+                const int jw = (int)(__float_as_uint(b) & 0xffu);
+                const int pw = (jw >> 1) & 3, qw = (jw >> 3) & 3;
+                float xg[kC];
+#pragma unroll
+                for (int w = 0; w < kC / 2; ++w) {
+                    const uint32_t ww = kC == 2 ? xwreg[mt][hf] : __shfl_sync(0xffffffffu, xwreg[mt][hf], (lane & ~3) | w);
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&ww));
+                    xg[2 * w] = f.x;
+                    xg[(2 * w + 1) % kC] = f.y;
+                }
+                float dbest = kInfBits;
+                int code = 0;
+#pragma unroll
+                for (int tt = 0; tt < 2; ++tt) {
+                    const int j0 = (qw + 4 * (2 * p + tt)) * 8 + 2 * pw;       // centroids j0, j0 + 1 (ascending over tt)
+                    float cc[2 * kC];
+#pragma unroll
+                    for (int w = 0; w < 2 * kC; w += 4) {
+                        const float4 t4 = *reinterpret_cast<const float4*>(cb_g + j0 * kC + w);
+                        cc[w] = t4.x; cc[w + 1] = t4.y; cc[w + 2] = t4.z; cc[w + 3] = t4.w;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float dd = 0.f;
+#pragma unroll
+                        for (int i = 0; i < kC; ++i) {
+                            const float diff = xg[i] - cc[e * kC + i];
+                            dd = fmaf(diff, diff, dd);
+                        }
+                        if (dd < dbest) { dbest = dd; code = j0 + e; }         // ascending j: strict < keeps the lowest
+                    }
+                }
+#pragma unroll
+                for (int o = 1; o <= 2; o <<= 1) {
+                    const float od = __shfl_xor_sync(0xffffffffu, dbest, o);
+                    const int oc = __shfl_xor_sync(0xffffffffu, code, o);
+                    if (od < dbest || (od == dbest && oc < code)) { dbest = od; code = oc; }
+                }
                 const int64_t v = v0 + mt * 16 + r + 8 * hf;
-                const float sb = __uint_as_float(__float_as_uint(b) & keep);
                 const float ss = __uint_as_float(__float_as_uint(s2) & keep);
                 // Evaluation error of a score: fp32 accumulation of up to ~20 terms bounded by
-                // 2 (X + N) in magnitude, plus the mantissa byte given to the index.
-                const float tau = 3.1e-5f * (Xrow[mt][hf] + nmax) + 1.3e-4f * fmaxf(fabsf(ss), fabsf(sb));
-                const bool certain = !out_of_range && (ss - sb > tau);
-                int code = (int)(__float_as_uint(b) & 0xffu);
+                // 2 (X + N) in magnitude, plus the mantissa byte given to the index.  dbest is exact.
+                const float tau = 1.6e-5f * (Xrow[mt][hf] + nmax) + 6.2e-5f * fabsf(ss);
+                const bool certain = !out_of_range && (ss - dbest > tau);
                 // exact recomputation of the uncertain rows, one row at a time by the whole warp
                 unsigned pending = __ballot_sync(0xffffffffu, !certain && p == 0 && v < n_vec);
                 while (pending) {
@@ -357,7 +408,7 @@ encode_tuned_kernel(const __half* __restrict__ x, const float* __restrict__ cb, 
                     float xg[kC];
 #pragma unroll
                     for (int w = 0; w < kC / 2; ++w) {
-                        const uint32_t ww = __shfl_sync(0xffffffffu, a[mt][0][hf], src + (kC == 2 ? 0 : w));
+                        const uint32_t ww = __shfl_sync(0xffffffffu, xwreg[mt][hf], src + (kC == 2 ? 0 : w));
                         const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&ww));
                         xg[2 * w] = f.x;
                         xg[(2 * w + 1) % kC] = f.y;
