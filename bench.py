@@ -318,6 +318,14 @@ def extra_encode_cfg3(cq, dev, reps=5):
     res = {"workload": w.name, "ms": ms, "tokens_per_s": tokens / (ms * 1e-3), "vectors_per_s": vectors / (ms * 1e-3),
            "useful_tflops": vectors * 2 * D * (1 << w.b) / (ms * 1e-3) / 1e12,
            "gbs": (vectors * (D * 2 + w.G) + 2 * w.n_kv_heads * D * (1 << w.b) * 4) / (ms * 1e-3) / 1e9}
+    # The selection over the 2^b scores of every (vector, group) bounds this kernel: at least 1.5
+    # ALU-pipe operations per score (two index packs and one 3-input min per two scores) on a pipe of
+    # 64 lanes per clock and SM (148 SMs, nominal 1965 MHz).
+    pairs = vectors * w.G * (1 << w.b)
+    alu_peak = 148 * 64 * 1965e6
+    res["roofline"] = {"bound": "alu", "achieved": 1.5 * pairs / (ms * 1e-3), "peak": alu_peak, "unit": "lane-ops/s",
+                       "frac": 1.5 * pairs / (ms * 1e-3) / alu_peak, "traffic": None,
+                       "peak_source": "64 ALU lanes/clk/SM x 148 SMs x 1965 MHz"}
     return res
 
 
