@@ -702,7 +702,7 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
 }
 
 // Context chunk per CTA.  The table build and the bins x centroids product are paid once per
-// chunk, so chunks are long (up to 16384 tokens); they are halved only while the grid would not
+// chunk, so chunks are long (up to 65536 tokens); they are halved only while the grid would not
 // give the CTA slots of the 148 SMs one and a half CTAs each, and never below 2048 tokens.
 template <int G, int R>
 int chunk_for(const Shape& sh)
@@ -715,7 +715,7 @@ int chunk_for(const Shape& sh)
     const int64_t items = sh.n_seq * sh.n_kv_heads;
     const int64_t slots = 148 * C::kMinBlocks;
     int64_t chunk = (sh.max_tokens + round - 1) / round * round;
-    if (chunk > 16384) chunk = 16384;
+    if (chunk > 65536) chunk = 65536;
     while (chunk > 2048 && 2 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
         chunk = (chunk / 2 + round - 1) / round * round;
     return (int)chunk;
