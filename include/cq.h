@@ -14,7 +14,8 @@
  * General rules
  *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The
  *     caller owns all buffers, including the workspace; the library allocates
- *     nothing and keeps no state between calls.
+ *     nothing and keeps no state between calls (cq_decode_attn_static, below, is
+ *     the one exception: it remembers the address of its built-in array).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *     enqueue work and return; they never synchronise, except cq_decode_step_host.
  *   - Every function that returns int returns a cq_status: arguments are checked
@@ -22,8 +23,9 @@
  *     and a CUDA launch error is reported as CQ_ERR_CUDA.  Nothing aborts or traps.
  *   - Supported shapes: c divides head_dim, head_dim <= 256, 1 <= b <= 8 (codes
  *     are one uint8 each), n_q_heads a multiple of n_kv_heads.  Tuned kernels
- *     exist for head_dim 128 with CQ-2c8b, CQ-4c8b and CQ-8c8b; every other
- *     supported shape runs on generic sm_100a kernels (never on the CPU).
+ *     exist for head_dim 128 and b = 8: encode for c = 2, 4, 8; decode attention
+ *     for c = 8 with 1, 2 or 4 query heads per KV head and c = 4 with 1 or 2.
+ *     Every other supported shape runs on generic sm_100a kernels (never on the CPU).
  *   - Inputs must be finite.
  *
  * Code layout (version cq_layout_version() == 1).  Codes of one (sequence, head)

@@ -249,6 +249,34 @@ def test_attention_multi_chunk_gqa_and_mha_long():
         H.check_attn(out, ref, f"long c={c} Hq={n_q} Hkv={n_kv}")
 
 
+def test_encode_codebooks_beyond_fp16_range_take_the_exact_path():
+    # centroids too large for the fp16 term splits of the tensor-core path: the tuned kernel must
+    # notice and recompute those groups exactly
+    for c in (2, 4, 8):
+        b, D, nh, n = 8, 128, 2, 48
+        xk, _, kcb, _, _ = H.generic_case(500 + c, 1, n, nh, nh, D, c, b)
+        kcb = kcb.clone()
+        kcb[0, 1] *= 3.0e4                      # one group of head 0 far outside the range
+        kcb[1, 0, 5] = 7.0e4                    # one centroid of another group
+        _, rm = encode_both(xk, kcb, c, b, n, 0)
+        H.check_codes(xk.numpy().reshape(-1, nh, D), kcb.numpy(), rm.reshape(-1, nh, D // c), c, b)
+
+
+def test_attention_table_entries_beyond_fp16_range_are_prescaled():
+    # |scale * <q_g, C>| far above 2^15: the table is rebuilt with a power-of-two prescale
+    c, b, D, cap = 8, 8, 128, 300
+    w = H.small_workload("t", 91, c, b, 2, 2, 1, cap)
+    xk = synth.layer_activations(w, 0, False, 2, cap)
+    xv = synth.layer_activations(w, 0, True, 2, cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False) * 300.0, synth.layer_codebooks(w, 0, True)
+    kc_rm, _ = H.oracle_encode_rowmajor((xk.float() * 300.0).clamp(-6e4, 6e4).to(torch.float16), kcb, c, b)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, c, b)
+    q = (synth.queries(91, 0, 2, 2).float() * 4).to(torch.float16)
+    for variant in (1, 0):
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [cap, 77], 1.0, c, b, variant)
+        H.check_attn(out, ref, f"prescaled table variant={variant}")
+
+
 def test_token_permutation_and_seq_len_padding_invariance():
     c, b, D, cap, n = 8, 8, 128, 640, 600
     w = H.small_workload("t", 55, c, b, 1, 4, 1, cap)
