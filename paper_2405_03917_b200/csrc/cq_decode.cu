@@ -150,13 +150,21 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
-// D += A * ones: sums, per fragment row, the 16 halves the quad holds for that row.
-__device__ __forceinline__ void mma_rowsum(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
+// D = A * ones (+ C): sums, per fragment row, the 16 halves the quad holds for that row.
+// Rows r (registers a0, a2) and r + 8 (a1, a3) carry two different tokens.
+__device__ __forceinline__ void mma_rowsum_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
 {
     const uint32_t ones = 0x3c003c00u;   // half2(1, 1)
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(ones), "r"(ones), "f"(0.f));
+}
+__device__ __forceinline__ void mma_rowsum_acc(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
+{
+    const uint32_t ones = 0x3c003c00u;
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(ones), "r"(ones));
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(ones), "r"(ones));
 }
 
 template <int kC>
@@ -456,9 +464,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         const int64_t blk = blk_warp + qb;
         load_words(vw, vbase, blk);
 
-        // K side: scores of this quad's 16 tokens for the query heads this lane serves.  One MMA
-        // per (token, head) and per 4 code words: fragment rows r and r + 8 carry two halves of
-        // the same token's lookups, so the token's score is the sum of both row sums.
+        // K side: scores of this quad's 16 tokens for the query heads this lane serves.
         float sc[C::kLaneHeads][16];
 #pragma unroll
         for (int k0 = 0; k0 < 16; k0 += kBatch) {
@@ -474,18 +480,18 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     for (int u = 0; u < C::kLaneHeads; ++u)
                         a[kk][u][m] = *reinterpret_cast<const volatile uint32_t*>(smem + u * 128 + idx);
                 }
+            // two tokens per MMA chain: fragment rows r and r + 8; two code words per MMA
 #pragma unroll
-            for (int kk = 0; kk < kBatch; ++kk)
+            for (int kk = 0; kk < kBatch; kk += 2)
 #pragma unroll
                 for (int u = 0; u < C::kLaneHeads; ++u) {
-                    float tot = 0.f;
+                    float d[4];
+                    mma_rowsum_first(d, a[kk][u][0], a[kk + 1][u][0], a[kk][u][1], a[kk + 1][u][1]);
 #pragma unroll
-                    for (int m = 0; m < C::kSlots; m += 4) {
-                        float d[4] = {0.f, 0.f, 0.f, 0.f};
-                        mma_rowsum(d, a[kk][u][m], a[kk][u][m + 1], a[kk][u][m + 2], a[kk][u][m + 3]);
-                        tot += d[0] + d[2];
-                    }
-                    sc[u][k0 + kk] = tot;
+                    for (int m = 2; m < C::kSlots; m += 2)
+                        mma_rowsum_acc(d, a[kk][u][m], a[kk + 1][u][m], a[kk][u][m + 1], a[kk + 1][u][m + 1]);
+                    sc[u][k0 + kk] = d[0];
+                    sc[u][k0 + kk + 1] = d[2];
                 }
         }
 
