@@ -1,7 +1,8 @@
 /*
  * CPU oracle for Coupled Quantization (CQ) of LLM KV caches -- TEST INFRASTRUCTURE.
  *
- * Plain, slow, fp64.  It exists to check the CUDA library and to be timed as a
+ * Plain, slow, fp64 (encode, decode attention, and the centroid-learning steps of
+ * Section 3.2.1).  It exists to check the CUDA library and to be timed as a
  * CPU baseline; it shares no code with the CUDA path and the product never
  * calls it.  Every function states the passage of the paper it follows.
  *
@@ -289,6 +290,128 @@ void oracle_decode_lut(const uint16_t *q, const int32_t *k_codes, const int32_t 
             free(bins);
             free(acc);
             free(tot);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Centroid learning (Section 3.2.1).  For every (head, group) one independent k-means
+ * problem over the n_vec group vectors: Eq. 5 (uniform) or Eq. 6 (every group vector carries
+ * a non-negative weight, the paper's g^T g of that group).  The paper runs k-means++
+ * initialisation followed by a fixed number of k-means iterations (Section 4.3).
+ *   x         fp16 bits [n_vec][n_heads][D]
+ *   weights   fp32 [n_vec][n_heads][G], or NULL for all-ones (Eq. 5)
+ *   codebooks fp32 [n_heads][G][K][c]
+ * ------------------------------------------------------------------------------------------ */
+
+/*
+ * k-means++ (Arthur and Vassilvitskii 2007) with the random draws passed in:
+ * uniforms [n_heads][G][K], each in [0, 1).  Centre 0 of a problem is vector
+ * floor(u_0 * n_vec).  Centre k >= 1 is vector i*, the first index whose running sum
+ * sum_{i <= i*} w_i D_i reaches u_k * sum_i w_i D_i, where D_i is the squared distance of
+ * vector i to its nearest already chosen centre; sums run in index order, in fp64; if the
+ * total is 0 (fewer distinct vectors than centres) the draw falls back to floor(u_k * n_vec).
+ * chosen (may be NULL) receives the picked vector indices [n_heads][G][K].
+ */
+void oracle_kmeanspp_init(const uint16_t *x, const float *weights, const double *uniforms,
+                          int64_t n_vec, int n_heads, int D, int c, int b,
+                          float *codebooks, int64_t *chosen)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int h = 0; h < n_heads; ++h) {
+        for (int g = 0; g < G; ++g) {
+            double *dist = (double *)malloc(sizeof(double) * (size_t)n_vec);
+            float *cb = codebooks + ((int64_t)h * G + g) * K * c;
+            const double *u = uniforms + ((int64_t)h * G + g) * K;
+            for (int k = 0; k < K; ++k) {
+                int64_t pick;
+                if (k == 0) {
+                    pick = (int64_t)(u[0] * (double)n_vec);
+                } else {
+                    double total = 0.0;
+                    for (int64_t i = 0; i < n_vec; ++i) {
+                        double w = weights ? (double)weights[(i * n_heads + h) * G + g] : 1.0;
+                        total += w * dist[i];
+                    }
+                    if (total > 0.0) {
+                        const double target = u[k] * total;
+                        double run = 0.0;
+                        pick = n_vec - 1;
+                        for (int64_t i = 0; i < n_vec; ++i) {
+                            double w = weights ? (double)weights[(i * n_heads + h) * G + g] : 1.0;
+                            run += w * dist[i];
+                            if (run >= target && w * dist[i] > 0.0) { pick = i; break; }
+                        }
+                    } else {
+                        pick = (int64_t)(u[k] * (double)n_vec);
+                    }
+                }
+                if (pick >= n_vec) pick = n_vec - 1;
+                if (chosen) chosen[((int64_t)h * G + g) * K + k] = pick;
+                for (int i = 0; i < c; ++i)
+                    cb[k * c + i] = (float)half_to_double(x[(pick * n_heads + h) * (int64_t)D + g * c + i]);
+                for (int64_t i = 0; i < n_vec; ++i) {
+                    double d = 0.0;
+                    for (int j = 0; j < c; ++j) {
+                        double diff = half_to_double(x[(i * n_heads + h) * (int64_t)D + g * c + j]) - (double)cb[k * c + j];
+                        d += diff * diff;
+                    }
+                    if (k == 0 || d < dist[i]) dist[i] = d;
+                }
+            }
+            free(dist);
+        }
+    }
+}
+
+/*
+ * One k-means (Lloyd) iteration: assign every group vector to its nearest centroid (the map
+ * CQ(.), lowest index on ties), then move every centroid to the weighted mean of its members;
+ * a centroid without members (or with zero total weight) stays where it is.
+ * codes_out (may be NULL) [n_vec][n_heads][G]; objective_out (may be NULL) [n_heads][G] receives
+ * sum_i w_i ||x_i - CQ(x_i)||^2 of the assignment, i.e. the objective of Eq. 5 / Eq. 6 for the
+ * INPUT codebooks.
+ */
+void oracle_lloyd_step(const uint16_t *x, const float *weights, const float *codebooks_in,
+                       int64_t n_vec, int n_heads, int D, int c, int b,
+                       float *codebooks_out, int32_t *codes_out, double *objective_out)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int h = 0; h < n_heads; ++h) {
+        for (int g = 0; g < G; ++g) {
+            const float *cb = codebooks_in + ((int64_t)h * G + g) * K * c;
+            float *out = codebooks_out + ((int64_t)h * G + g) * K * c;
+            double *sum = (double *)calloc((size_t)K * c, sizeof(double));
+            double *wsum = (double *)calloc((size_t)K, sizeof(double));
+            double obj = 0.0;
+            for (int64_t i = 0; i < n_vec; ++i) {
+                const uint16_t *xv = x + (i * n_heads + h) * (int64_t)D + g * c;
+                double best = INFINITY;
+                int arg = 0;
+                for (int j = 0; j < K; ++j) {
+                    double d = 0.0;
+                    for (int q = 0; q < c; ++q) {
+                        double diff = half_to_double(xv[q]) - (double)cb[j * c + q];
+                        d += diff * diff;
+                    }
+                    if (d < best) { best = d; arg = j; }
+                }
+                double w = weights ? (double)weights[(i * n_heads + h) * G + g] : 1.0;
+                obj += w * best;
+                wsum[arg] += w;
+                for (int q = 0; q < c; ++q) sum[arg * c + q] += w * half_to_double(xv[q]);
+                if (codes_out) codes_out[(i * n_heads + h) * G + g] = arg;
+            }
+            for (int j = 0; j < K; ++j)
+                for (int q = 0; q < c; ++q)
+                    out[j * c + q] = wsum[j] > 0.0 ? (float)(sum[j * c + q] / wsum[j]) : cb[j * c + q];
+            if (objective_out) objective_out[h * G + g] = obj;
+            free(sum);
+            free(wsum);
         }
     }
 }

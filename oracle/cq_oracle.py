@@ -42,6 +42,10 @@ def _load():
         L.oracle_dequant.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp]
         L.oracle_decode_dense.argtypes = [vp, vp, vp, vp, vp, vp, f64, i32, i32, i32, i32, i32, i32, i64, vp]
         L.oracle_decode_lut.argtypes = [vp, vp, vp, vp, vp, vp, f64, i32, i32, i32, i32, i32, i32, i64, i32, vp]
+        L.oracle_kmeanspp_init.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp]
+        L.oracle_lloyd_step.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp]
+        L.oracle_kmeanspp_init.restype = None
+        L.oracle_lloyd_step.restype = None
         for f in (L.oracle_set_num_threads, L.oracle_encode, L.oracle_code_distance, L.oracle_dequant,
                   L.oracle_decode_dense, L.oracle_decode_lut):
             f.restype = None
@@ -153,3 +157,44 @@ def decode_lut(q, k_codes, v_codes, k_cb, v_cb, seq_lens, scale: float, c: int, 
     _load().oracle_decode_lut(_p(qb), _p(kc), _p(vc), _p(kcb), _p(vcb), _p(sl), float(scale),
                               n_seq, hq, hkv, D, c, b, mt, int(n_chunks), _p(out))
     return out
+
+
+def _weights(weights, n_vec, n_heads, G):
+    if weights is None:
+        return None
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    if w.shape != (n_vec, n_heads, G):
+        raise ValueError(f"weights shape {w.shape}, expected {(n_vec, n_heads, G)}")
+    assert (w >= 0).all()
+    return w
+
+
+def kmeanspp_init(x, weights, uniforms, c: int, b: int):
+    """k-means++ with the draws passed in.  x fp16 (n_vec, n_heads, D); weights fp32
+    (n_vec, n_heads, G) or None; uniforms fp64 (n_heads, G, 2^b) in [0, 1).
+    Returns (codebooks fp32 (n_heads, G, 2^b, c), chosen int64 (n_heads, G, 2^b))."""
+    xb = _half_bits(x)
+    n_vec, n_heads, D = xb.shape
+    G, K = D // c, 1 << b
+    w = _weights(weights, n_vec, n_heads, G)
+    u = np.ascontiguousarray(uniforms, dtype=np.float64)
+    assert u.shape == (n_heads, G, K) and (u >= 0).all() and (u < 1).all()
+    cb = np.empty((n_heads, G, K, c), dtype=np.float32)
+    chosen = np.empty((n_heads, G, K), dtype=np.int64)
+    _load().oracle_kmeanspp_init(_p(xb), _p(w), _p(u), n_vec, n_heads, D, c, b, _p(cb), _p(chosen))
+    return cb, chosen
+
+
+def lloyd_step(x, weights, codebooks, c: int, b: int):
+    """One k-means iteration.  Returns (new codebooks fp32, codes int32 (n_vec, n_heads, G),
+    objective fp64 (n_heads, G) of the assignment under the input codebooks)."""
+    xb = _half_bits(x)
+    n_vec, n_heads, D = xb.shape
+    G = D // c
+    w = _weights(weights, n_vec, n_heads, G)
+    cb = _cb(codebooks, n_heads, D, c, b)
+    out = np.empty_like(cb)
+    codes = np.empty((n_vec, n_heads, G), dtype=np.int32)
+    obj = np.empty((n_heads, G), dtype=np.float64)
+    _load().oracle_lloyd_step(_p(xb), _p(w), _p(cb), n_vec, n_heads, D, c, b, _p(out), _p(codes), _p(obj))
+    return out, codes, obj

@@ -276,3 +276,125 @@ def test_scale_is_applied_to_scores_only():
     b2 = oracle.decode_dense(q, kc, vc, (0.25 * kcb.astype(np.float64)).astype(np.float32), vcb, sl, 1.0, c, b)
     np.testing.assert_allclose(a, b2, rtol=1e-6)      # 0.25 is a power of two: kcb scaling is exact
     assert np.abs(a - oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 1.0, c, b)).max() > 1e-3
+
+
+# ----------------------------------------------------------------------------- centroid learning
+
+def _golden_kmeans():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "kmeans_hand_worked.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, *cols = [f.strip() for f in line.split("|")]
+        rows.append((head.split(), [np.array(col.split(), dtype=np.float64) for col in cols]))
+    return rows
+
+
+def _as_problem(points):
+    """1-D points as a (n, 1 head, D = 1) fp16 array: one head, one group of one channel."""
+    return np.asarray(points, dtype=np.float16).reshape(-1, 1, 1)
+
+
+def test_lloyd_step_hand_worked_cases():
+    n_cases = 0
+    for (kind, name), cols in _golden_kmeans():
+        if kind != "lloyd":
+            continue
+        pts, w, cin, cout, obj = cols
+        K = len(cin)
+        b = int(np.log2(K)) if K & (K - 1) == 0 else None
+        if b is None:                 # pad a 3-centroid case to 4 with a far copy that stays empty
+            cin = np.append(cin, 1e4)
+            cout = np.append(cout, 1e4)
+            b = 2
+        new, codes, o = oracle.lloyd_step(_as_problem(pts), w.reshape(-1, 1, 1).astype(np.float32),
+                                          cin.reshape(1, 1, -1, 1).astype(np.float32), 1, b)
+        np.testing.assert_allclose(new.reshape(-1), cout, rtol=0, atol=1e-6, err_msg=name)
+        assert abs(o[0, 0] - obj[0]) < 1e-9, name
+        n_cases += 1
+    assert n_cases == 4
+
+
+def test_kmeanspp_hand_worked_cases():
+    n_cases = 0
+    for (kind, name), cols in _golden_kmeans():
+        if kind != "kmeanspp":
+            continue
+        pts, w, u, chosen = cols
+        K = 4                          # 3 draws checked; a fourth centre pads to a power of two
+        uu = np.append(u, 0.5).reshape(1, 1, K)
+        cb, ch = oracle.kmeanspp_init(_as_problem(pts), w.reshape(-1, 1, 1).astype(np.float32), uu, 1, 2)
+        assert ch[0, 0, :3].tolist() == chosen.astype(int).tolist(), name
+        np.testing.assert_array_equal(cb[0, 0, :3, 0], pts[chosen.astype(int)])
+        n_cases += 1
+    assert n_cases == 3
+
+
+def test_lloyd_step_matches_sklearn_one_iteration():
+    from sklearn.cluster import KMeans
+    r = np.random.default_rng(7)
+    for c, b, weighted in ((2, 3, False), (4, 4, True), (8, 3, True)):
+        n, K = 600, 1 << b
+        x = r.standard_normal((n, 1, c)).astype(np.float16)
+        w = (r.random((n, 1, 1)) + 0.1).astype(np.float32) if weighted else None
+        init = x[r.choice(n, K, replace=False), 0].astype(np.float32)            # members guaranteed: no empty cluster
+        new, codes, obj = oracle.lloyd_step(x, w, init.reshape(1, 1, K, c), c, b)
+        km = KMeans(n_clusters=K, init=init.astype(np.float64), n_init=1, max_iter=1, tol=0.0, algorithm="lloyd")
+        km.fit(x[:, 0].astype(np.float64), sample_weight=None if w is None else w[:, 0, 0].astype(np.float64))
+        np.testing.assert_allclose(new[0, 0], km.cluster_centers_, rtol=1e-6, atol=1e-6)
+
+
+def test_lloyd_objective_never_increases_and_means_are_optimal():
+    r = np.random.default_rng(8)
+    c, b, n = 4, 4, 800
+    x = r.standard_normal((n, 2, 8)).astype(np.float16)
+    w = r.random((n, 2, 2)).astype(np.float32)
+    cb, _ = oracle.kmeanspp_init(x, w, r.random((2, 2, 16)), c, b)
+    last = None
+    for _ in range(6):
+        new, codes, obj = oracle.lloyd_step(x, w, cb, c, b)
+        if last is not None:
+            assert (obj <= last * (1 + 1e-12)).all()
+        last = obj
+        # for the fixed assignment, moving any centroid away from the weighted mean raises the objective
+        xf = x.astype(np.float64)
+        for h, g in ((0, 0), (1, 1)):
+            grp = xf[:, h, g * c:(g + 1) * c]
+            cost = lambda cc: float((w[:, h, g] * ((grp - cc[codes[:, h, g]]) ** 2).sum(1)).sum())
+            base = cost(new[h, g].astype(np.float64))
+            for _t in range(5):
+                pert = new[h, g].astype(np.float64).copy()
+                pert[r.integers(16), r.integers(c)] += r.choice([-1, 1]) * 0.05
+                assert cost(pert) >= base - 1e-9
+        cb = new
+
+
+def test_kmeanspp_picks_every_point_once_when_points_equal_centres():
+    r = np.random.default_rng(9)
+    c, b = 2, 4
+    x = (np.arange(16)[:, None, None] * 3.0 + r.random((16, 1, c))).astype(np.float16)     # 16 distinct, separated points
+    for _ in range(5):
+        _, ch = oracle.kmeanspp_init(x, None, r.random((1, 1, 16)), c, b)
+        assert sorted(ch[0, 0].tolist()) == list(range(16))
+
+
+def test_centroid_learning_batches_are_independent_problems():
+    # the batched call over heads and groups equals separate calls on each (head, group) slice
+    r = np.random.default_rng(10)
+    c, b, n, H_, G = 2, 2, 50, 3, 2
+    x = r.standard_normal((n, H_, G * c)).astype(np.float16)
+    w = r.random((n, H_, G)).astype(np.float32)
+    u = r.random((H_, G, 4))
+    cb, ch = oracle.kmeanspp_init(x, w, u, c, b)
+    new, codes, obj = oracle.lloyd_step(x, w, cb, c, b)
+    for h in range(H_):
+        for g in range(G):
+            xs = np.ascontiguousarray(x[:, h:h + 1, g * c:(g + 1) * c])
+            ws = np.ascontiguousarray(w[:, h:h + 1, g:g + 1])
+            cb1, ch1 = oracle.kmeanspp_init(xs, ws, u[h:h + 1, g:g + 1], c, b)
+            assert ch1[0, 0].tolist() == ch[h, g].tolist()
+            n1, c1, o1 = oracle.lloyd_step(xs, ws, cb1, c, b)
+            np.testing.assert_array_equal(n1[0, 0], new[h, g])
+            np.testing.assert_array_equal(c1[:, 0, 0], codes[:, h, g])
+            assert o1[0, 0] == obj[h, g]
