@@ -191,6 +191,40 @@ int cq_encode_variant(const void *x_fp16, const float *codebooks, const int32_t 
                       void *stream);
 
 /*
+ * Centroid learning (Section 3.2.1): for every (head, group) an independent k-means problem
+ * over the n_vec group vectors of a calibration tensor -- Eq. 5, or Eq. 6 when `weights` gives
+ * every group vector its importance (the paper's g^T g of that group) -- with k-means++
+ * initialisation and a fixed number of k-means iterations (Section 4.3).
+ *
+ *   x_fp16     [n_vec][n_heads][head_dim] fp16, 16-byte aligned
+ *   weights    NULL (Eq. 5), or [n_vec][n_heads][G] fp32, non-negative (Eq. 6)
+ *   uniforms   [n_heads][G][2^b] fp64 in [0, 1): the random draws of k-means++, supplied by the
+ *              caller (the library draws nothing).  Centre 0 of a problem is vector
+ *              floor(u_0 n_vec); centre k is the first vector whose running sum of w_i D_i, in
+ *              index order and in fp64, reaches u_k times the total (D_i: squared distance to
+ *              the nearest centre chosen so far)
+ *   codebooks  [n_heads][G][2^b][c] fp32, 16-byte aligned
+ *   objective_out  NULL, or [n_heads][G] fp64: sum_i w_i ||x_i - CQ(x_i)||^2 of the last
+ *              assignment (measured against the codebooks that assignment used)
+ *   workspace  at least cq_learn_workspace_bytes(...) bytes, 16-byte aligned
+ *
+ * cq_kmeanspp_init writes the initial centroids; cq_lloyd_step performs one iteration
+ * (assignment = cq_encode, then every centroid moves to the weighted mean of its members; a
+ * centroid without members stays; codebooks_in and codebooks_out must differ);
+ * cq_learn_centroids runs the initialisation and n_iters iterations.
+ */
+size_t cq_learn_workspace_bytes(int64_t n_vec, int n_heads, int head_dim, int c, int b);
+int cq_kmeanspp_init(const void *x_fp16, const float *weights, const double *uniforms, int64_t n_vec,
+                     int n_heads, int head_dim, int c, int b, float *codebooks_out, void *workspace,
+                     size_t workspace_bytes, void *stream);
+int cq_lloyd_step(const void *x_fp16, const float *weights, const float *codebooks_in, int64_t n_vec,
+                  int n_heads, int head_dim, int c, int b, float *codebooks_out, double *objective_out,
+                  void *workspace, size_t workspace_bytes, void *stream);
+int cq_learn_centroids(const void *x_fp16, const float *weights, const double *uniforms, int64_t n_vec,
+                       int n_heads, int head_dim, int c, int b, int n_iters, float *codebooks_out,
+                       double *objective_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * One decode step of one layer driven from HOST buffers (the end-to-end path):
  * copies the step's query and the new token's key and value vectors to the
  * device, appends the new token's codes at position seq_lens_host[s] of every

@@ -19,7 +19,7 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
            "cq_decode_attn_variant", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
-           "cq_decode_step_host"]
+           "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
 
 
 class CQError(RuntimeError):
@@ -65,6 +65,14 @@ def lib() -> ctypes.CDLL:
                                              sz, i32, vp]
         L.cq_decode_attn_static.restype = i32
         L.cq_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp]
+        L.cq_learn_workspace_bytes.restype = sz
+        L.cq_learn_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
+        L.cq_kmeanspp_init.restype = i32
+        L.cq_kmeanspp_init.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, sz, vp]
+        L.cq_lloyd_step.restype = i32
+        L.cq_lloyd_step.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.cq_learn_centroids.restype = i32
+        L.cq_learn_centroids.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.cq_decode_step_host_workspace_bytes.restype = sz
         L.cq_decode_step_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
         L.cq_decode_step_host.restype = i32
@@ -231,3 +239,57 @@ def cq_decode_step_host(q_host: torch.Tensor, k_new_host: torch.Tensor, v_new_ho
                                    _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream())
     _check(st, "cq_decode_step_host")
     return out_host
+
+
+# ------------------------------------------------------------------------------ centroid learning
+
+def cq_learn_workspace_bytes(n_vec: int, n_heads: int, head_dim: int, c: int, b: int) -> int:
+    return int(lib().cq_learn_workspace_bytes(n_vec, n_heads, head_dim, c, b))
+
+
+def _learn_common(x, weights, c, b):
+    n_vec, n_heads, head_dim = x.shape
+    G = head_dim // max(c, 1)
+    if weights is not None and tuple(weights.shape) != (n_vec, n_heads, G):
+        raise ValueError(f"weights shape {tuple(weights.shape)}, expected {(n_vec, n_heads, G)}")
+    wp = None if weights is None else _dev(weights, torch.float32, "weights")
+    ws = torch.empty(max(256, cq_learn_workspace_bytes(n_vec, n_heads, head_dim, c, b)), dtype=torch.uint8, device=x.device)
+    return n_vec, n_heads, head_dim, G, wp, ws
+
+
+def cq_kmeanspp_init(x: torch.Tensor, weights: Optional[torch.Tensor], uniforms: torch.Tensor, c: int, b: int) -> torch.Tensor:
+    """x fp16 (n_vec, n_heads, head_dim); weights fp32 (n_vec, n_heads, G) or None; uniforms fp64
+    (n_heads, G, 2^b).  Returns the initial codebooks fp32 (n_heads, G, 2^b, c)."""
+    n_vec, n_heads, head_dim, G, wp, ws = _learn_common(x, weights, c, b)
+    if tuple(uniforms.shape) != (n_heads, G, 1 << b):
+        raise ValueError("uniforms must be (n_heads, G, 2^b)")
+    out = torch.empty(n_heads, G, 1 << b, c, dtype=torch.float32, device=x.device)
+    st = lib().cq_kmeanspp_init(_dev(x, torch.float16, "x"), wp, _dev(uniforms, torch.float64, "uniforms"), n_vec, n_heads,
+                                head_dim, c, b, out.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "cq_kmeanspp_init")
+    return out
+
+
+def cq_lloyd_step(x: torch.Tensor, weights: Optional[torch.Tensor], codebooks: torch.Tensor, c: int, b: int):
+    """One k-means iteration.  Returns (new codebooks, objective fp64 (n_heads, G) of the assignment)."""
+    n_vec, n_heads, head_dim, G, wp, ws = _learn_common(x, weights, c, b)
+    out = torch.empty_like(codebooks)
+    obj = torch.empty(n_heads, G, dtype=torch.float64, device=x.device)
+    st = lib().cq_lloyd_step(_dev(x, torch.float16, "x"), wp, _dev(codebooks, torch.float32, "codebooks"), n_vec, n_heads,
+                             head_dim, c, b, out.data_ptr(), obj.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "cq_lloyd_step")
+    return out, obj
+
+
+def cq_learn_centroids(x: torch.Tensor, weights: Optional[torch.Tensor], uniforms: torch.Tensor, c: int, b: int,
+                       n_iters: int):
+    """k-means++ initialisation and n_iters k-means iterations.  Returns (codebooks, objective of the
+    last assignment)."""
+    n_vec, n_heads, head_dim, G, wp, ws = _learn_common(x, weights, c, b)
+    out = torch.empty(n_heads, G, 1 << b, c, dtype=torch.float32, device=x.device)
+    obj = torch.zeros(n_heads, G, dtype=torch.float64, device=x.device)
+    st = lib().cq_learn_centroids(_dev(x, torch.float16, "x"), wp, _dev(uniforms, torch.float64, "uniforms"), n_vec,
+                                  n_heads, head_dim, c, b, n_iters, out.data_ptr(), obj.data_ptr(), ws.data_ptr(),
+                                  ws.numel(), _stream())
+    _check(st, "cq_learn_centroids")
+    return out, obj

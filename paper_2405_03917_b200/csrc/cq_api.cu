@@ -232,6 +232,72 @@ int cq_decode_attn_static(const void* q_fp16, const void* k_codes, const void* v
                           head_dim, c, b, max_tokens, out, ws, (size_t)CQ_STATIC_WORKSPACE_BYTES, stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Centroid learning (Section 3.2.1): k-means++ initialisation and k-means iterations.
+// ---------------------------------------------------------------------------------------------
+namespace {
+int learn_shape(int64_t n_vec, int n_heads, int head_dim, int c, int b, Shape* sh)
+{
+    if (n_vec <= 0) return CQ_ERR_SHAPE;
+    return make_shape(1, n_vec, n_heads, n_heads, head_dim, c, b, sh);
+}
+}  // namespace
+
+size_t cq_learn_workspace_bytes(int64_t n_vec, int n_heads, int head_dim, int c, int b)
+{
+    Shape sh;
+    if (learn_shape(n_vec, n_heads, head_dim, c, b, &sh) != CQ_OK) return 0;
+    return learn_workspace_bytes(sh, n_vec);
+}
+
+int cq_kmeanspp_init(const void* x_fp16, const float* weights, const double* uniforms, int64_t n_vec, int n_heads,
+                     int head_dim, int c, int b, float* codebooks_out, void* workspace, size_t workspace_bytes,
+                     void* stream)
+{
+    if (!x_fp16 || !uniforms || !codebooks_out || !workspace) return CQ_ERR_NULL;
+    Shape sh;
+    int st = learn_shape(n_vec, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (!aligned16(x_fp16) || !aligned16(codebooks_out) || !aligned16(workspace)) return CQ_ERR_ALIGN;
+    if (workspace_bytes < learn_workspace_bytes(sh, n_vec)) return CQ_ERR_WORKSPACE;
+    cudaError_t e = launch_kmeanspp_init(static_cast<const __half*>(x_fp16), weights, uniforms, sh, n_vec, codebooks_out,
+                                         workspace, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_lloyd_step(const void* x_fp16, const float* weights, const float* codebooks_in, int64_t n_vec, int n_heads,
+                  int head_dim, int c, int b, float* codebooks_out, double* objective_out, void* workspace,
+                  size_t workspace_bytes, void* stream)
+{
+    if (!x_fp16 || !codebooks_in || !codebooks_out || !workspace) return CQ_ERR_NULL;
+    if (codebooks_in == codebooks_out) return CQ_ERR_SHAPE;
+    Shape sh;
+    int st = learn_shape(n_vec, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (!aligned16(x_fp16) || !aligned16(codebooks_in) || !aligned16(codebooks_out) || !aligned16(workspace))
+        return CQ_ERR_ALIGN;
+    if (workspace_bytes < learn_workspace_bytes(sh, n_vec)) return CQ_ERR_WORKSPACE;
+    cudaError_t e = launch_lloyd_step(static_cast<const __half*>(x_fp16), weights, codebooks_in, sh, n_vec, codebooks_out,
+                                      objective_out, workspace, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_learn_centroids(const void* x_fp16, const float* weights, const double* uniforms, int64_t n_vec, int n_heads,
+                       int head_dim, int c, int b, int n_iters, float* codebooks_out, double* objective_out,
+                       void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!x_fp16 || !uniforms || !codebooks_out || !workspace) return CQ_ERR_NULL;
+    if (n_iters < 0) return CQ_ERR_SHAPE;
+    Shape sh;
+    int st = learn_shape(n_vec, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (!aligned16(x_fp16) || !aligned16(codebooks_out) || !aligned16(workspace)) return CQ_ERR_ALIGN;
+    if (workspace_bytes < learn_workspace_bytes(sh, n_vec)) return CQ_ERR_WORKSPACE;
+    cudaError_t e = launch_learn(static_cast<const __half*>(x_fp16), weights, uniforms, sh, n_vec, n_iters, codebooks_out,
+                                 objective_out, workspace, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
 // Staging area of cq_decode_step_host inside the caller's workspace (all 256-byte aligned):
 //   [q fp16][k_new fp16][v_new fp16][seq_lens int32][seq_lens+1 int32][out fp32][attention workspace]
 size_t cq_decode_step_host_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,

@@ -60,6 +60,15 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
 // dst[i] = src[i] + 1 for i < n (context length after one appended token).
 cudaError_t launch_add_one(const int32_t* src, int32_t* dst, int n, cudaStream_t st);
 
+// Centroid learning (cq_learn.cu): the vectors are [n_vec][n_heads][head_dim], weights [n_vec][n_heads][G] or null.
+size_t learn_workspace_bytes(const Shape& sh, int64_t n_vec);
+cudaError_t launch_kmeanspp_init(const __half* x, const float* weights, const double* uniforms, const Shape& sh,
+                                 int64_t n_vec, float* codebooks, void* workspace, cudaStream_t st);
+cudaError_t launch_lloyd_step(const __half* x, const float* weights, const float* cb_in, const Shape& sh, int64_t n_vec,
+                              float* cb_out, double* objective, void* workspace, cudaStream_t st);
+cudaError_t launch_learn(const __half* x, const float* weights, const double* uniforms, const Shape& sh, int64_t n_vec,
+                         int n_iters, float* codebooks, double* objective, void* workspace, cudaStream_t st);
+
 // Merge of split-K partials into out (shared by both decode variants).
 cudaError_t launch_merge(const float* partials, int n_parts, const Shape& sh, float* out, cudaStream_t st);
 

@@ -1,0 +1,199 @@
+// Centroid learning (Section 3.2.1 of the paper): k-means++ initialisation and k-means
+// iterations, uniform (Eq. 5) or weighted per group vector (Eq. 6), for every (head, group)
+// problem of a key or value tensor at once.  The assignment step of an iteration is cq_encode.
+//
+// k-means++ decides integers (which vector becomes the next centre) from sums of squared
+// distances.  Those sums are formed in fp64, in index order, with the same operation order as
+// the definition (one multiply and one add per term, no fused multiply-add), so that the
+// decision does not depend on the machine: one thread per problem runs the two sequential
+// passes of a draw, while the distance update between draws runs over all (vector, problem)
+// pairs in parallel.  The mean update of an iteration accumulates in fp32 in shared memory.
+#include "cq_common.cuh"
+
+namespace cq {
+
+namespace {
+
+// problem p = h * G + g; vector i.  dist and weights are stored [i][p] (p fastest).
+__global__ void pp_pick_kernel(const __half* __restrict__ x, const float* __restrict__ weights,
+                               const double* __restrict__ uniforms, const double* __restrict__ dist, int64_t n_vec,
+                               int n_prob, int D, int c, int K, int k, float* __restrict__ codebooks)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n_prob) return;
+    const double u = uniforms[(int64_t)p * K + k];
+    int64_t pick;
+    if (k == 0) {
+        pick = (int64_t)__dmul_rn(u, (double)n_vec);
+    } else {
+        double total = 0.0;
+        for (int64_t i = 0; i < n_vec; ++i) {
+            const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
+            total = __dadd_rn(total, __dmul_rn(w, dist[i * n_prob + p]));
+        }
+        if (total > 0.0) {
+            const double target = __dmul_rn(u, total);
+            double run = 0.0;
+            pick = n_vec - 1;
+            for (int64_t i = 0; i < n_vec; ++i) {
+                const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
+                const double contrib = __dmul_rn(w, dist[i * n_prob + p]);
+                run = __dadd_rn(run, contrib);
+                if (run >= target && contrib > 0.0) { pick = i; break; }
+            }
+        } else {
+            pick = (int64_t)__dmul_rn(u, (double)n_vec);
+        }
+    }
+    if (pick >= n_vec) pick = n_vec - 1;
+    // x row of vector `pick`: all problems of a vector are contiguous (p * c = h * D + g * c)
+    const __half* xv = x + pick * (int64_t)n_prob * c + (int64_t)p * c;
+    float* cb = codebooks + ((int64_t)p * K + k) * c;
+    for (int q = 0; q < c; ++q) cb[q] = __half2float(xv[q]);
+}
+
+__global__ void pp_dist_kernel(const __half* __restrict__ x, const float* __restrict__ codebooks, int64_t n_vec,
+                               int n_prob, int c, int K, int k, double* __restrict__ dist)
+{
+    const int64_t total = n_vec * n_prob;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int p = (int)(idx % n_prob);
+        const __half* xv = x + idx * c;                       // (i * n_prob + p) * c
+        const float* cb = codebooks + ((int64_t)p * K + k) * c;
+        double d = 0.0;
+        for (int q = 0; q < c; ++q) {
+            const double diff = __dsub_rn((double)__half2float(xv[q]), (double)cb[q]);
+            d = __dadd_rn(d, __dmul_rn(diff, diff));
+        }
+        if (k == 0 || d < dist[idx]) dist[idx] = d;
+    }
+}
+
+// One CTA per problem: weighted sums of the members of every centroid in shared memory, then the
+// new centroids; the objective of the assignment (against the input codebooks) in fp64.
+constexpr int kUpdThreads = 256;
+__global__ void __launch_bounds__(kUpdThreads)
+lloyd_update_kernel(const __half* __restrict__ x, const float* __restrict__ weights, const uint8_t* __restrict__ codes,
+                    const float* __restrict__ cb_in, Shape sh, int64_t n_vec, float* __restrict__ cb_out,
+                    double* __restrict__ objective)
+{
+    extern __shared__ float upd_smem[];            // [K][c] sums, [K] weight sums, [K][c] input centroids
+    const int p = blockIdx.x, h = p / sh.G, g = p % sh.G, c = sh.c, K = sh.K;
+    const int n_prob = sh.n_kv_heads * sh.G;
+    float* sums = upd_smem;
+    float* wsum = sums + K * c;
+    float* cin = wsum + K;
+    for (int e = threadIdx.x; e < K * c; e += kUpdThreads) { sums[e] = 0.f; cin[e] = cb_in[(int64_t)p * K * c + e]; }
+    for (int e = threadIdx.x; e < K; e += kUpdThreads) wsum[e] = 0.f;
+    __syncthreads();
+    double obj = 0.0;
+    for (int64_t i = threadIdx.x; i < n_vec; i += kUpdThreads) {
+        const int code = codes[code_word_offset(sh, sh.n_kv_heads, 0, h, i / kTokenBlock, g) + i % kTokenBlock];
+        const float w = weights ? weights[i * n_prob + p] : 1.f;
+        const __half* xv = x + (i * n_prob + p) * (int64_t)c;
+        double d = 0.0;
+        for (int q = 0; q < c; ++q) {
+            const float xf = __half2float(xv[q]);
+            const double diff = (double)xf - (double)cin[code * c + q];
+            d += diff * diff;
+            atomicAdd(&sums[code * c + q], w * xf);
+        }
+        atomicAdd(&wsum[code], w);
+        obj += (double)w * d;
+    }
+    // objective: block reduction in fp64
+    __shared__ double red[kUpdThreads / 32];
+    for (int o = 16; o > 0; o >>= 1) obj += __shfl_xor_sync(0xffffffffu, obj, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = obj;
+    __syncthreads();
+    if (threadIdx.x == 0 && objective) {
+        double t = 0.0;
+        for (int wv = 0; wv < kUpdThreads / 32; ++wv) t += red[wv];
+        objective[p] = t;
+    }
+    for (int e = threadIdx.x; e < K * c; e += kUpdThreads) {
+        const float ws = wsum[e / c];
+        cb_out[(int64_t)p * K * c + e] = ws > 0.f ? sums[e] / ws : cin[e];
+    }
+}
+
+size_t round256(size_t v) { return (v + 255) / 256 * 256; }
+
+struct LearnLayout {
+    size_t codes, dist, tmp_cb, total;
+};
+
+LearnLayout learn_layout(const Shape& sh, int64_t n_vec)
+{
+    LearnLayout l;
+    const size_t n_prob = (size_t)sh.n_kv_heads * sh.G;
+    l.codes = round256((size_t)sh.n_kv_heads * ((n_vec + kTokenBlock - 1) / kTokenBlock) * sh.G * kTokenBlock);
+    l.dist = round256((size_t)n_vec * n_prob * sizeof(double));
+    l.tmp_cb = round256(n_prob * sh.K * sh.c * sizeof(float));
+    l.total = l.codes + l.dist + l.tmp_cb;
+    return l;
+}
+
+}  // namespace
+
+size_t learn_workspace_bytes(const Shape& sh, int64_t n_vec) { return learn_layout(sh, n_vec).total; }
+
+cudaError_t launch_kmeanspp_init(const __half* x, const float* weights, const double* uniforms, const Shape& sh,
+                                 int64_t n_vec, float* codebooks, void* workspace, cudaStream_t st)
+{
+    const LearnLayout l = learn_layout(sh, n_vec);
+    double* dist = reinterpret_cast<double*>(static_cast<char*>(workspace) + l.codes);
+    const int n_prob = sh.n_kv_heads * sh.G;
+    const int64_t pairs = n_vec * n_prob;
+    const int dist_grid = (int)((pairs + 255) / 256 < 148 * 16 ? (pairs + 255) / 256 : 148 * 16);
+    for (int k = 0; k < sh.K; ++k) {
+        pp_pick_kernel<<<(n_prob + 63) / 64, 64, 0, st>>>(x, weights, uniforms, dist, n_vec, n_prob, sh.head_dim, sh.c, sh.K,
+                                                          k, codebooks);
+        pp_dist_kernel<<<dist_grid, 256, 0, st>>>(x, codebooks, n_vec, n_prob, sh.c, sh.K, k, dist);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lloyd_step(const __half* x, const float* weights, const float* cb_in, const Shape& sh, int64_t n_vec,
+                              float* cb_out, double* objective, void* workspace, cudaStream_t st)
+{
+    const LearnLayout l = learn_layout(sh, n_vec);
+    uint8_t* codes = static_cast<uint8_t*>(workspace);
+    // assignment: the vectors are one sequence of n_vec tokens
+    Shape es = sh;
+    es.n_seq = 1;
+    es.max_tokens = n_vec;
+    es.n_blocks = (n_vec + kTokenBlock - 1) / kTokenBlock;
+    cudaError_t e = encode_tuned_supported(es) ? launch_encode_tuned(x, cb_in, nullptr, es, n_vec, 0, codes, st)
+                                               : launch_encode_generic(x, cb_in, nullptr, es, n_vec, 0, codes, st);
+    if (e != cudaSuccess) return e;
+    const size_t smem = (size_t)(2 * sh.K * sh.c + sh.K) * sizeof(float);
+    e = cudaFuncSetAttribute(lloyd_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    lloyd_update_kernel<<<sh.n_kv_heads * sh.G, kUpdThreads, smem, st>>>(x, weights, codes, cb_in, es, n_vec, cb_out,
+                                                                         objective);
+    (void)l;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_learn(const __half* x, const float* weights, const double* uniforms, const Shape& sh, int64_t n_vec,
+                         int n_iters, float* codebooks, double* objective, void* workspace, cudaStream_t st)
+{
+    const LearnLayout l = learn_layout(sh, n_vec);
+    float* tmp = reinterpret_cast<float*>(static_cast<char*>(workspace) + l.codes + l.dist);
+    cudaError_t e = launch_kmeanspp_init(x, weights, uniforms, sh, n_vec, codebooks, workspace, st);
+    if (e != cudaSuccess) return e;
+    float* cur = codebooks;
+    float* nxt = tmp;
+    for (int it = 0; it < n_iters; ++it) {
+        e = launch_lloyd_step(x, weights, cur, sh, n_vec, nxt, objective, workspace, st);
+        if (e != cudaSuccess) return e;
+        float* t = cur; cur = nxt; nxt = t;
+    }
+    if (cur != codebooks)
+        e = cudaMemcpyAsync(codebooks, cur, (size_t)sh.n_kv_heads * sh.G * sh.K * sh.c * sizeof(float),
+                            cudaMemcpyDeviceToDevice, st);
+    return e;
+}
+
+}  // namespace cq
