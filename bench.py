@@ -329,6 +329,33 @@ def extra_encode_cfg3(cq, dev, reps=5):
     return res
 
 
+def extra_learn(cq, dev, iters=100):
+    """Centroid learning (Section 3.2.1) on one layer's key tensor of a LLaMA-2-7B-shaped model with the
+    paper's calibration size (16 sequences x 2048 tokens): CQ-8c8b, k-means++ and `iters` k-means iterations
+    for all 32 heads x 16 groups.  The paper's Table 4 quotes 14 minutes for all 64 (layer, K|V) tensors of
+    this model on one A100-40GB: context, another machine."""
+    n_vec, n_heads, c, b = 16 * 2048, 32, 8, 8
+    w = synth.Workload("learn_llama2_7b_8c8b", 7, c, b, 1, 1, n_heads, n_heads, n_vec)
+    x = synth.layer_activations(w, 0, False, 1, n_vec, device=dev)[0].contiguous()
+    g = torch.Generator(device="cpu").manual_seed(77)
+    u = torch.rand(n_heads, 128 // c, 1 << b, dtype=torch.float64, generator=g).to(dev)
+    cq.cq_learn_centroids(x, None, u, c, b, 2)                      # warm-up
+    torch.cuda.synchronize()
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    e0.record()
+    cb0 = cq.cq_kmeanspp_init(x, None, u, c, b)
+    e1.record()
+    cb, obj = cq.cq_learn_centroids(x, None, u, c, b, iters)
+    e2.record()
+    torch.cuda.synchronize()
+    init_ms, total_ms = e0.elapsed_time(e1), e1.elapsed_time(e2)
+    _, obj0 = cq.cq_lloyd_step(x, None, cb0, c, b)
+    return {"workload": w.name, "n_vec": n_vec, "problems": n_heads * (128 // c), "iters": iters,
+            "init_ms": init_ms, "init_plus_iters_ms": total_ms, "ms_per_iter": (total_ms - init_ms) / iters,
+            "objective_init": float(obj0.sum().item()), "objective_final": float(obj.sum().item()),
+            "paper_context": "Table 4: 14 min for 64 such tensors (LLaMA-2-7b, CQ-8c8b) on one A100-40GB"}
+
+
 def extra_decode(cq, dev, w, reps=20):
     st = DecodeState(w, 0, dev, cq)
     for _ in range(3):
@@ -483,6 +510,7 @@ def main():
             if args.extras == "all":
                 extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
                 extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
+                extras["learn"] = extra_learn(cq, dev)
         except Exception as e:      # extras never hide the headline number
             extras["error"] = repr(e)
         line["extras"] = extras

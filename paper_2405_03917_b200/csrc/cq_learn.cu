@@ -5,67 +5,95 @@
 // k-means++ decides integers (which vector becomes the next centre) from sums of squared
 // distances.  Those sums are formed in fp64, in index order, with the same operation order as
 // the definition (one multiply and one add per term, no fused multiply-add), so that the
-// decision does not depend on the machine: one thread per problem runs the two sequential
-// passes of a draw, while the distance update between draws runs over all (vector, problem)
-// pairs in parallel.  The mean update of an iteration accumulates in fp32 in shared memory.
+// decision does not depend on the machine: one CTA per problem stages the terms in shared
+// memory and one of its threads adds them up in order (two passes per draw), while the distance
+// update between draws runs over all (vector, problem) pairs in parallel.  The mean update of an iteration accumulates in fp32 in shared memory.
 #include "cq_common.cuh"
 
 namespace cq {
 
 namespace {
 
-// problem p = h * G + g; vector i.  dist and weights are stored [i][p] (p fastest).
-__global__ void pp_pick_kernel(const __half* __restrict__ x, const float* __restrict__ weights,
-                               const double* __restrict__ uniforms, const double* __restrict__ dist, int64_t n_vec,
-                               int n_prob, int D, int c, int K, int k, float* __restrict__ codebooks)
+// problem p = h * G + g; vector i.  dist[p][i]: squared distance of vector i to its nearest centre
+// so far; contrib[p][i] = w_i * dist[p][i], the term of the k-means++ draw.
+
+// One CTA per problem.  The CTA stages tiles of contributions in shared memory (coalesced loads);
+// thread 0 adds them up in index order, so the fp64 running sum is the sequential one.
+constexpr int kPickThreads = 128;
+constexpr int kPickTile = 2048;
+__global__ void __launch_bounds__(kPickThreads)
+pp_pick_kernel(const __half* __restrict__ x, const double* __restrict__ uniforms, const double* __restrict__ contrib,
+               int64_t n_vec, int n_prob, int c, int K, int k, float* __restrict__ codebooks)
 {
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= n_prob) return;
+    __shared__ double tile[kPickTile];
+    __shared__ double s_total;
+    __shared__ long long s_pick;
+    const int p = blockIdx.x;
     const double u = uniforms[(int64_t)p * K + k];
-    int64_t pick;
-    if (k == 0) {
-        pick = (int64_t)__dmul_rn(u, (double)n_vec);
-    } else {
+    const double* cp = contrib + (int64_t)p * n_vec;
+    if (threadIdx.x == 0) s_pick = -1;
+    if (k > 0) {
         double total = 0.0;
-        for (int64_t i = 0; i < n_vec; ++i) {
-            const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
-            total = __dadd_rn(total, __dmul_rn(w, dist[i * n_prob + p]));
+        for (int64_t t0 = 0; t0 < n_vec; t0 += kPickTile) {
+            const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
+            __syncthreads();
+            for (int e = threadIdx.x; e < m; e += kPickThreads) tile[e] = cp[t0 + e];
+            __syncthreads();
+            if (threadIdx.x == 0)
+                for (int e = 0; e < m; ++e) total = __dadd_rn(total, tile[e]);
         }
-        if (total > 0.0) {
-            const double target = __dmul_rn(u, total);
+        if (threadIdx.x == 0) s_total = total;
+        __syncthreads();
+        if (s_total > 0.0) {
+            const double target = __dmul_rn(u, s_total);
             double run = 0.0;
-            pick = n_vec - 1;
-            for (int64_t i = 0; i < n_vec; ++i) {
-                const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
-                const double contrib = __dmul_rn(w, dist[i * n_prob + p]);
-                run = __dadd_rn(run, contrib);
-                if (run >= target && contrib > 0.0) { pick = i; break; }
+            for (int64_t t0 = 0; t0 < n_vec; t0 += kPickTile) {
+                const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
+                __syncthreads();
+                if (s_pick >= 0) break;                     // same value in every thread: read after the barrier
+                for (int e = threadIdx.x; e < m; e += kPickThreads) tile[e] = cp[t0 + e];
+                __syncthreads();
+                if (threadIdx.x == 0)
+                    for (int e = 0; e < m; ++e) {
+                        run = __dadd_rn(run, tile[e]);
+                        if (run >= target && tile[e] > 0.0) { s_pick = t0 + e; break; }
+                    }
             }
-        } else {
-            pick = (int64_t)__dmul_rn(u, (double)n_vec);
+            __syncthreads();
+            if (threadIdx.x == 0 && s_pick < 0) s_pick = n_vec - 1;
         }
     }
-    if (pick >= n_vec) pick = n_vec - 1;
-    // x row of vector `pick`: all problems of a vector are contiguous (p * c = h * D + g * c)
-    const __half* xv = x + pick * (int64_t)n_prob * c + (int64_t)p * c;
-    float* cb = codebooks + ((int64_t)p * K + k) * c;
-    for (int q = 0; q < c; ++q) cb[q] = __half2float(xv[q]);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long pick = s_pick;
+        if (pick < 0) pick = (long long)__dmul_rn(u, (double)n_vec);       // first centre, or no vector left to draw
+        if (pick >= n_vec) pick = n_vec - 1;
+        // x row of vector `pick`: all problems of a vector are contiguous (p * c = h * D + g * c)
+        const __half* xv = x + pick * (int64_t)n_prob * c + (int64_t)p * c;
+        float* cb = codebooks + ((int64_t)p * K + k) * c;
+        for (int q = 0; q < c; ++q) cb[q] = __half2float(xv[q]);
+    }
 }
 
-__global__ void pp_dist_kernel(const __half* __restrict__ x, const float* __restrict__ codebooks, int64_t n_vec,
-                               int n_prob, int c, int K, int k, double* __restrict__ dist)
+__global__ void pp_dist_kernel(const __half* __restrict__ x, const float* __restrict__ weights,
+                               const float* __restrict__ codebooks, int64_t n_vec, int n_prob, int c, int K, int k,
+                               double* __restrict__ dist, double* __restrict__ contrib)
 {
     const int64_t total = n_vec * n_prob;
     for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-        const int p = (int)(idx % n_prob);
-        const __half* xv = x + idx * c;                       // (i * n_prob + p) * c
+        const int p = (int)(idx / n_vec);
+        const int64_t i = idx % n_vec;
+        const __half* xv = x + (i * n_prob + p) * c;
         const float* cb = codebooks + ((int64_t)p * K + k) * c;
         double d = 0.0;
         for (int q = 0; q < c; ++q) {
             const double diff = __dsub_rn((double)__half2float(xv[q]), (double)cb[q]);
             d = __dadd_rn(d, __dmul_rn(diff, diff));
         }
-        if (k == 0 || d < dist[idx]) dist[idx] = d;
+        if (k > 0 && !(d < dist[idx])) d = dist[idx];
+        dist[idx] = d;
+        const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
+        contrib[idx] = __dmul_rn(w, d);
     }
 }
 
@@ -130,7 +158,7 @@ LearnLayout learn_layout(const Shape& sh, int64_t n_vec)
     l.codes = round256((size_t)sh.n_kv_heads * ((n_vec + kTokenBlock - 1) / kTokenBlock) * sh.G * kTokenBlock);
     l.dist = round256((size_t)n_vec * n_prob * sizeof(double));
     l.tmp_cb = round256(n_prob * sh.K * sh.c * sizeof(float));
-    l.total = l.codes + l.dist + l.tmp_cb;
+    l.total = l.codes + 2 * l.dist + l.tmp_cb;      // dist and contrib
     return l;
 }
 
@@ -146,10 +174,10 @@ cudaError_t launch_kmeanspp_init(const __half* x, const float* weights, const do
     const int n_prob = sh.n_kv_heads * sh.G;
     const int64_t pairs = n_vec * n_prob;
     const int dist_grid = (int)((pairs + 255) / 256 < 148 * 16 ? (pairs + 255) / 256 : 148 * 16);
+    double* contrib = reinterpret_cast<double*>(static_cast<char*>(workspace) + l.codes + l.dist);
     for (int k = 0; k < sh.K; ++k) {
-        pp_pick_kernel<<<(n_prob + 63) / 64, 64, 0, st>>>(x, weights, uniforms, dist, n_vec, n_prob, sh.head_dim, sh.c, sh.K,
-                                                          k, codebooks);
-        pp_dist_kernel<<<dist_grid, 256, 0, st>>>(x, codebooks, n_vec, n_prob, sh.c, sh.K, k, dist);
+        pp_pick_kernel<<<n_prob, kPickThreads, 0, st>>>(x, uniforms, contrib, n_vec, n_prob, sh.c, sh.K, k, codebooks);
+        pp_dist_kernel<<<dist_grid, 256, 0, st>>>(x, weights, codebooks, n_vec, n_prob, sh.c, sh.K, k, dist, contrib);
     }
     return cudaGetLastError();
 }
@@ -180,7 +208,7 @@ cudaError_t launch_learn(const __half* x, const float* weights, const double* un
                          int n_iters, float* codebooks, double* objective, void* workspace, cudaStream_t st)
 {
     const LearnLayout l = learn_layout(sh, n_vec);
-    float* tmp = reinterpret_cast<float*>(static_cast<char*>(workspace) + l.codes + l.dist);
+    float* tmp = reinterpret_cast<float*>(static_cast<char*>(workspace) + l.codes + 2 * l.dist);
     cudaError_t e = launch_kmeanspp_init(x, weights, uniforms, sh, n_vec, codebooks, workspace, st);
     if (e != cudaSuccess) return e;
     float* cur = codebooks;
