@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
                     const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                    float* __restrict__ partials)
+                    int tail_first, float* __restrict__ partials)
 {
     using C = Cfg<G, R>;
     constexpr int kC = C::kC;
@@ -261,19 +261,35 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int r = lane >> 2, p = lane & 3;
 
-    // work item: (context part, sequence, KV head); parts are the slowest index so that the
-    // always-populated first parts start first
-    const int hkv = blockIdx.x % sh.n_kv_heads;
-    const int64_t s = (blockIdx.x / sh.n_kv_heads) % sh.n_seq;
-    const int part = (int)(blockIdx.x / (sh.n_kv_heads * sh.n_seq));
+    // Work item: (context part, sequence, KV head); parts are the slowest index so that the
+    // always-populated first parts start first.  With a tail (tail_first >= 0) the items before
+    // tail_first take their whole context in one CTA, and each later item is spread over n_parts
+    // CTAs of chunk_tokens each: those shorter CTAs start last and fill the last, partly empty
+    // wave of the grid.
+    const int n_items = (int)(sh.n_kv_heads * sh.n_seq);
+    int item = blockIdx.x % n_items;
+    int part = (int)(blockIdx.x / n_items);
+    bool whole = false;
+    if (tail_first >= 0) {
+        whole = (int)blockIdx.x < tail_first;
+        item = whole ? blockIdx.x : tail_first + (blockIdx.x - tail_first) / n_parts;
+        part = whole ? 0 : (blockIdx.x - tail_first) % n_parts;
+    }
+    const int hkv = item % sh.n_kv_heads;
+    const int64_t s = item / sh.n_kv_heads;
 
     int64_t n = seq_lens[s];
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
     const int64_t t_begin = (int64_t)part * chunk_tokens;
-    const int64_t t_end = (t_begin + chunk_tokens < n) ? t_begin + chunk_tokens : n;
+    const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
     const int stride = partial_stride(128);
     float* part_base = partials + ((s * sh.n_q_heads + (int64_t)hkv * R) * n_parts + part) * stride;
     // partial of query head hkv*R + h: part_base + h * n_parts * stride
+    if (whole)          // the other partial slots of this item hold the neutral element of the merge
+        for (int i = threadIdx.x; i < R * (n_parts - 1) * stride; i += C::kThreads) {
+            const int h = i / ((n_parts - 1) * stride), d = i % ((n_parts - 1) * stride);
+            part_base[(int64_t)h * n_parts * stride + stride + d] = d % stride == 0 ? -INFINITY : 0.f;
+        }
     if (t_begin >= t_end) {
         for (int i = threadIdx.x; i < R * stride; i += C::kThreads) {
             const int h = i / stride, d = i % stride;
@@ -692,49 +708,79 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     }
 }
 
-template <int G, int R>
-cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
-                       const int32_t* seq_lens, float scale, const Shape& sh, int chunk_tokens, int n_parts,
-                       float* partials, cudaStream_t st)
-{
-    using C = Cfg<G, R>;
-    cudaError_t e = cudaFuncSetAttribute(decode_tuned_kernel<G, R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)(sh.n_seq * sh.n_kv_heads * n_parts);
-    decode_tuned_kernel<G, R><<<grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
-                                                                        chunk_tokens, n_parts, partials);
-    return cudaGetLastError();
-}
+// Launch plan of one call: context chunk per CTA, partial slots per (sequence, query head), and
+// the first item of the tail (-1: none).
+struct Plan {
+    int chunk;
+    int n_parts;
+    int tail_first;
+    unsigned grid;
+};
 
-// Context chunk per CTA.  The table build and the bins x centroids product are paid once per
-// chunk, so chunks are long (up to 65536 tokens); they are halved only while the grid would not
-// give the CTA slots of the 148 SMs one and a half CTAs each, and never below 2048 tokens.
+// The table build and the bins x centroids product are paid once per CTA, so chunks are long (up
+// to 65536 tokens); they are halved only while the grid would not give the CTA slots of the 148
+// SMs one and a half CTAs each, and never below 2048 tokens.  When every context fits one chunk
+// and the last wave of CTAs would fill at most half of the slots, the items of that wave are
+// spread over 2 to 4 CTAs each instead, which shortens the wave by that factor.  This applies
+// where one CTA fills an SM; with two CTAs per SM a CTA whose neighbour has finished already runs
+// faster, and the split was measured to gain nothing.
 template <int G, int R>
-int chunk_for(const Shape& sh)
+Plan plan_for(const Shape& sh)
 {
     using C = Cfg<G, R>;
-#ifdef CQ_TUNE_CHUNK_TOKENS
-    return CQ_TUNE_CHUNK_TOKENS;
-#endif
+    Plan pl;
     const int64_t round = C::kRoundTokens;
     const int64_t items = sh.n_seq * sh.n_kv_heads;
     const int64_t slots = 148 * C::kMinBlocks;
     int64_t chunk = (sh.max_tokens + round - 1) / round * round;
     if (chunk > 65536) chunk = 65536;
+#ifdef CQ_TUNE_CHUNK_TOKENS
+    chunk = CQ_TUNE_CHUNK_TOKENS;
+#else
     while (chunk > 2048 && 2 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
         chunk = (chunk / 2 + round - 1) / round * round;
-    return (int)chunk;
+#endif
+    pl.chunk = (int)chunk;
+    pl.n_parts = (int)((sh.max_tokens + chunk - 1) / chunk);
+    pl.tail_first = -1;
+    pl.grid = (unsigned)(items * pl.n_parts);
+#ifndef CQ_TUNE_NO_TAIL
+    const int64_t rest = items % slots;               // CTAs of the last wave
+    if (C::kMinBlocks == 1 && pl.n_parts == 1 && items > slots && rest > 0 && 2 * rest <= slots && chunk >= 4 * 2048) {
+        int64_t k = slots / rest;
+        if (k > 4) k = 4;
+        const int64_t part_chunk = ((chunk + k - 1) / k + round - 1) / round * round;
+        pl.chunk = (int)part_chunk;
+        pl.n_parts = (int)((sh.max_tokens + part_chunk - 1) / part_chunk);
+        pl.tail_first = (int)(items - rest);
+        pl.grid = (unsigned)(pl.tail_first + rest * pl.n_parts);
+    }
+#endif
+    return pl;
 }
 
-int chunk_dispatch(const Shape& sh)
+template <int G, int R>
+cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
+                       const int32_t* seq_lens, float scale, const Shape& sh, const Plan& pl, float* partials,
+                       cudaStream_t st)
 {
-    if (sh.G == 16 && sh.R == 1) return chunk_for<16, 1>(sh);
-    if (sh.G == 16 && sh.R == 2) return chunk_for<16, 2>(sh);
-    if (sh.G == 16 && sh.R == 4) return chunk_for<16, 4>(sh);
-    if (sh.G == 32 && sh.R == 1) return chunk_for<32, 1>(sh);
-    if (sh.G == 32 && sh.R == 2) return chunk_for<32, 2>(sh);
-    return 0;
+    using C = Cfg<G, R>;
+    cudaError_t e = cudaFuncSetAttribute(decode_tuned_kernel<G, R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    decode_tuned_kernel<G, R><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
+                                                                          pl.chunk, pl.n_parts, pl.tail_first, partials);
+    return cudaGetLastError();
+}
+
+Plan plan_dispatch(const Shape& sh)
+{
+    if (sh.G == 16 && sh.R == 1) return plan_for<16, 1>(sh);
+    if (sh.G == 16 && sh.R == 2) return plan_for<16, 2>(sh);
+    if (sh.G == 16 && sh.R == 4) return plan_for<16, 4>(sh);
+    if (sh.G == 32 && sh.R == 1) return plan_for<32, 1>(sh);
+    if (sh.G == 32 && sh.R == 2) return plan_for<32, 2>(sh);
+    return Plan{0, 1, -1, 0u};
 }
 
 }  // namespace
@@ -746,28 +792,22 @@ bool decode_tuned_supported(const Shape& sh)
     return (sh.G == 16 && (sh.R == 1 || sh.R == 2 || sh.R == 4)) || (sh.G == 32 && (sh.R == 1 || sh.R == 2));
 }
 
-int decode_tuned_parts(const Shape& sh)
-{
-    const int chunk = chunk_dispatch(sh);
-    if (chunk <= 0) return 1;
-    return (int)((sh.max_tokens + chunk - 1) / chunk);
-}
+int decode_tuned_parts(const Shape& sh) { return plan_dispatch(sh).n_parts; }
 
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh, float* out,
                                 float* partials, cudaStream_t st)
 {
-    const int chunk = chunk_dispatch(sh);
-    if (chunk <= 0) return cudaErrorNotSupported;
-    const int n_parts = decode_tuned_parts(sh);
+    const Plan pl = plan_dispatch(sh);
+    if (pl.chunk <= 0) return cudaErrorNotSupported;
     cudaError_t e = cudaErrorNotSupported;
-    if (sh.G == 16 && sh.R == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, chunk, n_parts, partials, st);
-    else if (sh.G == 16 && sh.R == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, chunk, n_parts, partials, st);
-    else if (sh.G == 16 && sh.R == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, chunk, n_parts, partials, st);
-    else if (sh.G == 32 && sh.R == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, chunk, n_parts, partials, st);
-    else if (sh.G == 32 && sh.R == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, chunk, n_parts, partials, st);
+    if (sh.G == 16 && sh.R == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 16 && sh.R == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 16 && sh.R == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 32 && sh.R == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 32 && sh.R == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     if (e != cudaSuccess) return e;
-    return launch_merge(partials, n_parts, sh, out, st);
+    return launch_merge(partials, pl.n_parts, sh, out, st);
 }
 
 }  // namespace cq

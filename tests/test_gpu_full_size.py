@@ -100,7 +100,9 @@ def test_config1_llama2_7b_4c8b_decode_full_size():
 def test_config2_mistral_gqa_8c8b_decode_full_size():
     w = synth.WORKLOADS[2]
     st = bench.DecodeState(w, 0, torch.device(DEV), cq)
-    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 6, 202))        # 6 KV heads = 24 query heads x 16384 tokens
+    # 6 KV heads = 24 query heads x 16384 tokens; one of them among the last items, whose context the
+    # launch plan spreads over two CTAs
+    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 6, 202, must=[(w.n_seq - 1, 3)]))
     assert ties <= total // 500
     print(f"config 2: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
 

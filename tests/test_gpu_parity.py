@@ -249,6 +249,25 @@ def test_attention_multi_chunk_gqa_and_mha_long():
         H.check_attn(out, ref, f"long c={c} Hq={n_q} Hkv={n_kv}")
 
 
+def test_attention_when_the_last_wave_of_items_is_spread_over_several_ctas():
+    # 160 (sequence, KV head) items with one CTA per SM: the items beyond a multiple of the SM count
+    # are spread over several CTAs each while the others take their whole context in one.  The spread
+    # ones include a full-length sequence, a short one (its later parts are empty) and an empty one.
+    c, b, D, n_q, n_kv = 8, 8, 128, 32, 8
+    rng = np.random.default_rng(77)
+    for lens_tail in ([8200, 100], [0, 8200]):
+        lens = [int(v) for v in rng.integers(1, 8200, size=18)] + lens_tail
+        n_seq, cap = len(lens), 8200
+        kcb, vcb = (torch.from_numpy(rng.standard_normal((n_kv, D // c, 256, c)).astype(np.float32)) for _ in range(2))
+        q = torch.from_numpy(rng.standard_normal((n_seq, n_q, D)).astype(np.float16))
+        kc_rm = rng.integers(0, 256, size=(n_seq, cap, n_kv, D // c)).astype(np.int32)
+        vc_rm = rng.integers(0, 256, size=(n_seq, cap, n_kv, D // c)).astype(np.int32)
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, D ** -0.5, c, b, 0)
+        H.check_attn(out, ref, f"spread tail, lens of the last sequences {lens_tail}")
+        for s_ in (n_seq - 2, n_seq - 1):
+            H.check_attn(out[s_], ref[s_], f"spread tail, sequence {s_}")
+
+
 def test_encode_codebooks_beyond_fp16_range_take_the_exact_path():
     # centroids too large for the fp16 term splits of the tensor-core path: the tuned kernel must
     # notice and recompute those groups exactly
