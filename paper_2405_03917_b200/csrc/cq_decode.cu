@@ -167,14 +167,22 @@ __device__ __forceinline__ void mma_rowsum_acc(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(ones), "r"(ones));
 }
 
+// One centroid into registers.  The asm statements keep the loads where the code puts them: the
+// units of a codebook are loaded one unit ahead of their use, not all at once.
+__device__ __forceinline__ float4 ldg_f4(const float* p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
+}
 template <int kC>
 __device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC])
 {
     static_assert(kC == 4 || kC == 8, "centroids of 4 or 8 channels");
-    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 a = ldg_f4(p);
     cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
     if (kC == 8) {
-        const float4 b = *reinterpret_cast<const float4*>(p + 4);
+        const float4 b = ldg_f4(p + 4);
         cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
     }
 }
@@ -298,6 +306,46 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         return;
     }
 
+    // ---------------------------------------------------------------- addresses; the first centroids travel during the set-up
+    const int64_t blk0 = t_begin / kTokenBlock;
+    const int64_t blk_lim = (t_end + kTokenBlock - 1) / kTokenBlock;       // blocks holding a valid token
+    const int n_iters = (int)((t_end - t_begin + C::kRoundTokens - 1) / C::kRoundTokens);
+    const int qb = (C::kBlocksPerIter == 8) ? r : (r & 3);                 // block of this quad inside the warp's iteration
+    uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a plane, per code word
+#pragma unroll
+    for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m);
+    // code words of this lane: word (block, group) sits at (block * G + group) * 16 bytes
+    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+
+    uint4 kw[C::kSlots], vw[C::kSlots];
+    auto load_words = [&](uint4 (&dst)[C::kSlots], const uint8_t* base, int64_t blk) {
+        if (blk < blk_lim) {
+            const uint8_t* bp = base + blk * (G * kTokenBlock);
+#pragma unroll
+            for (int m = 0; m < C::kSlots; ++m)
+                dst[m] = ldg_codes(reinterpret_cast<const uint4*>(bp + C::group_of(lane_off[m] >> 2) * kTokenBlock));
+        } else {
+#pragma unroll
+            for (int m = 0; m < C::kSlots; ++m) dst[m] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+
+    // Codebooks are read in units of kJb * 32 centroids (32 registers per lane): a warp owns whole
+    // groups, its lanes walk the code values, and the next unit is loaded while the current one is used.
+    constexpr int kJb = (kC == 8) ? 4 : 8;
+    constexpr int kUnitsPerGroup = (kRows / 32) / kJb;
+    constexpr int kUnits = C::kGroupsPerWarp * kUnitsPerGroup;
+    static_assert(kUnits % 2 == 0, "units are taken in pairs");
+    auto load_unit = [&](float (&cv)[kJb][kC], const float* cb, int u) {
+        const int g = warp * C::kGroupsPerWarp + u / kUnitsPerGroup;
+        const float* cg = cb + (((int64_t)hkv * G + g) * kRows + (u % kUnitsPerGroup) * kJb * 32 + lane) * kC;
+#pragma unroll
+        for (int jb = 0; jb < kJb; ++jb) load_centroid<kC>(cg + jb * 32 * kC, cv[jb]);
+    };
+    float cva[kJb][kC], cvb[kJb][kC];
+    load_unit(cva, kcb, 0);
+
     // ---------------------------------------------------------------- set-up: query, LUT, bins
     if (threadIdx.x < 4) {
         ctl->e_cur[threadIdx.x] = kUnset;
@@ -323,25 +371,21 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     for (int attempt = 0; attempt < 2; ++attempt) {
         const float inv = 1.f / lut_scale;
         float absmax = 0.f;
-#pragma unroll 1
-        for (int gi = 0; gi < C::kGroupsPerWarp; ++gi) {
-            const int g = warp * C::kGroupsPerWarp + gi;
+        auto build_unit = [&](const float (&cv)[kJb][kC], int u) {
+            const int g = warp * C::kGroupsPerWarp + u / kUnitsPerGroup;
             float qreg[R][kC];
 #pragma unroll
             for (int h = 0; h < R; ++h)
 #pragma unroll
                 for (int i = 0; i < kC; ++i) qreg[h][i] = qs[h * 128 + g * kC + i] * inv;
-            const float* cg = kcb + ((int64_t)hkv * G + g) * kRows * kC;
 #pragma unroll
-            for (int jb = 0; jb < kRows / 32; ++jb) {
-                const int j = jb * 32 + lane;
-                float cv[kC];
-                load_centroid<kC>(cg + j * kC, cv);
+            for (int jb = 0; jb < kJb; ++jb) {
+                const int j = ((u % kUnitsPerGroup) * kJb + jb) * 32 + lane;
 #pragma unroll
                 for (int h = 0; h < R; ++h) {
                     float dot = 0.f;
 #pragma unroll
-                    for (int i = 0; i < kC; ++i) dot = fmaf(qreg[h][i], cv[i], dot);
+                    for (int i = 0; i < kC; ++i) dot = fmaf(qreg[h][i], cv[jb][i], dot);
                     absmax = fmaxf(absmax, fabsf(dot));
                     const uint32_t e = pack_hi_lo(dot);
                     uint8_t* row = smem + j * kRowBytes + C::plane_of(h) * 128;
@@ -349,6 +393,14 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     if (C::kReplica) *reinterpret_cast<uint32_t*>(row + ((16 + g + j) & 31) * 4) = e;
                 }
             }
+        };
+        if (attempt == 1) load_unit(cva, kcb, 0);
+#pragma unroll 1
+        for (int u = 0; u < kUnits; u += 2) {
+            load_unit(cvb, kcb, u + 1);
+            build_unit(cva, u);
+            if (u + 2 < kUnits) load_unit(cva, kcb, u + 2);
+            build_unit(cvb, u + 1);
         }
         absmax = fmaxf(absmax, __shfl_xor_sync(0xffffffffu, absmax, 16));
         absmax = fmaxf(absmax, __shfl_xor_sync(0xffffffffu, absmax, 8));
@@ -366,46 +418,34 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         if (threadIdx.x == 0) ctl->lut_absmax = 0.f;
         __syncthreads();
     }
-    for (int j = warp; j < kRows; j += C::kWarps)
+    // un-rotate: a warp owns rows warp, warp + kWarps, ...; eight (row, plane) pairs per step
+    constexpr int kOwnRowPlanes = kRows / C::kWarps * C::kPlanes;
+    static_assert(kOwnRowPlanes % 8 == 0, "row batches");
+#pragma unroll 1
+    for (int i0 = 0; i0 < kOwnRowPlanes; i0 += 8) {
+        uint32_t e[8];
 #pragma unroll
-        for (int pl = 0; pl < C::kPlanes; ++pl) {
-            uint8_t* row = smem + j * kRowBytes + pl * 128;
-            const uint32_t e = *reinterpret_cast<const uint32_t*>(row + ((lane + j) & 31) * 4);
-            __syncwarp();
-            *reinterpret_cast<uint32_t*>(row + lane * 4) = e;
+        for (int k = 0; k < 8; ++k) {
+            const int j = warp + (i0 + k) / C::kPlanes * C::kWarps;
+            const uint8_t* row = smem + j * kRowBytes + (i0 + k) % C::kPlanes * 128;
+            e[k] = *reinterpret_cast<const uint32_t*>(row + ((lane + j) & 31) * 4);
         }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int j = warp + (i0 + k) / C::kPlanes * C::kWarps;
+            uint8_t* row = smem + j * kRowBytes + (i0 + k) % C::kPlanes * 128;
+            *reinterpret_cast<uint32_t*>(row + lane * 4) = e[k];
+        }
+    }
     __syncthreads();
 
     // ---------------------------------------------------------------- main loop over the chunk
-    const int64_t blk0 = t_begin / kTokenBlock;
-    const int64_t blk_lim = (t_end + kTokenBlock - 1) / kTokenBlock;       // blocks holding a valid token
-    const int n_iters = (int)((t_end - t_begin + C::kRoundTokens - 1) / C::kRoundTokens);
-    const int qb = (C::kBlocksPerIter == 8) ? r : (r & 3);                 // block of this quad inside the warp's iteration
 #ifdef CQ_TUNE_KBATCH
     constexpr int kBatch = CQ_TUNE_KBATCH;
 #else
     constexpr int kBatch = (C::kSlots * C::kLaneHeads >= 8) ? 2 : 4;       // tokens whose lookups are in flight together
 #endif
-
-    uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a plane, per code word
-#pragma unroll
-    for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m);
-    // code words of this lane: word (block, group) sits at (block * G + group) * 16 bytes
-    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
-    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
-
-    uint4 kw[C::kSlots], vw[C::kSlots];
-    auto load_words = [&](uint4 (&dst)[C::kSlots], const uint8_t* base, int64_t blk) {
-        if (blk < blk_lim) {
-            const uint8_t* bp = base + blk * (G * kTokenBlock);
-#pragma unroll
-            for (int m = 0; m < C::kSlots; ++m)
-                dst[m] = ldg_codes(reinterpret_cast<const uint4*>(bp + C::group_of(lane_off[m] >> 2) * kTokenBlock));
-        } else {
-#pragma unroll
-            for (int m = 0; m < C::kSlots; ++m) dst[m] = make_uint4(0u, 0u, 0u, 0u);
-        }
-    };
 
     // Weight units.  Each query head's bins count in units of 2^e_cur[h].  A warp adds its tokens'
     // weights without waiting for the others as long as (a) its largest score fits the unit
@@ -636,6 +676,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         }
     }
     // Warps that are done keep joining coarsening events until every warp is done.
+    load_unit(cva, vcb, 0);                       // the first V centroids travel meanwhile
     for (int guard = 0; guard < 4096; ++guard) {
         event_barrier(C::kThreads);
         if (*reinterpret_cast<volatile int*>(&ctl->want) == 0) break;
@@ -646,32 +687,39 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     // ---------------------------------------------------------------- epilogue: bins x V centroids
     // Same ownership as the table build: a warp owns whole groups, lanes walk the code values.
     // Rows are first rotated by their index so that a column read is bank-conflict free.
-    for (int j = warp; j < kRows; j += C::kWarps)
-#pragma unroll
-        for (int pl = 0; pl < C::kPlanes; ++pl) {
-            uint8_t* row = smem + C::kVOffset + j * kRowBytes + pl * 128;
-            const uint32_t v = *reinterpret_cast<const uint32_t*>(row + lane * 4);
-            __syncwarp();
-            *reinterpret_cast<uint32_t*>(row + ((lane + j) & 31) * 4) = v;
-        }
-    __syncthreads();
 #pragma unroll 1
-    for (int gi = 0; gi < C::kGroupsPerWarp; ++gi) {
-        const int g = warp * C::kGroupsPerWarp + gi;
-        const float* cg = vcb + ((int64_t)hkv * G + g) * kRows * kC;
-        float acc[R][kC];
-        float lsum[R];                        // sum of the group's bins (the normaliser)
+    for (int i0 = 0; i0 < kOwnRowPlanes; i0 += 8) {
+        uint32_t v[8];
 #pragma unroll
-        for (int h = 0; h < R; ++h) {
-            lsum[h] = 0.f;
+        for (int k = 0; k < 8; ++k) {
+            const int j = warp + (i0 + k) / C::kPlanes * C::kWarps;
+            const uint8_t* row = smem + C::kVOffset + j * kRowBytes + (i0 + k) % C::kPlanes * 128;
+            v[k] = *reinterpret_cast<const uint32_t*>(row + lane * 4);
+        }
+        __syncwarp();
 #pragma unroll
-            for (int i = 0; i < kC; ++i) acc[h][i] = 0.f;
+        for (int k = 0; k < 8; ++k) {
+            const int j = warp + (i0 + k) / C::kPlanes * C::kWarps;
+            uint8_t* row = smem + C::kVOffset + j * kRowBytes + (i0 + k) % C::kPlanes * 128;
+            *reinterpret_cast<uint32_t*>(row + ((lane + j) & 31) * 4) = v[k];
+        }
+    }
+    __syncthreads();
+    float acc[R][kC];
+    float lsum[R];                            // sum of the bins of group 0 (the normaliser)
+#pragma unroll
+    for (int h = 0; h < R; ++h) lsum[h] = 0.f;
+    auto use_unit = [&](const float (&cv)[kJb][kC], int u) {
+        const int gi = u / kUnitsPerGroup, g = warp * C::kGroupsPerWarp + gi;
+        if (u % kUnitsPerGroup == 0) {
+#pragma unroll
+            for (int h = 0; h < R; ++h)
+#pragma unroll
+                for (int i = 0; i < kC; ++i) acc[h][i] = 0.f;
         }
 #pragma unroll
-        for (int jb = 0; jb < kRows / 32; ++jb) {
-            const int j = jb * 32 + lane;
-            float cv[kC];
-            load_centroid<kC>(cg + j * kC, cv);
+        for (int jb = 0; jb < kJb; ++jb) {
+            const int j = ((u % kUnitsPerGroup) * kJb + jb) * 32 + lane;
 #pragma unroll
             for (int h = 0; h < R; ++h) {
                 const uint8_t* row = smem + C::kVOffset + j * kRowBytes + C::plane_of(h) * 128;
@@ -680,9 +728,10 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 const float bv = (float)bi;
                 if (gi == 0) lsum[h] += bv;
 #pragma unroll
-                for (int i = 0; i < kC; ++i) acc[h][i] = fmaf(bv, cv[i], acc[h][i]);
+                for (int i = 0; i < kC; ++i) acc[h][i] = fmaf(bv, cv[jb][i], acc[h][i]);
             }
         }
+        if (u % kUnitsPerGroup != kUnitsPerGroup - 1) return;
         // Sum over the 32 lanes.  The kC channel sums are folded while they are exchanged: after
         // the steps with lane masks 16, 8 (and 4 for kC = 8) a lane holds one channel, the
         // remaining steps finish that channel.
@@ -705,8 +754,16 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 }
             }
         }
+    };
+#pragma unroll 1
+    for (int u = 0; u < kUnits; u += 2) {
+        load_unit(cvb, vcb, u + 1);
+        use_unit(cva, u);
+        if (u + 2 < kUnits) load_unit(cva, vcb, u + 2);
+        use_unit(cvb, u + 1);
     }
 }
+
 
 // Launch plan of one call: context chunk per CTA, partial slots per (sequence, query head), and
 // the first item of the tail (-1: none).
