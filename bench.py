@@ -7,7 +7,7 @@ key and value vectors are CQ-encoded and appended (cq_encode, K and V), then eve
 head attends over the coded cache (cq_decode_attn).  Inputs are seeded and synthetic.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg2|cfg1|cfg4|cfg0] [--extras none|default|all]
+                    [--workload cfg2|cfg1|cfg4|cfg0] [--extras none|default|decode|all]
 
 Prints ONE JSON line (rank 0).  `value` is KV tokens/s with everything resident in HBM;
 `e2e` is the same metric through cq_decode_step_host with host buffers; `roofline` is the
@@ -381,7 +381,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg4"])
-    ap.add_argument("--extras", default="default", choices=["none", "default", "all"])
+    ap.add_argument("--extras", default="default", choices=["none", "default", "decode", "all"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -506,10 +506,12 @@ def main():
     if args.extras != "none" and world == 1:
         extras = {}
         try:
-            extras["encode"] = extra_encode_cfg3(cq, dev)
-            if args.extras == "all":
+            if args.extras != "decode":
+                extras["encode"] = extra_encode_cfg3(cq, dev)
+            if args.extras in ("decode", "all"):
                 extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
                 extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
+            if args.extras == "all":
                 extras["learn"] = extra_learn(cq, dev)
         except Exception as e:      # extras never hide the headline number
             extras["error"] = repr(e)
