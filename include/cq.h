@@ -21,8 +21,12 @@
  *   - Every function that returns int returns a cq_status: arguments are checked
  *     on the host before anything is launched, a failed check launches nothing,
  *     and a CUDA launch error is reported as CQ_ERR_CUDA.  Nothing aborts or traps.
- *   - Supported shapes: c divides head_dim, head_dim <= 256, 1 <= b <= 8 (codes
- *     are one uint8 each), n_q_heads a multiple of n_kv_heads.  Tuned kernels
+ *   - Supported shapes: c divides head_dim, head_dim <= 256, n_q_heads a multiple
+ *     of n_kv_heads, and b bits per code with 1 <= b <= 8 (one byte per code) or
+ *     b = 9, 10, 12 or 16 (the low byte as for b <= 8 plus b - 8 packed upper bits,
+ *     see the layout below; CQ-8c10b of the paper's Section 4 is the case b = 10:
+ *     1.25 bytes per code).  Decode attention needs (head_dim / c) * 2^b <= 24576
+ *     table entries (CQ_ERR_UNSUPPORTED otherwise).  Tuned kernels
  *     exist for head_dim 128 and b = 8: encode for c = 2, 4, 8; decode attention
  *     for c = 8 with 1, 2 or 4 query heads per KV head and c = 4 with 1 or 2.
  *     Every other supported shape runs on generic sm_100a kernels (never on the CPU).
@@ -35,8 +39,18 @@
  *       (((s * n_heads + h) * NB + t / 16) * G + g) * 16 + t % 16,   NB = ceil(max_tokens / 16)
  *
  * so the 16 codes of one group for 16 consecutive tokens are one aligned 16-byte
- * word.  cq_codes_to_rowmajor / cq_codes_from_rowmajor convert to and from the
- * plain [n_seq][max_tokens][n_heads][G] order.
+ * word.  For b > 8 a block of one head is G * (16 + 2 * (b - 8)) bytes: first the
+ * G 16-byte words above, holding the low byte of every code, then G words of
+ * 2 * (b - 8) bytes, word g holding the upper b - 8 bits of group g's 16 codes,
+ * token k at bits [k * (b - 8), (k + 1) * (b - 8)) of the little-endian word:
+ *
+ *   block start of (s, h, t)  = ((s * n_heads + h) * NB + t / 16) * G * (16 + 2 * (b - 8))
+ *   low byte of (.., g)       = block start + g * 16 + t % 16
+ *   upper bits of (.., g)     = block start + G * 16 + g * 2 * (b - 8), bit (t % 16) * (b - 8) onwards
+ *
+ * cq_codes_to_rowmajor / cq_codes_from_rowmajor convert to and from the plain
+ * [n_seq][max_tokens][n_heads][G] order (uint8 per code for b <= 8, uint16 for b > 8).
+ * cq_codes_bytes() is the size of a code buffer (a multiple of 16).
  */
 #ifndef CQ_H_
 #define CQ_H_
@@ -55,7 +69,8 @@ typedef enum {
     CQ_ERR_NULL = -1,        /* a required pointer is NULL                                  */
     CQ_ERR_SHAPE = -2,       /* zero / negative dims, c does not divide head_dim, Hq % Hkv, */
                              /* token range outside [0, max_tokens]                         */
-    CQ_ERR_UNSUPPORTED = -3, /* b outside [1, 8], head_dim > 256                            */
+    CQ_ERR_UNSUPPORTED = -3, /* b not in {1..8, 9, 10, 12, 16}, head_dim > 256, tables too  */
+                             /* large for shared memory                                     */
     CQ_ERR_ALIGN = -4,       /* a pointer is not aligned as documented                      */
     CQ_ERR_WORKSPACE = -5,   /* workspace smaller than the matching *_workspace_bytes()     */
     CQ_ERR_CUDA = -6         /* a CUDA runtime call or launch failed                        */

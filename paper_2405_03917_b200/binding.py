@@ -141,7 +141,9 @@ def cq_encode(x: torch.Tensor, codebooks: torch.Tensor, c: int, b: int, codes_ou
 
 def cq_codes_to_rowmajor(codes: torch.Tensor, n_seq: int, max_tokens: int, n_heads: int, head_dim: int, c: int,
                          b: int) -> torch.Tensor:
-    out = torch.empty(n_seq, max_tokens, n_heads, head_dim // c, dtype=torch.uint8, device=codes.device)
+    # one byte per code for b <= 8, else two (returned as int16 holding the unsigned 16-bit pattern)
+    out = torch.empty(n_seq, max_tokens, n_heads, head_dim // c, dtype=torch.uint8 if b <= 8 else torch.int16,
+                      device=codes.device)
     st = lib().cq_codes_to_rowmajor(_dev(codes, torch.uint8, "codes"), n_seq, max_tokens, n_heads, head_dim, c, b,
                                     out.data_ptr(), _stream())
     _check(st, "cq_codes_to_rowmajor")
@@ -154,7 +156,7 @@ def cq_codes_from_rowmajor(rowmajor: torch.Tensor, head_dim: int, c: int, b: int
         raise ValueError("last dimension must be head_dim / c")
     out = torch.empty(cq_codes_bytes(n_seq, max_tokens, n_heads, head_dim, c, b), dtype=torch.uint8,
                       device=rowmajor.device)
-    st = lib().cq_codes_from_rowmajor(_dev(rowmajor, torch.uint8, "rowmajor"), n_seq, max_tokens, n_heads, head_dim,
+    st = lib().cq_codes_from_rowmajor(_dev(rowmajor, torch.uint8 if b <= 8 else torch.int16, "rowmajor"), n_seq, max_tokens, n_heads, head_dim,
                                       c, b, out.data_ptr(), _stream())
     _check(st, "cq_codes_from_rowmajor")
     return out

@@ -19,7 +19,9 @@ int make_shape(int64_t n_seq, int64_t max_tokens, int n_q_heads, int n_kv_heads,
     if (n_seq <= 0 || max_tokens <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0 || c <= 0)
         return CQ_ERR_SHAPE;
     if (head_dim % c != 0 || n_q_heads % n_kv_heads != 0) return CQ_ERR_SHAPE;
-    if (b < 1 || b > 8 || head_dim > kMaxHeadDim) return CQ_ERR_UNSUPPORTED;
+    // codes wider than a byte keep their upper bits in a separate word of the block; only widths
+    // whose upper part never straddles a byte are laid out
+    if (b < 1 || (b > 8 && b != 9 && b != 10 && b != 12 && b != 16) || head_dim > kMaxHeadDim) return CQ_ERR_UNSUPPORTED;
     if (n_seq * (int64_t)n_q_heads > (int64_t)1 << 24) return CQ_ERR_UNSUPPORTED;
     sh->n_seq = n_seq;
     sh->max_tokens = max_tokens;
@@ -32,6 +34,8 @@ int make_shape(int64_t n_seq, int64_t max_tokens, int n_q_heads, int n_kv_heads,
     sh->G = head_dim / c;
     sh->K = 1 << b;
     sh->R = n_q_heads / n_kv_heads;
+    sh->hb = high_bits(b);
+    sh->block_bytes = block_bytes_for(sh->G, b);
     return CQ_OK;
 }
 
@@ -77,7 +81,7 @@ size_t cq_codes_bytes(int64_t n_seq, int64_t max_tokens, int n_heads, int head_d
 {
     Shape sh;
     if (make_shape(n_seq, max_tokens, n_heads, n_heads, head_dim, c, b, &sh) != CQ_OK) return 0;
-    return (size_t)sh.n_seq * n_heads * sh.n_blocks * sh.G * kTokenBlock;
+    return round_up((size_t)sh.n_seq * n_heads * sh.n_blocks * sh.block_bytes, 16);
 }
 
 int cq_encode_variant(const void* x_fp16, const float* codebooks, const int32_t* seq_offsets, int64_t n_seq,
@@ -239,7 +243,11 @@ namespace {
 int learn_shape(int64_t n_vec, int n_heads, int head_dim, int c, int b, Shape* sh)
 {
     if (n_vec <= 0) return CQ_ERR_SHAPE;
-    return make_shape(1, n_vec, n_heads, n_heads, head_dim, c, b, sh);
+    const int st = make_shape(1, n_vec, n_heads, n_heads, head_dim, c, b, sh);
+    if (st != CQ_OK) return st;
+    // the update step keeps sums, counts and the old centroids of one problem in shared memory
+    if ((size_t)(2 * sh->K * sh->c + sh->K) * sizeof(float) > (size_t)200 * 1024) return CQ_ERR_UNSUPPORTED;
+    return CQ_OK;
 }
 }  // namespace
 

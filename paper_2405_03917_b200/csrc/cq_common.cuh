@@ -25,13 +25,41 @@ struct Shape {
     int G;                // head_dim / c
     int K;                // 2^b
     int R;                // n_q_heads / n_kv_heads
+    int hb;               // code bits above the low byte: 0 for b <= 8, else b - 8 (1, 2, 4 or 8)
+    int block_bytes;      // bytes of one 16-token block of one head: G * (16 + 2 * hb)
 };
 
-// Byte offset of the 16-byte code word of (sequence s, head h, block blk, group g).
+// Bits of a code above its low byte, and the bytes of a block, for b bits per code.
+__host__ __device__ inline int high_bits(int b) { return b > 8 ? b - 8 : 0; }
+__host__ __device__ inline int block_bytes_for(int G, int b) { return G * (kTokenBlock + 2 * high_bits(b)); }
+
+// Layout of a block (16 tokens of one head): first the G low words (16 bytes: the low byte of the
+// code of each token), then, for b > 8, the G high words (2 * hb bytes: the remaining hb bits of
+// token k at bits [k * hb, (k + 1) * hb), little endian).
+// Byte offset of the low word of (sequence s, head h, block blk, group g).
 __host__ __device__ inline int64_t code_word_offset(const Shape& sh, int n_heads, int64_t s, int h, int64_t blk, int g)
 {
-    return (((s * n_heads + h) * sh.n_blocks + blk) * sh.G + g) * (int64_t)kTokenBlock;
+    return ((s * n_heads + h) * sh.n_blocks + blk) * (int64_t)sh.block_bytes + (int64_t)g * kTokenBlock;
 }
+// Byte offset of the high word of the same (block, group); only for b > 8.
+__host__ __device__ inline int64_t code_high_offset(const Shape& sh, int n_heads, int64_t s, int h, int64_t blk, int g)
+{
+    return ((s * n_heads + h) * sh.n_blocks + blk) * (int64_t)sh.block_bytes + (int64_t)sh.G * kTokenBlock +
+           (int64_t)g * 2 * sh.hb;
+}
+#ifdef __CUDACC__
+// Code of token k (0..15) of group g in the block that starts at `block`.
+__device__ inline int read_code(const uint8_t* __restrict__ block, const Shape& sh, int g, int k)
+{
+    int code = block[g * kTokenBlock + k];
+    if (sh.hb) {
+        const int bit = k * sh.hb;
+        const int hi = (block[sh.G * kTokenBlock + g * 2 * sh.hb + (bit >> 3)] >> (bit & 7)) & ((1 << sh.hb) - 1);
+        code |= hi << 8;
+    }
+    return code;
+}
+#endif
 
 // A split-K partial: running max (log2 domain), normaliser, head_dim accumulators.
 __host__ __device__ inline int partial_stride(int head_dim) { return head_dim + 2; }

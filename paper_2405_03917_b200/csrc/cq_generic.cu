@@ -40,7 +40,19 @@ __global__ void encode_generic_kernel(const __half* __restrict__ x, const float*
                 arg = j;
             }
         }
-        codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + pos % kTokenBlock] = (uint8_t)arg;
+        const int k = (int)(pos % kTokenBlock);
+        codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + k] = (uint8_t)arg;
+        if (sh.hb) {
+            // The upper bits share a byte with other tokens, which other threads write: the bits are
+            // replaced with atomics on the aligned 32-bit word that holds the byte.
+            const int bit = k * sh.hb;
+            const uintptr_t a = reinterpret_cast<uintptr_t>(codes) +
+                                (uintptr_t)code_high_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + (bit >> 3);
+            unsigned int* w = reinterpret_cast<unsigned int*>(a & ~(uintptr_t)3);
+            const int shift = (int)(a & 3) * 8 + (bit & 7);
+            atomicAnd(w, ~((unsigned int)((1 << sh.hb) - 1) << shift));
+            atomicOr(w, (unsigned int)(arg >> 8) << shift);
+        }
     }
 }
 
@@ -71,10 +83,14 @@ __global__ void to_rowmajor_kernel(const uint8_t* __restrict__ codes, Shape sh, 
         rest /= sh.n_blocks;
         const int h = (int)(rest % n_heads);
         const int64_t s = rest / n_heads;
-        const uint8_t* src = codes + w * kTokenBlock;
+        const uint8_t* block = codes + code_word_offset(sh, n_heads, s, h, blk, 0);
         for (int k = 0; k < kTokenBlock; ++k) {
             const int64_t t = blk * kTokenBlock + k;
-            if (t < sh.max_tokens) rm[((s * sh.max_tokens + t) * n_heads + h) * sh.G + g] = src[k];
+            if (t >= sh.max_tokens) continue;
+            const int code = read_code(block, sh, g, k);
+            const int64_t e = ((s * sh.max_tokens + t) * n_heads + h) * sh.G + g;
+            if (sh.hb) reinterpret_cast<uint16_t*>(rm)[e] = (uint16_t)code;
+            else rm[e] = (uint8_t)code;
         }
     }
 }
@@ -90,10 +106,23 @@ __global__ void from_rowmajor_kernel(const uint8_t* __restrict__ rm, Shape sh, u
         rest /= sh.n_blocks;
         const int h = (int)(rest % n_heads);
         const int64_t s = rest / n_heads;
-        uint8_t* dst = codes + w * kTokenBlock;
+        uint8_t* dst = codes + code_word_offset(sh, n_heads, s, h, blk, g);
+        uint8_t* dst_hi = codes + code_high_offset(sh, n_heads, s, h, blk, g);     // this thread owns the whole high word
+        unsigned int hi_byte = 0;
         for (int k = 0; k < kTokenBlock; ++k) {
             const int64_t t = blk * kTokenBlock + k;
-            dst[k] = t < sh.max_tokens ? rm[((s * sh.max_tokens + t) * n_heads + h) * sh.G + g] : (uint8_t)0;
+            const int64_t e = ((s * sh.max_tokens + t) * n_heads + h) * sh.G + g;
+            int code = 0;
+            if (t < sh.max_tokens) code = sh.hb ? (int)reinterpret_cast<const uint16_t*>(rm)[e] : (int)rm[e];
+            dst[k] = (uint8_t)code;
+            if (sh.hb) {
+                const int bit = k * sh.hb;
+                hi_byte |= (unsigned int)((code >> 8) & ((1 << sh.hb) - 1)) << (bit & 7);
+                if (((bit + sh.hb) & 7) == 0) {
+                    dst_hi[bit >> 3] = (uint8_t)hi_byte;
+                    hi_byte = 0;
+                }
+            }
         }
     }
 }
@@ -210,11 +239,12 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
     for (int64_t t0 = t_begin; t0 < t_end; t0 += blockDim.x) {
         const int64_t t = t0 + threadIdx.x;
         const bool valid = t < t_end;
-        const int64_t word0 = (t / kTokenBlock) * sh.G * kTokenBlock + t % kTokenBlock;
+        const int64_t block0 = (t / kTokenBlock) * sh.block_bytes;
+        const int k16 = (int)(t % kTokenBlock);
         float sc = -INFINITY;
         if (valid) {
             sc = 0.f;
-            for (int g = 0; g < sh.G; ++g) sc += lut[g * sh.K + kbase[word0 + g * kTokenBlock]];
+            for (int g = 0; g < sh.G; ++g) sc += lut[g * sh.K + read_code(kbase + block0, sh, g, k16)];
         }
         const float m_tile = block_reduce_max(sc, red);
         if (m_tile > m_run) {
@@ -227,7 +257,7 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
         if (valid) {
             const float p = exp2f(sc - m_run);
             l_thr += p;
-            for (int g = 0; g < sh.G; ++g) atomicAdd(&bins[g * sh.K + vbase[word0 + g * kTokenBlock]], p);
+            for (int g = 0; g < sh.G; ++g) atomicAdd(&bins[g * sh.K + read_code(vbase + block0, sh, g, k16)], p);
         }
         __syncthreads();
     }

@@ -116,7 +116,8 @@ lloyd_update_kernel(const __half* __restrict__ x, const float* __restrict__ weig
     __syncthreads();
     double obj = 0.0;
     for (int64_t i = threadIdx.x; i < n_vec; i += kUpdThreads) {
-        const int code = codes[code_word_offset(sh, sh.n_kv_heads, 0, h, i / kTokenBlock, g) + i % kTokenBlock];
+        const int code = read_code(codes + code_word_offset(sh, sh.n_kv_heads, 0, h, i / kTokenBlock, 0), sh, g,
+                                   (int)(i % kTokenBlock));
         const float w = weights ? weights[i * n_prob + p] : 1.f;
         const __half* xv = x + (i * n_prob + p) * (int64_t)c;
         double d = 0.0;
@@ -155,7 +156,7 @@ LearnLayout learn_layout(const Shape& sh, int64_t n_vec)
 {
     LearnLayout l;
     const size_t n_prob = (size_t)sh.n_kv_heads * sh.G;
-    l.codes = round256((size_t)sh.n_kv_heads * ((n_vec + kTokenBlock - 1) / kTokenBlock) * sh.G * kTokenBlock);
+    l.codes = round256((size_t)sh.n_kv_heads * ((n_vec + kTokenBlock - 1) / kTokenBlock) * sh.block_bytes);
     l.dist = round256((size_t)n_vec * n_prob * sizeof(double));
     l.tmp_cb = round256(n_prob * sh.K * sh.c * sizeof(float));
     l.total = l.codes + 2 * l.dist + l.tmp_cb;      // dist and contrib

@@ -50,7 +50,14 @@ def test_code_buffer_sizes():
     assert cq.cq_codes_bytes(2, 17, 3, 64, 4, 5) == 2 * 3 * 2 * 16 * 16               # 17 tokens -> 2 blocks
     # invalid shapes give 0
     assert cq.cq_codes_bytes(1, 16, 1, 128, 3, 8) == 0      # c does not divide head_dim
-    assert cq.cq_codes_bytes(1, 16, 1, 128, 8, 9) == 0      # b > 8
+    # codes wider than a byte: 16 low bytes + 2 (b - 8) bytes of upper bits per (block, group);
+    # CQ-8c10b is 10 bits per 8 channels = 1.25 bits per channel (Table 1)
+    assert cq.cq_codes_bytes(1, 16, 1, 128, 8, 10) == 16 * 20
+    assert cq.cq_codes_bytes(1, 16, 1, 128, 8, 10) * 8 / (16 * 128) == 1.25
+    assert cq.cq_codes_bytes(2, 17, 3, 64, 8, 12) == 2 * 3 * 2 * 8 * 24
+    assert cq.cq_codes_bytes(1, 16, 1, 8, 8, 9) == 32       # 18 bytes, rounded up to a multiple of 16
+    assert cq.cq_codes_bytes(1, 16, 1, 128, 8, 11) == 0     # widths whose upper bits would straddle bytes
+    assert cq.cq_codes_bytes(1, 16, 1, 128, 8, 17) == 0
     assert cq.cq_codes_bytes(0, 16, 1, 128, 8, 8) == 0
     assert cq.cq_codes_bytes(1, 16, 1, 512, 8, 8) == 0      # head_dim > 256
 
@@ -76,7 +83,7 @@ def test_argument_validation_happens_on_the_host(L):
     assert enc(n_tok=17) == -2                 # past capacity
     assert enc(off=-1) == -2
     assert enc(b=0) == -3
-    assert enc(b=9) == -3
+    assert enc(b=11) == -3                     # a width whose upper bits would straddle bytes
     assert enc(D=512, c=8) == -3
     assert enc(x=p + 2) == -4
     assert enc(n_tok=0) == 0                   # nothing to do, nothing launched

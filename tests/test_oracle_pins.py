@@ -108,7 +108,7 @@ def test_c1_reduces_to_scalar_bucketing():
         assert np.array_equal(codes[:, 0, ch], want)
 
 
-@pytest.mark.parametrize("c,b", [(2, 8), (4, 6), (8, 8)])
+@pytest.mark.parametrize("c,b", [(2, 8), (4, 6), (8, 8), (8, 10), (4, 9)])
 def test_matches_torch_cdist_argmin(c, b):
     D, n_heads = 64, 3
     x, cb = rand_case(40, n_heads, D, c, b)
@@ -189,7 +189,7 @@ def torch_dense(q, kc, vc, kcb, vcb, sl, scale, c, b):
     return out
 
 
-@pytest.mark.parametrize("c,b,Hq,Hkv", [(8, 8, 4, 2), (4, 8, 2, 2), (2, 5, 6, 2)])
+@pytest.mark.parametrize("c,b,Hq,Hkv", [(8, 8, 4, 2), (4, 8, 2, 2), (2, 5, 6, 2), (8, 10, 2, 1)])
 def test_dense_matches_torch_softmax(c, b, Hq, Hkv):
     D = 32
     args = attn_case(3, Hq, Hkv, D, c, b, 37, lens=[37, 5, 0])
