@@ -186,7 +186,8 @@ class DecodeState:
         """Bytes decode attention must read per call: one byte per (token, KV head, group) for K
         and for V, both codebooks once per KV head, queries; plus the output it writes."""
         w = self.w
-        codes = 2 * self.kv_tokens() * w.n_kv_heads * w.G
+        code_bytes_x16 = 16 + 2 * max(0, w.b - 8)               # bytes of 16 codes of one group
+        codes = 2 * self.kv_tokens() * w.n_kv_heads * w.G * code_bytes_x16 // 16
         books = 2 * w.n_kv_heads * w.G * (1 << w.b) * w.c * 4
         qo = w.n_seq * w.n_q_heads * w.head_dim * (2 + 4)
         return codes + books + qo
@@ -511,6 +512,7 @@ def main():
             if args.extras in ("decode", "all"):
                 extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
                 extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
+                extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
             if args.extras == "all":
                 extras["learn"] = extra_learn(cq, dev)
         except Exception as e:      # extras never hide the headline number

@@ -8,6 +8,7 @@ using namespace cq;
 namespace {
 
 constexpr int kMaxHeadDim = 256;
+constexpr int64_t kSmallEncodeVectors = 128;         // appends up to this many vectors per head may take the few-vector kernel
 constexpr int64_t kGenericMaxTableEntries = 24576;   // (G * 2^b) floats x 2 tables must fit shared memory
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -95,12 +96,22 @@ int cq_encode_variant(const void* x_fp16, const float* codebooks, const int32_t*
     if (n_tokens < 0 || token_offset < 0) return CQ_ERR_SHAPE;
     if (!seq_offsets && token_offset + n_tokens > max_tokens) return CQ_ERR_SHAPE;
     if (!aligned16(x_fp16) || !aligned16(codebooks) || !aligned16(codes_out)) return CQ_ERR_ALIGN;
-    if (variant < 0 || variant > 2) return CQ_ERR_SHAPE;
+    if (variant < 0 || variant > 3) return CQ_ERR_SHAPE;
     if (n_tokens == 0) return CQ_OK;
     const bool tuned_ok = encode_tuned_supported(sh);
     if (variant == 2 && !tuned_ok) return CQ_ERR_UNSUPPORTED;
-    const bool use_tuned = variant == 2 || (variant == 0 && tuned_ok);
+    const bool small_ok = encode_small_supported(sh);
+    if (variant == 3 && !small_ok) return CQ_ERR_UNSUPPORTED;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    // An append (a few vectors per head) is latency-bound.  Shapes without a tuned kernel take the
+    // few-vector kernel for it (13 us against 300 us of the generic kernel for 64 vectors x 8 heads of
+    // CQ-8c8b); the tuned kernel's single-tile form is still faster where it exists (9 us).
+    if (variant == 3 || (variant == 0 && !tuned_ok && small_ok && n_seq * n_tokens <= kSmallEncodeVectors)) {
+        cudaError_t es = launch_encode_small(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh, n_tokens,
+                                             token_offset, static_cast<uint8_t*>(codes_out), cs);
+        return es == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    }
+    const bool use_tuned = variant == 2 || (variant == 0 && tuned_ok);
     cudaError_t e = use_tuned
                         ? launch_encode_tuned(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh, n_tokens,
                                               token_offset, static_cast<uint8_t*>(codes_out), cs)

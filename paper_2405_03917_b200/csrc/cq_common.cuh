@@ -67,6 +67,9 @@ __host__ __device__ inline int partial_stride(int head_dim) { return head_dim + 
 // ---- launchers implemented in the .cu files (return cudaGetLastError()) ----
 cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                   int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
+bool encode_small_supported(const Shape& sh);       // few-vector kernel: the group's codebook fits 48 KiB
+cudaError_t launch_encode_small(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
+                                int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
 bool encode_tuned_supported(const Shape& sh);
 cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                 int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);

@@ -69,6 +69,98 @@ cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_
 }
 
 // ------------------------------------------------------------------------------------------
+// Encode of a few vectors per head (the append of a decode step).  One CTA per (head, group,
+// run of 8 vectors): the group's codebook is staged in shared memory, channel-major, together
+// with one vector per warp, and the lanes of a warp share the 2^b centroids.  Distances are
+// formed exactly as in encode_generic_kernel; the lowest index wins ties.  The kernel is
+// latency-bound, so everything it reads from global memory is requested before the one barrier.
+// ------------------------------------------------------------------------------------------
+constexpr int kSmallWarps = 8;
+constexpr int kSmallVecPerCta = kSmallWarps;
+
+__global__ void __launch_bounds__(kSmallWarps * 32)
+encode_small_kernel(const __half* __restrict__ x, const float* __restrict__ cb, const int32_t* __restrict__ seq_offsets,
+                    Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes)
+{
+    extern __shared__ __align__(16) float cbt[];            // [c][K], then [warps][c] for the vectors
+    const int n_heads = sh.n_kv_heads;
+    const int prob = blockIdx.x % (n_heads * sh.G);
+    const int64_t run = blockIdx.x / (n_heads * sh.G);
+    const int h = prob / sh.G, g = prob % sh.G;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* xs = cbt + sh.K * sh.c + warp * sh.c;
+    const int64_t n_vec = sh.n_seq * n_tokens;
+    const int64_t v = run * kSmallVecPerCta + warp;
+    const int64_t s = v / n_tokens, i = v % n_tokens;
+    int64_t pos = -1;
+    const __half* xv = x + ((s * n_tokens + i) * n_heads + h) * (int64_t)sh.head_dim + g * sh.c;
+    __half x_first = __float2half(0.f);          // requested now, stored after the codebook has been requested too
+    if (v < n_vec) {
+        pos = token_offset + (seq_offsets ? seq_offsets[s] : 0) + i;
+        if (lane < sh.c) x_first = xv[lane];
+    }
+    const float* cg = cb + (int64_t)prob * sh.K * sh.c;
+    for (int e = threadIdx.x; e < sh.K * sh.c; e += blockDim.x) cbt[(e % sh.c) * sh.K + e / sh.c] = cg[e];
+    if (v < n_vec) {
+        if (lane < sh.c) xs[lane] = __half2float(x_first);
+        for (int k = lane + 32; k < sh.c; k += 32) xs[k] = __half2float(xv[k]);
+    }
+    __syncthreads();
+    if (pos >= 0 && pos < sh.max_tokens) {                                  // same decision in every lane
+        float best = INFINITY;
+        int arg = 0;
+        for (int j = lane; j < sh.K; j += 32) {
+            float d = 0.f;
+            for (int k = 0; k < sh.c; ++k) {
+                const float diff = xs[k] - cbt[k * sh.K + j];
+                d = fmaf(diff, diff, d);
+            }
+            if (d < best) {       // j rises: the lowest index of this lane wins ties
+                best = d;
+                arg = j;
+            }
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+            if (ob < best || (ob == best && oa < arg)) {
+                best = ob;
+                arg = oa;
+            }
+        }
+        if (lane == 0) {
+            const int k = (int)(pos % kTokenBlock);
+            codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + k] = (uint8_t)arg;
+            if (sh.hb) {
+                const int bit = k * sh.hb;
+                const uintptr_t a = reinterpret_cast<uintptr_t>(codes) +
+                                    (uintptr_t)code_high_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + (bit >> 3);
+                unsigned int* w = reinterpret_cast<unsigned int*>(a & ~(uintptr_t)3);
+                const int shift = (int)(a & 3) * 8 + (bit & 7);
+                atomicAnd(w, ~((unsigned int)((1 << sh.hb) - 1) << shift));
+                atomicOr(w, (unsigned int)(arg >> 8) << shift);
+            }
+        }
+    }
+}
+
+static size_t small_smem(const Shape& sh) { return (size_t)(sh.K + kSmallWarps) * sh.c * sizeof(float); }
+bool encode_small_supported(const Shape& sh) { return small_smem(sh) <= 48 * 1024; }
+
+cudaError_t launch_encode_small(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
+                                int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st)
+{
+    const int64_t n_vec = sh.n_seq * n_tokens;
+    if (n_vec == 0) return cudaSuccess;
+    const int64_t runs = (n_vec + kSmallVecPerCta - 1) / kSmallVecPerCta;
+    const int64_t grid = runs * sh.n_kv_heads * sh.G;
+    if (grid > 0x7fffffff) return cudaErrorInvalidValue;
+    encode_small_kernel<<<(unsigned)grid, kSmallWarps * 32, small_smem(sh), st>>>(
+        x, cb, seq_offsets, sh, n_tokens, token_offset, codes);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
 // Layout converters between the library layout and [n_seq][max_tokens][n_heads][G].
 // One thread per code word (16 tokens of one group).
 // ------------------------------------------------------------------------------------------

@@ -135,6 +135,9 @@ WORKLOADS: List[Workload] = [
     Workload("cfg2_mistral_7b_gqa_8c8b_decode", 2, 8, 8, 1, 64, 32, 8, 16384),
     Workload("cfg3_2c8b_prefill_encode", 3, 2, 8, 1, 8, 32, 32, 8192),
     Workload("cfg4_llama2_13b_8c8b_full_step", 4, 8, 8, 40, 32, 40, 40, 32768, min_tokens=8192),
+    # CQ-8c10b (1024 centroids per group, 1.25 bytes per code), Llama-2-7B-shaped heads; not one of the
+    # measured configurations of the headline metric: a workload for the wide-code path
+    Workload("cfg5_llama2_7b_8c10b_decode", 5, 8, 10, 1, 16, 32, 32, 8192),
 ]
 
 

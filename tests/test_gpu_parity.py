@@ -44,8 +44,9 @@ def test_config0_encode_bit_exact(variant):
 ])
 def test_encode_shapes_and_ragged_tails(c, b, head_dim, n_heads, n_tokens):
     xk, xv, kcb, vcb, _ = H.generic_case(11 * c + b, 2, n_tokens, n_heads, n_heads, head_dim, c, b)
+    tuned = head_dim == 128 and b == 8 and c in (2, 4, 8)
     for x, cb in ((xk, kcb), (xv, vcb)):
-        for variant in (1, 0):
+        for variant in (1, 0, 3) + ((2,) if tuned else ()):       # generic, automatic, few-vector, tuned
             _, rm = encode_both(x, cb, c, b, n_tokens, variant)
             H.check_codes(x.numpy().reshape(-1, n_heads, head_dim), cb.numpy(),
                           rm.reshape(-1, n_heads, head_dim // c), c, b)
@@ -61,7 +62,7 @@ def test_encode_codebook_contains_inputs_and_exact_ties():
     hh = torch.arange(H_)[None, :, None]
     gg = torch.arange(D // c)[None, None, :]
     x = cb[hh, gg, pick[0]].reshape(1, 64, H_, D)        # group g of token t = centroid pick[t, h, g]
-    for variant in (1, 0):
+    for variant in (1, 0, 2, 3):
         _, rm = encode_both(x.to(torch.float16), cb, c, b, 64, variant)
         want = torch.where(pick == 200, torch.tensor(7), pick).numpy()
         assert np.array_equal(rm.astype(np.int64), want)
@@ -277,8 +278,9 @@ def test_encode_codebooks_beyond_fp16_range_take_the_exact_path():
         kcb = kcb.clone()
         kcb[0, 1] *= 3.0e4                      # one group of head 0 far outside the range
         kcb[1, 0, 5] = 7.0e4                    # one centroid of another group
-        _, rm = encode_both(xk, kcb, c, b, n, 0)
-        H.check_codes(xk.numpy().reshape(-1, nh, D), kcb.numpy(), rm.reshape(-1, nh, D // c), c, b)
+        for variant in (2, 0):
+            _, rm = encode_both(xk, kcb, c, b, n, variant)
+            H.check_codes(xk.numpy().reshape(-1, nh, D), kcb.numpy(), rm.reshape(-1, nh, D // c), c, b)
 
 
 def test_attention_table_entries_beyond_fp16_range_are_prescaled():
