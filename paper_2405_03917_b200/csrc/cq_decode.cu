@@ -765,6 +765,420 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 }
 
 
+// ---------------------------------------------------------------------------------------------
+// CQ-8c10b (Section 4 of the paper: groups of 8 channels, 1024 centroids per group, 1.25 bytes per
+// code).  The formulation and the weight-unit protocol are those of decode_tuned_kernel; what
+// changes is the size of the tables.  One CTA of 16 warps serves one QUERY head (query heads that
+// share a KV head read the same codes again, from L2):
+//   K table: row j (128 bytes) holds the 16 groups' entries of code value j twice, words g and
+//            16 + g, so that the two half warps of a lookup use different banks (128 KiB);
+//   V bins:  row j (64 bytes) holds the 16 groups' bins of code value j (64 KiB): bins of even and
+//            odd code values fall into different halves of the banks, so a bin update of a warp
+//            takes two wavefronts when two of its lanes meet, one otherwise.
+// Code words: the low bytes of a (block, group) are one 16-byte word as for b = 8; the upper two
+// bits of its 16 tokens are one 32-bit word, 256 bytes into the block.
+// ---------------------------------------------------------------------------------------------
+struct WideCfg {
+    static constexpr int kC = 8, kG = 16, kRows = 1024;
+    static constexpr int kWarps = 16, kThreads = kWarps * 32;
+    static constexpr int kSlots = 4, kBlocksPerIter = 8;
+    static constexpr int kRoundTokens = kWarps * kBlocksPerIter * 16;
+    static constexpr int kKRowBytes = 128, kVRowBytes = 64;
+    static constexpr int kVOffset = kRows * kKRowBytes;
+    static constexpr int kTableBytes = kVOffset + kRows * kVRowBytes;
+    static constexpr int kSmemBytes = kTableBytes + 128 + 128 * 4;      // tables, control block, scaled query
+    static constexpr int kBlockBytes = kG * (16 + 4);
+    static constexpr int kLog2Groups = 4;
+    __device__ static __forceinline__ int word(int r, int p, int m) { return 16 * (r >> 2) + 4 * ((r + m) & 3) + p; }
+};
+
+__device__ __forceinline__ uint32_t ldg_u32(const uint8_t* p)
+{
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+// table byte offset (code << row_shift) + lane_off for token k of a code word: low byte from `w`,
+// upper two bits from `hw`
+__device__ __forceinline__ uint32_t wide_index(const uint4& w, uint32_t hw, int k, uint32_t lane_off, int row_shift)
+{
+    const uint32_t low = __byte_perm(word32(w, k), 0u, 0x4440u | (uint32_t)(k & 3));
+    const uint32_t hi = (hw >> (2 * k)) & 3u;
+    return (low << row_shift) + (hi << (row_shift + 8)) + lane_off;
+}
+
+__global__ void __launch_bounds__(WideCfg::kThreads, 1)
+decode_wide_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
+                   const float* __restrict__ kcb, const float* __restrict__ vcb,
+                   const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
+                   int tail_first, float* __restrict__ partials)
+{
+    using C = WideCfg;
+    constexpr int kC = C::kC;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + C::kTableBytes);
+    float* qs = reinterpret_cast<float*>(smem + C::kTableBytes + 128);     // [128], scaled by scale*log2(e)
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int r = lane >> 2, p = lane & 3;
+
+    // work item: (context part, sequence, query head), with the same tail rule as decode_tuned_kernel
+    const int n_items = (int)(sh.n_q_heads * sh.n_seq);
+    int item = blockIdx.x % n_items;
+    int part = (int)(blockIdx.x / n_items);
+    bool whole = false;
+    if (tail_first >= 0) {
+        whole = (int)blockIdx.x < tail_first;
+        item = whole ? blockIdx.x : tail_first + (blockIdx.x - tail_first) / n_parts;
+        part = whole ? 0 : (blockIdx.x - tail_first) % n_parts;
+    }
+    const int hq = item % sh.n_q_heads;
+    const int64_t s = item / sh.n_q_heads;
+    const int hkv = hq / sh.R;
+
+    int64_t n = seq_lens[s];
+    n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
+    const int64_t t_begin = (int64_t)part * chunk_tokens;
+    const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
+    const int stride = partial_stride(128);
+    float* part_base = partials + ((s * sh.n_q_heads + hq) * n_parts + part) * stride;
+    if (whole)
+        for (int i = threadIdx.x; i < (n_parts - 1) * stride; i += C::kThreads)
+            part_base[stride + i] = i % stride == 0 ? -INFINITY : 0.f;
+    if (t_begin >= t_end) {
+        for (int i = threadIdx.x; i < stride; i += C::kThreads) part_base[i] = i == 0 ? -INFINITY : 0.f;
+        return;
+    }
+
+    // ---------------------------------------------------------------- addresses; the first centroids travel during the set-up
+    const int64_t blk0 = t_begin / kTokenBlock;
+    const int64_t blk_lim = (t_end + kTokenBlock - 1) / kTokenBlock;
+    const int n_iters = (int)((t_end - t_begin + C::kRoundTokens - 1) / C::kRoundTokens);
+    uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a K row, per code word
+#pragma unroll
+    for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m);
+    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+
+    uint4 kw[C::kSlots], vw[C::kSlots];
+    uint32_t kh[C::kSlots], vh[C::kSlots];
+    auto load_words = [&](uint4 (&dst)[C::kSlots], uint32_t (&dsth)[C::kSlots], const uint8_t* base, int64_t blk) {
+        if (blk < blk_lim) {
+            const uint8_t* bp = base + blk * C::kBlockBytes;
+#pragma unroll
+            for (int m = 0; m < C::kSlots; ++m) {
+                const int gm = (lane_off[m] >> 2) & 15;
+                dst[m] = ldg_codes(reinterpret_cast<const uint4*>(bp + gm * kTokenBlock));
+                dsth[m] = ldg_u32(bp + C::kG * kTokenBlock + gm * 4);
+            }
+        } else {
+#pragma unroll
+            for (int m = 0; m < C::kSlots; ++m) {
+                dst[m] = make_uint4(0u, 0u, 0u, 0u);
+                dsth[m] = 0u;
+            }
+        }
+    };
+
+    // Codebooks: warp g owns group g; its lanes walk the code values in units of 4 x 32 centroids
+    // (32 registers per lane), the next unit loaded while the current one is used.
+    constexpr int kJb = 4;
+    constexpr int kUnits = C::kRows / 32 / kJb;
+    const int g = warp;
+    auto load_unit = [&](float (&cv)[kJb][kC], const float* cb, int u) {
+        const float* cg = cb + (((int64_t)hkv * C::kG + g) * C::kRows + u * kJb * 32 + lane) * kC;
+#pragma unroll
+        for (int jb = 0; jb < kJb; ++jb) load_centroid<kC>(cg + jb * 32 * kC, cv[jb]);
+    };
+    float cva[kJb][kC], cvb[kJb][kC];
+    load_unit(cva, kcb, 0);
+
+    // ---------------------------------------------------------------- set-up: query, LUT, bins
+    if (threadIdx.x < 4) {
+        ctl->e_cur[threadIdx.x] = kUnset;
+        ctl->total[threadIdx.x] = 0u;
+        ctl->req_ref[threadIdx.x] = kUnset;
+        ctl->req_need[threadIdx.x] = kUnset;
+    }
+    if (threadIdx.x == 4) { ctl->want = 0; ctl->lut_absmax = 0.f; }
+    if (threadIdx.x < 128)
+        qs[threadIdx.x] = __half2float(q[(s * sh.n_q_heads + hq) * 128 + threadIdx.x]) * scale_log2e;
+    for (int i = threadIdx.x; i < C::kRows * C::kVRowBytes / 16; i += C::kThreads)
+        *reinterpret_cast<uint4*>(smem + C::kVOffset + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+
+    // K table: row j is written rotated by j words (a column would fall into one bank), both copies,
+    // then every row is un-rotated.  Entries are half2 (hi, lo) of LUT * 2^-kexp as in decode_tuned_kernel.
+    float lut_scale = 1.f;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        const float inv = 1.f / lut_scale;
+        float absmax = 0.f;
+        float qreg[kC];
+#pragma unroll
+        for (int i = 0; i < kC; ++i) qreg[i] = qs[g * kC + i] * inv;
+        auto build_unit = [&](const float (&cv)[kJb][kC], int u) {
+#pragma unroll
+            for (int jb = 0; jb < kJb; ++jb) {
+                const int j = (u * kJb + jb) * 32 + lane;
+                float dot = 0.f;
+#pragma unroll
+                for (int i = 0; i < kC; ++i) dot = fmaf(qreg[i], cv[jb][i], dot);
+                absmax = fmaxf(absmax, fabsf(dot));
+                const uint32_t e = pack_hi_lo(dot);
+                uint8_t* row = smem + j * C::kKRowBytes;
+                *reinterpret_cast<uint32_t*>(row + ((g + j) & 31) * 4) = e;
+                *reinterpret_cast<uint32_t*>(row + ((16 + g + j) & 31) * 4) = e;
+            }
+        };
+        if (attempt == 1) load_unit(cva, kcb, 0);
+#pragma unroll 1
+        for (int u = 0; u < kUnits; u += 2) {
+            load_unit(cvb, kcb, u + 1);
+            build_unit(cva, u);
+            if (u + 2 < kUnits) load_unit(cva, kcb, u + 2);
+            build_unit(cvb, u + 1);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) absmax = fmaxf(absmax, __shfl_xor_sync(0xffffffffu, absmax, o));
+        if (lane == 0) atomicMax(reinterpret_cast<int*>(&ctl->lut_absmax), __float_as_int(absmax));
+        __syncthreads();
+        const float amax = ctl->lut_absmax;
+        if (attempt == 1 || amax < 32768.f) break;       // same decision in every thread
+        int ex;
+        frexpf(amax, &ex);
+        lut_scale = exp2f((float)(ex - 15));
+        __syncthreads();
+        if (threadIdx.x == 0) ctl->lut_absmax = 0.f;
+        __syncthreads();
+    }
+#pragma unroll 1
+    for (int i0 = 0; i0 < C::kRows / C::kWarps; i0 += 8) {
+        uint32_t e[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int j = warp + (i0 + k) * C::kWarps;
+            e[k] = *reinterpret_cast<const uint32_t*>(smem + j * C::kKRowBytes + ((lane + j) & 31) * 4);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int j = warp + (i0 + k) * C::kWarps;
+            *reinterpret_cast<uint32_t*>(smem + j * C::kKRowBytes + lane * 4) = e[k];
+        }
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- main loop over the chunk
+    constexpr int kBatch = 4;
+    auto coarsen = [&]() {                       // entered by every thread, right after the event's first barrier
+        const int e = ctl->e_cur[0], cmr = ctl->req_ref[0], need = ctl->req_need[0];
+        const unsigned int tot = ctl->total[0];
+        int e_new = e, shift = 0;
+        unsigned int t_next = tot;
+        if (cmr != kUnset) {
+            if (e == kUnset || cmr - e > kMaxWeightBits) e_new = cmr - kUnitBits;
+            const int room = need + C::kLog2Groups - 31;
+            if (need != kUnset && room > e_new) e_new = room;
+        }
+        if (e != kUnset) {
+            for (int tries = 0; tries < 24; ++tries) {              // 2 bits per try: bounded
+                const int k = e_new - e;
+                if ((k >= 32 ? 0u : tot >> k) < kBinLimit256 / 16u) break;
+                e_new += 2;
+            }
+            shift = e_new - e;
+            t_next = (shift >= 32 ? 0u : tot >> shift) + 1u;
+        }
+        if (shift > 0) {
+            for (int i = threadIdx.x; i < C::kRows * C::kVRowBytes / 4; i += C::kThreads) {
+                uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset) + i;
+                const uint32_t v = *bp;
+                *bp = shift >= 32 ? 0u : (v >> shift) + ((v >> (shift - 1)) & 1u);
+            }
+        }
+        event_barrier(C::kThreads);                         // every thread has read the request and rescaled its bins
+        if (threadIdx.x == 0) {
+            ctl->e_cur[0] = e_new;
+            ctl->total[0] = t_next;
+            ctl->req_ref[0] = kUnset;
+            ctl->req_need[0] = kUnset;
+            ctl->want = 0;
+        }
+        event_barrier(C::kThreads);                         // the new state is visible
+    };
+    load_words(kw, kh, kbase, blk0 + (int64_t)warp * C::kBlocksPerIter + r);
+
+    for (int it = 0; it < n_iters; ++it) {
+        const int64_t blk_warp = blk0 + ((int64_t)it * C::kWarps + warp) * C::kBlocksPerIter;
+        const int64_t blk = blk_warp + r;
+        load_words(vw, vh, vbase, blk);
+
+        // K side: scores of this quad's 16 tokens
+        float sc[16];
+#pragma unroll
+        for (int k0 = 0; k0 < 16; k0 += kBatch) {
+            uint32_t a[kBatch][C::kSlots];
+#pragma unroll
+            for (int kk = 0; kk < kBatch; ++kk)
+#pragma unroll
+                for (int m = 0; m < C::kSlots; ++m)
+                    a[kk][m] = *reinterpret_cast<const volatile uint32_t*>(smem + wide_index(kw[m], kh[m], k0 + kk, lane_off[m], 7));
+#pragma unroll
+            for (int kk = 0; kk < kBatch; kk += 2) {
+                float d[4];
+                mma_rowsum_first(d, a[kk][0], a[kk + 1][0], a[kk][1], a[kk + 1][1]);
+                mma_rowsum_acc(d, a[kk][2], a[kk + 1][2], a[kk][3], a[kk + 1][3]);
+                sc[k0 + kk] = d[0];
+                sc[k0 + kk + 1] = d[2];
+            }
+        }
+        if ((blk_warp + C::kBlocksPerIter) * kTokenBlock > t_end) {
+            const int64_t tok0 = blk * kTokenBlock;
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+                if (tok0 + k >= t_end) sc[k] = -INFINITY;
+        }
+        // reference exponent of the warp, weights of this lane's own four tokens (see decode_tuned_kernel)
+        float mx = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) mx = fmaxf(mx, sc[k]);
+        const float gm = dec_float(__reduce_max_sync(0xffffffffu, enc_float(mx * lut_scale)));
+        const bool any_tokens = gm > -INFINITY;
+        const int ref = any_tokens ? (int)fminf(fmaxf(ceilf(gm), -1.0e9f), 1.0e9f) : kUnset;
+        const float fref = any_tokens ? (float)ref : 0.f;
+        float wown[4], zsum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float s01 = (p & 1) ? sc[4 * j + 1] : sc[4 * j];
+            const float s23 = (p & 1) ? sc[4 * j + 3] : sc[4 * j + 2];
+            const float own = (p & 2) ? s23 : s01;
+            wown[j] = ex2(fmaf(own, lut_scale, -fref));
+            zsum += wown[j];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) zsum += __shfl_xor_sync(0xffffffffu, zsum, o);
+
+        // reserve room for this warp's weights, or ask for a coarser unit (bounded: see decode_tuned_kernel)
+        int eu = kUnset;
+        for (int attempt = 0; attempt < 64; ++attempt) {
+            if (*reinterpret_cast<volatile int*>(&ctl->want) != 0) {
+                if (lane == 0 && ref != kUnset) {
+                    atomicMax(&ctl->req_ref[0], ref);
+                    atomicMax(&ctl->req_need[0], ref + ilogbf(fmaxf(zsum, 1e-30f)) + 1);
+                }
+                event_barrier(C::kThreads);
+                coarsen();
+                continue;
+            }
+            if (!any_tokens) break;
+            bool ok = true;
+            unsigned int mine = 0u;
+            eu = *reinterpret_cast<volatile int*>(&ctl->e_cur[0]);
+            if (eu == kUnset || ref - eu > kMaxWeightBits) {
+                ok = false;
+            } else {
+                const float cw = (zsum * pow2i(ref - eu) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
+                const unsigned int ci = (unsigned int)fminf(cw, 6.7e7f);
+                unsigned int old = 0u;
+                if (lane == 0) old = atomicAdd(&ctl->total[0], ci);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                mine = ci;
+                if (old + ci >= kBinLimit256) ok = false;
+            }
+            if (ok) break;
+            if (lane == 0) {
+                if (mine) atomicSub(&ctl->total[0], mine);
+                atomicMax(&ctl->req_ref[0], ref);
+                atomicMax(&ctl->req_need[0], ref + ilogbf(fmaxf(zsum, 1e-30f)) + 1);
+                atomicExch(&ctl->want, 1);
+            }
+            event_barrier(C::kThreads);
+            coarsen();
+        }
+
+        load_words(kw, kh, kbase, blk + (int64_t)C::kWarps * C::kBlocksPerIter);
+        if (!any_tokens) continue;
+
+        // V side: integer weights, handed round the quad, into the bins of this lane's groups
+        uint32_t wint[4];
+        {
+            const float f = pow2i(ref - eu);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) wint[j] = __float2uint_rn(wown[j] * f);
+        }
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const uint32_t wk = __shfl_sync(0xffffffffu, wint[k >> 2], (lane & ~3) | (k & 3));
+#pragma unroll
+            for (int m = 0; m < C::kSlots; ++m)
+                atomicAdd(reinterpret_cast<unsigned int*>(smem + C::kVOffset + wide_index(vw[m], vh[m], k, lane_off[m] & 63u, 6)), wk);
+        }
+    }
+    load_unit(cva, vcb, 0);                       // the first V centroids travel meanwhile
+    for (int guard = 0; guard < 4096; ++guard) {
+        event_barrier(C::kThreads);
+        if (*reinterpret_cast<volatile int*>(&ctl->want) == 0) break;
+        coarsen();
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- epilogue: bins x V centroids
+    // The bins are 512 rows of 32 words (two code values per row); each is rotated by its index so
+    // that the column read of a warp (its group, 32 consecutive code values) is conflict-free.
+#pragma unroll 1
+    for (int i0 = 0; i0 < C::kRows / 2 / C::kWarps; i0 += 8) {
+        uint32_t v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int rho = warp + (i0 + k) * C::kWarps;
+            v[k] = *reinterpret_cast<const uint32_t*>(smem + C::kVOffset + rho * 128 + lane * 4);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int rho = warp + (i0 + k) * C::kWarps;
+            *reinterpret_cast<uint32_t*>(smem + C::kVOffset + rho * 128 + ((lane + rho) & 31) * 4) = v[k];
+        }
+    }
+    __syncthreads();
+    float acc[kC];
+#pragma unroll
+    for (int i = 0; i < kC; ++i) acc[i] = 0.f;
+    float lsum = 0.f;
+#pragma unroll 1
+    for (int u = 0; u < kUnits; u += 2) {
+        load_unit(cvb, vcb, u + 1);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            if (half == 1 && u + 2 < kUnits) load_unit(cva, vcb, u + 2);
+#pragma unroll
+            for (int jb = 0; jb < kJb; ++jb) {
+                const int j = ((u + half) * kJb + jb) * 32 + lane;
+                const int rho = j >> 1;
+                const uint32_t bi = *reinterpret_cast<const uint32_t*>(smem + C::kVOffset + rho * 128 + ((16 * (j & 1) + g + rho) & 31) * 4);
+                const float bv = (float)bi;
+                lsum += bv;
+#pragma unroll
+                for (int i = 0; i < kC; ++i) acc[i] = fmaf(bv, half == 0 ? cva[jb][i] : cvb[jb][i], acc[i]);
+            }
+        }
+    }
+    {
+        const float v = fold_channels<kC>(acc, lane);
+        const int ch = fold_channel_of<kC>(lane);
+        if ((lane & 3) == 0) part_base[2 + g * kC + ch] = v;
+    }
+    if (g == 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+        if (lane == 0) {
+            part_base[0] = (float)ctl->e_cur[0];      // reference exponent (log2 domain)
+            part_base[1] = lsum;                      // normaliser, in the same unit
+        }
+    }
+}
+
 // Launch plan of one call: context chunk per CTA, partial slots per (sequence, query head), and
 // the first item of the tail (-1: none).
 struct Plan {
@@ -781,14 +1195,10 @@ struct Plan {
 // spread over 2 to 4 CTAs each instead, which shortens the wave by that factor.  This applies
 // where one CTA fills an SM; with two CTAs per SM a CTA whose neighbour has finished already runs
 // faster, and the split was measured to gain nothing.
-template <int G, int R>
-Plan plan_for(const Shape& sh)
+Plan plan_from(const Shape& sh, int64_t round, int min_blocks, int64_t items)
 {
-    using C = Cfg<G, R>;
     Plan pl;
-    const int64_t round = C::kRoundTokens;
-    const int64_t items = sh.n_seq * sh.n_kv_heads;
-    const int64_t slots = 148 * C::kMinBlocks;
+    const int64_t slots = 148 * min_blocks;
     int64_t chunk = (sh.max_tokens + round - 1) / round * round;
     if (chunk > 65536) chunk = 65536;
 #ifdef CQ_TUNE_CHUNK_TOKENS
@@ -803,7 +1213,7 @@ Plan plan_for(const Shape& sh)
     pl.grid = (unsigned)(items * pl.n_parts);
 #ifndef CQ_TUNE_NO_TAIL
     const int64_t rest = items % slots;               // CTAs of the last wave
-    if (C::kMinBlocks == 1 && pl.n_parts == 1 && items > slots && rest > 0 && 2 * rest <= slots && chunk >= 4 * 2048) {
+    if (min_blocks == 1 && pl.n_parts == 1 && items > slots && rest > 0 && 2 * rest <= slots && chunk >= 4 * 2048) {
         int64_t k = slots / rest;
         if (k > 4) k = 4;
         const int64_t part_chunk = ((chunk + k - 1) / k + round - 1) / round * round;
@@ -814,6 +1224,12 @@ Plan plan_for(const Shape& sh)
     }
 #endif
     return pl;
+}
+
+template <int G, int R>
+Plan plan_for(const Shape& sh)
+{
+    return plan_from(sh, Cfg<G, R>::kRoundTokens, Cfg<G, R>::kMinBlocks, sh.n_seq * sh.n_kv_heads);
 }
 
 template <int G, int R>
@@ -830,8 +1246,11 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
     return cudaGetLastError();
 }
 
+bool wide_shape(const Shape& sh) { return sh.head_dim == 128 && sh.c == 8 && sh.b == 10; }
+
 Plan plan_dispatch(const Shape& sh)
 {
+    if (wide_shape(sh)) return plan_from(sh, WideCfg::kRoundTokens, 1, sh.n_seq * sh.n_q_heads);
     if (sh.G == 16 && sh.R == 1) return plan_for<16, 1>(sh);
     if (sh.G == 16 && sh.R == 2) return plan_for<16, 2>(sh);
     if (sh.G == 16 && sh.R == 4) return plan_for<16, 4>(sh);
@@ -844,8 +1263,9 @@ Plan plan_dispatch(const Shape& sh)
 
 bool decode_tuned_supported(const Shape& sh)
 {
-    if (sh.head_dim != 128 || sh.b != 8) return false;
     if (sh.max_tokens > ((int64_t)1 << 30)) return false;
+    if (wide_shape(sh)) return true;
+    if (sh.head_dim != 128 || sh.b != 8) return false;
     return (sh.G == 16 && (sh.R == 1 || sh.R == 2 || sh.R == 4)) || (sh.G == 32 && (sh.R == 1 || sh.R == 2));
 }
 
@@ -858,7 +1278,14 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
     const Plan pl = plan_dispatch(sh);
     if (pl.chunk <= 0) return cudaErrorNotSupported;
     cudaError_t e = cudaErrorNotSupported;
-    if (sh.G == 16 && sh.R == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    if (wide_shape(sh)) {
+        e = cudaFuncSetAttribute(decode_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WideCfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        decode_wide_kernel<<<pl.grid, WideCfg::kThreads, WideCfg::kSmemBytes, st>>>(
+            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, partials);
+        e = cudaGetLastError();
+    }
+    else if (sh.G == 16 && sh.R == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     else if (sh.G == 16 && sh.R == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     else if (sh.G == 16 && sh.R == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     else if (sh.G == 32 && sh.R == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);

@@ -78,28 +78,80 @@ def test_append_into_shared_upper_words():
     assert np.array_equal(rm2, want)
 
 
-@pytest.mark.parametrize("c,b,n_q,n_kv,lens", [
-    (8, 10, 2, 2, [700, 33, 0]),               # CQ-8c10b, MHA
-    (8, 10, 4, 1, [1, 16, 17, 1200]),          # GQA R = 4
-    (8, 9, 2, 1, [300, 257]),
-    (16, 10, 1, 1, [500]),
-])
-def test_attention_wide_codes(c, b, n_q, n_kv, lens):
-    D, n_seq, cap = 128, len(lens), max(lens) + 5
-    rng = np.random.default_rng(40 + b + n_q)
-    G = D // c
+def random_attention_case(seed, c, b, n_q, n_kv, lens, cap, D=128):
+    rng = np.random.default_rng(seed)
+    G, n_seq = D // c, len(lens)
     kcb, vcb = (torch.from_numpy(rng.standard_normal((n_kv, G, 1 << b, c)).astype(np.float32)) for _ in range(2))
     q = torch.from_numpy(rng.standard_normal((n_seq, n_q, D)).astype(np.float16))
     kc_rm = rng.integers(0, 1 << b, size=(n_seq, cap, n_kv, G)).astype(np.int32)
     vc_rm = rng.integers(0, 1 << b, size=(n_seq, cap, n_kv, G)).astype(np.int32)
+    return q, kc_rm, vc_rm, kcb, vcb
+
+
+def attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, scale, c, b, variant):
+    n_seq, cap, n_kv, G = kc_rm.shape
+    D = G * c
     kb = cq.cq_codes_from_rowmajor(to_dev_rowmajor(kc_rm), D, c, b)
     vb = cq.cq_codes_from_rowmajor(to_dev_rowmajor(vc_rm), D, c, b)
     sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
-    out = cq.cq_decode_attn(q.to(DEV), kb, vb, kcb.to(DEV), vcb.to(DEV), sl, D ** -0.5, c, b, cap).cpu().numpy()
-    ref = oracle.decode_dense(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32), D ** -0.5, c, b)
-    H.check_attn(out, ref, f"c={c} b={b} Hq={n_q} Hkv={n_kv}")
-    for s_ in range(n_seq):
-        H.check_attn(out[s_], ref[s_], f"sequence {s_}")
+    out = cq.cq_decode_attn(q.to(DEV), kb, vb, kcb.to(DEV), vcb.to(DEV), sl, scale, c, b, cap, variant=variant)
+    ref = oracle.decode_dense(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32), scale, c, b)
+    return out.cpu().numpy(), ref
+
+
+@pytest.mark.parametrize("c,b,n_q,n_kv,lens", [
+    (8, 10, 2, 2, [700, 33, 0]),               # CQ-8c10b, MHA
+    (8, 10, 4, 1, [1, 16, 17, 1200]),          # GQA R = 4
+    (8, 10, 3, 3, [15, 2049, 128, 2048]),      # block and round edges of the tuned kernel
+    (8, 9, 2, 1, [300, 257]),
+    (16, 10, 1, 1, [500]),
+])
+def test_attention_wide_codes(c, b, n_q, n_kv, lens):
+    D, cap = 128, max(lens) + 5
+    q, kc_rm, vc_rm, kcb, vcb = random_attention_case(40 + b + n_q, c, b, n_q, n_kv, lens, cap)
+    for variant in (1, 0):                      # generic; automatic (the tuned kernel for 8c10b)
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, D ** -0.5, c, b, variant)
+        H.check_attn(out, ref, f"c={c} b={b} Hq={n_q} Hkv={n_kv} variant={variant}")
+        for s_ in range(len(lens)):
+            H.check_attn(out[s_], ref[s_], f"sequence {s_} variant={variant}")
+
+
+def test_attention_8c10b_long_contexts_and_several_chunks():
+    # few items, so the launch plan cuts the contexts into chunks of a few rounds; ragged ends
+    lens = [9000, 4097, 20000]
+    q, kc_rm, vc_rm, kcb, vcb = random_attention_case(5, 8, 10, 2, 1, lens, 20011)
+    out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, 128 ** -0.5, 8, 10, 2)
+    H.check_attn(out, ref, "8c10b long")
+    for s_ in range(3):
+        H.check_attn(out[s_], ref[s_], f"8c10b long, sequence {s_}")
+
+
+def test_attention_8c10b_weight_unit_is_coarsened():
+    # zero query (every weight is the maximum), scores rising along the context, scores falling
+    c, b, cap, n_kv, n_q = 8, 10, 20000, 1, 2
+    q, kc_rm, vc_rm, kcb, vcb = random_attention_case(6, c, b, n_q, n_kv, [cap] * 3, cap)
+    q[0] = 0
+    q[2] = q[1]
+    kc_rm[1] = kc_rm[2]
+    vc_rm[1] = vc_rm[2]
+    khat = oracle.dequant(kc_rm[1].reshape(cap, n_kv, -1), kcb.numpy(), c, b)[:, 0]
+    order = np.argsort(khat @ q[1, 0].double().numpy(), kind="stable")
+    kc_rm[2], vc_rm[2] = kc_rm[1][order[::-1]], vc_rm[1][order[::-1]]
+    kc_rm[1], vc_rm[1] = kc_rm[1][order], vc_rm[1][order]
+    for variant in (1, 2):
+        out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, [cap, cap - 3, cap - 17], 0.7, c, b, variant)
+        H.check_attn(out, ref, f"flat/rising/falling variant={variant}")
+        for s_ in range(3):
+            H.check_attn(out[s_], ref[s_], f"flat/rising/falling sequence {s_} variant={variant}")
+
+
+def test_attention_8c10b_spread_tail():
+    # 152 (sequence, query head) items on 148 SMs: the last four are spread over several CTAs each
+    lens = [int(v) for v in np.random.default_rng(8).integers(1, 8200, size=18)] + [8200]
+    q, kc_rm, vc_rm, kcb, vcb = random_attention_case(9, 8, 10, 8, 2, lens, 8200)
+    out, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, 128 ** -0.5, 8, 10, 2)
+    H.check_attn(out, ref, "8c10b spread tail")
+    H.check_attn(out[-1], ref[-1], "8c10b spread tail, last sequence")
 
 
 def test_encode_then_attention_8c10b_end_to_end():
