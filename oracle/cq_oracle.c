@@ -214,6 +214,87 @@ void oracle_decode_dense(const uint16_t *q, const int32_t *k_codes, const int32_
 }
 
 /*
+ * Decode attention when the cache holds codes of the keys as they were BEFORE the
+ * rotary position embedding (last sentence of Section 3.2: CQ quantises keys before
+ * RoPE; Section 2.1: the key transformation f_K includes the positional encoding).
+ * The key that enters Eq. 1 is then the rotated reconstruction:
+ *   Khat_t = dequant(k_codes[t]);   K_t = rotate(Khat_t, position t)
+ *   s_t = scale * <q, K_t>,  p = softmax(s),  out = sum_t p_t Vhat_t
+ * rotate acts on channel pairs (a, b) with the angle of pair i at position t given by
+ * its cosine and sine, rope_cos[t][i] and rope_sin[t][i] (fp32 [max_tokens][D/2], as
+ * models cache them):
+ *   K_a = Khat_a cos - Khat_b sin,   K_b = Khat_b cos + Khat_a sin
+ * pairing 0: (a, b) = (i, i + D/2)   ("rotate half", the LLaMA / Mistral convention)
+ * pairing 1: (a, b) = (2i, 2i + 1)   (interleaved)
+ * The query is taken as given (already rotated for its own position).  Values are
+ * not rotated.  The paper states neither the pairing nor how the angles are stored:
+ * both are this library's reading.
+ */
+void oracle_decode_dense_rope(const uint16_t *q, const int32_t *k_codes, const int32_t *v_codes,
+                              const float *k_cb, const float *v_cb, const int32_t *seq_lens,
+                              const float *rope_cos, const float *rope_sin, int pairing,
+                              double scale, int n_seq, int n_q_heads, int n_kv_heads, int D,
+                              int c, int b, int64_t max_tokens, double *out)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+    const int R = n_q_heads / n_kv_heads;
+    const int P = D / 2;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int s = 0; s < n_seq; ++s) {
+        for (int hq = 0; hq < n_q_heads; ++hq) {
+            const int hkv = hq / R;
+            const int64_t n = seq_lens[s];
+            double *o = out + ((int64_t)s * n_q_heads + hq) * D;
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+            if (n <= 0) continue;
+            double *qd = (double *)malloc(sizeof(double) * D);
+            double *khat = (double *)malloc(sizeof(double) * D);
+            double *krot = (double *)malloc(sizeof(double) * D);
+            double *score = (double *)malloc(sizeof(double) * n);
+            for (int d = 0; d < D; ++d)
+                qd[d] = half_to_double(q[((int64_t)s * n_q_heads + hq) * D + d]);
+            double smax = -INFINITY;
+            for (int64_t t = 0; t < n; ++t) {
+                const int32_t *kc = k_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                for (int g = 0; g < G; ++g) {
+                    const float *cj = k_cb + (((int64_t)hkv * G + g) * K + kc[g]) * c;
+                    for (int i = 0; i < c; ++i) khat[g * c + i] = (double)cj[i];
+                }
+                for (int i = 0; i < P; ++i) {
+                    const int a = pairing == 0 ? i : 2 * i;
+                    const int bb = pairing == 0 ? i + P : 2 * i + 1;
+                    const double cs = (double)rope_cos[t * P + i], sn = (double)rope_sin[t * P + i];
+                    krot[a] = khat[a] * cs - khat[bb] * sn;
+                    krot[bb] = khat[bb] * cs + khat[a] * sn;
+                }
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d) dot += qd[d] * krot[d];
+                score[t] = scale * dot;
+                if (score[t] > smax) smax = score[t];
+            }
+            double denom = 0.0;
+            for (int64_t t = 0; t < n; ++t) {
+                score[t] = exp(score[t] - smax);
+                denom += score[t];
+            }
+            for (int64_t t = 0; t < n; ++t) {
+                const int32_t *vc = v_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                double p = score[t] / denom;
+                for (int g = 0; g < G; ++g) {
+                    const float *cj = v_cb + (((int64_t)hkv * G + g) * K + vc[g]) * c;
+                    for (int i = 0; i < c; ++i) o[g * c + i] += p * (double)cj[i];
+                }
+            }
+            free(qd);
+            free(khat);
+            free(krot);
+            free(score);
+        }
+    }
+}
+
+/*
  * The same attention in the lookup-table form the CUDA library is asked to
  * use: a per-query table LUT[g][j] = scale * <q_g, Ck[g][j]>, scores as sums
  * of table entries, softmax online over n_chunks contiguous context chunks,

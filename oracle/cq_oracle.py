@@ -42,6 +42,8 @@ def _load():
         L.oracle_dequant.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp]
         L.oracle_decode_dense.argtypes = [vp, vp, vp, vp, vp, vp, f64, i32, i32, i32, i32, i32, i32, i64, vp]
         L.oracle_decode_lut.argtypes = [vp, vp, vp, vp, vp, vp, f64, i32, i32, i32, i32, i32, i32, i64, i32, vp]
+        L.oracle_decode_dense_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f64, i32, i32, i32, i32, i32, i32, i64, vp]
+        L.oracle_decode_dense_rope.restype = None
         L.oracle_kmeanspp_init.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp]
         L.oracle_lloyd_step.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp]
         L.oracle_kmeanspp_init.restype = None
@@ -147,6 +149,20 @@ def decode_dense(q, k_codes, v_codes, k_cb, v_cb, seq_lens, scale: float, c: int
     qb, kc, vc, kcb, vcb, sl, n_seq, hq, hkv, D, mt, out = _attn_args(q, k_codes, v_codes, k_cb, v_cb, seq_lens, c, b)
     _load().oracle_decode_dense(_p(qb), _p(kc), _p(vc), _p(kcb), _p(vcb), _p(sl), float(scale),
                                 n_seq, hq, hkv, D, c, b, mt, _p(out))
+    return out
+
+
+def decode_dense_rope(q, k_codes, v_codes, k_cb, v_cb, seq_lens, rope_cos, rope_sin, scale: float, c: int, b: int,
+                      pairing: int = 0) -> np.ndarray:
+    """Attention over codes of pre-RoPE keys: every reconstructed key is rotated by its position
+    before the dot product.  rope_cos / rope_sin fp32 (max_tokens, D/2); pairing 0 = (i, i + D/2),
+    1 = (2i, 2i + 1).  Returns fp64 (n_seq, Hq, D)."""
+    qb, kc, vc, kcb, vcb, sl, n_seq, hq, hkv, D, mt, out = _attn_args(q, k_codes, v_codes, k_cb, v_cb, seq_lens, c, b)
+    cs = np.ascontiguousarray(rope_cos, dtype=np.float32)
+    sn = np.ascontiguousarray(rope_sin, dtype=np.float32)
+    assert cs.shape == sn.shape == (mt, D // 2) and pairing in (0, 1) and D % 2 == 0
+    _load().oracle_decode_dense_rope(_p(qb), _p(kc), _p(vc), _p(kcb), _p(vcb), _p(sl), _p(cs), _p(sn), int(pairing),
+                                     float(scale), n_seq, hq, hkv, D, c, b, mt, _p(out))
     return out
 
 

@@ -296,6 +296,101 @@ def _as_problem(points):
     return np.asarray(points, dtype=np.float16).reshape(-1, 1, 1)
 
 
+# ----------------------------------------------------------------------------- keys coded before RoPE
+
+def rope_tables(max_tokens, P, base=10000.0, offset=0):
+    """cos / sin of t * base^(-i/P) as models cache them (fp32), positions offset .. offset + max_tokens - 1."""
+    t = np.arange(offset, offset + max_tokens, dtype=np.float64)[:, None]
+    ang = t * base ** (-np.arange(P, dtype=np.float64) / P)[None, :]
+    return np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+
+
+def test_rope_identity_tables_give_the_plain_attention():
+    args = attn_case(2, 4, 2, 32, 8, 8, 29, lens=[29, 6])
+    cs, sn = np.ones((29, 16), np.float32), np.zeros((29, 16), np.float32)
+    for pairing in (0, 1):
+        got = oracle.decode_dense_rope(*args, cs, sn, 0.4, 8, 8, pairing)
+        assert np.array_equal(got, oracle.decode_dense(*args, 0.4, 8, 8))
+
+
+def test_rope_hand_worked_quarter_turns():
+    # D = 2, one pair, c = 1 (two groups of one channel), two code values per group: centroids {1, 3} and {2, 5}.
+    # Token 0 = (1, 2) at angle 0, token 1 = (3, 5) turned by 90 degrees = (-5, 3).  q = (1, 1), scale 1:
+    # scores (3, -2); values are the V centroids (10, 20) and (30, 40).
+    q = np.array([[[1.0, 1.0]]], np.float16)
+    kcb = np.array([[[[1.0], [3.0]], [[2.0], [5.0]]]], np.float32)          # (1 head, 2 groups, 2 codes, c = 1)
+    vcb = np.array([[[[10.0], [30.0]], [[20.0], [40.0]]]], np.float32)
+    codes = np.array([[[[0, 0]], [[1, 1]]]], np.int32)                        # (1 seq, 2 tokens, 1 head, 2 groups)
+    cs = np.array([[1.0], [0.0]], np.float32)
+    sn = np.array([[0.0], [1.0]], np.float32)
+    got = oracle.decode_dense_rope(q, codes, codes, kcb, vcb, [2], cs, sn, 1.0, 1, 1, 0)
+    p0 = 1.0 / (1.0 + np.exp(-5.0))
+    np.testing.assert_allclose(got[0, 0], [10 * p0 + 30 * (1 - p0), 20 * p0 + 40 * (1 - p0)], rtol=1e-14)
+    # with D = 2 both pairings name the same pair
+    assert np.array_equal(got, oracle.decode_dense_rope(q, codes, codes, kcb, vcb, [2], cs, sn, 1.0, 1, 1, 1))
+
+
+@pytest.mark.parametrize("pairing", [0, 1])
+def test_rope_matches_torch_rotation(pairing):
+    D, c, b, n = 32, 4, 6, 41
+    q, kc, vc, kcb, vcb, sl = attn_case(2, 2, 1, D, c, b, n, lens=[41, 17])
+    cs, sn = rope_tables(n, D // 2)
+    got = oracle.decode_dense_rope(q, kc, vc, kcb, vcb, sl, cs, sn, 0.3, c, b, pairing)
+    G = D // c
+    gi = torch.arange(G)
+    for s in range(2):
+        m = int(sl[s])
+        K = torch.from_numpy(kcb[0].astype(np.float64))[gi[None, :], torch.from_numpy(kc[s, :m, 0].astype(np.int64))].reshape(m, D)
+        V = torch.from_numpy(vcb[0].astype(np.float64))[gi[None, :], torch.from_numpy(vc[s, :m, 0].astype(np.int64))].reshape(m, D)
+        C, S = torch.from_numpy(cs[:m].astype(np.float64)), torch.from_numpy(sn[:m].astype(np.float64))
+        if pairing == 0:      # rotate_half: x * [cos, cos] + [-x2, x1] * [sin, sin]
+            Kr = K * torch.cat([C, C], 1) + torch.cat([-K[:, D // 2:], K[:, :D // 2]], 1) * torch.cat([S, S], 1)
+        else:                 # complex multiplication of (x_2i + i x_2i+1) by e^{i angle}
+            z = torch.view_as_complex(K.reshape(m, D // 2, 2).contiguous()) * torch.complex(C, S)
+            Kr = torch.view_as_real(z).reshape(m, D)
+        for hq in range(2):
+            p = torch.softmax(0.3 * (Kr @ torch.from_numpy(q[s, hq].astype(np.float64))), dim=0)
+            np.testing.assert_allclose(got[s, hq], (p[None, :] @ V).numpy()[0], rtol=1e-11, atol=1e-13)
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    # Quarter-turn angles are exact in fp32 (cos, sin in {0, 1, -1}): pair i turns by (i % 4) quarter turns per
+    # position.  Turning the query by the angles of position Delta and shifting every key position by Delta
+    # leaves every score, hence the output, unchanged.
+    D, c, b, n, delta = 16, 4, 5, 23, 5
+    q, kc, vc, kcb, vcb, sl = attn_case(1, 1, 1, D, c, b, n)
+    P = D // 2
+    def tables(offset):
+        k = ((np.arange(offset, offset + n)[:, None]) * (np.arange(P)[None, :] % 4)) % 4
+        return np.array([1, 0, -1, 0], np.float32)[k], np.array([0, 1, 0, -1], np.float32)[k]
+    base = oracle.decode_dense_rope(q, kc, vc, kcb, vcb, sl, *tables(0), 0.5, c, b, 0)
+    # the query turned by delta positions (exact: a signed permutation of its channels)
+    cd, sd = tables(delta)[0][0], tables(delta)[1][0]
+    qf = q.astype(np.float64)[0, 0]
+    qr = np.concatenate([qf[:P] * cd - qf[P:] * sd, qf[P:] * cd + qf[:P] * sd]).astype(np.float16)[None, None]
+    shifted = oracle.decode_dense_rope(qr, kc, vc, kcb, vcb, sl, *tables(delta), 0.5, c, b, 0)
+    np.testing.assert_allclose(shifted, base, rtol=1e-12, atol=1e-14)
+
+
+def test_rope_pairings_differ_by_a_channel_permutation():
+    # interleaved pairs (2i, 2i+1) of permuted inputs = half-split pairs (i, i + D/2) of the original ones
+    D, b, n = 16, 4, 19
+    q, kc, vc, kcb, vcb, sl = attn_case(1, 2, 1, D, 1, b, n)               # c = 1: any channel order is a valid grouping
+    cs, sn = rope_tables(n, D // 2)
+    perm = np.empty(D, np.int64)
+    perm[0::2], perm[1::2] = np.arange(D // 2), np.arange(D // 2) + D // 2  # new channel 2i <- i, 2i+1 <- i + D/2
+    half = oracle.decode_dense_rope(q, kc, vc, kcb, vcb, sl, cs, sn, 0.7, 1, b, 0)
+    inter = oracle.decode_dense_rope(q[..., perm], kc[..., perm], vc, kcb[:, perm], vcb, sl, cs, sn, 0.7, 1, b, 1)
+    np.testing.assert_allclose(inter, half, rtol=1e-12, atol=1e-14)
+
+
+def test_rope_single_token_returns_its_value():
+    q, kc, vc, kcb, vcb, _ = attn_case(1, 1, 1, 16, 4, 4, 9)
+    cs, sn = rope_tables(9, 8)
+    got = oracle.decode_dense_rope(q, kc, vc, kcb, vcb, [1], cs, sn, 1.0, 4, 4, 0)
+    np.testing.assert_allclose(got[0, 0], oracle.dequant(vc[0, :1], vcb, 4, 4)[0, 0], rtol=1e-15)
+
+
 def test_lloyd_step_hand_worked_cases():
     n_cases = 0
     for (kind, name), cols in _golden_kmeans():
