@@ -373,6 +373,31 @@ def extra_decode(cq, dev, w, reps=20):
             "query_heads_per_s": w.n_seq * w.n_q_heads / (ms * 1e-3), "gbs": gbs, "frac_of_measured_hbm": gbs / hbm}
 
 
+def extra_decode_rope(cq, dev, w, reps=5):
+    """Attention over codes of pre-RoPE keys (generic kernel) on the shape of a decode workload."""
+    st = DecodeState(w, 0, dev, cq)
+    P = w.head_dim // 2
+    ang = torch.arange(st.cap, dtype=torch.float64, device=dev)[:, None] * \
+        (10000.0 ** (-torch.arange(P, dtype=torch.float64, device=dev) / P))[None, :]
+    cs, sn = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    run = lambda: cq.cq_decode_attn_rope(st.q, st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.seq_lens, cs, sn, st.scale,
+                                         w.c, w.b, st.cap, out=st.out, workspace=st.ws)
+    for _ in range(2):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    hbm, _ = measured_peaks()
+    gbs = (st.algorithmic_bytes() + 2 * cs.numel() * 4) / (ms * 1e-3) / 1e9
+    return {"workload": w.name + " with pre-RoPE key codes", "decode_ms": ms, "kv_tokens_per_s": st.kv_tokens() / (ms * 1e-3),
+            "gbs": gbs, "frac_of_measured_hbm": gbs / hbm}
+
+
 # --------------------------------------------------------------------------------- main
 
 def main():
@@ -513,6 +538,7 @@ def main():
                 extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
                 extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
                 extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
+                extras["decode_rope_cfg1"] = extra_decode_rope(cq, dev, synth.WORKLOADS[1])
             if args.extras == "all":
                 extras["learn"] = extra_learn(cq, dev)
         except Exception as e:      # extras never hide the headline number

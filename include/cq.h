@@ -190,6 +190,32 @@ int cq_decode_attn_static(const void *q_fp16, const void *k_codes, const void *v
                           int64_t max_tokens, float *out, void *stream);
 
 /*
+ * Decode attention over a cache whose KEY codes were taken before the rotary position
+ * embedding (last sentence of Section 3.2: CQ quantises keys before RoPE; Section 2.1:
+ * the key transformation includes the positional encoding).  The key that enters Eq. 1
+ * is the reconstructed key of token t rotated by the angles of position t:
+ *   K_a = k_a cos - k_b sin,  K_b = k_b cos + k_a sin    for every channel pair (a, b),
+ * with pair i's cosine and sine at position t read from rope_cos[t][i], rope_sin[t][i]
+ * (fp32 [max_tokens][head_dim / 2], the tables a model caches; position = token index in
+ * the cache).  pairing CQ_ROPE_HALF: (a, b) = (i, i + head_dim/2), the LLaMA / Mistral
+ * convention; CQ_ROPE_INTERLEAVED: (2i, 2i + 1).  The paper fixes neither; both are
+ * readings of this library.  q is used as given (already rotated for its own position);
+ * values are not rotated.  Every other argument, the workspace size
+ * (cq_decode_attn_workspace_bytes) and the output are those of cq_decode_attn.
+ * CQ_ERR_UNSUPPORTED when a pair would not lie in whole groups (odd number of groups for
+ * CQ_ROPE_HALF, odd c for CQ_ROPE_INTERLEAVED).  Runs on a generic sm_100a kernel: the
+ * score of a token is no longer a sum of per-code table entries.
+ */
+#define CQ_ROPE_HALF 0
+#define CQ_ROPE_INTERLEAVED 1
+int cq_decode_attn_rope(const void *q_fp16, const void *k_codes, const void *v_codes,
+                        const float *k_cb, const float *v_cb, const int32_t *seq_lens,
+                        const float *rope_cos, const float *rope_sin, int pairing, float scale,
+                        int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                        int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
+                        void *stream);
+
+/*
  * Same operation with an explicit kernel choice, for tests and benchmarks:
  * variant 0 = automatic (what cq_decode_attn uses), 1 = generic kernel,
  * 2 = tuned kernel (CQ_ERR_UNSUPPORTED when the shape has none).

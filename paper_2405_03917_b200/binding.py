@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 # Every symbol include/cq.h declares.
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
-           "cq_decode_attn_variant", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
+           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
            "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
 
 
@@ -63,6 +63,9 @@ def lib() -> ctypes.CDLL:
         L.cq_decode_attn_variant.restype = i32
         L.cq_decode_attn_variant.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp,
                                              sz, i32, vp]
+        L.cq_decode_attn_rope.restype = i32
+        L.cq_decode_attn_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, i32, i32, i32, i32, i32, i64,
+                                          vp, vp, sz, vp]
         L.cq_decode_attn_static.restype = i32
         L.cq_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp]
         L.cq_learn_workspace_bytes.restype = sz
@@ -199,6 +202,38 @@ def cq_decode_attn(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor
 
 
 STATIC_WORKSPACE_BYTES = 4 << 20      # CQ_STATIC_WORKSPACE_BYTES of include/cq.h
+
+
+ROPE_HALF, ROPE_INTERLEAVED = 0, 1
+
+
+def cq_decode_attn_rope(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor,
+                        v_cb: torch.Tensor, seq_lens: torch.Tensor, rope_cos: torch.Tensor, rope_sin: torch.Tensor,
+                        scale: float, c: int, b: int, max_tokens: int, pairing: int = ROPE_HALF,
+                        out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """cq_decode_attn for key codes taken before RoPE: rope_cos / rope_sin fp32 (max_tokens, head_dim / 2)."""
+    n_seq, n_q_heads, head_dim = q.shape
+    n_kv_heads = k_cb.shape[0]
+    for nm, t in (("rope_cos", rope_cos), ("rope_sin", rope_sin)):
+        if tuple(t.shape) != (max_tokens, head_dim // 2):
+            raise ValueError(f"{nm} shape {tuple(t.shape)}, expected {(max_tokens, head_dim // 2)}")
+    need_codes = cq_codes_bytes(n_seq, max_tokens, n_kv_heads, head_dim, c, b)
+    if need_codes and (k_codes.numel() < need_codes or v_codes.numel() < need_codes):
+        raise ValueError(f"code buffers must hold {need_codes} bytes")
+    if out is None:
+        out = torch.empty(n_seq, n_q_heads, head_dim, dtype=torch.float32, device=q.device)
+    if workspace is None:
+        nbytes = cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens)
+        workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    st = lib().cq_decode_attn_rope(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+                                   _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
+                                   _dev(v_cb, torch.float32, "v_cb"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                   _dev(rope_cos, torch.float32, "rope_cos"), _dev(rope_sin, torch.float32, "rope_sin"),
+                                   int(pairing), float(scale), n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
+                                   _dev(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
+                                   workspace.numel(), _stream())
+    _check(st, "cq_decode_attn_rope")
+    return out
 
 
 def cq_decode_attn_static(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor,

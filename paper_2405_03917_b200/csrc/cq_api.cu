@@ -198,6 +198,33 @@ int cq_decode_attn(const void* q_fp16, const void* k_codes, const void* v_codes,
                                   head_dim, c, b, max_tokens, out, workspace, workspace_bytes, 0, stream);
 }
 
+int cq_decode_attn_rope(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
+                        const float* v_cb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
+                        int pairing, float scale, int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                        int64_t max_tokens, float* out, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!q_fp16 || !k_codes || !v_codes || !k_cb || !v_cb || !seq_lens || !rope_cos || !rope_sin || !out || !workspace)
+        return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (pairing != CQ_ROPE_HALF && pairing != CQ_ROPE_INTERLEAVED) return CQ_ERR_SHAPE;
+    if (head_dim % 2 != 0) return CQ_ERR_SHAPE;
+    // a pair must lie in whole groups: (i, i + D/2) needs an even number of groups, (2i, 2i+1) an even c
+    if (pairing == CQ_ROPE_HALF ? sh.G % 2 != 0 : c % 2 != 0) return CQ_ERR_UNSUPPORTED;
+    if (!aligned16(k_codes) || !aligned16(v_codes) || !aligned16(workspace) || !aligned16(k_cb) || !aligned16(v_cb) ||
+        (reinterpret_cast<uintptr_t>(q_fp16) & 1u) || (reinterpret_cast<uintptr_t>(out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(rope_cos) & 3u) || (reinterpret_cast<uintptr_t>(rope_sin) & 3u))
+        return CQ_ERR_ALIGN;
+    if (workspace_bytes < round_up(partial_bytes(sh), 256)) return CQ_ERR_WORKSPACE;
+    if ((int64_t)sh.G * sh.K > 2 * kGenericMaxTableEntries) return CQ_ERR_UNSUPPORTED;     // one table (the bins) only
+    cudaError_t e = launch_decode_rope(static_cast<const __half*>(q_fp16), static_cast<const uint8_t*>(k_codes),
+                                       static_cast<const uint8_t*>(v_codes), k_cb, v_cb, seq_lens, rope_cos, rope_sin,
+                                       pairing, scale, sh, out, static_cast<float*>(workspace),
+                                       static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
 // ---------------------------------------------------------------------------------------------
 // cq_decode_attn_static: the split-K partials live in this array instead of a caller workspace.
 // In host code the name `g_static_workspace` is only a handle for the runtime, not a device

@@ -82,6 +82,10 @@ int decode_generic_splits(const Shape& sh);
 cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                   const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
                                   float* out, float* partials, cudaStream_t st);
+// Attention over codes of pre-RoPE keys (generic kernel; uses decode_generic_splits partial slots).
+cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
+                               const float* vcb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
+                               int pairing, float scale, const Shape& sh, float* out, float* partials, cudaStream_t st);
 bool decode_tuned_supported(const Shape& sh);
 int decode_tuned_parts(const Shape& sh);      // partial slots per (sequence, query head)
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,

@@ -364,6 +364,121 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Decode attention over codes of keys that were quantised BEFORE the rotary position embedding
+// (last sentence of Section 3.2).  The key of Eq. 1 is the reconstruction rotated by its position,
+// so the score is no longer a sum of per-(group, code) table entries: for the channel pair (a, b)
+// with cosine cs and sine sn at the token's position,
+//   q_a K_a + q_b K_b = cs (q_a k_a + q_b k_b) + sn (q_b k_a - q_a k_b),   k = reconstructed key.
+// One thread per token gathers the token's centroids and forms that sum over the D/2 pairs; the
+// V side, the online softmax and the partials are those of decode_generic_kernel.
+// pairing 0: (a, b) = (i, i + D/2); pairing 1: (a, b) = (2i, 2i + 1).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kGenericThreads)
+decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
+                   const float* __restrict__ kcb, const float* __restrict__ vcb,
+                   const int32_t* __restrict__ seq_lens, const float* __restrict__ rope_cos,
+                   const float* __restrict__ rope_sin, int pairing, float scale_log2e, Shape sh, int n_splits,
+                   float* __restrict__ partials)
+{
+    extern __shared__ __align__(16) float smem_f[];
+    float* bins = smem_f;                      // [G][K]
+    float* qsm = bins + sh.G * sh.K;           // [D]
+    __shared__ float red[kGenericThreads / 32];
+
+    const int split = blockIdx.x % n_splits;
+    const int hq = (blockIdx.x / n_splits) % sh.n_q_heads;
+    const int64_t s = blockIdx.x / (n_splits * sh.n_q_heads);
+    const int hkv = hq / sh.R;
+    const int GK = sh.G * sh.K;
+    const int P = sh.head_dim / 2;
+
+    int64_t n = seq_lens[s];
+    n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
+    const int64_t nblk = (n + kTokenBlock - 1) / kTokenBlock;
+    const int64_t t_begin = nblk * split / n_splits * kTokenBlock;
+    int64_t t_end = nblk * (split + 1) / n_splits * kTokenBlock;
+    if (t_end > n) t_end = n;
+
+    float* part = partials + ((s * sh.n_q_heads + hq) * n_splits + split) * (int64_t)partial_stride(sh.head_dim);
+    if (t_end <= t_begin) {          // empty split: neutral element of the merge
+        if (threadIdx.x == 0) { part[0] = -INFINITY; part[1] = 0.f; }
+        for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) part[2 + d] = 0.f;
+        return;
+    }
+
+    const __half* qv = q + (s * sh.n_q_heads + hq) * (int64_t)sh.head_dim;
+    for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) qsm[d] = __half2float(qv[d]);
+    for (int e = threadIdx.x; e < GK; e += blockDim.x) bins[e] = 0.f;
+    __syncthreads();
+
+    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
+    const float* kcb_h = kcb + (int64_t)hkv * GK * sh.c;
+    float m_run = -INFINITY;
+    float l_thr = 0.f;
+    for (int64_t t0 = t_begin; t0 < t_end; t0 += blockDim.x) {
+        const int64_t t = t0 + threadIdx.x;
+        const bool valid = t < t_end;
+        const int64_t block0 = (t / kTokenBlock) * sh.block_bytes;
+        const int k16 = (int)(t % kTokenBlock);
+        float sc = -INFINITY;
+        if (valid) {
+            const float* cs = rope_cos + t * P;
+            const float* sn = rope_sin + t * P;
+            float acc = 0.f;
+            if (pairing == 0) {
+                const int half_groups = sh.G / 2;
+                for (int g = 0; g < half_groups; ++g) {
+                    const float* ca = kcb_h + ((int64_t)g * sh.K + read_code(kbase + block0, sh, g, k16)) * sh.c;
+                    const float* cb2 = kcb_h + ((int64_t)(g + half_groups) * sh.K +
+                                                read_code(kbase + block0, sh, g + half_groups, k16)) * sh.c;
+                    for (int k = 0; k < sh.c; ++k) {
+                        const int i = g * sh.c + k;
+                        const float ka = ca[k], kb = cb2[k], qa = qsm[i], qb = qsm[i + P];
+                        acc = fmaf(cs[i], fmaf(qa, ka, qb * kb), acc);
+                        acc = fmaf(sn[i], fmaf(qb, ka, -qa * kb), acc);
+                    }
+                }
+            } else {
+                for (int g = 0; g < sh.G; ++g) {
+                    const float* cg = kcb_h + ((int64_t)g * sh.K + read_code(kbase + block0, sh, g, k16)) * sh.c;
+                    for (int k = 0; k < sh.c; k += 2) {
+                        const int a = g * sh.c + k, i = a >> 1;
+                        const float ka = cg[k], kb = cg[k + 1], qa = qsm[a], qb = qsm[a + 1];
+                        acc = fmaf(cs[i], fmaf(qa, ka, qb * kb), acc);
+                        acc = fmaf(sn[i], fmaf(qb, ka, -qa * kb), acc);
+                    }
+                }
+            }
+            sc = acc * scale_log2e;
+        }
+        const float m_tile = block_reduce_max(sc, red);
+        if (m_tile > m_run) {
+            const float f = exp2f(m_run - m_tile);      // 0 when m_run is -inf
+            for (int e = threadIdx.x; e < GK; e += blockDim.x) bins[e] *= f;
+            l_thr *= f;
+            m_run = m_tile;
+            __syncthreads();
+        }
+        if (valid) {
+            const float p = exp2f(sc - m_run);
+            l_thr += p;
+            for (int g = 0; g < sh.G; ++g) atomicAdd(&bins[g * sh.K + read_code(vbase + block0, sh, g, k16)], p);
+        }
+        __syncthreads();
+    }
+    const float l = block_reduce_sum(l_thr, red);
+    if (threadIdx.x == 0) { part[0] = m_run; part[1] = l; }
+    for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) {
+        const int g = d / sh.c, k = d % sh.c;
+        const float* cv = vcb + ((int64_t)hkv * GK + g * sh.K) * sh.c + k;
+        float a = 0.f;
+        for (int j = 0; j < sh.K; ++j) a = fmaf(bins[g * sh.K + j], cv[j * sh.c], a);
+        part[2 + d] = a;
+    }
+}
+
 int decode_generic_splits(const Shape& sh)
 {
     // enough CTAs for a few waves of 148 SMs, at least 256 tokens per split
@@ -423,6 +538,22 @@ cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint
     const unsigned grid = (unsigned)(n_splits * sh.n_q_heads * sh.n_seq);
     decode_generic_kernel<<<grid, kGenericThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
                                                                n_splits, partials);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_merge(partials, n_splits, sh, out, st);
+}
+
+cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
+                               const float* vcb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
+                               int pairing, float scale, const Shape& sh, float* out, float* partials, cudaStream_t st)
+{
+    const int n_splits = decode_generic_splits(sh);
+    const size_t smem = ((size_t)sh.G * sh.K + sh.head_dim) * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)(n_splits * sh.n_q_heads * sh.n_seq);
+    decode_rope_kernel<<<grid, kGenericThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, rope_cos, rope_sin, pairing,
+                                                            scale * kLog2e, sh, n_splits, partials);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return launch_merge(partials, n_splits, sh, out, st);
