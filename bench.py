@@ -195,10 +195,9 @@ class DecodeState:
     def step(self, cq, ev=None):
         """Append-encode the new token (K, V) at the last position, then attend."""
         w = self.w
-        cq.cq_encode(self.k_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim), self.k_cb, w.c, w.b, self.k_codes,
-                     self.cap, seq_offsets=self.append_pos)
-        cq.cq_encode(self.v_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim), self.v_cb, w.c, w.b, self.v_codes,
-                     self.cap, seq_offsets=self.append_pos)
+        cq.cq_encode_kv(self.k_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim),
+                        self.v_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim), self.k_cb, self.v_cb, w.c, w.b,
+                        self.k_codes, self.v_codes, self.cap, seq_offsets=self.append_pos)
         if ev is not None:
             ev[0].record()
         cq.cq_decode_attn(self.q, self.k_codes, self.v_codes, self.k_cb, self.v_cb, self.seq_lens, self.scale,
@@ -526,7 +525,7 @@ def main():
             "clocks": clocks,
             "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": args.steps * 4 * len(states),
+            "gpu_launches": args.steps * 3 * len(states),      # per layer: append-encode (K and V), attention, merge
             "roofline": roofline, "shared_memory": shared}
 
     if args.extras != "none" and world == 1:

@@ -112,7 +112,18 @@ int cq_encode(const void *x_fp16, const float *codebooks, const int32_t *seq_off
               int n_heads, int head_dim, int c, int b, void *codes_out, void *stream);
 
 /*
- * Layout converters.  rowmajor is uint8 [n_seq][max_tokens][n_heads][G].
+ * cq_encode for the key and the value embeddings of the same tokens (Section 3.2 quantises
+ * both, each with its own codebooks): the result is that of two cq_encode calls, in one
+ * launch where the shape has a tuned encode kernel.  k_fp16 / v_fp16, k_cb / v_cb and the two
+ * code buffers are laid out as in cq_encode; the two code buffers must differ.
+ */
+int cq_encode_kv(const void *k_fp16, const void *v_fp16, const float *k_cb, const float *v_cb,
+                 const int32_t *seq_offsets, int64_t n_seq, int64_t n_tokens, int64_t token_offset,
+                 int64_t max_tokens, int n_heads, int head_dim, int c, int b,
+                 void *k_codes_out, void *v_codes_out, void *stream);
+
+/*
+ * Layout converters.  rowmajor is uint8 [n_seq][max_tokens][n_heads][G] (uint16 for b > 8).
  * to_rowmajor reads every position < max_tokens of the library layout;
  * from_rowmajor writes every position < max_tokens (block padding is zeroed).
  */

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libcq.so")
 
 # Every symbol include/cq.h declares.
-EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant",
+EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant", "cq_encode_kv",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
            "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
            "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.cq_decode_attn_variant.restype = i32
         L.cq_decode_attn_variant.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp,
                                              sz, i32, vp]
+        L.cq_encode_kv.restype = i32
+        L.cq_encode_kv.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp]
         L.cq_decode_attn_rope.restype = i32
         L.cq_decode_attn_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, i32, i32, i32, i32, i32, i64,
                                           vp, vp, sz, vp]
@@ -140,6 +142,21 @@ def cq_encode(x: torch.Tensor, codebooks: torch.Tensor, c: int, b: int, codes_ou
                                  _dev(codes_out, torch.uint8, "codes_out"), variant, _stream())
     _check(st, "cq_encode")
     return codes_out
+
+
+def cq_encode_kv(k: torch.Tensor, v: torch.Tensor, k_cb: torch.Tensor, v_cb: torch.Tensor, c: int, b: int,
+                 k_codes_out: torch.Tensor, v_codes_out: torch.Tensor, max_tokens: int, token_offset: int = 0,
+                 seq_offsets: Optional[torch.Tensor] = None) -> None:
+    """cq_encode of the key and the value embeddings of the same tokens; k, v fp16 (n_seq, n_tokens, n_heads, head_dim)."""
+    n_seq, n_tokens, n_heads, head_dim = k.shape
+    if tuple(v.shape) != tuple(k.shape):
+        raise ValueError("k and v must have the same shape")
+    so = None if seq_offsets is None else _dev(seq_offsets, torch.int32, "seq_offsets")
+    st = lib().cq_encode_kv(_dev(k, torch.float16, "k"), _dev(v, torch.float16, "v"), _dev(k_cb, torch.float32, "k_cb"),
+                            _dev(v_cb, torch.float32, "v_cb"), so, n_seq, n_tokens, token_offset, max_tokens, n_heads,
+                            head_dim, c, b, _dev(k_codes_out, torch.uint8, "k_codes_out"),
+                            _dev(v_codes_out, torch.uint8, "v_codes_out"), _stream())
+    _check(st, "cq_encode_kv")
 
 
 def cq_codes_to_rowmajor(codes: torch.Tensor, n_seq: int, max_tokens: int, n_heads: int, head_dim: int, c: int,

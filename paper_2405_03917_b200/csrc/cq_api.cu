@@ -128,6 +128,34 @@ int cq_encode(const void* x_fp16, const float* codebooks, const int32_t* seq_off
                              head_dim, c, b, codes_out, 0, stream);
 }
 
+int cq_encode_kv(const void* k_fp16, const void* v_fp16, const float* k_cb, const float* v_cb,
+                 const int32_t* seq_offsets, int64_t n_seq, int64_t n_tokens, int64_t token_offset, int64_t max_tokens,
+                 int n_heads, int head_dim, int c, int b, void* k_codes_out, void* v_codes_out, void* stream)
+{
+    if (!k_fp16 || !v_fp16 || !k_cb || !v_cb || !k_codes_out || !v_codes_out) return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_heads, n_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (n_tokens < 0 || token_offset < 0) return CQ_ERR_SHAPE;
+    if (!seq_offsets && token_offset + n_tokens > max_tokens) return CQ_ERR_SHAPE;
+    if (!aligned16(k_fp16) || !aligned16(v_fp16) || !aligned16(k_cb) || !aligned16(v_cb) || !aligned16(k_codes_out) ||
+        !aligned16(v_codes_out))
+        return CQ_ERR_ALIGN;
+    if (k_codes_out == v_codes_out) return CQ_ERR_SHAPE;
+    if (n_tokens == 0) return CQ_OK;
+    if (encode_tuned_supported(sh)) {       // one launch for both tensors
+        cudaError_t e = launch_encode_tuned(static_cast<const __half*>(k_fp16), k_cb, seq_offsets, sh, n_tokens, token_offset,
+                                            static_cast<uint8_t*>(k_codes_out), static_cast<cudaStream_t>(stream),
+                                            static_cast<const __half*>(v_fp16), v_cb, static_cast<uint8_t*>(v_codes_out));
+        return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    }
+    st = cq_encode(k_fp16, k_cb, seq_offsets, n_seq, n_tokens, token_offset, max_tokens, n_heads, head_dim, c, b,
+                   k_codes_out, stream);
+    if (st != CQ_OK) return st;
+    return cq_encode(v_fp16, v_cb, seq_offsets, n_seq, n_tokens, token_offset, max_tokens, n_heads, head_dim, c, b,
+                     v_codes_out, stream);
+}
+
 int cq_codes_to_rowmajor(const void* codes, int64_t n_seq, int64_t max_tokens, int n_heads, int head_dim, int c,
                          int b, void* rowmajor_out, void* stream)
 {
@@ -397,9 +425,8 @@ int cq_decode_step_host(const void* q_host, const void* k_new_host, const void* 
     if (cudaMemcpyAsync(d_k, k_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
     if (cudaMemcpyAsync(d_v, v_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
     if (cudaMemcpyAsync(d_sl, seq_lens_host, slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
-    int st = cq_encode(d_k, k_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, k_codes, stream);
-    if (st != CQ_OK) return st;
-    st = cq_encode(d_v, v_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, v_codes, stream);
+    int st = cq_encode_kv(d_k, d_v, k_cb, v_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, k_codes, v_codes,
+                          stream);
     if (st != CQ_OK) return st;
     if (launch_add_one(d_sl, d_sl1, n_seq, cs) != cudaSuccess) return CQ_ERR_CUDA;
     st = cq_decode_attn(d_q, k_codes, v_codes, k_cb, v_cb, d_sl1, scale, n_seq, n_q_heads, n_kv_heads, head_dim, c, b,

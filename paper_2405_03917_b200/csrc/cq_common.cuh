@@ -71,8 +71,10 @@ bool encode_small_supported(const Shape& sh);       // few-vector kernel: the gr
 cudaError_t launch_encode_small(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                 int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
 bool encode_tuned_supported(const Shape& sh);
+// (x2, cb2, codes2): an optional second tensor of the same shape, encoded by the same launch.
 cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
-                                int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
+                                int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st,
+                                const __half* x2 = nullptr, const float* cb2 = nullptr, uint8_t* codes2 = nullptr);
 
 cudaError_t launch_to_rowmajor(const uint8_t* codes, const Shape& sh, uint8_t* rowmajor, cudaStream_t st);
 cudaError_t launch_from_rowmajor(const uint8_t* rowmajor, const Shape& sh, uint8_t* codes, cudaStream_t st);

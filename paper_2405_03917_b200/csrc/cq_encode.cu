@@ -214,11 +214,17 @@ __device__ __forceinline__ int exact_code(const float (&xg)[kC], const float* __
 }
 
 // kMT: 16-vector m-tiles per warp (4 for bulk encode, 1 when there are few vectors).
+// A launch covers one tensor, or two of the same shape (the key and the value of an append):
+// blockIdx.y picks (x, cb, codes) or (x2, cb2, codes2).
 template <int kC, int kMT>
 __global__ void __launch_bounds__(kEncThreads, 2)
-encode_tuned_kernel(const __half* __restrict__ x, const float* __restrict__ cb, const int32_t* __restrict__ seq_offsets,
-                    Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes, int groups_per_cta)
+encode_tuned_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, const int32_t* __restrict__ seq_offsets,
+                    Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes1, int groups_per_cta,
+                    const __half* __restrict__ x2, const float* __restrict__ cb2, uint8_t* __restrict__ codes2)
 {
+    const __half* x = blockIdx.y ? x2 : x1;
+    const float* cb = blockIdx.y ? cb2 : cb1;
+    uint8_t* codes = blockIdx.y ? codes2 : codes1;
     using C = EncCfg<kC>;
     constexpr int G = C::G;
     constexpr int kTileVecs = kEncWarps * kMT * 16;
@@ -428,7 +434,8 @@ encode_tuned_kernel(const __half* __restrict__ x, const float* __restrict__ cb, 
 
 template <int kC, int kMT>
 cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh, int64_t n_tokens,
-                       int64_t token_offset, uint8_t* codes, cudaStream_t st)
+                       int64_t token_offset, uint8_t* codes, cudaStream_t st, const __half* x2 = nullptr,
+                       const float* cb2 = nullptr, uint8_t* codes2 = nullptr)
 {
     using C = EncCfg<kC>;
     constexpr int kTileVecs = kEncWarps * kMT * 16;
@@ -445,8 +452,8 @@ cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offs
     const size_t smem = (size_t)2 * C::kBufWords * 4 + sizeof(EncCtl);
     cudaError_t e = cudaFuncSetAttribute(encode_tuned_kernel<kC, kMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    encode_tuned_kernel<kC, kMT><<<(unsigned)grid, kEncThreads, smem, st>>>(x, cb, seq_offsets, sh, n_tokens, token_offset,
-                                                                          codes, groups_per_cta);
+    encode_tuned_kernel<kC, kMT><<<dim3((unsigned)grid, x2 ? 2u : 1u), kEncThreads, smem, st>>>(
+        x, cb, seq_offsets, sh, n_tokens, token_offset, codes, groups_per_cta, x2, cb2, codes2);
     return cudaGetLastError();
 }
 
@@ -458,18 +465,19 @@ bool encode_tuned_supported(const Shape& sh)
 }
 
 cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
-                                int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st)
+                                int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st,
+                                const __half* x2, const float* cb2, uint8_t* codes2)
 {
     const int64_t n_vec = sh.n_seq * n_tokens;
     if (n_vec == 0) return cudaSuccess;
     const bool few = n_vec * sh.n_kv_heads < (int64_t)148 * 512 * 2;    // not enough vectors for 64 per warp
     switch (sh.c) {
-        case 2: return few ? launch_enc<2, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st)
-                           : launch_enc<2, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st);
-        case 4: return few ? launch_enc<4, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st)
-                           : launch_enc<4, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st);
-        case 8: return few ? launch_enc<8, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st)
-                           : launch_enc<8, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st);
+        case 2: return few ? launch_enc<2, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
+                           : launch_enc<2, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
+        case 4: return few ? launch_enc<4, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
+                           : launch_enc<4, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
+        case 8: return few ? launch_enc<8, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
+                           : launch_enc<8, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
         default: return cudaErrorNotSupported;
     }
 }

@@ -97,6 +97,23 @@ def test_append_positions_and_untouched_bytes():
     assert np.array_equal(rm3, want3)
 
 
+@pytest.mark.parametrize("c,b,head_dim", [(8, 8, 128), (2, 8, 128), (4, 5, 64), (8, 10, 128)])
+def test_encode_kv_equals_two_encodes(c, b, head_dim):
+    nh, cap = 2, 50
+    xk, xv, kcb, vcb, _ = H.generic_case(70 + c + b, 3, cap, nh, nh, head_dim, c, b)
+    nbytes = cq.cq_codes_bytes(3, cap, nh, head_dim, c, b)
+    want_k, want_v, got_k, got_v = (torch.zeros(nbytes, dtype=torch.uint8, device=DEV) for _ in range(4))
+    offs = torch.tensor([3, 49, 0], dtype=torch.int32, device=DEV)
+    for x, cb, buf in ((xk, kcb, want_k), (xv, vcb, want_v)):
+        cq.cq_encode(x[:, :30].contiguous().to(DEV), cb.to(DEV), c, b, buf, cap)                      # prefill
+        cq.cq_encode(x[:, 30:31].contiguous().to(DEV), cb.to(DEV), c, b, buf, cap, seq_offsets=offs)  # append
+    cq.cq_encode_kv(xk[:, :30].contiguous().to(DEV), xv[:, :30].contiguous().to(DEV), kcb.to(DEV), vcb.to(DEV), c, b,
+                    got_k, got_v, cap)
+    cq.cq_encode_kv(xk[:, 30:31].contiguous().to(DEV), xv[:, 30:31].contiguous().to(DEV), kcb.to(DEV), vcb.to(DEV), c, b,
+                    got_k, got_v, cap, seq_offsets=offs)
+    assert torch.equal(got_k, want_k) and torch.equal(got_v, want_v)
+
+
 def test_layout_roundtrip_matches_documented_offsets():
     n_seq, cap, nh, D, c, b = 2, 37, 3, 64, 4, 8
     G = D // c
