@@ -355,12 +355,14 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
     }
     const float l = block_reduce_sum(l_thr, red);
     if (threadIdx.x == 0) { part[0] = m_run; part[1] = l; }
-    for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) {
+    // bins x V centroids: a warp per output channel, its lanes share the code values
+    for (int d = threadIdx.x >> 5; d < sh.head_dim; d += blockDim.x >> 5) {
         const int g = d / sh.c, k = d % sh.c;
         const float* cv = vcb + ((int64_t)hkv * GK + g * sh.K) * sh.c + k;
         float a = 0.f;
-        for (int j = 0; j < sh.K; ++j) a = fmaf(bins[g * sh.K + j], cv[j * sh.c], a);
-        part[2 + d] = a;
+        for (int j = threadIdx.x & 31; j < sh.K; j += 32) a = fmaf(bins[g * sh.K + j], cv[j * sh.c], a);
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if ((threadIdx.x & 31) == 0) part[2 + d] = a;
     }
 }
 
@@ -374,17 +376,20 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
 // V side, the online softmax and the partials are those of decode_generic_kernel.
 // pairing 0: (a, b) = (i, i + D/2); pairing 1: (a, b) = (2i, 2i + 1).
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kGenericThreads)
+constexpr int kRopeThreads = 512;
+
+__global__ void __launch_bounds__(kRopeThreads)
 decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                    const float* __restrict__ kcb, const float* __restrict__ vcb,
                    const int32_t* __restrict__ seq_lens, const float* __restrict__ rope_cos,
                    const float* __restrict__ rope_sin, int pairing, float scale_log2e, Shape sh, int n_splits,
-                   float* __restrict__ partials)
+                   int stage_codebook, float* __restrict__ partials)
 {
     extern __shared__ __align__(16) float smem_f[];
     float* bins = smem_f;                      // [G][K]
     float* qsm = bins + sh.G * sh.K;           // [D]
-    __shared__ float red[kGenericThreads / 32];
+    float* kcb_s = qsm + sh.head_dim;          // [G][K][c]: the KV head's key codebook, when it fits
+    __shared__ float red[kRopeThreads / 32];
 
     const int split = blockIdx.x % n_splits;
     const int hq = (blockIdx.x / n_splits) % sh.n_q_heads;
@@ -410,11 +415,21 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     const __half* qv = q + (s * sh.n_q_heads + hq) * (int64_t)sh.head_dim;
     for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) qsm[d] = __half2float(qv[d]);
     for (int e = threadIdx.x; e < GK; e += blockDim.x) bins[e] = 0.f;
+    const float* kcb_h = kcb + (int64_t)hkv * GK * sh.c;
+    if (stage_codebook) {                      // centroid gathers then come from shared memory
+        const float4* src = reinterpret_cast<const float4*>(kcb_h);
+        float4* dst = reinterpret_cast<float4*>(kcb_s);
+        for (int e = threadIdx.x; e < GK * sh.c / 4; e += blockDim.x) dst[e] = src[e];
+        kcb_h = kcb_s;
+    }
     __syncthreads();
 
     const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
     const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
-    const float* kcb_h = kcb + (int64_t)hkv * GK * sh.c;
+    // 16-byte accesses need c and D/2 to be multiples of 4 and 16-byte aligned tables and codebooks
+    const bool vec4 = sh.c % 4 == 0 && P % 4 == 0 &&
+                      ((reinterpret_cast<uintptr_t>(rope_cos) | reinterpret_cast<uintptr_t>(rope_sin) |
+                        reinterpret_cast<uintptr_t>(kcb_h)) & 15u) == 0;
     float m_run = -INFINITY;
     float l_thr = 0.f;
     for (int64_t t0 = t_begin; t0 < t_end; t0 += blockDim.x) {
@@ -427,7 +442,42 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             const float* cs = rope_cos + t * P;
             const float* sn = rope_sin + t * P;
             float acc = 0.f;
-            if (pairing == 0) {
+            if (pairing == 0 && vec4) {
+                // Four pairs per 16-byte load of the token's cos / sin row and of the two centroids; the
+                // loads of 32 pairs are issued together, since their latency is what this loop waits for.
+                constexpr int kAhead = 8;
+                const int half_groups = sh.G / 2;
+                for (int i0 = 0; i0 < P; i0 += 4 * kAhead) {
+                    float4 c4[kAhead], s4[kAhead];
+#pragma unroll
+                    for (int u = 0; u < kAhead; ++u)
+                        if (i0 + 4 * u < P) {
+                            c4[u] = *reinterpret_cast<const float4*>(cs + i0 + 4 * u);
+                            s4[u] = *reinterpret_cast<const float4*>(sn + i0 + 4 * u);
+                        }
+#pragma unroll
+                    for (int u = 0; u < kAhead; ++u) {
+                        const int i = i0 + 4 * u;
+                        if (i >= P) break;
+                        const int g = i / sh.c, k = i % sh.c;
+                        const float* ca = kcb_h + ((int64_t)g * sh.K + read_code(kbase + block0, sh, g, k16)) * sh.c;
+                        const float* cb2 = kcb_h + ((int64_t)(g + half_groups) * sh.K +
+                                                    read_code(kbase + block0, sh, g + half_groups, k16)) * sh.c;
+                        const float4 a4 = *reinterpret_cast<const float4*>(ca + k);
+                        const float4 b4 = *reinterpret_cast<const float4*>(cb2 + k);
+                        const float4 qa4 = *reinterpret_cast<const float4*>(qsm + i);
+                        const float4 qb4 = *reinterpret_cast<const float4*>(qsm + i + P);
+                        acc = fmaf(c4[u].x, fmaf(qa4.x, a4.x, qb4.x * b4.x), acc);
+                        acc = fmaf(s4[u].x, fmaf(qb4.x, a4.x, -qa4.x * b4.x), acc);
+                        acc = fmaf(c4[u].y, fmaf(qa4.y, a4.y, qb4.y * b4.y), acc);
+                        acc = fmaf(s4[u].y, fmaf(qb4.y, a4.y, -qa4.y * b4.y), acc);
+                        acc = fmaf(c4[u].z, fmaf(qa4.z, a4.z, qb4.z * b4.z), acc);
+                        acc = fmaf(s4[u].z, fmaf(qb4.z, a4.z, -qa4.z * b4.z), acc);
+                        acc = fmaf(c4[u].w, fmaf(qa4.w, a4.w, qb4.w * b4.w), acc);
+                        acc = fmaf(s4[u].w, fmaf(qb4.w, a4.w, -qa4.w * b4.w), acc);
+                    }
+                }
+            } else if (pairing == 0) {
                 const int half_groups = sh.G / 2;
                 for (int g = 0; g < half_groups; ++g) {
                     const float* ca = kcb_h + ((int64_t)g * sh.K + read_code(kbase + block0, sh, g, k16)) * sh.c;
@@ -470,12 +520,14 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     }
     const float l = block_reduce_sum(l_thr, red);
     if (threadIdx.x == 0) { part[0] = m_run; part[1] = l; }
-    for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) {
+    // bins x V centroids: a warp per output channel, its lanes share the code values
+    for (int d = threadIdx.x >> 5; d < sh.head_dim; d += blockDim.x >> 5) {
         const int g = d / sh.c, k = d % sh.c;
         const float* cv = vcb + ((int64_t)hkv * GK + g * sh.K) * sh.c + k;
         float a = 0.f;
-        for (int j = 0; j < sh.K; ++j) a = fmaf(bins[g * sh.K + j], cv[j * sh.c], a);
-        part[2 + d] = a;
+        for (int j = threadIdx.x & 31; j < sh.K; j += 32) a = fmaf(bins[g * sh.K + j], cv[j * sh.c], a);
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if ((threadIdx.x & 31) == 0) part[2 + d] = a;
     }
 }
 
@@ -547,13 +599,26 @@ cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t
                                const float* vcb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
                                int pairing, float scale, const Shape& sh, float* out, float* partials, cudaStream_t st)
 {
-    const int n_splits = decode_generic_splits(sh);
-    const size_t smem = ((size_t)sh.G * sh.K + sh.head_dim) * sizeof(float);
+    // One CTA fills an SM and stages a codebook, so contexts are split only as far as the SMs need it
+    // (and never into more partial slots than the workspace holds: those of decode_generic_splits).
+    int n_splits = decode_generic_splits(sh);
+    {
+        const int64_t items = sh.n_seq * sh.n_q_heads;
+        int64_t want = (2 * 148 + items - 1) / items;
+        const int64_t cap = (sh.max_tokens + kRopeThreads - 1) / kRopeThreads;
+        if (want > cap) want = cap;
+        if (want < 1) want = 1;
+        if (want < n_splits) n_splits = (int)want;
+    }
+    size_t smem = ((size_t)sh.G * sh.K + sh.head_dim) * sizeof(float);
+    const size_t book = (size_t)sh.G * sh.K * sh.c * sizeof(float);
+    const int stage = (sh.G * sh.K * sh.c) % 4 == 0 && smem + book <= (size_t)220 * 1024;
+    if (stage) smem += book;
     cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(n_splits * sh.n_q_heads * sh.n_seq);
-    decode_rope_kernel<<<grid, kGenericThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, rope_cos, rope_sin, pairing,
-                                                            scale * kLog2e, sh, n_splits, partials);
+    decode_rope_kernel<<<grid, kRopeThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, rope_cos, rope_sin, pairing,
+                                                         scale * kLog2e, sh, n_splits, stage, partials);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return launch_merge(partials, n_splits, sh, out, st);
