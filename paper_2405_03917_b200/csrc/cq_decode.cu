@@ -175,10 +175,20 @@ __device__ __forceinline__ float4 ldg_f4(const float* p)
     asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
     return v;
 }
+// `wide`: an 8-channel centroid is one 32-byte load (the lanes of a warp then read one contiguous
+// KiB; two 16-byte loads at a 32-byte lane stride touch every sector twice).  Needs 32-byte
+// aligned codebooks, which the launcher checks.
 template <int kC>
-__device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC])
+__device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC], bool wide)
 {
     static_assert(kC == 4 || kC == 8, "centroids of 4 or 8 channels");
+    if (kC == 8 && wide) {
+        asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(cv[0]), "=f"(cv[1]), "=f"(cv[2]), "=f"(cv[3]), "=f"(cv[4 % kC]), "=f"(cv[5 % kC]),
+                       "=f"(cv[6 % kC]), "=f"(cv[7 % kC])
+                     : "l"(p) : "memory");
+        return;
+    }
     const float4 a = ldg_f4(p);
     cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
     if (kC == 8) {
@@ -258,7 +268,7 @@ __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
                     const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                    int tail_first, float* __restrict__ partials)
+                    int tail_first, int cb_aligned32, float* __restrict__ partials)
 {
     using C = Cfg<G, R>;
     constexpr int kC = C::kC;
@@ -341,7 +351,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         const int g = warp * C::kGroupsPerWarp + u / kUnitsPerGroup;
         const float* cg = cb + (((int64_t)hkv * G + g) * kRows + (u % kUnitsPerGroup) * kJb * 32 + lane) * kC;
 #pragma unroll
-        for (int jb = 0; jb < kJb; ++jb) load_centroid<kC>(cg + jb * 32 * kC, cv[jb]);
+        for (int jb = 0; jb < kJb; ++jb) load_centroid<kC>(cg + jb * 32 * kC, cv[jb], cb_aligned32 != 0);
     };
     float cva[kJb][kC], cvb[kJb][kC];
     load_unit(cva, kcb, 0);
@@ -812,7 +822,7 @@ __global__ void __launch_bounds__(WideCfg::kThreads, 1)
 decode_wide_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                    const float* __restrict__ kcb, const float* __restrict__ vcb,
                    const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                   int tail_first, float* __restrict__ partials)
+                   int tail_first, int cb_aligned32, float* __restrict__ partials)
 {
     using C = WideCfg;
     constexpr int kC = C::kC;
@@ -889,7 +899,7 @@ decode_wide_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     auto load_unit = [&](float (&cv)[kJb][kC], const float* cb, int u) {
         const float* cg = cb + (((int64_t)hkv * C::kG + g) * C::kRows + u * kJb * 32 + lane) * kC;
 #pragma unroll
-        for (int jb = 0; jb < kJb; ++jb) load_centroid<kC>(cg + jb * 32 * kC, cv[jb]);
+        for (int jb = 0; jb < kJb; ++jb) load_centroid<kC>(cg + jb * 32 * kC, cv[jb], cb_aligned32 != 0);
     };
     float cva[kJb][kC], cvb[kJb][kC];
     load_unit(cva, kcb, 0);
@@ -1179,6 +1189,11 @@ decode_wide_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     }
 }
 
+int aligned32(const float* a, const float* b)
+{
+    return ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) & 31u) == 0 ? 1 : 0;
+}
+
 // Launch plan of one call: context chunk per CTA, partial slots per (sequence, query head), and
 // the first item of the tail (-1: none).
 struct Plan {
@@ -1242,7 +1257,8 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
                                          C::kSmemBytes);
     if (e != cudaSuccess) return e;
     decode_tuned_kernel<G, R><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
-                                                                          pl.chunk, pl.n_parts, pl.tail_first, partials);
+                                                                          pl.chunk, pl.n_parts, pl.tail_first,
+                                                                          aligned32(kcb, vcb), partials);
     return cudaGetLastError();
 }
 
@@ -1282,7 +1298,8 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
         e = cudaFuncSetAttribute(decode_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WideCfg::kSmemBytes);
         if (e != cudaSuccess) return e;
         decode_wide_kernel<<<pl.grid, WideCfg::kThreads, WideCfg::kSmemBytes, st>>>(
-            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, partials);
+            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
+            partials);
         e = cudaGetLastError();
     }
     else if (sh.G == 16 && sh.R == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);

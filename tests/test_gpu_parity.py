@@ -286,6 +286,32 @@ def test_attention_when_the_last_wave_of_items_is_spread_over_several_ctas():
             H.check_attn(out[s_], ref[s_], f"spread tail, sequence {s_}")
 
 
+def test_attention_with_codebooks_at_16_byte_offsets():
+    # the tuned kernels read 8-channel centroids with 32-byte loads when both codebooks are 32-byte aligned
+    # and with pairs of 16-byte loads otherwise: both paths must give the oracle's result
+    c, b, D, n_q, n_kv, lens = 8, 8, 128, 4, 1, [3000, 77]
+    cap = 3000
+    w = H.small_workload("t", 131, c, b, 2, n_q, n_kv, cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    q = synth.queries(w.config, 0, 2, n_q)
+    rng = np.random.default_rng(4)
+    kc_rm = rng.integers(0, 256, size=(2, cap, n_kv, D // c)).astype(np.int32)
+    vc_rm = rng.integers(0, 256, size=(2, cap, n_kv, D // c)).astype(np.int32)
+    kb = cq.cq_codes_from_rowmajor(torch.from_numpy(kc_rm.astype(np.uint8)).to(DEV), D, c, b)
+    vb = cq.cq_codes_from_rowmajor(torch.from_numpy(vc_rm.astype(np.uint8)).to(DEV), D, c, b)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    ref = oracle.decode_dense(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32), D ** -0.5, c, b)
+    def shifted(t):                      # same values, 16 bytes past a 256-byte aligned allocation
+        buf = torch.empty(t.numel() + 4, dtype=torch.float32, device=DEV)
+        v = buf[4:].view(t.shape)
+        v.copy_(t)
+        assert v.data_ptr() % 32 == 16
+        return v
+    for kd, vd in ((kcb.to(DEV), vcb.to(DEV)), (shifted(kcb), shifted(vcb)), (kcb.to(DEV), shifted(vcb))):
+        out = cq.cq_decode_attn(q.to(DEV), kb, vb, kd, vd, sl, D ** -0.5, c, b, cap, variant=2).cpu().numpy()
+        H.check_attn(out, ref, "codebook alignment")
+
+
 def test_encode_codebooks_beyond_fp16_range_take_the_exact_path():
     # centroids too large for the fp16 term splits of the tensor-core path: the tuned kernel must
     # notice and recompute those groups exactly
