@@ -27,7 +27,8 @@
  *     see the layout below; CQ-8c10b of the paper's Section 4 is the case b = 10:
  *     1.25 bytes per code).  Decode attention needs (head_dim / c) * 2^b <= 24576
  *     table entries (CQ_ERR_UNSUPPORTED otherwise).  Tuned kernels
- *     exist for head_dim 128 and b = 8: encode for c = 2, 4, 8; decode attention
+ *     exist for head_dim 128: encode for c = 2, 4, 8 with b = 8, 9, 10, 12 (codebooks
+ *     of more than 256 centroids are taken in chunks of 256); for b = 8 decode attention
  *     for c = 8 with 1, 2 or 4 query heads per KV head and c = 4 with 1 or 2;
  *     and for decode attention of CQ-8c10b (head_dim 128, c = 8, b = 10).
  *     Every other supported shape runs on generic sm_100a kernels (never on the CPU).

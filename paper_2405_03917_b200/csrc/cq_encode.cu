@@ -189,7 +189,7 @@ __device__ __forceinline__ void build_a(const uint32_t (&xw)[2], const float (&X
 // Exact nearest centroid of one group of one vector, computed by the whole warp:
 // d_j = sum_i (x_i - C_ji)^2 in fp32 (same operation order as the generic kernel), lowest j on ties.
 template <int kC>
-__device__ __forceinline__ int exact_code(const float (&xg)[kC], const float* __restrict__ cb_g, int lane)
+__device__ __forceinline__ int exact_code(const float (&xg)[kC], const float* __restrict__ cb_g, int lane, float* dist)
 {
     float best = kInfBits;
     int arg = 0;
@@ -210,13 +210,17 @@ __device__ __forceinline__ int exact_code(const float (&xg)[kC], const float* __
         const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
         if (ob < best || (ob == best && oa < arg)) { best = ob; arg = oa; }
     }
+    *dist = best;
     return arg;
 }
 
 // kMT: 16-vector m-tiles per warp (4 for bulk encode, 1 when there are few vectors).
 // A launch covers one tensor, or two of the same shape (the key and the value of an append):
 // blockIdx.y picks (x, cb, codes) or (x2, cb2, codes2).
-template <int kC, int kMT>
+// kWide: 2^b > 256 centroids per group (b = 9, 10, 12): the group's codebook is taken in chunks of
+// 256 centroids, each chunk exactly as a codebook of b = 8, and the chunk winners are compared by
+// their exact distances (the earlier chunk wins ties, so the lowest index still does).
+template <int kC, int kMT, bool kWide>
 __global__ void __launch_bounds__(kEncThreads, 2)
 encode_tuned_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, const int32_t* __restrict__ seq_offsets,
                     Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes1, int groups_per_cta,
@@ -253,18 +257,27 @@ encode_tuned_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1
 
     if (threadIdx.x < 2) { ctl->range_flag[threadIdx.x] = 0; ctl->nmax[threadIdx.x] = 0.f; }
     __syncthreads();
-    prepare_group<kC>(cb + ((int64_t)h * G + g_begin) * 256 * kC, bbuf[0], ctl, 0);
+    const int n_chunks = kWide ? sh.K / 256 : 1;
+    const int n_steps = (g_end - g_begin) * n_chunks;
+    // centroids of step st: chunk st % n_chunks of group g_begin + st / n_chunks
+    auto chunk_ptr = [&](int st) {
+        return cb + (((int64_t)h * G + g_begin + st / n_chunks) * n_chunks + st % n_chunks) * 256 * kC;
+    };
+    prepare_group<kC>(chunk_ptr(0), bbuf[0], ctl, 0);
+    float dkeep[kWide ? kMT : 1][2];           // best exact distance and code over the chunks seen so far
+    int ckeep[kWide ? kMT : 1][2];
 
-    for (int g = g_begin; g < g_end; ++g) {
-        const int cur = (g - g_begin) & 1;
+    for (int st = 0; st < n_steps; ++st) {
+        const int g = g_begin + st / n_chunks, ch = st % n_chunks;
+        const int cur = st & 1;
         __syncthreads();                       // bbuf[cur] is complete; bbuf[cur ^ 1] is no longer read
         const bool out_of_range = ctl->range_flag[cur] != 0;
         const float nmax = ctl->nmax[cur];
         __syncthreads();                       // everyone has read the control words of `cur`
         if (threadIdx.x == 0) { ctl->range_flag[cur ^ 1] = 0; ctl->nmax[cur ^ 1] = 0.f; }
         __syncthreads();
-        if (g + 1 < g_end) prepare_group<kC>(cb + ((int64_t)h * G + g + 1) * 256 * kC, bbuf[cur ^ 1], ctl, cur ^ 1);
-        const float* cb_g = cb + ((int64_t)h * G + g) * 256 * kC;
+        if (st + 1 < n_steps) prepare_group<kC>(chunk_ptr(st + 1), bbuf[cur ^ 1], ctl, cur ^ 1);
+        const float* cb_g = chunk_ptr(st);
 
         // A operands of this warp's m-tiles
         uint32_t a[kMT][C::kSteps][4];
@@ -419,20 +432,39 @@ encode_tuned_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1
                         xg[2 * w] = f.x;
                         xg[(2 * w + 1) % kC] = f.y;
                     }
-                    const int ec = exact_code<kC>(xg, cb_g, lane);
-                    if ((lane & ~3) == src) code = ec;
+                    float ed;
+                    const int ec = exact_code<kC>(xg, cb_g, lane, &ed);
+                    if ((lane & ~3) == src) { code = ec; dbest = ed; }
+                }
+                if (kWide) {
+                    // dbest is the exact distance of `code` within this chunk: keep the best chunk so far
+                    const int m = kWide ? mt : 0;
+                    if (ch == 0 || dbest < dkeep[m][hf]) { dkeep[m][hf] = dbest; ckeep[m][hf] = code + 256 * ch; }
+                    if (ch + 1 < n_chunks) continue;
+                    code = ckeep[m][hf];
                 }
                 if (p == 0 && v < n_vec) {
                     const int64_t s = v / n_tokens, i = v % n_tokens;
                     const int64_t pos = token_offset + (seq_offsets ? seq_offsets[s] : 0) + i;
-                    if (pos >= 0 && pos < sh.max_tokens)
-                        codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + pos % kTokenBlock] = (uint8_t)code;
+                    if (pos >= 0 && pos < sh.max_tokens) {
+                        const int k = (int)(pos % kTokenBlock);
+                        codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + k] = (uint8_t)code;
+                        if (kWide) {        // upper bits: replaced in the 32-bit word that other tokens share
+                            const int bit = k * sh.hb;
+                            const uintptr_t a = reinterpret_cast<uintptr_t>(codes) +
+                                                (uintptr_t)code_high_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + (bit >> 3);
+                            unsigned int* w = reinterpret_cast<unsigned int*>(a & ~(uintptr_t)3);
+                            const int shift = (int)(a & 3) * 8 + (bit & 7);
+                            atomicAnd(w, ~((unsigned int)((1 << sh.hb) - 1) << shift));
+                            atomicOr(w, (unsigned int)(code >> 8) << shift);
+                        }
+                    }
                 }
             }
     }
 }
 
-template <int kC, int kMT>
+template <int kC, int kMT, bool kWide = false>
 cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh, int64_t n_tokens,
                        int64_t token_offset, uint8_t* codes, cudaStream_t st, const __half* x2 = nullptr,
                        const float* cb2 = nullptr, uint8_t* codes2 = nullptr)
@@ -450,9 +482,9 @@ cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offs
     const int64_t grid = tiles * sh.n_kv_heads * n_gsplit;
     if (grid > 0x7fffffff) return cudaErrorInvalidConfiguration;
     const size_t smem = (size_t)2 * C::kBufWords * 4 + sizeof(EncCtl);
-    cudaError_t e = cudaFuncSetAttribute(encode_tuned_kernel<kC, kMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(encode_tuned_kernel<kC, kMT, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    encode_tuned_kernel<kC, kMT><<<dim3((unsigned)grid, x2 ? 2u : 1u), kEncThreads, smem, st>>>(
+    encode_tuned_kernel<kC, kMT, kWide><<<dim3((unsigned)grid, x2 ? 2u : 1u), kEncThreads, smem, st>>>(
         x, cb, seq_offsets, sh, n_tokens, token_offset, codes, groups_per_cta, x2, cb2, codes2);
     return cudaGetLastError();
 }
@@ -461,7 +493,8 @@ cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offs
 
 bool encode_tuned_supported(const Shape& sh)
 {
-    return sh.head_dim == 128 && sh.b == 8 && (sh.c == 2 || sh.c == 4 || sh.c == 8);
+    if (sh.head_dim != 128 || !(sh.c == 2 || sh.c == 4 || sh.c == 8)) return false;
+    return sh.b == 8 || sh.b == 9 || sh.b == 10 || sh.b == 12;       // whole chunks of 256 centroids
 }
 
 cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
@@ -471,6 +504,17 @@ cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t*
     const int64_t n_vec = sh.n_seq * n_tokens;
     if (n_vec == 0) return cudaSuccess;
     const bool few = n_vec * sh.n_kv_heads < (int64_t)148 * 512 * 2;    // not enough vectors for 64 per warp
+    if (sh.b > 8) {
+        switch (sh.c) {
+            case 2: return few ? launch_enc<2, 1, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
+                               : launch_enc<2, 4, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
+            case 4: return few ? launch_enc<4, 1, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
+                               : launch_enc<4, 4, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
+            case 8: return few ? launch_enc<8, 1, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
+                               : launch_enc<8, 4, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
+            default: return cudaErrorNotSupported;
+        }
+    }
     switch (sh.c) {
         case 2: return few ? launch_enc<2, 1>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)
                            : launch_enc<2, 4>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);

@@ -30,13 +30,33 @@ def encode_rowmajor(x, cb, c, b, cap, **kw):
 
 
 @pytest.mark.parametrize("c,b,head_dim,n_heads,n_tokens", [(8, 10, 128, 2, 70), (8, 9, 128, 1, 33), (4, 12, 32, 2, 21),
-                                                         (8, 10, 64, 3, 16), (16, 10, 128, 1, 50)])
+                                                         (8, 10, 64, 3, 16), (16, 10, 128, 1, 50), (4, 10, 128, 2, 300),
+                                                         (2, 9, 128, 1, 130), (8, 12, 128, 1, 90)])
 def test_encode_wide_codes(c, b, head_dim, n_heads, n_tokens):
     xk, xv, kcb, vcb, _ = H.generic_case(900 + b + c, 2, n_tokens, n_heads, n_heads, head_dim, c, b)
+    tuned = head_dim == 128 and c in (2, 4, 8) and b in (9, 10, 12)      # chunks of 256 centroids on the tensor cores
+    small = (1 << b) * c * 4 + 8 * c * 4 <= 48 * 1024
     for x, cb in ((xk, kcb), (xv, vcb)):
-        _, rm = encode_rowmajor(x, cb, c, b, n_tokens)
-        assert rm.max() >= 256                                    # the upper bits are in use
-        H.check_codes(x.numpy().reshape(-1, n_heads, head_dim), cb.numpy(), rm.reshape(-1, n_heads, head_dim // c), c, b)
+        for variant in (1, 0) + ((2,) if tuned else ()) + ((3,) if small else ()):
+            _, rm = encode_rowmajor(x, cb, c, b, n_tokens, variant=variant)
+            assert rm.max() >= 256                                    # the upper bits are in use
+            H.check_codes(x.numpy().reshape(-1, n_heads, head_dim), cb.numpy(), rm.reshape(-1, n_heads, head_dim // c), c, b)
+
+
+def test_encode_8c10b_bulk_and_duplicate_centroids_across_chunks():
+    # enough vectors for the 64-per-warp form of the tuned kernel; centroids duplicated in a later chunk of 256
+    # must lose the tie to their first copy (lowest index)
+    c, b, D, nh, n_tok = 8, 10, 128, 8, 2500
+    g = torch.Generator().manual_seed(12)
+    cb = torch.randn(nh, D // c, 1 << b, c, generator=g)
+    cb[:, :, 700] = cb[:, :, 40]
+    cb[:, :, 300] = cb[:, :, 299]
+    x = torch.randn(8, n_tok, nh, D, generator=g).to(torch.float16)
+    x[0, :64, :, :] = cb[:, :, 40].reshape(1, nh, D).to(torch.float16)          # vectors that sit (nearly) on centroid 40 / 700
+    for variant in (2, 1):
+        _, rm = encode_rowmajor(x, cb, c, b, n_tok, variant=variant)
+        assert not (rm == 700).any() and not (rm == 300).any()
+        H.check_codes(x.numpy().reshape(-1, nh, D), cb.numpy(), rm.reshape(-1, nh, D // c), c, b)
 
 
 @pytest.mark.parametrize("b", [9, 10, 12, 16])
