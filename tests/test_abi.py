@@ -101,3 +101,23 @@ def test_argument_validation_happens_on_the_host(L):
     assert dec(ws_bytes=16) == -5
     conv = L.cq_codes_to_rowmajor(None, 1, 16, 1, 128, 8, 8, p, None)
     assert conv == -1
+    # cq_encode_kv: the two code buffers must differ; the same checks as cq_encode otherwise
+    kv = lambda **kw: L.cq_encode_kv(*[kw.get(k, d) for k, d in [
+        ("k", p), ("v", p), ("kcb", p), ("vcb", p), ("so", None), ("n_seq", 1), ("n_tok", 4), ("off", 0), ("cap", 16),
+        ("heads", 1), ("D", 128), ("c", 8), ("b", 8), ("ko", p), ("vo", p + 4096), ("stream", None)]])
+    assert kv(v=None) == -1
+    assert kv(vo=p) == -2
+    assert kv(n_tok=17) == -2
+    assert kv(b=11) == -3
+    assert kv(ko=p + 4) == -4
+    # cq_decode_attn_rope: tables are required, the pairing is 0 or 1, a pair must lie in whole groups
+    rope = lambda **kw: L.cq_decode_attn_rope(*[kw.get(k, d) for k, d in [
+        ("q", p), ("kc", p), ("vc", p), ("kcb", p), ("vcb", p), ("sl", p), ("cos", p), ("sin", p), ("pairing", 0),
+        ("scale", ctypes.c_float(0.1)), ("n_seq", 2), ("hq", 4), ("hkv", 2), ("D", 128), ("c", 8), ("b", 8), ("cap", 64),
+        ("out", p), ("ws", p), ("ws_bytes", 1 << 30), ("stream", None)]])
+    assert rope(cos=None) == -1
+    assert rope(pairing=2) == -2
+    assert rope(c=128, b=2) == -3              # one group: channel i + 64 cannot be in another group's code
+    assert rope(c=1, b=2, pairing=1) == -3     # an interleaved pair would span two groups
+    assert rope(cos=p + 2) == -4
+    assert rope(ws_bytes=16) == -5
