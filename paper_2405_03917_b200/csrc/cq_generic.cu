@@ -378,6 +378,35 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
 // ------------------------------------------------------------------------------------------
 constexpr int kRopeThreads = 512;
 
+// Bulk asynchronous copy global -> shared memory (the TMA engine; no tensor map, no multicast) with
+// an mbarrier that counts the bytes.  Source, destination and size are multiples of 16 bytes.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+// Waits for the phase with the given parity; gives up after a bounded number of polls (returns false).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+{
+    for (int poll = 0; poll < (1 << 22); ++poll) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
 __global__ void __launch_bounds__(kRopeThreads)
 decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                    const float* __restrict__ kcb, const float* __restrict__ vcb,
@@ -390,6 +419,7 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     float* qsm = bins + sh.G * sh.K;           // [D]
     float* kcb_s = qsm + sh.head_dim;          // [G][K][c]: the KV head's key codebook, when it fits
     __shared__ float red[kRopeThreads / 32];
+    __shared__ __align__(8) uint64_t book_bar;      // counts the bytes of the staged codebook
 
     const int split = blockIdx.x % n_splits;
     const int hq = (blockIdx.x / n_splits) % sh.n_q_heads;
@@ -416,10 +446,28 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) qsm[d] = __half2float(qv[d]);
     for (int e = threadIdx.x; e < GK; e += blockDim.x) bins[e] = 0.f;
     const float* kcb_h = kcb + (int64_t)hkv * GK * sh.c;
-    if (stage_codebook) {                      // centroid gathers then come from shared memory
-        const float4* src = reinterpret_cast<const float4*>(kcb_h);
-        float4* dst = reinterpret_cast<float4*>(kcb_s);
-        for (int e = threadIdx.x; e < GK * sh.c / 4; e += blockDim.x) dst[e] = src[e];
+    if (stage_codebook) {
+        // Centroid gathers then come from shared memory.  One thread hands the copy to the bulk-copy
+        // engine in pieces of 32 KiB; if the barrier does not complete within its poll limit, the
+        // threads copy the codebook themselves (the same bytes, so a late bulk copy does no harm).
+        const uint32_t book_bytes = (uint32_t)GK * sh.c * sizeof(float);
+        if (threadIdx.x == 0) {
+            mbar_init(&book_bar, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            mbar_expect_tx(&book_bar, book_bytes);
+            for (uint32_t off = 0; off < book_bytes; off += 32768u) {
+                const uint32_t piece = book_bytes - off < 32768u ? book_bytes - off : 32768u;
+                bulk_copy_g2s(reinterpret_cast<char*>(kcb_s) + off, reinterpret_cast<const char*>(kcb_h) + off, piece, &book_bar);
+            }
+        }
+        if (__syncthreads_or(mbar_wait(&book_bar, 0) ? 0 : 1)) {      // same decision in every thread
+            const float4* src = reinterpret_cast<const float4*>(kcb_h);
+            float4* dst = reinterpret_cast<float4*>(kcb_s);
+            for (int e = threadIdx.x; e < GK * sh.c / 4; e += blockDim.x) dst[e] = src[e];
+        }
         kcb_h = kcb_s;
     }
     __syncthreads();
