@@ -356,6 +356,27 @@ def extra_learn(cq, dev, iters=100):
             "paper_context": "Table 4: 14 min for 64 such tensors (LLaMA-2-7b, CQ-8c8b) on one A100-40GB"}
 
 
+def extra_encode_wide(cq, dev, w, reps=3):
+    """Bulk encode of one tensor of a wide-code workload (chunks of 256 centroids on the tensor cores)."""
+    D = w.head_dim
+    n_seq = min(w.n_seq, 4)
+    x = synth.layer_activations(w, 0, False, n_seq, w.n_tokens, device=dev)
+    cb = synth.layer_codebooks(w, 0, False).to(dev)
+    buf = torch.zeros(cq.cq_codes_bytes(n_seq, w.n_tokens, w.n_kv_heads, D, w.c, w.b), dtype=torch.uint8, device=dev)
+    cq.cq_encode(x, cb, w.c, w.b, buf, w.n_tokens)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        cq.cq_encode(x, cb, w.c, w.b, buf, w.n_tokens)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    vectors = n_seq * w.n_tokens * w.n_kv_heads
+    return {"workload": f"{w.name}: {n_seq} x {w.n_tokens} tokens x {w.n_kv_heads} heads, one tensor", "ms": ms,
+            "vectors_per_s": vectors / (ms * 1e-3), "useful_tflops": vectors * 2 * D * (1 << w.b) / (ms * 1e-3) / 1e12}
+
+
 def extra_decode(cq, dev, w, reps=20):
     st = DecodeState(w, 0, dev, cq)
     for _ in range(3):
@@ -538,6 +559,7 @@ def main():
                 extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
                 extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
                 extras["decode_rope_cfg1"] = extra_decode_rope(cq, dev, synth.WORKLOADS[1])
+                extras["encode_cfg5_8c10b"] = extra_encode_wide(cq, dev, synth.WORKLOADS[5])
             if args.extras == "all":
                 extras["learn"] = extra_learn(cq, dev)
         except Exception as e:      # extras never hide the headline number
