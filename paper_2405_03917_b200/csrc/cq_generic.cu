@@ -660,7 +660,9 @@ cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t
     }
     size_t smem = ((size_t)sh.G * sh.K + sh.head_dim) * sizeof(float);
     const size_t book = (size_t)sh.G * sh.K * sh.c * sizeof(float);
-    const int stage = (sh.G * sh.K * sh.c) % 4 == 0 && smem + book <= (size_t)220 * 1024;
+    // the staged copy starts after the bins and the query and moves 16-byte pieces: both must be 16-byte multiples
+    const int stage = (sh.G * sh.K + sh.head_dim) % 4 == 0 && (sh.G * sh.K * sh.c) % 4 == 0 &&
+                      smem + book <= (size_t)220 * 1024;
     if (stage) smem += book;
     cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -40,6 +40,8 @@ def to_lib(rm, D, c, b):
     (4, 8, 2, 1, [300, 257], 128),
     (2, 6, 3, 3, [90], 64),
     (8, 10, 2, 1, [500, 123], 128),              # CQ-8c10b
+    (2, 1, 1, 1, [40], 4),                       # tiny shapes: the staged codebook would not be 16-byte aligned
+    (2, 3, 2, 1, [70, 5], 12),
 ])
 @pytest.mark.parametrize("pairing", [0, 1])
 def test_rope_attention_matches_the_oracle(c, b, n_q, n_kv, lens, D, pairing):
