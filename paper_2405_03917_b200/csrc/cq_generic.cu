@@ -258,7 +258,8 @@ cudaError_t launch_from_rowmajor(const uint8_t* rowmajor, const Shape& sh, uint8
 //   acc[g*c+i] = sum_j bins[g][j] * Cv[g][j][i];  partial = (m, l, acc)
 // The partials of all splits are merged by merge_kernel.
 // ------------------------------------------------------------------------------------------
-constexpr int kGenericThreads = 256;
+constexpr int kGenericThreads = 256;        // CTA size when several CTAs fit an SM
+constexpr int kGenericThreadsMax = 1024;    // CTA size when the tables leave room for one CTA only
 
 __device__ inline float block_reduce_max(float v, float* red)
 {
@@ -282,7 +283,7 @@ __device__ inline float block_reduce_sum(float v, float* red)
     return r;
 }
 
-__global__ void __launch_bounds__(kGenericThreads)
+__global__ void __launch_bounds__(kGenericThreadsMax)
 decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                       const float* __restrict__ kcb, const float* __restrict__ vcb,
                       const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int n_splits,
@@ -291,7 +292,7 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
     extern __shared__ __align__(16) float smem_f[];
     float* lut = smem_f;                       // [G][K]
     float* bins = lut + sh.G * sh.K;           // [G][K]
-    __shared__ float red[kGenericThreads / 32];
+    __shared__ float red[kGenericThreadsMax / 32];
 
     const int split = blockIdx.x % n_splits;
     const int hq = (blockIdx.x / n_splits) % sh.n_q_heads;
@@ -631,12 +632,24 @@ cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint
                                   const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
                                   float* out, float* partials, cudaStream_t st)
 {
-    const int n_splits = decode_generic_splits(sh);
+    int n_splits = decode_generic_splits(sh);
     const size_t smem = (size_t)2 * sh.G * sh.K * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(decode_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    // tables of more than a third of an SM's shared memory: fewer, larger CTAs keep the SM's warps busy
+    const int threads = smem > 72 * 1024 ? (smem > 110 * 1024 ? kGenericThreadsMax : 512) : kGenericThreads;
+    if (threads == kGenericThreadsMax) {
+        // one CTA per SM, each paying a table build over the whole codebook: split the contexts only as far
+        // as two CTAs per SM need it (never into more partial slots than the workspace holds)
+        const int64_t items = sh.n_seq * sh.n_q_heads;
+        int64_t want = (2 * 148 + items - 1) / items;
+        const int64_t cap = (sh.max_tokens + threads - 1) / threads;
+        if (want > cap) want = cap;
+        if (want < 1) want = 1;
+        if (want < n_splits) n_splits = (int)want;
+    }
     const unsigned grid = (unsigned)(n_splits * sh.n_q_heads * sh.n_seq);
-    decode_generic_kernel<<<grid, kGenericThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
+    decode_generic_kernel<<<grid, threads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
                                                                n_splits, partials);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
