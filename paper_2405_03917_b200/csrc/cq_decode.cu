@@ -47,14 +47,17 @@ constexpr int kUnset = INT_MIN;                    // no score seen yet
 
 template <int G, int R>
 struct Cfg {
-    static_assert(G == 16 || G == 32, "tuned decode kernels cover 16 and 32 groups");
+    static_assert(G == 16 || G == 32 || (G == 64 && R == 1), "tuned decode kernels cover 16, 32 and (one query head) 64 groups");
     static constexpr int kC = 128 / G;                                  // channels per group
+    // 64 groups: the two half warps take the same four 16-token blocks, quads 0-3 the groups 0-31 and quads
+    // 4-7 the groups 32-63 (second plane of a table row); they exchange their partial scores with one shuffle.
+    static constexpr bool kHalfGroups = (G == 64);
     static constexpr bool kHalfRows = (G == 16);                         // quads 0-3 / 4-7 use different 16-word halves
     static constexpr bool kReplica = (G == 16 && R == 1);                // the two halves are copies of one table
     static constexpr int kLaneHeads = (G == 16 && R >= 2) ? R / 2 : R;   // query heads a lane serves
-    static constexpr int kPlanes = kLaneHeads;                           // 32-word planes per table row
-    static constexpr int kSlots = G / 4;                                 // code words (16 tokens each) per lane
-    static constexpr int kBlocksPerIter = (G == 16 && R >= 2) ? 4 : 8;   // 16-token blocks per warp iteration
+    static constexpr int kPlanes = kHalfGroups ? 2 : kLaneHeads;         // 32-word planes per table row
+    static constexpr int kSlots = kHalfGroups ? 8 : G / 4;               // code words (16 tokens each) per lane
+    static constexpr int kBlocksPerIter = ((G == 16 && R >= 2) || kHalfGroups) ? 4 : 8;   // 16-token blocks per warp iteration
 #ifdef CQ_TUNE_WARPS1
     static constexpr int kWarps = (kPlanes == 1) ? CQ_TUNE_WARPS1 : 16;
 #else
@@ -81,14 +84,22 @@ struct Cfg {
     }
     // group of a table word, and the (plane, word) that holds (group g, query head h of the KV head)
     __device__ static __forceinline__ int group_of(int w) { return kHalfRows ? (w & 15) : w; }
-    __device__ static __forceinline__ int plane_of(int h) { return kHalfRows ? (R <= 2 ? 0 : h >> 1) : h; }
-    __device__ static __forceinline__ int word_of(int g, int h) { return kHalfRows ? (R == 1 ? 0 : (h & 1) * 16) + g : g; }
+    __device__ static __forceinline__ int plane_of(int g, int h)
+    {
+        return kHalfGroups ? g >> 5 : (kHalfRows ? (R <= 2 ? 0 : h >> 1) : h);
+    }
+    __device__ static __forceinline__ int word_of(int g, int h)
+    {
+        return kHalfGroups ? (g & 31) : (kHalfRows ? (R == 1 ? 0 : (h & 1) * 16) + g : g);
+    }
+    // byte offset, inside a table row, of the plane that lane row r uses by itself (64 groups only)
+    __device__ static __forceinline__ unsigned lane_plane_bytes(int r) { return kHalfGroups ? 128u * (unsigned)(r >> 2) : 0u; }
     // query head (of the KV head) that lane row r serves as its u-th head, and the head a table word belongs to
     __device__ static __forceinline__ int lane_head(int u, int r) { return kHalfRows ? (R == 1 ? 0 : 2 * u + (r >> 2)) : u; }
     __device__ static __forceinline__ int head_of_word(int word_in_row)
     {
         const int plane = word_in_row >> 5, w = word_in_row & 31;
-        return kHalfRows ? (R == 1 ? 0 : 2 * plane + (w >> 4)) : plane;
+        return kHalfGroups ? 0 : (kHalfRows ? (R == 1 ? 0 : 2 * plane + (w >> 4)) : plane);
     }
     // v[lane_head(u, r)] without indexing a register array by a run-time value
     template <int N>
@@ -181,7 +192,11 @@ __device__ __forceinline__ float4 ldg_f4(const float* p)
 template <int kC>
 __device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC], bool wide)
 {
-    static_assert(kC == 4 || kC == 8, "centroids of 4 or 8 channels");
+    static_assert(kC == 2 || kC == 4 || kC == 8, "centroids of 2, 4 or 8 channels");
+    if (kC == 2) {
+        asm volatile("ld.global.nc.v2.f32 {%0,%1}, [%2];" : "=f"(cv[0]), "=f"(cv[1 % kC]) : "l"(p) : "memory");
+        return;
+    }
     if (kC == 8 && wide) {
         asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                      : "=f"(cv[0]), "=f"(cv[1]), "=f"(cv[2]), "=f"(cv[3]), "=f"(cv[4 % kC]), "=f"(cv[5 % kC]),
@@ -190,7 +205,7 @@ __device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC], b
         return;
     }
     const float4 a = ldg_f4(p);
-    cv[0] = a.x; cv[1] = a.y; cv[2] = a.z; cv[3] = a.w;
+    cv[0] = a.x; cv[1 % kC] = a.y; cv[2 % kC] = a.z; cv[3 % kC] = a.w;
     if (kC == 8) {
         const float4 b = ldg_f4(p + 4);
         cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
@@ -323,7 +338,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     const int qb = (C::kBlocksPerIter == 8) ? r : (r & 3);                 // block of this quad inside the warp's iteration
     uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a plane, per code word
 #pragma unroll
-    for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m);
+    for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m) + C::lane_plane_bytes(r);
     // code words of this lane: word (block, group) sits at (block * G + group) * 16 bytes
     const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
     const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
@@ -398,7 +413,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     for (int i = 0; i < kC; ++i) dot = fmaf(qreg[h][i], cv[jb][i], dot);
                     absmax = fmaxf(absmax, fabsf(dot));
                     const uint32_t e = pack_hi_lo(dot);
-                    uint8_t* row = smem + j * kRowBytes + C::plane_of(h) * 128;
+                    uint8_t* row = smem + j * kRowBytes + C::plane_of(g, h) * 128;
                     *reinterpret_cast<uint32_t*>(row + ((C::word_of(g, h) + j) & 31) * 4) = e;
                     if (C::kReplica) *reinterpret_cast<uint32_t*>(row + ((16 + g + j) & 31) * 4) = e;
                 }
@@ -561,6 +576,10 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 }
         }
 
+        if (C::kHalfGroups) {            // the other half warp summed the other 32 groups of the same tokens
+#pragma unroll
+            for (int k = 0; k < 16; ++k) sc[0][k] += __shfl_xor_sync(0xffffffffu, sc[0][k], 16);
+        }
         // tokens past the end of the context get -inf (only the warp that holds the ragged end pays)
         if ((blk_warp + C::kBlocksPerIter) * kTokenBlock > t_end) {
             const int64_t tok0 = blk * kTokenBlock;
@@ -597,7 +616,8 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                 z += wown[u][j];
             }
 #pragma unroll
-            for (int o = kSplit ? 8 : 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+            // (with 64 groups both half warps hold the same tokens: each counts them once)
+            for (int o = (kSplit || C::kHalfGroups) ? 8 : 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
             zsum[u] = z;
         }
         any_tokens = __any_sync(0xffffffffu, any_tokens);
@@ -732,7 +752,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             const int j = ((u % kUnitsPerGroup) * kJb + jb) * 32 + lane;
 #pragma unroll
             for (int h = 0; h < R; ++h) {
-                const uint8_t* row = smem + C::kVOffset + j * kRowBytes + C::plane_of(h) * 128;
+                const uint8_t* row = smem + C::kVOffset + j * kRowBytes + C::plane_of(g, h) * 128;
                 uint32_t bi = *reinterpret_cast<const uint32_t*>(row + ((C::word_of(g, h) + j) & 31) * 4);
                 if (C::kReplica) bi += *reinterpret_cast<const uint32_t*>(row + ((16 + g + j) & 31) * 4);
                 const float bv = (float)bi;
@@ -747,10 +767,19 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         // remaining steps finish that channel.
 #pragma unroll
         for (int h = 0; h < R; ++h) {
-            float v = fold_channels<kC>(acc[h], lane);
-            // lane holds channel fold_channel_of<kC>(lane) summed over the lanes that share it
-            const int ch = fold_channel_of<kC>(lane);
-            if ((lane & (kC == 8 ? 3 : 7)) == 0) part_base[(int64_t)h * n_parts * stride + 2 + g * kC + ch] = v;
+            if constexpr (kC == 2) {
+                // one exchange gives each half warp one of the two channels, four more steps finish it
+                const bool up = (lane & 16) != 0;
+                float v = (up ? acc[h][1] : acc[h][0]) + __shfl_xor_sync(0xffffffffu, up ? acc[h][0] : acc[h][1], 16);
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if ((lane & 15) == 0) part_base[(int64_t)h * n_parts * stride + 2 + g * kC + (up ? 1 : 0)] = v;
+            } else {
+                float v = fold_channels<kC>(acc[h], lane);
+                // lane holds channel fold_channel_of<kC>(lane) summed over the lanes that share it
+                const int ch = fold_channel_of<kC>(lane);
+                if ((lane & (kC == 8 ? 3 : 7)) == 0) part_base[(int64_t)h * n_parts * stride + 2 + g * kC + ch] = v;
+            }
         }
         if (g == 0) {
 #pragma unroll
@@ -1272,6 +1301,7 @@ Plan plan_dispatch(const Shape& sh)
     if (sh.G == 16 && sh.R == 4) return plan_for<16, 4>(sh);
     if (sh.G == 32 && sh.R == 1) return plan_for<32, 1>(sh);
     if (sh.G == 32 && sh.R == 2) return plan_for<32, 2>(sh);
+    if (sh.G == 64 && sh.R == 1) return plan_for<64, 1>(sh);
     return Plan{0, 1, -1, 0u};
 }
 
@@ -1282,7 +1312,8 @@ bool decode_tuned_supported(const Shape& sh)
     if (sh.max_tokens > ((int64_t)1 << 30)) return false;
     if (wide_shape(sh)) return true;
     if (sh.head_dim != 128 || sh.b != 8) return false;
-    return (sh.G == 16 && (sh.R == 1 || sh.R == 2 || sh.R == 4)) || (sh.G == 32 && (sh.R == 1 || sh.R == 2));
+    return (sh.G == 16 && (sh.R == 1 || sh.R == 2 || sh.R == 4)) || (sh.G == 32 && (sh.R == 1 || sh.R == 2)) ||
+           (sh.G == 64 && sh.R == 1);
 }
 
 int decode_tuned_parts(const Shape& sh) { return plan_dispatch(sh).n_parts; }
@@ -1307,6 +1338,7 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
     else if (sh.G == 16 && sh.R == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     else if (sh.G == 32 && sh.R == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     else if (sh.G == 32 && sh.R == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 64 && sh.R == 1) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     if (e != cudaSuccess) return e;
     return launch_merge(partials, pl.n_parts, sh, out, st);
 }

@@ -222,7 +222,7 @@ def test_attention_peaked_and_flat_softmax():
         H.check_attn(out, ref, f"peaked/flat variant={variant}")
 
 
-@pytest.mark.parametrize("c,n_q,n_kv", [(8, 1, 1), (8, 4, 1), (8, 2, 1), (4, 1, 1), (4, 2, 1)])
+@pytest.mark.parametrize("c,n_q,n_kv", [(8, 1, 1), (8, 4, 1), (8, 2, 1), (4, 1, 1), (4, 2, 1), (2, 1, 1)])
 def test_weight_unit_is_coarsened_on_flat_and_on_rising_scores(c, n_q, n_kv):
     # Stress of the integer weight unit, for every tuned kernel shape.  Sequence 0: zero queries over
     # a long context (every weight equals the maximum, so the bins must coarsen their unit instead of
@@ -253,7 +253,8 @@ def test_weight_unit_is_coarsened_on_flat_and_on_rising_scores(c, n_q, n_kv):
 
 def test_attention_multi_chunk_gqa_and_mha_long():
     # contexts long enough for several chunks per (sequence, KV head) and ragged ends
-    for c, n_q, n_kv, lens in ((8, 4, 1, [9000, 4097]), (4, 1, 1, [5000]), (8, 2, 1, [6001]), (4, 2, 1, [4500])):
+    for c, n_q, n_kv, lens in ((8, 4, 1, [9000, 4097]), (4, 1, 1, [5000]), (8, 2, 1, [6001]), (4, 2, 1, [4500]),
+                               (2, 2, 2, [4100, 1025, 0])):
         b, D = 8, 128
         cap = max(lens) + 11
         w = H.small_workload("t", 120 + c + n_q, c, b, len(lens), n_q, n_kv, cap)
