@@ -558,6 +558,7 @@ def main():
                 extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
                 extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
                 extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
+                extras["decode_cfg6_2c8b"] = extra_decode(cq, dev, synth.WORKLOADS[6])
                 extras["decode_rope_cfg1"] = extra_decode_rope(cq, dev, synth.WORKLOADS[1])
                 extras["encode_cfg5_8c10b"] = extra_encode_wide(cq, dev, synth.WORKLOADS[5])
             if args.extras == "all":

@@ -138,6 +138,8 @@ WORKLOADS: List[Workload] = [
     # CQ-8c10b (1024 centroids per group, 1.25 bytes per code), Llama-2-7B-shaped heads; not one of the
     # measured configurations of the headline metric: a workload for the wide-code path
     Workload("cfg5_llama2_7b_8c10b_decode", 5, 8, 10, 1, 16, 32, 32, 8192),
+    # CQ-2c8b (64 groups, 4 bits per channel) decode on config 1's shape: the workload of the 64-group decode kernel
+    Workload("cfg6_llama2_7b_2c8b_decode", 6, 2, 8, 1, 16, 32, 32, 4096),
 ]
 
 

@@ -159,3 +159,12 @@ def test_config5_llama2_7b_8c10b_decode_full_size():
     ties, total, a, r = check_items(w, 0, st, seeded_items(w, 4, 505))
     assert ties <= total // 500
     print(f"config 5: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
+
+
+def test_config6_llama2_7b_2c8b_decode_full_size():
+    # CQ-2c8b decode (64 groups) at the size the benchmark times it: eight sampled (sequence, head) items
+    w = synth.WORKLOADS[6]
+    st = bench.DecodeState(w, 0, torch.device(DEV), cq)
+    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 8, 606))
+    assert ties <= total // 500
+    print(f"config 6: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
