@@ -1257,7 +1257,7 @@ Plan plan_from(const Shape& sh, int64_t round, int min_blocks, int64_t items)
     pl.grid = (unsigned)(items * pl.n_parts);
 #ifndef CQ_TUNE_NO_TAIL
     const int64_t rest = items % slots;               // CTAs of the last wave
-    if (min_blocks == 1 && pl.n_parts == 1 && items > slots && rest > 0 && 2 * rest <= slots && chunk >= 4 * 2048) {
+    if (min_blocks == 1 && pl.n_parts == 1 && items > slots && rest > 0 && 2 * rest <= slots && chunk >= 2 * 2048) {
         int64_t k = slots / rest;
         if (k > 4) k = 4;
         const int64_t part_chunk = ((chunk + k - 1) / k + round - 1) / round * round;
