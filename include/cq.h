@@ -29,7 +29,7 @@
  *     table entries (CQ_ERR_UNSUPPORTED otherwise).  Tuned kernels
  *     exist for head_dim 128: encode for c = 2, 4, 8 with b = 8, 9, 10, 12 (codebooks
  *     of more than 256 centroids are taken in chunks of 256); for b = 8 decode attention
- *     for c = 8 with 1, 2 or 4 query heads per KV head, c = 4 with 1 or 2 and c = 2 with 1;
+ *     for c = 8, 4 and 2 with any number of query heads per KV head (a CTA serves up to 4, 2, 1 of them);
  *     and for decode attention of CQ-8c10b (head_dim 128, c = 8, b = 10).
  *     Every other supported shape runs on generic sm_100a kernels (never on the CPU).
  *   - Inputs must be finite.

@@ -283,8 +283,10 @@ __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
                     const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                    int tail_first, int cb_aligned32, float* __restrict__ partials)
+                    int tail_first, int cb_aligned32, int kv_share, float* __restrict__ partials)
 {
+    // R is the number of query heads one CTA serves.  A KV head with more query heads than that
+    // (kv_share groups of R) is served by kv_share CTAs, which read the same codes and codebooks.
     using C = Cfg<G, R>;
     constexpr int kC = C::kC;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -299,7 +301,8 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     // tail_first take their whole context in one CTA, and each later item is spread over n_parts
     // CTAs of chunk_tokens each: those shorter CTAs start last and fill the last, partly empty
     // wave of the grid.
-    const int n_items = (int)(sh.n_kv_heads * sh.n_seq);
+    const int n_head_groups = sh.n_q_heads / R;
+    const int n_items = (int)(n_head_groups * sh.n_seq);
     int item = blockIdx.x % n_items;
     int part = (int)(blockIdx.x / n_items);
     bool whole = false;
@@ -308,16 +311,17 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         item = whole ? blockIdx.x : tail_first + (blockIdx.x - tail_first) / n_parts;
         part = whole ? 0 : (blockIdx.x - tail_first) % n_parts;
     }
-    const int hkv = item % sh.n_kv_heads;
-    const int64_t s = item / sh.n_kv_heads;
+    const int head_group = item % n_head_groups;      // query heads head_group * R ... + R - 1
+    const int hkv = head_group / kv_share;
+    const int64_t s = item / n_head_groups;
 
     int64_t n = seq_lens[s];
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
     const int64_t t_begin = (int64_t)part * chunk_tokens;
     const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
     const int stride = partial_stride(128);
-    float* part_base = partials + ((s * sh.n_q_heads + (int64_t)hkv * R) * n_parts + part) * stride;
-    // partial of query head hkv*R + h: part_base + h * n_parts * stride
+    float* part_base = partials + ((s * sh.n_q_heads + (int64_t)head_group * R) * n_parts + part) * stride;
+    // partial of query head head_group*R + h: part_base + h * n_parts * stride
     if (whole)          // the other partial slots of this item hold the neutral element of the merge
         for (int i = threadIdx.x; i < R * (n_parts - 1) * stride; i += C::kThreads) {
             const int h = i / ((n_parts - 1) * stride), d = i % ((n_parts - 1) * stride);
@@ -380,7 +384,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     }
     if (threadIdx.x == 4) { ctl->want = 0; ctl->lut_absmax = 0.f; }
     for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
-        qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)hkv * R) * 128 + i]) * scale_log2e;
+        qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)head_group * R) * 128 + i]) * scale_log2e;
     // bins start at zero (16-byte stores over the V planes)
     for (int i = threadIdx.x; i < kRows * 8 * C::kPlanes; i += C::kThreads)
         *reinterpret_cast<uint4*>(smem + C::kVOffset + (i / (8 * C::kPlanes)) * kRowBytes + (i % (8 * C::kPlanes)) * 16) =
@@ -1273,7 +1277,7 @@ Plan plan_from(const Shape& sh, int64_t round, int min_blocks, int64_t items)
 template <int G, int R>
 Plan plan_for(const Shape& sh)
 {
-    return plan_from(sh, Cfg<G, R>::kRoundTokens, Cfg<G, R>::kMinBlocks, sh.n_seq * sh.n_kv_heads);
+    return plan_from(sh, Cfg<G, R>::kRoundTokens, Cfg<G, R>::kMinBlocks, sh.n_seq * sh.n_kv_heads * (sh.R / R));
 }
 
 template <int G, int R>
@@ -1287,21 +1291,31 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
     if (e != cudaSuccess) return e;
     decode_tuned_kernel<G, R><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
                                                                           pl.chunk, pl.n_parts, pl.tail_first,
-                                                                          aligned32(kcb, vcb), partials);
+                                                                          aligned32(kcb, vcb), sh.R / R, partials);
     return cudaGetLastError();
 }
 
 bool wide_shape(const Shape& sh) { return sh.head_dim == 128 && sh.c == 8 && sh.b == 10; }
 
+// Query heads one CTA of decode_tuned_kernel serves for this shape: the largest built width that divides
+// the number of query heads per KV head (16 groups: 4, 2, 1; 32 groups: 2, 1; 64 groups: 1).
+int heads_per_cta(const Shape& sh)
+{
+    if (sh.G == 16) return sh.R % 4 == 0 ? 4 : (sh.R % 2 == 0 ? 2 : 1);
+    if (sh.G == 32) return sh.R % 2 == 0 ? 2 : 1;
+    return 1;
+}
+
 Plan plan_dispatch(const Shape& sh)
 {
     if (wide_shape(sh)) return plan_from(sh, WideCfg::kRoundTokens, 1, sh.n_seq * sh.n_q_heads);
-    if (sh.G == 16 && sh.R == 1) return plan_for<16, 1>(sh);
-    if (sh.G == 16 && sh.R == 2) return plan_for<16, 2>(sh);
-    if (sh.G == 16 && sh.R == 4) return plan_for<16, 4>(sh);
-    if (sh.G == 32 && sh.R == 1) return plan_for<32, 1>(sh);
-    if (sh.G == 32 && sh.R == 2) return plan_for<32, 2>(sh);
-    if (sh.G == 64 && sh.R == 1) return plan_for<64, 1>(sh);
+    const int w = heads_per_cta(sh);
+    if (sh.G == 16 && w == 1) return plan_for<16, 1>(sh);
+    if (sh.G == 16 && w == 2) return plan_for<16, 2>(sh);
+    if (sh.G == 16 && w == 4) return plan_for<16, 4>(sh);
+    if (sh.G == 32 && w == 1) return plan_for<32, 1>(sh);
+    if (sh.G == 32 && w == 2) return plan_for<32, 2>(sh);
+    if (sh.G == 64) return plan_for<64, 1>(sh);
     return Plan{0, 1, -1, 0u};
 }
 
@@ -1312,8 +1326,7 @@ bool decode_tuned_supported(const Shape& sh)
     if (sh.max_tokens > ((int64_t)1 << 30)) return false;
     if (wide_shape(sh)) return true;
     if (sh.head_dim != 128 || sh.b != 8) return false;
-    return (sh.G == 16 && (sh.R == 1 || sh.R == 2 || sh.R == 4)) || (sh.G == 32 && (sh.R == 1 || sh.R == 2)) ||
-           (sh.G == 64 && sh.R == 1);
+    return sh.G == 16 || sh.G == 32 || sh.G == 64;      // any number of query heads per KV head
 }
 
 int decode_tuned_parts(const Shape& sh) { return plan_dispatch(sh).n_parts; }
@@ -1333,12 +1346,12 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
             partials);
         e = cudaGetLastError();
     }
-    else if (sh.G == 16 && sh.R == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 16 && sh.R == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 16 && sh.R == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 32 && sh.R == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 32 && sh.R == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 64 && sh.R == 1) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 16 && heads_per_cta(sh) == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 16 && heads_per_cta(sh) == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 16 && heads_per_cta(sh) == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 32 && heads_per_cta(sh) == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 32 && heads_per_cta(sh) == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 64) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
     if (e != cudaSuccess) return e;
     return launch_merge(partials, pl.n_parts, sh, out, st);
 }

@@ -169,8 +169,13 @@ def test_config0_end_to_end(variant):
     (4, 4, 2, [1000, 1]),
     (2, 2, 2, [129, 64]),
     (2, 2, 1, [300]),
-    (8, 8, 1, [90, 200]),                        # R = 8
+    (8, 8, 1, [90, 200]),                        # R = 8: two CTAs of four query heads per KV head
     (8, 3, 3, [50]),
+    (8, 6, 2, [700, 2500]),                      # R = 3: three CTAs of one query head
+    (8, 12, 2, [1300, 64]),                      # R = 6: three CTAs of two
+    (4, 8, 2, [900, 33]),                        # 32 groups, R = 4: two CTAs of two
+    (4, 3, 1, [515]),                            # 32 groups, R = 3
+    (2, 4, 1, [2100, 17]),                       # 64 groups, R = 4: four CTAs of one
 ])
 def test_attention_small_cases(c, n_q, n_kv, lens):
     b, D = 8, 128
@@ -222,7 +227,7 @@ def test_attention_peaked_and_flat_softmax():
         H.check_attn(out, ref, f"peaked/flat variant={variant}")
 
 
-@pytest.mark.parametrize("c,n_q,n_kv", [(8, 1, 1), (8, 4, 1), (8, 2, 1), (4, 1, 1), (4, 2, 1), (2, 1, 1)])
+@pytest.mark.parametrize("c,n_q,n_kv", [(8, 1, 1), (8, 4, 1), (8, 2, 1), (4, 1, 1), (4, 2, 1), (2, 1, 1), (8, 8, 1), (2, 2, 1)])
 def test_weight_unit_is_coarsened_on_flat_and_on_rising_scores(c, n_q, n_kv):
     # Stress of the integer weight unit, for every tuned kernel shape.  Sequence 0: zero queries over
     # a long context (every weight equals the maximum, so the bins must coarsen their unit instead of
