@@ -377,7 +377,7 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
 // V side, the online softmax and the partials are those of decode_generic_kernel.
 // pairing 0: (a, b) = (i, i + D/2); pairing 1: (a, b) = (2i, 2i + 1).
 // ------------------------------------------------------------------------------------------
-constexpr int kRopeThreads = 512;
+constexpr int kRopeThreads = 1024;
 
 // Bulk asynchronous copy global -> shared memory (the TMA engine; no tensor map, no multicast) with
 // an mbarrier that counts the bytes.  Source, destination and size are multiples of 16 bytes.
@@ -494,7 +494,7 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             if (pairing == 0 && vec4) {
                 // Four pairs per 16-byte load of the token's cos / sin row and of the two centroids; the
                 // loads of 32 pairs are issued together, since their latency is what this loop waits for.
-                constexpr int kAhead = 8;
+                constexpr int kAhead = 4;
                 const int half_groups = sh.G / 2;
                 for (int i0 = 0; i0 < P; i0 += 4 * kAhead) {
                     float4 c4[kAhead], s4[kAhead];
