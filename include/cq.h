@@ -11,6 +11,12 @@
  *   cq_decode_attn  single-query attention that reads only the codes
  *                   (Eq. 1 with K and V replaced by their CQ reconstructions)
  *
+ * and, around them: cq_encode_kv (key and value of the same tokens in one launch),
+ * cq_decode_attn_rope (key codes taken before the rotary embedding, Section 3.2),
+ * cq_decode_attn_static (no caller workspace), cq_decode_step_host (one decode
+ * step from host buffers) and the centroid learning of Section 3.2.1
+ * (cq_kmeanspp_init, cq_lloyd_step, cq_learn_centroids).
+ *
  * General rules
  *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The
  *     caller owns all buffers, including the workspace; the library allocates
