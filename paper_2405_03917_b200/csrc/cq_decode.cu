@@ -278,7 +278,7 @@ __device__ __forceinline__ uint32_t row_index(const uint4& w, int k, uint32_t la
     return __byte_perm(word32(w, k), lane_off, 0x5504u | ((uint32_t)(k & 3) << 4));
 }
 
-template <int G, int R>
+template <int G, int R, bool kShared>
 __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
@@ -286,7 +286,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     int tail_first, int cb_aligned32, int kv_share, float* __restrict__ partials)
 {
     // R is the number of query heads one CTA serves.  A KV head with more query heads than that
-    // (kv_share groups of R) is served by kv_share CTAs, which read the same codes and codebooks.
+    // (kv_share groups of R; kShared) is served by kv_share CTAs, which read the same codes and codebooks.
     using C = Cfg<G, R>;
     constexpr int kC = C::kC;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -301,7 +301,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     // tail_first take their whole context in one CTA, and each later item is spread over n_parts
     // CTAs of chunk_tokens each: those shorter CTAs start last and fill the last, partly empty
     // wave of the grid.
-    const int n_head_groups = sh.n_q_heads / R;
+    const int n_head_groups = kShared ? sh.n_q_heads / R : sh.n_kv_heads;
     const int n_items = (int)(n_head_groups * sh.n_seq);
     int item = blockIdx.x % n_items;
     int part = (int)(blockIdx.x / n_items);
@@ -312,7 +312,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         part = whole ? 0 : (blockIdx.x - tail_first) % n_parts;
     }
     const int head_group = item % n_head_groups;      // query heads head_group * R ... + R - 1
-    const int hkv = head_group / kv_share;
+    const int hkv = kShared ? head_group / kv_share : head_group;
     const int64_t s = item / n_head_groups;
 
     int64_t n = seq_lens[s];
@@ -1286,12 +1286,20 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
                        cudaStream_t st)
 {
     using C = Cfg<G, R>;
-    cudaError_t e = cudaFuncSetAttribute(decode_tuned_kernel<G, R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         C::kSmemBytes);
+    const int kv_share = sh.R / R;
+    cudaError_t e = kv_share > 1 ? cudaFuncSetAttribute(decode_tuned_kernel<G, R, true>,
+                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)
+                                 : cudaFuncSetAttribute(decode_tuned_kernel<G, R, false>,
+                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     if (e != cudaSuccess) return e;
-    decode_tuned_kernel<G, R><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh,
-                                                                          pl.chunk, pl.n_parts, pl.tail_first,
-                                                                          aligned32(kcb, vcb), sh.R / R, partials);
+    if (kv_share > 1)
+        decode_tuned_kernel<G, R, true><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
+            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
+            kv_share, partials);
+    else
+        decode_tuned_kernel<G, R, false><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
+            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
+            kv_share, partials);
     return cudaGetLastError();
 }
 
