@@ -214,6 +214,74 @@ void oracle_decode_dense(const uint16_t *q, const int32_t *k_codes, const int32_
 }
 
 /*
+ * Causal attention of a run of n_q new tokens per sequence over the CQ-coded cache
+ * (Section 2.1: Eq. 1 gives the output of "the current token" from the keys and values
+ * of all tokens up to and including it; a prompt, or a chunk of one, applies it to each
+ * of its tokens in turn, with K and V replaced by their CQ reconstructions, Section 3.2).
+ *
+ * The cache of sequence s holds seq_lens[s] tokens, the last n_q of which are the new
+ * ones.  Query i (0 <= i < n_q) therefore sits at position pos_i = seq_lens[s] - n_q + i
+ * and attends the cached tokens 0 .. pos_i:
+ *   s_t = scale * <q_i, Khat_t>,  p = softmax(s_0 .. s_{pos_i}),  out_i = sum_t p_t Vhat_t
+ * A query whose position is negative (seq_lens[s] < n_q: fewer cached tokens than
+ * queries) has nothing to attend and gives a zero row.
+ *
+ *   q    fp16 bits [n_seq][n_q][n_q_heads][D]
+ *   out  fp64      [n_seq][n_q][n_q_heads][D]
+ */
+void oracle_prefill_dense(const uint16_t *q, const int32_t *k_codes, const int32_t *v_codes,
+                          const float *k_cb, const float *v_cb, const int32_t *seq_lens,
+                          double scale, int n_seq, int n_q, int n_q_heads, int n_kv_heads, int D,
+                          int c, int b, int64_t max_tokens, double *out)
+{
+    const int G = D / c;
+    const int K = 1 << b;
+    const int R = n_q_heads / n_kv_heads;
+#pragma omp parallel for collapse(3) schedule(dynamic, 1)
+    for (int s = 0; s < n_seq; ++s) {
+        for (int i = 0; i < n_q; ++i) {
+            for (int hq = 0; hq < n_q_heads; ++hq) {
+                const int hkv = hq / R;
+                const int64_t n = (int64_t)seq_lens[s] - n_q + i + 1;      /* tokens 0 .. pos_i */
+                const int64_t row = ((int64_t)s * n_q + i) * n_q_heads + hq;
+                double *o = out + row * D;
+                for (int d = 0; d < D; ++d) o[d] = 0.0;
+                if (n <= 0) continue;
+                double *qd = (double *)malloc(sizeof(double) * D);
+                double *score = (double *)malloc(sizeof(double) * n);
+                for (int d = 0; d < D; ++d) qd[d] = half_to_double(q[row * D + d]);
+                double smax = -INFINITY;
+                for (int64_t t = 0; t < n; ++t) {
+                    const int32_t *kc = k_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                    double dot = 0.0;
+                    for (int g = 0; g < G; ++g) {
+                        const float *cj = k_cb + (((int64_t)hkv * G + g) * K + kc[g]) * c;
+                        for (int e = 0; e < c; ++e) dot += qd[g * c + e] * (double)cj[e];
+                    }
+                    score[t] = scale * dot;
+                    if (score[t] > smax) smax = score[t];
+                }
+                double denom = 0.0;
+                for (int64_t t = 0; t < n; ++t) {
+                    score[t] = exp(score[t] - smax);
+                    denom += score[t];
+                }
+                for (int64_t t = 0; t < n; ++t) {
+                    const int32_t *vc = v_codes + (((int64_t)s * max_tokens + t) * n_kv_heads + hkv) * G;
+                    const double p = score[t] / denom;
+                    for (int g = 0; g < G; ++g) {
+                        const float *cj = v_cb + (((int64_t)hkv * G + g) * K + vc[g]) * c;
+                        for (int e = 0; e < c; ++e) o[g * c + e] += p * (double)cj[e];
+                    }
+                }
+                free(qd);
+                free(score);
+            }
+        }
+    }
+}
+
+/*
  * Decode attention when the cache holds codes of the keys as they were BEFORE the
  * rotary position embedding (last sentence of Section 3.2: CQ quantises keys before
  * RoPE; Section 2.1: the key transformation f_K includes the positional encoding).

@@ -44,6 +44,8 @@ def _load():
         L.oracle_decode_lut.argtypes = [vp, vp, vp, vp, vp, vp, f64, i32, i32, i32, i32, i32, i32, i64, i32, vp]
         L.oracle_decode_dense_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f64, i32, i32, i32, i32, i32, i32, i64, vp]
         L.oracle_decode_dense_rope.restype = None
+        L.oracle_prefill_dense.argtypes = [vp, vp, vp, vp, vp, vp, f64, i32, i32, i32, i32, i32, i32, i32, i64, vp]
+        L.oracle_prefill_dense.restype = None
         L.oracle_kmeanspp_init.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp]
         L.oracle_lloyd_step.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp]
         L.oracle_kmeanspp_init.restype = None
@@ -149,6 +151,29 @@ def decode_dense(q, k_codes, v_codes, k_cb, v_cb, seq_lens, scale: float, c: int
     qb, kc, vc, kcb, vcb, sl, n_seq, hq, hkv, D, mt, out = _attn_args(q, k_codes, v_codes, k_cb, v_cb, seq_lens, c, b)
     _load().oracle_decode_dense(_p(qb), _p(kc), _p(vc), _p(kcb), _p(vcb), _p(sl), float(scale),
                                 n_seq, hq, hkv, D, c, b, mt, _p(out))
+    return out
+
+
+def prefill_dense(q, k_codes, v_codes, k_cb, v_cb, seq_lens, scale: float, c: int, b: int) -> np.ndarray:
+    """Causal attention of the last n_q cached tokens of every sequence.  q fp16 (n_seq, n_q, Hq, D);
+    codes int32 (n_seq, max_tokens, Hkv, G); seq_lens counts the cached tokens including the n_q new
+    ones; query i attends tokens 0 .. seq_lens[s] - n_q + i.  Returns fp64 (n_seq, n_q, Hq, D)."""
+    qb = _half_bits(q)
+    n_seq, n_q, n_q_heads, D = qb.shape
+    k_codes = np.ascontiguousarray(k_codes, dtype=np.int32)
+    v_codes = np.ascontiguousarray(v_codes, dtype=np.int32)
+    _, max_tokens, n_kv_heads, G = k_codes.shape
+    assert k_codes.shape == v_codes.shape == (n_seq, max_tokens, n_kv_heads, D // c)
+    assert n_q_heads % n_kv_heads == 0
+    for cd in (k_codes, v_codes):
+        assert cd.min(initial=0) >= 0 and cd.max(initial=0) < (1 << b)
+    kcb = _cb(k_cb, n_kv_heads, D, c, b)
+    vcb = _cb(v_cb, n_kv_heads, D, c, b)
+    sl = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    assert sl.shape == (n_seq,) and sl.min(initial=0) >= 0 and sl.max(initial=0) <= max_tokens
+    out = np.empty((n_seq, n_q, n_q_heads, D), dtype=np.float64)
+    _load().oracle_prefill_dense(_p(qb), _p(k_codes), _p(v_codes), _p(kcb), _p(vcb), _p(sl), float(scale),
+                                 n_seq, n_q, n_q_heads, n_kv_heads, D, c, b, max_tokens, _p(out))
     return out
 
 

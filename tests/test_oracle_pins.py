@@ -278,6 +278,87 @@ def test_scale_is_applied_to_scores_only():
     assert np.abs(a - oracle.decode_dense(q, kc, vc, kcb, vcb, sl, 1.0, c, b)).max() > 1e-3
 
 
+# ----------------------------------------------------------------------------- causal attention of a run of new tokens
+
+def prefill_case(n_seq, n_q, Hq, Hkv, D, c, b, max_tokens, lens):
+    _, kc, vc, kcb, vcb, sl = attn_case(n_seq, Hq, Hkv, D, c, b, max_tokens, lens=lens)
+    q = rng.standard_normal((n_seq, n_q, Hq, D)).astype(np.float16)
+    return q, kc, vc, kcb, vcb, sl
+
+
+@pytest.mark.parametrize("c,b,Hq,Hkv", [(8, 8, 4, 2), (4, 6, 2, 2), (2, 5, 6, 2)])
+def test_prefill_matches_torch_masked_softmax(c, b, Hq, Hkv):
+    # Eq. 1 for all queries at once with library routines: one score matrix, a causal mask, torch.softmax.
+    D, n_q = 32, 7
+    q, kc, vc, kcb, vcb, sl = prefill_case(3, n_q, Hq, Hkv, D, c, b, 29, lens=[29, 11, 4])
+    got = oracle.prefill_dense(q, kc, vc, kcb, vcb, sl, 0.23, c, b)
+    G, R = D // c, Hq // Hkv
+    gi = torch.arange(G)
+    for s in range(3):
+        n = int(sl[s])
+        for hq in range(Hq):
+            h = hq // R
+            K = torch.from_numpy(kcb[h].astype(np.float64))[gi[None, :], torch.from_numpy(kc[s, :n, h].astype(np.int64))].reshape(n, D)
+            V = torch.from_numpy(vcb[h].astype(np.float64))[gi[None, :], torch.from_numpy(vc[s, :n, h].astype(np.int64))].reshape(n, D)
+            Q = torch.from_numpy(q[s, :, hq].astype(np.float64))                       # (n_q, D)
+            S = 0.23 * (Q @ K.T)                                                         # (n_q, n)
+            pos = n - n_q + torch.arange(n_q)                                            # position of query i
+            mask = torch.arange(n)[None, :] > pos[:, None]
+            S = S.masked_fill(mask, float("-inf"))
+            want = torch.zeros(n_q, D, dtype=torch.float64)
+            ok = pos >= 0
+            want[ok] = torch.softmax(S[ok], dim=1) @ V
+            np.testing.assert_allclose(got[s, :, hq], want.numpy(), rtol=1e-11, atol=1e-13)
+    assert (got[2, :3] == 0).all()          # sequence 2 caches 4 tokens for 7 queries: the first three have no position
+
+
+def test_prefill_row_equals_single_query_attention_at_that_length():
+    # Row i is Eq. 1 for one query over the first pos_i + 1 tokens: the decode form, which has its own pins.
+    D, c, b, n_q = 32, 8, 6, 5
+    q, kc, vc, kcb, vcb, sl = prefill_case(2, n_q, 4, 2, D, c, b, 23, lens=[23, 9])
+    got = oracle.prefill_dense(q, kc, vc, kcb, vcb, sl, 0.2, c, b)
+    for i in range(n_q):
+        one = oracle.decode_dense(np.ascontiguousarray(q[:, i]), kc, vc, kcb, vcb, sl - n_q + i + 1, 0.2, c, b)
+        assert np.array_equal(got[:, i], one)
+
+
+def test_prefill_hand_worked_and_first_token():
+    # A prompt that is the whole cache: query 0 sees only token 0 and returns its value reconstruction
+    # exactly; query 1 sees two tokens: out = sigma(s0 - s1) V0 + (1 - sigma) V1.
+    D, c, b = 16, 4, 3
+    q, kc, vc, kcb, vcb, sl = prefill_case(1, 3, 1, 1, D, c, b, 3, lens=[3])
+    scale = 0.6
+    got = oracle.prefill_dense(q, kc, vc, kcb, vcb, sl, scale, c, b)
+    khat = oracle.dequant(kc[0], kcb, c, b)[:, 0]
+    vhat = oracle.dequant(vc[0], vcb, c, b)[:, 0]
+    assert np.array_equal(got[0, 0, 0], vhat[0])
+    s = scale * khat[:2] @ q[0, 1, 0].astype(np.float64)
+    w0 = 1 / (1 + np.exp(s[1] - s[0]))
+    np.testing.assert_allclose(got[0, 1, 0], w0 * vhat[0] + (1 - w0) * vhat[1], rtol=1e-12, atol=1e-14)
+
+
+def test_prefill_sees_no_future_token_and_no_order_in_the_past():
+    D, c, b, n_q = 32, 4, 5, 6
+    q, kc, vc, kcb, vcb, sl = prefill_case(1, n_q, 2, 1, D, c, b, 20, lens=[17])
+    base = oracle.prefill_dense(q, kc, vc, kcb, vcb, sl, 0.3, c, b)
+    # changing the codes of new token j changes rows j.. only; tokens past seq_len are never read
+    j = 3
+    k2, v2 = kc.copy(), vc.copy()
+    t = 17 - n_q + j
+    k2[0, t] = (k2[0, t] + 1) % (1 << b)
+    v2[0, t] = (v2[0, t] + 3) % (1 << b)
+    k2[0, 17:] = (k2[0, 17:] + 1) % (1 << b)
+    got = oracle.prefill_dense(q, k2, v2, kcb, vcb, sl, 0.3, c, b)
+    assert np.array_equal(got[0, :j], base[0, :j])
+    assert all(np.abs(got[0, i] - base[0, i]).max() > 1e-9 for i in range(j, n_q))
+    # permuting the tokens cached before the first query leaves every row unchanged
+    perm = rng.permutation(17 - n_q)
+    kp, vp = kc.copy(), vc.copy()
+    kp[0, :17 - n_q] = kc[0, perm]
+    vp[0, :17 - n_q] = vc[0, perm]
+    np.testing.assert_allclose(oracle.prefill_dense(q, kp, vp, kcb, vcb, sl, 0.3, c, b), base, rtol=1e-11, atol=1e-13)
+
+
 # ----------------------------------------------------------------------------- centroid learning
 
 def _golden_kmeans():
