@@ -5,6 +5,50 @@
 
 using namespace cq;
 
+namespace cq {
+
+namespace {
+constexpr int kDeviceSlots = 64;
+std::mutex g_device_mutex;
+int g_sm_count[kDeviceSlots] = {};                   // 0: not queried yet
+int g_smem_set[kDeviceSlots][64] = {};               // per device and call site: dynamic shared memory size already set
+}  // namespace
+
+int device_sm_count()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDeviceSlots) {
+        cudaGetLastError();                          // no usable device (size queries on a machine without a GPU): B200's count
+        return 148;
+    }
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    if (g_sm_count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = 148;
+        }
+        g_sm_count[dev] = n;
+    }
+    return g_sm_count[dev];
+}
+
+cudaError_t ensure_dynamic_smem(const void* func, int bytes, int slot)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kDeviceSlots || slot < 0 || slot >= 64)
+        return cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    if (g_smem_set[dev][slot] >= bytes && bytes > 0) return cudaSuccess;
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) g_smem_set[dev][slot] = bytes;
+    return e;
+}
+
+}  // namespace cq
+
 namespace {
 
 constexpr int kMaxHeadDim = 256;

@@ -64,6 +64,22 @@ __device__ inline int read_code(const uint8_t* __restrict__ block, const Shape& 
 // A split-K partial: running max (log2 domain), normaliser, head_dim accumulators.
 __host__ __device__ inline int partial_stride(int head_dim) { return head_dim + 2; }
 
+// ---- host helpers (cq_api.cu) ----
+// SM count of the current device (queried once per device and process).
+int device_sm_count();
+// cudaFuncAttributeMaxDynamicSharedMemorySize for `func`, set once per device and (func, bytes);
+// `slot` is a small integer unique to the call site (0 <= slot < 64).
+cudaError_t ensure_dynamic_smem(const void* func, int bytes, int slot);
+
+// Launch plan of one tuned decode call: context chunk per CTA, partial slots per (sequence, query
+// head), and the first item of the tail (-1: none).
+struct DecodePlan {
+    int chunk;
+    int n_parts;
+    int tail_first;
+    unsigned grid;
+};
+
 // ---- launchers implemented in the .cu files (return cudaGetLastError()) ----
 cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                   int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
@@ -93,6 +109,13 @@ int decode_tuned_parts(const Shape& sh);      // partial slots per (sequence, qu
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
                                 float* out, float* partials, cudaStream_t st);
+
+// CQ-8c8b with a multiple of four query heads per KV head: two query heads per table word (cq_decode_pair.cu).
+bool decode_pair_supported(const Shape& sh);
+DecodePlan decode_pair_plan(const Shape& sh);
+cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
+                               const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
+                               float* partials, cudaStream_t st);
 
 // dst[i] = src[i] + 1 for i < n (context length after one appended token).
 cudaError_t launch_add_one(const int32_t* src, int32_t* dst, int n, cudaStream_t st);

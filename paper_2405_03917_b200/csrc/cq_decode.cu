@@ -32,18 +32,12 @@
 // directly one register of an m16n8k16 A fragment: an MMA against an all-ones B matrix
 // sums the quad's lookups (all groups of a token) in fp32 and leaves the token's score in
 // every lane of the quad, which is exactly where the V-side bin updates need it.
-#include "cq_common.cuh"
+#include "cq_decode_util.cuh"
 
 namespace cq {
 
 namespace {
 
-constexpr int kRows = 256;            // code values
-constexpr int kRowBytes = 256;        // bytes per table row
-constexpr int kUnitBits = 27;         // weight of the running-maximum token: (2^26, 2^27]
-constexpr int kMaxWeightBits = 30;    // a score may exceed the unit exponent by at most this
-constexpr unsigned int kBinLimit256 = 16000000u;   // bins stay below 2^32: bound on their sum, in units of 256
-constexpr int kUnset = INT_MIN;                    // no score seen yet
 
 template <int G, int R>
 struct Cfg {
@@ -125,41 +119,6 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= 128, "control block");
 
-__device__ __forceinline__ int enc_float(float f)
-{
-    const int i = __float_as_int(f);
-    return i ^ ((i >> 31) & 0x7fffffff);
-}
-__device__ __forceinline__ float dec_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
-
-__device__ __forceinline__ uint4 ldg_codes(const uint4* p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-
-// Barrier 1 of the CTA, for the coarsening events: warps reach it from different places of the
-// code (bar.sync counts arrivals per barrier, whatever instruction they come from).
-__device__ __forceinline__ void event_barrier(int n_threads)
-{
-    asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory");
-}
-
-// 2^d for an integer d; 0 below the normal range, saturates at 2^127
-__device__ __forceinline__ float pow2i(int d)
-{
-    d = d > 127 ? 127 : d;
-    return d < -126 ? 0.f : __int_as_float((127 + d) << 23);
-}
-
-__device__ __forceinline__ float ex2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 
 // D = A * ones (+ C): sums, per fragment row, the 16 halves the quad holds for that row.
 // Rows r (registers a0, a2) and r + 8 (a1, a3) carry two different tokens.
@@ -178,39 +137,6 @@ __device__ __forceinline__ void mma_rowsum_acc(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(ones), "r"(ones));
 }
 
-// One centroid into registers.  The asm statements keep the loads where the code puts them: the
-// units of a codebook are loaded one unit ahead of their use, not all at once.
-__device__ __forceinline__ float4 ldg_f4(const float* p)
-{
-    float4 v;
-    asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
-    return v;
-}
-// `wide`: an 8-channel centroid is one 32-byte load (the lanes of a warp then read one contiguous
-// KiB; two 16-byte loads at a 32-byte lane stride touch every sector twice).  Needs 32-byte
-// aligned codebooks, which the launcher checks.
-template <int kC>
-__device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC], bool wide)
-{
-    static_assert(kC == 2 || kC == 4 || kC == 8, "centroids of 2, 4 or 8 channels");
-    if (kC == 2) {
-        asm volatile("ld.global.nc.v2.f32 {%0,%1}, [%2];" : "=f"(cv[0]), "=f"(cv[1 % kC]) : "l"(p) : "memory");
-        return;
-    }
-    if (kC == 8 && wide) {
-        asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                     : "=f"(cv[0]), "=f"(cv[1]), "=f"(cv[2]), "=f"(cv[3]), "=f"(cv[4 % kC]), "=f"(cv[5 % kC]),
-                       "=f"(cv[6 % kC]), "=f"(cv[7 % kC])
-                     : "l"(p) : "memory");
-        return;
-    }
-    const float4 a = ldg_f4(p);
-    cv[0] = a.x; cv[1 % kC] = a.y; cv[2 % kC] = a.z; cv[3 % kC] = a.w;
-    if (kC == 8) {
-        const float4 b = ldg_f4(p + 4);
-        cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
-    }
-}
 
 // half2 (hi, lo) with hi + lo ~= v to about 22 bits: hi in the low half, lo in the high half
 __device__ __forceinline__ uint32_t pack_hi_lo(float v)
@@ -267,16 +193,6 @@ __device__ __forceinline__ float fold_channels(const float (&a)[kC], int lane)
     return v;
 }
 
-// byte `k` (0..15) of a 16-byte code word
-__device__ __forceinline__ uint32_t word32(const uint4& w, int k)
-{
-    return (k >> 2) == 0 ? w.x : (k >> 2) == 1 ? w.y : (k >> 2) == 2 ? w.z : w.w;
-}
-// table byte offset code*256 + lane_off for token k of a code word (lane_off < 256)
-__device__ __forceinline__ uint32_t row_index(const uint4& w, int k, uint32_t lane_off)
-{
-    return __byte_perm(word32(w, k), lane_off, 0x5504u | ((uint32_t)(k & 3) << 4));
-}
 
 template <int G, int R, bool kShared>
 __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
@@ -1337,12 +1253,22 @@ bool decode_tuned_supported(const Shape& sh)
     return sh.G == 16 || sh.G == 32 || sh.G == 64;      // any number of query heads per KV head
 }
 
-int decode_tuned_parts(const Shape& sh) { return plan_dispatch(sh).n_parts; }
+int decode_tuned_parts(const Shape& sh)
+{
+    if (decode_pair_supported(sh)) return decode_pair_plan(sh).n_parts;
+    return plan_dispatch(sh).n_parts;
+}
 
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh, float* out,
                                 float* partials, cudaStream_t st)
 {
+    if (decode_pair_supported(sh)) {
+        const DecodePlan pp = decode_pair_plan(sh);
+        const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st);
+        if (ep != cudaSuccess) return ep;
+        return launch_merge(partials, pp.n_parts, sh, out, st);
+    }
     const Plan pl = plan_dispatch(sh);
     if (pl.chunk <= 0) return cudaErrorNotSupported;
     cudaError_t e = cudaErrorNotSupported;

@@ -1,0 +1,807 @@
+// Decode attention over CQ-8c8b codes for KV heads shared by four query heads (head_dim 128,
+// 16 groups of 8 channels, one byte per code): the kernel for grouped-query attention.
+//
+// Same re-association of Eq. 1 of the paper (K and V replaced by their CQ reconstructions,
+// Section 3.2) as decode_tuned_kernel:
+//   LUT[h][g][j]  = scale*log2(e) * <q_h,g , Ck[g][j]>
+//   s_t[h]        = sum_g LUT[h][g][kcode[t][g]]
+//   w_t[h]        = round(2^(s_t[h] - e_h))                      integer weight, unit 2^e_h
+//   bins[h][g][j] += w_t[h]   for j = vcode[t][g]
+//   acc[h][g*8+i] = sum_j bins[h][g][j] * Cv[g][j][i],  l[h] = sum_j bins[h][0][j]
+// Measured on sm_100a, what limits this path with four heads per KV head is the number of warp
+// instructions issued per token (the instruction issue slots of the four schedulers of an SM),
+// before the shared-memory pipe and long before HBM.  The kernel is built around that:
+//
+// * K side, four query heads per lookup.  Per (head, group) the smallest entry is taken out
+//   (softmax does not see a constant added to every score of a head) and the rest is stored as a
+//   16-bit fixed-point number in units of delta_h = (largest entry range of the head's groups) /
+//   65535.  A 32-bit word holds the entries of heads 2i and 2i+1 and the words of the two head
+//   pairs of a (code value, group) are neighbours, so ONE 64-bit lookup serves the four heads: 16
+//   lookup instructions per token instead of 64.  A looked-up word is one register of an
+//   m16n8k32 u8 A fragment; the B operand selects byte position n mod 4 into column n, so the
+//   integer MMA returns, exactly, the sums of the low bytes and of the high bytes of one head in
+//   the two accumulator columns of a lane: lanes 0 and 2 of a quad get the first head of a
+//   pair, lanes 1 and 3 the second.  score = low + 256 * high, an exact integer.
+// * A lane therefore holds the scores of its quad's tokens for TWO heads (one of each pair),
+//   turns them into weights itself and adds them to those heads' bins for 8 of the 16 groups, one
+//   index computation per two adds; no weight crosses lanes.
+// * Tables of 32 KiB (K) + 64 KiB (bins) let two CTAs share an SM, so one CTA's table build and
+//   bins x centroids product overlap the other's main loop.
+// * Code words reach the lanes through shared memory: a warp's four blocks are 1 KiB of
+//   contiguous codes per tensor, which one bulk asynchronous copy (no tensor map, no multicast)
+//   puts into the warp's staging tile while the previous tile is in use; the lanes then take their
+//   8-byte half words with 64-bit loads.  (Direct 16-byte global loads of this access pattern
+//   were measured 10 % slower.)
+//
+// Lane roles: lane = (r, p) = (lane / 4, lane % 4).  Quad r owns the tokens 8 (r % 2) ... + 7 of
+// block r / 2 of the warp's four 16-token blocks.  With hb = p % 2 and pu = p / 2:
+//   K row j (128 bytes): bytes 8 g ... 8 g + 7 = (pair 0 word, pair 1 word) of group g.  The
+//     lane's m-th K code word: group 4 ((r ^ m) % 4) + p  (16 lanes, 16 groups: distinct banks).
+//   bins row j (256 bytes): word 32 (h / 2) + 16 (h % 2) + g.  The lane serves heads hb and
+//     2 + hb; its m-th V code word: group 8 pu + ((r + 4 pu) % 8 ^ m), so that for every m the 32
+//     lanes touch 32 distinct banks (and the 64-bit reads of the staging tile do not collide).
+//   The eight bins offsets of a lane are bytes of two registers, and one PRMT builds
+//   code * 256 + offset from a code byte and an offset byte (every offset is below 128, so the
+//   byte's replicated sign supplies the zero upper bytes).
+//
+// The integer weight units, the reservation of bin room and the coarsening events are those of
+// decode_tuned_kernel (see there).  In the usual case (no request pending, the lane's scores fit
+// the unit, its sum is small and the total is far from its limit) a lane decides by itself, from
+// a control record it read at the top of the iteration, and adds its sum to the head's total
+// without waiting for the old value; no value crosses lanes.  Everything else - the first tokens
+// of a head, a large sum, a full total, a pending request - takes reserve_slow(), where the
+// sixteen lanes of a warp with the same hb act as one group.  That code and the coarsening are
+// kept out of line: inlined into the loop they cost a quarter of the kernel's time in
+// instruction fetches alone.
+#include <utility>
+
+#include "cq_bulk_copy.cuh"
+#include "cq_decode_util.cuh"
+
+namespace cq {
+
+namespace {
+
+struct PairCfg {
+    static constexpr int kHeads = 4;                  // query heads per CTA
+    static constexpr int kWarps = 8, kThreads = kWarps * 32;
+    static constexpr int kBlocksPerIter = 4;          // 16-token blocks per warp iteration
+    static constexpr int kRoundTokens = kWarps * kBlocksPerIter * 16;
+    static constexpr int kKRowBytes = 128, kVRowBytes = 256;
+    static constexpr int kKBytes = kRows * kKRowBytes;          // 32 KiB
+    static constexpr int kVOffset = kKBytes;
+    static constexpr int kVBytes = kRows * kVRowBytes;          // 64 KiB; also the fp32 staging area of the table build
+    static constexpr int kCtlOffset = kVOffset + kVBytes;
+    static constexpr int kCtlBytes = 512;
+    static constexpr int kStageOffset = kCtlOffset + kCtlBytes; // per warp: K tile (4 blocks x 256 bytes), then V tile
+    static constexpr int kTileBytes = kBlocksPerIter * 16 * 16;
+    static constexpr int kSmemBytes = kStageOffset + kWarps * 2 * kTileBytes;   // 112.5 KiB: two CTAs per SM
+    static constexpr int kQOffset = 0;                          // scaled query [4][128] fp32, in the K table's place until the table is written
+    static constexpr int kLog2Groups = 3;             // log2 of the warps that add to a head's bins per round
+};
+
+struct PairCtl {
+    // Per query head, one 16-byte record that a lane reads with one load at the top of an iteration:
+    // e_cur = log2 of the weight unit of the head's bins (kUnset before the first tokens); total = bound,
+    // in units of 256, on the weights added since the last coarsening; want_hint = copy of `want`.
+    struct Head { int e_cur; unsigned int total; int want_hint; int pad; } head[4];
+    int req_ref[4];            // coarsening request: largest score exponent the requesters need to represent
+    int req_need[4];           // coarsening request: log2 bound of the largest round sum of one lane group
+    int want;                  // non-zero: a warp asks every warp to stop adding and coarsen
+    int range_bits[4];         // per head: largest (max - min) over its groups' table entries, as float bits
+    float offset[4];           // per head: sum over groups of the entry taken out of each group
+    float mins[4][16];         // per (head, group): smallest table entry
+    uint64_t bar[PairCfg::kWarps];      // per warp: arrival of its code tiles (K and V of one iteration)
+};
+static_assert(sizeof(PairCtl) <= PairCfg::kCtlBytes, "control block");
+
+// D = A * B + C for u8 operands: A holds looked-up table words (four bytes = four k slots), B
+// selects byte position n % 4 into column n, so that columns 2p and 2p + 1 of lane p are the sums
+// of the low and of the high bytes of one head.  Rows r (a0, a2) and r + 8 (a1, a3) are two tokens.
+__device__ __forceinline__ void mma_bytesum_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b, int c_low)
+{
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%8}, {%9,%10,%9,%10};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b), "r"(c_low), "r"(0));
+}
+__device__ __forceinline__ void mma_bytesum_acc(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b)
+{
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%8}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b));
+}
+
+// byte k (0..7) of an 8-byte code half word
+__device__ __forceinline__ uint32_t word32(const uint2& w, int k) { return (k >> 2) == 0 ? w.x : w.y; }
+// code * 128 + lane_off as one multiply-add (byte offset into the K table)
+__device__ __forceinline__ uint32_t k_row_index(const uint2& w, int k, uint32_t lane_off)
+{
+    const uint32_t code = __byte_perm(word32(w, k), 0u, 0x4440u | (uint32_t)(k & 3));
+    uint32_t idx;
+    asm("mad.lo.u32 %0, %1, 128, %2;" : "=r"(idx) : "r"(code), "r"(lane_off));
+    return idx;
+}
+template <typename F, int... I>
+__device__ __forceinline__ void static_for_impl(F&& f, std::integer_sequence<int, I...>) { (f(std::integral_constant<int, I>{}), ...); }
+// f(integral_constant<int, 0>) ... f(integral_constant<int, N - 1>): a loop whose index is a compile-time constant
+template <int N, typename F>
+__device__ __forceinline__ void static_for(F&& f) { static_for_impl(f, std::make_integer_sequence<int, N>{}); }
+
+// code * 256 + (byte m % 4 of `offs`): byte offset into the bins.  Result bytes: the offset byte, the code
+// byte k of the half word, and twice the replicated sign of the offset byte (zero: offsets are below 128).
+template <int K, int M>
+__device__ __forceinline__ uint32_t v_row_index(const uint2& w, uint32_t offs)
+{
+    // (prmt in PTX form: the fourth bit of a selector digit asks for the byte's replicated sign)
+    constexpr uint32_t ob = 4u + (uint32_t)(M & 3);
+    constexpr uint32_t sel = ob | ((uint32_t)(K & 3) << 4) | ((ob | 8u) << 8) | ((ob | 8u) << 12);
+    uint32_t idx;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(idx) : "r"(K < 4 ? w.x : w.y), "r"(offs), "n"(sel));
+    return idx;
+}
+
+// Coarsening event (see decode_tuned_kernel): entered by every thread of the CTA, right after the
+// event's first barrier.  Per head: new unit from the published requests, bins shifted right with
+// rounding, total rescaled.  Out of line on purpose.
+__device__ __noinline__ void coarsen_bins(uint8_t* smem, PairCtl* ctl)
+{
+    using C = PairCfg;
+    constexpr int R = C::kHeads;
+    int shift[R], e_next[R];
+    unsigned int t_next[R];
+    bool any_shift = false;
+#pragma unroll
+    for (int h = 0; h < R; ++h) {
+        const int e = ctl->head[h].e_cur, cmr = ctl->req_ref[h], need = ctl->req_need[h];
+        const unsigned int tot = ctl->head[h].total;
+        int e_new = e;
+        shift[h] = 0;
+        t_next[h] = tot;
+        if (cmr != kUnset) {
+            // range: the largest score must fit; room: one round of every warp takes at most half of 2^32
+            if (e == kUnset || cmr - e > kMaxWeightBits) e_new = cmr - kUnitBits;
+            const int room = need + C::kLog2Groups - 31;
+            if (need != kUnset && room > e_new) e_new = room;
+        }
+        if (e != kUnset) {
+            // the weights already in the bins keep a sixteenth of the range at most after an event
+            for (int tries = 0; tries < 24; ++tries) {              // 2 bits per try: bounded
+                const int k = e_new - e;
+                if ((k >= 32 ? 0u : tot >> k) < kBinLimit256 / 16u) break;
+                e_new += 2;
+            }
+            shift[h] = e_new - e;
+            t_next[h] = (shift[h] >= 32 ? 0u : tot >> shift[h]) + 1u;
+            any_shift = any_shift || shift[h] > 0;
+        }
+        e_next[h] = e_new;
+    }
+    if (any_shift) {
+        for (int i = threadIdx.x; i < C::kVBytes / 4; i += C::kThreads) {
+            const int word = i & 63;                                // word 32 (h / 2) + 16 (h % 2) + g of a bins row
+            const int hw_ = 2 * (word >> 5) + ((word >> 4) & 1);
+            int k = shift[0];
+#pragma unroll
+            for (int h = 1; h < R; ++h) k = hw_ == h ? shift[h] : k;
+            if (k > 0) {
+                uint32_t* bp = reinterpret_cast<uint32_t*>(smem + C::kVOffset) + i;
+                const uint32_t v = *bp;
+                *bp = k >= 32 ? 0u : (v >> k) + ((v >> (k - 1)) & 1u);
+            }
+        }
+    }
+    event_barrier(C::kThreads);                         // every thread has read the request and rescaled its bins
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int h = 0; h < R; ++h) {
+            ctl->head[h].e_cur = e_next[h];
+            ctl->head[h].total = t_next[h];
+            ctl->head[h].want_hint = 0;
+            ctl->req_ref[h] = kUnset;
+            ctl->req_need[h] = kUnset;
+        }
+        ctl->want = 0;
+    }
+    event_barrier(C::kThreads);                         // the new state is visible
+}
+
+// A lane whose weights (for one head, one iteration) sum to less than kFastLane256 units of 256 adds them to
+// the head's total without asking, after a look at the total as it stood at the top of its iteration.  A warp
+// adds at most 8 such sums per head and iteration (2^19).  Once the total has passed the soft limit
+// kBinLimit256 - 2^19 - kFastSlack256, every later look sends its warp to reserve_slow; until then each of
+// the 8 warps can still be inside one iteration that looked earlier, plus the add that crossed the limit: at
+// most 9 * 2^19 = kFastSlack256 on top, so the total stays below kBinLimit256 and no bin can wrap.
+constexpr unsigned int kFastLane256 = 1u << 16;
+constexpr unsigned int kFastSlack256 = 9u << 19;
+
+// Room for a warp's weights when the usual case does not apply (entered by the whole warp).  The
+// sixteen lanes with the same hb = lane % 2 form a group that serves heads hb and 2 + hb.  Per
+// head: ref_lane = the lane's reference exponent (kUnset without tokens), z_lane = the sum of its
+// weights 2^(score - ref_lane).  The group reserves the sum of its weights on the head's total
+// with the old value in hand, or asks for a coarser unit and joins the event.  Bounded: every
+// event coarsens the refused head by at least two bits.  Returns the units to use for the two heads.
+// (Scalars in, scalars out: nothing the caller's loop keeps in registers is forced into memory.)
+__device__ __noinline__ int2 reserve_slow(uint8_t* smem, PairCtl* ctl, int ref_lane0, int ref_lane1, float z_lane0, float z_lane1)
+{
+    const int ref_lane[2] = {ref_lane0, ref_lane1};
+    const float z_lane[2] = {z_lane0, z_lane1};
+    int eu[2] = {kUnset, kUnset};
+    using C = PairCfg;
+    const int lane = threadIdx.x & 31, hb = lane & 1;
+    const unsigned grp_mask = hb ? 0xaaaaaaaau : 0x55555555u;
+    const bool grp_leader = lane == hb;
+    int ref[2];
+    float zsum[2];
+    bool any_tokens = false;                                            // the same in every lane of the warp
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        ref[u] = __reduce_max_sync(grp_mask, ref_lane[u]);
+        any_tokens = ref[u] != kUnset;
+        const float zrel = ref_lane[u] == kUnset ? 0.f : z_lane[u] * pow2i(ref_lane[u] - ref[u]);
+        // sum over the group in 2^-16 steps, rounded up (the lanes p and p + 2 of a quad hold the same
+        // tokens, so the group's sum counts every token twice)
+        zsum[u] = (float)__reduce_add_sync(grp_mask, __float2uint_ru(zrel * 65536.f)) * (0.5f / 65536.f);
+    }
+    for (int attempt = 0; attempt < 64; ++attempt) {
+        if (*reinterpret_cast<volatile int*>(&ctl->want) != 0) {
+            // someone needs a coarser unit: tell the event what this group will need, then join it
+            if (grp_leader) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    if (ref[u] != kUnset) {
+                        atomicMax(&ctl->req_ref[2 * u + hb], ref[u]);
+                        atomicMax(&ctl->req_need[2 * u + hb], ref[u] + ilogbf(fmaxf(zsum[u], 1e-30f)) + 1);
+                    }
+            }
+            event_barrier(C::kThreads);
+            coarsen_bins(smem, ctl);
+            continue;
+        }
+        if (!any_tokens) break;
+        bool ok = true;
+        unsigned int mine[2] = {0u, 0u};
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int h = 2 * u + hb;
+            eu[u] = *reinterpret_cast<volatile int*>(&ctl->head[h].e_cur);
+            if (eu[u] == kUnset || ref[u] - eu[u] > kMaxWeightBits) { ok = false; continue; }
+            // this group's weights in the current unit, rounded up, in units of 256
+            const float cw = (zsum[u] * pow2i(ref[u] - eu[u]) * 1.00002f + (float)(16 * C::kBlocksPerIter)) * (1.f / 256.f) + 1.f;
+            const unsigned int ci = (unsigned int)fminf(cw, 6.7e7f);
+            unsigned int old = 0u;
+            if (grp_leader) old = atomicAdd(&ctl->head[h].total, ci);
+            old = __shfl_sync(grp_mask, old, hb);
+            mine[u] = ci;
+            // (the sums that other warps add without asking are covered by kFastSlack256)
+            if (old + ci + kFastSlack256 >= kBinLimit256) ok = false;
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) break;
+        // give the reservations back, publish what is needed, raise the request, join the event
+        if (grp_leader) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int h = 2 * u + hb;
+                if (mine[u]) atomicSub(&ctl->head[h].total, mine[u]);
+                atomicMax(&ctl->req_ref[h], ref[u]);
+                atomicMax(&ctl->req_need[h], ref[u] + ilogbf(fmaxf(zsum[u], 1e-30f)) + 1);
+            }
+            atomicExch(&ctl->want, 1);
+#pragma unroll
+            for (int h = 0; h < C::kHeads; ++h) atomicExch(&ctl->head[h].want_hint, 1);
+        }
+        event_barrier(C::kThreads);
+        coarsen_bins(smem, ctl);
+    }
+    return make_int2(eu[0], eu[1]);
+}
+
+__global__ void __launch_bounds__(PairCfg::kThreads, 2)
+decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
+                   const float* __restrict__ kcb, const float* __restrict__ vcb,
+                   const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
+                   int tail_first, int cb_aligned32, float* __restrict__ partials)
+{
+    using C = PairCfg;
+    constexpr int R = C::kHeads;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    PairCtl* ctl = reinterpret_cast<PairCtl*>(smem + C::kCtlOffset);
+    float* qs = reinterpret_cast<float*>(smem + C::kQOffset);
+    float* stage = reinterpret_cast<float*>(smem + C::kVOffset);       // [4][16][256] fp32 during the table build
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int p = lane & 3, r = lane >> 2;
+    const int hb = p & 1, pu = p >> 1;
+
+    // Work item: (context part, sequence, group of four query heads).  Items before tail_first take
+    // their whole context in one CTA; each later item is spread over n_parts CTAs of chunk_tokens
+    // (see the launch plan).
+    const int n_head_groups = sh.n_q_heads / R;
+    const int kv_share = sh.R / R;                    // CTAs (of four query heads) that share one KV head
+    const int n_items = (int)(n_head_groups * sh.n_seq);
+    int item = blockIdx.x % n_items;
+    int part = (int)(blockIdx.x / n_items);
+    bool whole = false;
+    if (tail_first >= 0) {
+        whole = (int)blockIdx.x < tail_first;
+        item = whole ? blockIdx.x : tail_first + (blockIdx.x - tail_first) / n_parts;
+        part = whole ? 0 : (blockIdx.x - tail_first) % n_parts;
+    }
+    const int head_group = item % n_head_groups;
+    const int hkv = head_group / kv_share;
+    const int64_t s = item / n_head_groups;
+
+    int64_t n = seq_lens[s];
+    n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
+    const int64_t t_begin = (int64_t)part * chunk_tokens;
+    const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
+    const int stride = partial_stride(128);
+    float* part_base = partials + ((s * sh.n_q_heads + (int64_t)head_group * R) * n_parts + part) * stride;
+    // partial of query head head_group*4 + h: part_base + h * n_parts * stride
+    if (whole)          // the other partial slots of this item hold the neutral element of the merge
+        for (int i = threadIdx.x; i < R * (n_parts - 1) * stride; i += C::kThreads) {
+            const int h = i / ((n_parts - 1) * stride), d = i % ((n_parts - 1) * stride);
+            part_base[(int64_t)h * n_parts * stride + stride + d] = d % stride == 0 ? -INFINITY : 0.f;
+        }
+    if (t_begin >= t_end) {
+        for (int i = threadIdx.x; i < R * stride; i += C::kThreads) {
+            const int h = i / stride, d = i % stride;
+            part_base[(int64_t)h * n_parts * stride + d] = d == 0 ? -INFINITY : 0.f;
+        }
+        return;
+    }
+
+    const int64_t blk0 = t_begin / kTokenBlock;
+    const int n_tok = (int)(t_end - blk0 * kTokenBlock);                   // tokens of this CTA, counted from its first block
+    const int n_iters = (n_tok + C::kRoundTokens - 1) / C::kRoundTokens;
+    const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, blk0, 0);
+    const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, blk0, 0);
+
+    // Codebooks are read in units of 4 x 32 centroids (32 registers per lane): a warp owns two
+    // groups, its lanes walk the code values, the next unit is loaded while the current one is used.
+    constexpr int kJb = 4;
+    constexpr int kUnits = 2 * (kRows / 32 / kJb);          // 4 units per warp
+    auto load_unit = [&](float (&cv)[kJb][8], const float* cb, int u) {
+        const int g = warp * 2 + (u >> 1);
+        const float* cg = cb + (((int64_t)hkv * 16 + g) * kRows + (u & 1) * (kJb * 32) + lane) * 8;
+#pragma unroll
+        for (int jb = 0; jb < kJb; ++jb) load_centroid<8>(cg + jb * 32 * 8, cv[jb], cb_aligned32 != 0);
+    };
+    float cva[kJb][8], cvb[kJb][8];
+    load_unit(cva, kcb, 0);
+
+    // table offsets of this lane's code words (bytes inside a K row / inside plane 0 of a bins row)
+    const uint32_t koff0 = 8u * (4 * (r & 3) + p);                     // m-th K code word: koff0 ^ (32 m)
+    const int vx = (r + 4 * pu) & 7;
+    uint32_t voffs[2] = {0u, 0u};                                        // m-th V code word: byte m % 4 of voffs[m / 4]
+#pragma unroll
+    for (int m = 0; m < 8; ++m) voffs[m >> 2] |= (4u * (16 * hb + 8 * pu + (vx ^ m))) << (8 * (m & 3));
+    const uint32_t bsel = 1u << (8 * (r & 3));                          // B fragment: column n = lane / 4 takes byte n % 4
+
+    // Code tiles.  Tile `it` of this warp = its four blocks of iteration `it`, 1 KiB of contiguous
+    // codes per tensor (less at the end of the chunk; blocks past the end are not copied and keep
+    // whatever the tile held: any byte is a valid table row, and those tokens are masked).  Lane 0
+    // asks for the next tile as soon as every lane has taken its words of the current one.
+    uint8_t* ktile = smem + C::kStageOffset + warp * 2 * C::kTileBytes;
+    uint8_t* vtile = ktile + C::kTileBytes;
+    // this lane's half word of its first code word in the K tile and in the V tile; word m is 64 m / 16 m bytes
+    // away in the XOR sense (the tiles are 128-byte aligned)
+    const uint8_t* my_ktile = ktile + (r >> 1) * 256 + 8 * (r & 1) + 2 * koff0;
+    const uint8_t* my_vtile = vtile + (r >> 1) * 256 + 8 * (r & 1) + 16 * (8 * pu + vx);
+    uint64_t* tbar = &ctl->bar[warp];
+    uint32_t tphase = 0u;
+    bool bulk = true;                       // false after a wait that gave up: plain loads from then on
+    bool t_out = false;                     // copies into the tiles have been requested and not yet awaited
+    const int n_blocks_cta = (n_tok + kTokenBlock - 1) / kTokenBlock;   // blocks holding a valid token
+    // bytes of this warp's tile of iteration `it` (per tensor)
+    auto tile_bytes = [&](int it) -> uint32_t {
+        int nb = n_blocks_cta - (it * C::kWarps + warp) * C::kBlocksPerIter;
+        nb = nb < 0 ? 0 : (nb > C::kBlocksPerIter ? C::kBlocksPerIter : nb);
+        return (uint32_t)nb * 256u;
+    };
+    auto request_tiles = [&](int it) {      // lane 0 only
+        const uint32_t bytes = tile_bytes(it);
+        if (bytes == 0u) return;
+        const int64_t off = (int64_t)(it * C::kWarps + warp) * (C::kBlocksPerIter * 256);
+        fence_async_smem();
+        mbar_expect_tx(tbar, 2u * bytes);
+        bulk_copy_g2s(ktile, kbase + off, bytes, tbar);
+        bulk_copy_g2s(vtile, vbase + off, bytes, tbar);
+    };
+    uint2 kw[4], vw[8];
+    // the words of tile `it` into registers; then the tiles are free for iteration it + 1
+    auto take_tiles = [&](int it) {
+        bool have = false;
+        const uint32_t bytes = tile_bytes(it);
+        if (bulk && bytes != 0u) {
+            have = mbar_wait(tbar, tphase);
+            have = __all_sync(0xffffffffu, have);
+            if (have) { tphase ^= 1u; t_out = false; } else bulk = false;
+        }
+        if (have || bytes == 0u) {
+#pragma unroll
+            for (int m = 0; m < 4; ++m)
+                kw[m] = *reinterpret_cast<const uint2*>(smem + ((uint32_t)(my_ktile - smem) ^ (64u * m)));
+#pragma unroll
+            for (int m = 0; m < 8; ++m)
+                vw[m] = *reinterpret_cast<const uint2*>(smem + ((uint32_t)(my_vtile - smem) ^ (16u * m)));
+        } else {
+            const int64_t off = (int64_t)((it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1)) * 256 + 8 * (r & 1);
+            const bool in = ((it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1)) < n_blocks_cta;
+#pragma unroll
+            for (int m = 0; m < 4; ++m)
+                kw[m] = in ? __ldg(reinterpret_cast<const uint2*>(kbase + off + 2u * (koff0 ^ (32u * m)))) : make_uint2(0u, 0u);
+#pragma unroll
+            for (int m = 0; m < 8; ++m)
+                vw[m] = in ? __ldg(reinterpret_cast<const uint2*>(vbase + off + 16u * (8 * pu + (vx ^ m)))) : make_uint2(0u, 0u);
+        }
+        __syncwarp();
+        if (bulk && it + 1 < n_iters && tile_bytes(it + 1) != 0u) {
+            t_out = true;
+            if (lane == 0) request_tiles(it + 1);
+        }
+    };
+
+    // ---------------------------------------------------------------- set-up: query, control block
+    if (threadIdx.x < 4) {
+        ctl->head[threadIdx.x].e_cur = kUnset;
+        ctl->head[threadIdx.x].total = 0u;
+        ctl->head[threadIdx.x].want_hint = 0;
+        ctl->req_ref[threadIdx.x] = kUnset;
+        ctl->req_need[threadIdx.x] = kUnset;
+        ctl->range_bits[threadIdx.x] = 0;
+    }
+    if (threadIdx.x == 4) ctl->want = 0;
+    if (threadIdx.x == 5) {
+        for (int w = 0; w < C::kWarps; ++w) mbar_init(&ctl->bar[w], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
+        qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)head_group * R) * 128 + i]) * scale_log2e;
+    __syncthreads();
+    // the first code tiles travel during the table build
+    t_out = tile_bytes(0) != 0u;
+    if (lane == 0) request_tiles(0);
+
+    // Table build, first pass: fp32 entries into the staging area (the later bins), entry (h, g, j)
+    // at word (h*16 + g)*256 + (j ^ (16*(h/2) + g)): a warp writing 32 consecutive j of one (h, g)
+    // and a warp reading one j of the 32 (h/2, g) both touch 32 distinct banks.  Per (head, group)
+    // the smallest and the largest entry are kept.
+    {
+        float qreg[R][8];
+        float vmin[R], vmax[R];
+        auto build_unit = [&](const float (&cv)[kJb][8], int u) {
+            const int g = warp * 2 + (u >> 1);
+            if ((u & 1) == 0) {
+#pragma unroll
+                for (int h = 0; h < R; ++h) {
+                    vmin[h] = INFINITY;
+                    vmax[h] = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) qreg[h][i] = qs[h * 128 + g * 8 + i];
+                }
+            }
+#pragma unroll
+            for (int jb = 0; jb < kJb; ++jb) {
+                const int j = (u & 1) * (kJb * 32) + jb * 32 + lane;
+#pragma unroll
+                for (int h = 0; h < R; ++h) {
+                    float dot = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dot = fmaf(qreg[h][i], cv[jb][i], dot);
+                    vmin[h] = fminf(vmin[h], dot);
+                    vmax[h] = fmaxf(vmax[h], dot);
+                    stage[(h * 16 + g) * kRows + (j ^ (16 * (h >> 1) + g))] = dot;
+                }
+            }
+            if ((u & 1) == 1) {
+#pragma unroll
+                for (int h = 0; h < R; ++h) {
+                    const float mn = dec_float(__reduce_min_sync(0xffffffffu, enc_float(vmin[h])));
+                    const float mx = dec_float(__reduce_max_sync(0xffffffffu, enc_float(vmax[h])));
+                    if (lane == 0) {
+                        ctl->mins[h][g] = mn;
+                        const float range = mx - mn;                     // >= 0 (or NaN / inf for non-finite inputs)
+                        atomicMax(&ctl->range_bits[h], __float_as_int(range >= 0.f ? range : 0.f));
+                    }
+                }
+            }
+        };
+#pragma unroll 1
+        for (int u = 0; u < kUnits; u += 2) {
+            load_unit(cvb, kcb, u + 1);
+            build_unit(cva, u);
+            if (u + 2 < kUnits) load_unit(cva, kcb, u + 2);
+            build_unit(cvb, u + 1);
+        }
+    }
+    __syncthreads();
+
+    // Second pass: lane = (head pair hp = lane / 16, group g = lane % 16) writes word 2 g + hp of the
+    // rows warp*32 ... +31: a row's 32 words, one per lane.
+    {
+        const int hp = lane >> 4, g = lane & 15;
+        const float r0 = __int_as_float(ctl->range_bits[2 * hp]), r1 = __int_as_float(ctl->range_bits[2 * hp + 1]);
+        const float inv0 = r0 > 1e-30f ? 65535.f / r0 : 0.f, inv1 = r1 > 1e-30f ? 65535.f / r1 : 0.f;
+        const float m0 = ctl->mins[2 * hp][g], m1 = ctl->mins[2 * hp + 1][g];
+        const float* s0 = stage + ((2 * hp) * 16 + g) * kRows;
+        const float* s1 = stage + ((2 * hp + 1) * 16 + g) * kRows;
+#pragma unroll 8
+        for (int i = 0; i < kRows / C::kWarps; ++i) {
+            const int j = warp * (kRows / C::kWarps) + i;
+            const float u0 = fminf(rintf((s0[j ^ lane] - m0) * inv0), 65535.f);
+            const float u1 = fminf(rintf((s1[j ^ lane] - m1) * inv1), 65535.f);
+            *reinterpret_cast<uint32_t*>(smem + j * C::kKRowBytes + (2 * g + hp) * 4) =
+                (uint32_t)fmaxf(u0, 0.f) | ((uint32_t)fmaxf(u1, 0.f) << 16);
+        }
+        if (threadIdx.x < R) {
+            float o = 0.f;
+            for (int gg = 0; gg < 16; ++gg) o += ctl->mins[threadIdx.x][gg];
+            ctl->offset[threadIdx.x] = o;
+        }
+    }
+    __syncthreads();
+    // bins start at zero
+    for (int i = threadIdx.x; i < C::kVBytes / 16; i += C::kThreads)
+        *reinterpret_cast<uint4*>(smem + C::kVOffset + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+
+    // ---------------------------------------------------------------- main loop over the chunk
+    // This lane's heads: hb (pair 0) and 2 + hb (pair 1); index u = 0, 1 below.
+    float delta[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const float rng = __int_as_float(ctl->range_bits[2 * u + hb]);
+        delta[u] = rng > 1e-30f ? rng * (1.f / 65535.f) : 0.f;
+    }
+    const uint32_t head_rec = smem_addr(&ctl->head[hb]);                // record of head hb; head 2 + hb is 32 bytes on
+
+    for (int it = 0; it < n_iters; ++it) {
+        take_tiles(it);
+        // the heads' control records as they stand now (used after the K side)
+        int4 seen[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            asm volatile("ld.volatile.shared.v4.s32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(seen[u].x), "=r"(seen[u].y), "=r"(seen[u].z), "=r"(seen[u].w) : "r"(head_rec + 32u * u));
+
+        // K side: the scores of this quad's eight tokens for the lane's two heads, as exact integers
+        // held in floats.  One 64-bit lookup per (token, code word) serves both head pairs.
+        float sc[2][8];
+        uint2 a[2][2][4];                        // [buffer][token][code word]
+        auto lookups = [&](uint2 (&dst)[2][4], int k0) {
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+                for (int m = 0; m < 4; ++m)
+                    dst[kk][m] = *reinterpret_cast<const uint2*>(smem + k_row_index(kw[m], k0 + kk, koff0 ^ (32u * m)));
+        };
+        // One MMA chain per token: fragment row r takes the words of pair 0, row r + 8 the words of pair 1
+        // (the two halves of a 64-bit lookup are neighbours in the A fragment), two code words per MMA.
+        auto scores = [&](const uint2 (&src)[2][4], int k0) {
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+                int d[4];
+                // columns start at 2^23 as float bits (low sums) and 0 (high sums): low + 256 * high < 2^21, so
+                // the float with these bits, minus 2^23, is the integer score, exactly
+                mma_bytesum_first(d, src[kk][0].x, src[kk][0].y, src[kk][1].x, src[kk][1].y, bsel, 0x4b000000);
+                mma_bytesum_acc(d, src[kk][2].x, src[kk][2].y, src[kk][3].x, src[kk][3].y, bsel);
+                sc[0][k0 + kk] = __int_as_float(d[0] + (d[1] << 8)) - 8388608.f;
+                sc[1][k0 + kk] = __int_as_float(d[2] + (d[3] << 8)) - 8388608.f;
+            }
+        };
+        lookups(a[0], 0);
+        lookups(a[1], 2);
+        scores(a[0], 0);
+        lookups(a[0], 4);
+        scores(a[1], 2);
+        lookups(a[1], 6);
+        scores(a[0], 4);
+        scores(a[1], 6);
+
+        // tokens past the end of the context (only the warp that holds the ragged end pays)
+        const int tok0 = ((it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1)) * kTokenBlock + 8 * (r & 1);
+        const bool ragged = ((it * C::kWarps + warp) * C::kBlocksPerIter + C::kBlocksPerIter) * kTokenBlock > n_tok;
+        if (ragged) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (tok0 + k >= n_tok) sc[0][k] = sc[1][k] = -1.f;
+        }
+        // Per head, from this lane's own eight tokens: reference exponent ref = ceil(largest score),
+        // weights 2^(score - ref) <= 1 and their sum.  Usual case, decided from the records read at the
+        // top of the iteration: no request pending, the scores fit the unit, the sum is small and the
+        // total far from its limit -> the sum goes to the total without waiting for the old value.  (No
+        // event can have happened since the records were read: an event needs this warp.)
+        int ref[2], eu[2];
+        float y[2][8], zlane[2];
+        unsigned int ci[2];
+        bool fast = true, have = false;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            float mx = -1.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) mx = fmaxf(mx, sc[u][k]);
+            have = mx >= 0.f;                                           // this lane holds a token of the context
+            ref[u] = have ? (int)ceilf(mx * delta[u]) : kUnset;
+            const float fref = have ? (float)ref[u] : 0.f;
+            float z = 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                y[u][k] = ex2(fmaf(sc[u][k], delta[u], -fref));
+                z += y[u][k];
+            }
+            if (ragged) {
+                z = 0.f;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (sc[u][k] < 0.f) y[u][k] = 0.f;
+                    z += y[u][k];
+                }
+            }
+            zlane[u] = z;
+            eu[u] = seen[u].x;
+            ci[u] = 0u;
+            bool f = seen[u].z == 0 && eu[u] != kUnset;
+            if (f && have) {
+                f = ref[u] - eu[u] <= kMaxWeightBits;
+                // this lane's weights in the current unit, rounded up, in units of 256
+                const float cw = (z * pow2i(ref[u] - eu[u]) * 1.00002f + 8.f) * (1.f / 256.f) + 1.f;
+                ci[u] = (unsigned int)fminf(cw, 6.7e7f);
+                f = f && ci[u] < kFastLane256 && (unsigned int)seen[u].y + 8u * kFastLane256 + kFastSlack256 < kBinLimit256;
+            }
+            fast = fast && f;
+        }
+        if (__all_sync(0xffffffffu, fast)) {
+            if (have && pu == 0) {                   // (the lanes p and p + 2 of a quad hold the same tokens)
+                atomicAdd(&ctl->head[hb].total, ci[0]);
+                atomicAdd(&ctl->head[2 + hb].total, ci[1]);
+            }
+        } else {
+            const int2 e2 = reserve_slow(smem, ctl, ref[0], ref[1], zlane[0], zlane[1]);
+            eu[0] = e2.x;
+            eu[1] = e2.y;
+        }
+        if (!have) continue;
+
+        // V side: this lane's integer weights into the bins of its two heads, for its eight groups
+        const float f0 = pow2i(ref[0] - eu[0]), f1 = pow2i(ref[1] - eu[1]);   // powers of two <= 2^kMaxWeightBits
+        static_for<8>([&](auto kc_) {
+            constexpr int k = decltype(kc_)::value;
+            const uint32_t w0 = __float2uint_rn(y[0][k] * f0), w1 = __float2uint_rn(y[1][k] * f1);
+            static_for<8>([&](auto mc_) {
+                constexpr int m = decltype(mc_)::value;
+                unsigned int* bin = reinterpret_cast<unsigned int*>(smem + C::kVOffset + v_row_index<k, m>(vw[m], voffs[m >> 2]));
+                atomicAdd(bin, w0);
+                atomicAdd(bin + 32, w1);
+            });
+        });
+    }
+    // (after a wait that gave up, a requested copy may still be on its way: it must land before the CTA ends)
+    if (!bulk && t_out) mbar_wait(tbar, tphase);
+    // Warps that are done keep joining coarsening events until every warp is done.
+    for (int guard = 0; guard < 4096; ++guard) {
+        event_barrier(C::kThreads);
+        if (*reinterpret_cast<volatile int*>(&ctl->want) == 0) break;
+        coarsen_bins(smem, ctl);
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- epilogue: bins x V centroids
+    // Lane = (hb', g) reads words `lane` of both planes of row j (heads hb' and 2 + hb', group g): a
+    // conflict-free row read; the centroid (g, j) is one 32-byte load.  A warp takes 32 rows; the
+    // eight warps' partial sums meet in shared memory (the K table is no longer needed).
+    {
+        const int g = lane & 15;
+        float acc0[8], acc1[8], l0 = 0.f, l1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc0[i] = acc1[i] = 0.f;
+        const float* cg = vcb + (((int64_t)hkv * 16 + g) * kRows + warp * (kRows / C::kWarps)) * 8;
+        const uint8_t* brow = smem + C::kVOffset + warp * (kRows / C::kWarps) * C::kVRowBytes + lane * 4;
+#pragma unroll 1
+        for (int i0 = 0; i0 < kRows / C::kWarps; i0 += 4) {
+            float cv[4][8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) load_centroid<8>(cg + (i0 + i) * 8, cv[i], cb_aligned32 != 0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float b0 = (float)*reinterpret_cast<const uint32_t*>(brow + (i0 + i) * C::kVRowBytes);
+                const float b1 = (float)*reinterpret_cast<const uint32_t*>(brow + (i0 + i) * C::kVRowBytes + 128);
+                l0 += b0;
+                l1 += b1;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    acc0[c] = fmaf(b0, cv[i][c], acc0[c]);
+                    acc1[c] = fmaf(b1, cv[i][c], acc1[c]);
+                }
+            }
+        }
+        float* red = reinterpret_cast<float*>(smem);                      // [warp][18][32]
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            red[(warp * 18 + c) * 32 + lane] = acc0[c];
+            red[(warp * 18 + 8 + c) * 32 + lane] = acc1[c];
+        }
+        red[(warp * 18 + 16) * 32 + lane] = l0;
+        red[(warp * 18 + 17) * 32 + lane] = l1;
+        __syncthreads();
+        // 18 x 32 sums of eight terms: slot k < 16 of lane (hb', g) is channel g*8 + k%8 of head 2 (k/8) + hb';
+        // slots 16, 17 of the lanes with g = 0 are the normalisers (sum of the bins of group 0)
+        for (int o = threadIdx.x; o < 18 * 32; o += C::kThreads) {
+            const int slot = o >> 5, ln = o & 31;
+            float v = 0.f;
+#pragma unroll
+            for (int w = 0; w < C::kWarps; ++w) v += red[(w * 18 + slot) * 32 + ln];
+            const int hb2 = ln >> 4, g2 = ln & 15;
+            if (slot < 16) {
+                const int h = 2 * (slot >> 3) + hb2;
+                part_base[(int64_t)h * n_parts * stride + 2 + g2 * 8 + (slot & 7)] = v;
+            } else if (g2 == 0) {
+                const int h = 2 * (slot - 16) + hb2;
+                part_base[(int64_t)h * n_parts * stride + 0] = (float)ctl->head[h].e_cur + ctl->offset[h];   // reference exponent (log2 domain)
+                part_base[(int64_t)h * n_parts * stride + 1] = v;                                            // normaliser, in the same unit
+            }
+        }
+    }
+}
+
+}  // namespace
+
+bool decode_pair_supported(const Shape& sh)
+{
+    return sh.head_dim == 128 && sh.b == 8 && sh.G == 16 && sh.R % PairCfg::kHeads == 0 &&
+           sh.max_tokens <= ((int64_t)1 << 30);
+}
+
+// Launch plan.  Two CTAs share an SM.  The table build and the bins x centroids product are paid
+// once per CTA, so a CTA takes its whole context (up to 65536 tokens) unless the grid would leave
+// CTA slots idle.  When every context fits one CTA, the items beyond the last full wave of CTAs are
+// spread over k <= 4 CTAs each, k chosen so that this last wave ends as early as possible.
+DecodePlan decode_pair_plan(const Shape& sh)
+{
+    using C = PairCfg;
+    DecodePlan pl;
+    const int64_t items = sh.n_seq * (sh.n_q_heads / C::kHeads);
+    const int64_t slots = 2 * (int64_t)device_sm_count();
+    const int64_t round = C::kRoundTokens;
+    int64_t chunk = (sh.max_tokens + round - 1) / round * round;
+    if (chunk > 65536) chunk = 65536;
+    while (chunk > 2048 && 2 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
+        chunk = (chunk / 2 + round - 1) / round * round;
+    pl.chunk = (int)chunk;
+    pl.n_parts = (int)((sh.max_tokens + chunk - 1) / chunk);
+    pl.tail_first = -1;
+    pl.grid = (unsigned)(items * pl.n_parts);
+    const int64_t rest = items % slots;
+    if (pl.n_parts == 1 && items > slots && rest > 0) {
+        int best_k = 1;
+        double best = 1.0;
+        for (int k = 2; k <= 4; ++k) {
+            if (chunk / k < 2048) break;
+            const double cost = (double)((rest * k + slots - 1) / slots) / k + 0.02 * (k - 1);
+            if (cost < best - 1e-9) { best = cost; best_k = k; }
+        }
+        if (best_k > 1) {
+            const int64_t part_chunk = ((chunk + best_k - 1) / best_k + round - 1) / round * round;
+            pl.chunk = (int)part_chunk;
+            pl.n_parts = (int)((sh.max_tokens + part_chunk - 1) / part_chunk);
+            pl.tail_first = (int)(items - rest);
+            pl.grid = (unsigned)(pl.tail_first + rest * pl.n_parts);
+        }
+    }
+    return pl;
+}
+
+cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
+                               const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
+                               float* partials, cudaStream_t st)
+{
+    using C = PairCfg;
+    const cudaError_t attr = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_pair_kernel), C::kSmemBytes, 0);
+    if (attr != cudaSuccess) return attr;
+    const int aligned = ((reinterpret_cast<uintptr_t>(kcb) | reinterpret_cast<uintptr_t>(vcb)) & 31u) == 0 ? 1 : 0;
+    decode_pair_kernel<<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk,
+                                                                    pl.n_parts, pl.tail_first, aligned, partials);
+    return cudaGetLastError();
+}
+
+}  // namespace cq

@@ -1,6 +1,7 @@
 // Generic sm_100a kernels of the CQ library: they accept every supported (head_dim, c, b)
 // and favour plainness over speed.  The tuned kernels live in cq_encode.cu / cq_decode.cu.
 #include "cq_common.cuh"
+#include "cq_bulk_copy.cuh"
 
 namespace cq {
 
@@ -379,34 +380,6 @@ decode_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ 
 // ------------------------------------------------------------------------------------------
 constexpr int kRopeThreads = 1024;
 
-// Bulk asynchronous copy global -> shared memory (the TMA engine; no tensor map, no multicast) with
-// an mbarrier that counts the bytes.  Source, destination and size are multiples of 16 bytes.
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int arrivals)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-// Waits for the phase with the given parity; gives up after a bounded number of polls (returns false).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
-{
-    for (int poll = 0; poll < (1 << 22); ++poll) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-        if (done) return true;
-    }
-    return false;
-}
 
 __global__ void __launch_bounds__(kRopeThreads)
 decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
