@@ -52,17 +52,9 @@ struct Cfg {
     static constexpr int kPlanes = kHalfGroups ? 2 : kLaneHeads;         // 32-word planes per table row
     static constexpr int kSlots = kHalfGroups ? 8 : G / 4;               // code words (16 tokens each) per lane
     static constexpr int kBlocksPerIter = ((G == 16 && R >= 2) || kHalfGroups) ? 4 : 8;   // 16-token blocks per warp iteration
-#ifdef CQ_TUNE_WARPS1
-    static constexpr int kWarps = (kPlanes == 1) ? CQ_TUNE_WARPS1 : 16;
-#else
     static constexpr int kWarps = (kPlanes == 1) ? 8 : 16;
-#endif
     static constexpr int kThreads = kWarps * 32;
-#ifdef CQ_TUNE_MINBLK
-    static constexpr int kMinBlocks = (kPlanes == 1) ? CQ_TUNE_MINBLK : 1;
-#else
     static constexpr int kMinBlocks = (kPlanes == 1) ? 2 : 1;     // 128 registers per thread in every configuration
-#endif
     static constexpr int kRoundTokens = kWarps * kBlocksPerIter * 16;    // tokens a CTA handles per iteration
     static_assert(kPlanes == 1 || kPlanes == 2, "table rows hold one or two planes");
     // One plane: K and V planes share a row (K at +0, V at +128).  Two planes: separate tables.
@@ -386,11 +378,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     __syncthreads();
 
     // ---------------------------------------------------------------- main loop over the chunk
-#ifdef CQ_TUNE_KBATCH
-    constexpr int kBatch = CQ_TUNE_KBATCH;
-#else
     constexpr int kBatch = (C::kSlots * C::kLaneHeads >= 8) ? 2 : 4;       // tokens whose lookups are in flight together
-#endif
 
     // Weight units.  Each query head's bins count in units of 2^e_cur[h].  A warp adds its tokens'
     // weights without waiting for the others as long as (a) its largest score fits the unit
@@ -1153,7 +1141,7 @@ struct Plan {
 };
 
 // The table build and the bins x centroids product are paid once per CTA, so chunks are long (up
-// to 65536 tokens); they are halved only while the grid would not give the CTA slots of the 148
+// to 65536 tokens); they are halved only while the grid would not give the CTA slots of the
 // SMs one and a half CTAs each, and never below 2048 tokens.  When every context fits one chunk
 // and the last wave of CTAs would fill at most half of the slots, the items of that wave are
 // spread over 2 to 4 CTAs each instead, which shortens the wave by that factor.  This applies
@@ -1162,20 +1150,15 @@ struct Plan {
 Plan plan_from(const Shape& sh, int64_t round, int min_blocks, int64_t items)
 {
     Plan pl;
-    const int64_t slots = 148 * min_blocks;
+    const int64_t slots = (int64_t)device_sm_count() * min_blocks;
     int64_t chunk = (sh.max_tokens + round - 1) / round * round;
     if (chunk > 65536) chunk = 65536;
-#ifdef CQ_TUNE_CHUNK_TOKENS
-    chunk = CQ_TUNE_CHUNK_TOKENS;
-#else
     while (chunk > 2048 && 2 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
         chunk = (chunk / 2 + round - 1) / round * round;
-#endif
     pl.chunk = (int)chunk;
     pl.n_parts = (int)((sh.max_tokens + chunk - 1) / chunk);
     pl.tail_first = -1;
     pl.grid = (unsigned)(items * pl.n_parts);
-#ifndef CQ_TUNE_NO_TAIL
     const int64_t rest = items % slots;               // CTAs of the last wave
     if (min_blocks == 1 && pl.n_parts == 1 && items > slots && rest > 0 && 2 * rest <= slots && chunk >= 2 * 2048) {
         int64_t k = slots / rest;
@@ -1186,7 +1169,6 @@ Plan plan_from(const Shape& sh, int64_t round, int min_blocks, int64_t items)
         pl.tail_first = (int)(items - rest);
         pl.grid = (unsigned)(pl.tail_first + rest * pl.n_parts);
     }
-#endif
     return pl;
 }
 
@@ -1203,10 +1185,10 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
 {
     using C = Cfg<G, R>;
     const int kv_share = sh.R / R;
-    cudaError_t e = kv_share > 1 ? cudaFuncSetAttribute(decode_tuned_kernel<G, R, true>,
-                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes)
-                                 : cudaFuncSetAttribute(decode_tuned_kernel<G, R, false>,
-                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    // call-site slots of ensure_dynamic_smem: 1 is the wide kernel, 2 ... 13 the template instances
+    constexpr int kSlot = 2 + 2 * ((G == 16 ? 0 : G == 32 ? 3 : 5) + (R == 1 ? 0 : R == 2 ? 1 : 2));
+    cudaError_t e = kv_share > 1 ? ensure_dynamic_smem(reinterpret_cast<const void*>(decode_tuned_kernel<G, R, true>), C::kSmemBytes, kSlot)
+                                 : ensure_dynamic_smem(reinterpret_cast<const void*>(decode_tuned_kernel<G, R, false>), C::kSmemBytes, kSlot + 1);
     if (e != cudaSuccess) return e;
     if (kv_share > 1)
         decode_tuned_kernel<G, R, true><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
@@ -1273,7 +1255,7 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
     if (pl.chunk <= 0) return cudaErrorNotSupported;
     cudaError_t e = cudaErrorNotSupported;
     if (wide_shape(sh)) {
-        e = cudaFuncSetAttribute(decode_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WideCfg::kSmemBytes);
+        e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_wide_kernel), WideCfg::kSmemBytes, 1);
         if (e != cudaSuccess) return e;
         decode_wide_kernel<<<pl.grid, WideCfg::kThreads, WideCfg::kSmemBytes, st>>>(
             q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),

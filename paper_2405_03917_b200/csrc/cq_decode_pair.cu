@@ -72,12 +72,13 @@ struct PairCfg {
     static constexpr int kVOffset = kKBytes;
     static constexpr int kVBytes = kRows * kVRowBytes;          // 64 KiB; also the fp32 staging area of the table build
     static constexpr int kCtlOffset = kVOffset + kVBytes;
-    static constexpr int kCtlBytes = 512;
+    static constexpr int kCtlBytes = 768;                       // keeps the tiles 256-byte aligned (their words are addressed with XOR)
     static constexpr int kStageOffset = kCtlOffset + kCtlBytes; // per warp: K tile (4 blocks x 256 bytes), then V tile
     static constexpr int kTileBytes = kBlocksPerIter * 16 * 16;
-    static constexpr int kSmemBytes = kStageOffset + kWarps * 2 * kTileBytes;   // 112.5 KiB: two CTAs per SM
+    static constexpr int kSmemBytes = kStageOffset + kWarps * 2 * kTileBytes;   // 112.75 KiB: two CTAs per SM
     static constexpr int kQOffset = 0;                          // scaled query [4][128] fp32, in the K table's place until the table is written
     static constexpr int kLog2Groups = 3;             // log2 of the warps that add to a head's bins per round
+    static_assert(kStageOffset % 256 == 0, "tile alignment");
 };
 
 struct PairCtl {
@@ -91,7 +92,7 @@ struct PairCtl {
     int range_bits[4];         // per head: largest (max - min) over its groups' table entries, as float bits
     float offset[4];           // per head: sum over groups of the entry taken out of each group
     float mins[4][16];         // per (head, group): smallest table entry
-    uint64_t bar[PairCfg::kWarps];      // per warp: arrival of its code tiles (K and V of one iteration)
+    uint64_t bar[PairCfg::kWarps][2];   // per warp: arrival of its K tile and of its V tile
 };
 static_assert(sizeof(PairCtl) <= PairCfg::kCtlBytes, "control block");
 
@@ -381,17 +382,19 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     // Code tiles.  Tile `it` of this warp = its four blocks of iteration `it`, 1 KiB of contiguous
     // codes per tensor (less at the end of the chunk; blocks past the end are not copied and keep
     // whatever the tile held: any byte is a valid table row, and those tokens are masked).  Lane 0
-    // asks for the next tile as soon as every lane has taken its words of the current one.
+    // asks for a tensor's next tile as soon as every lane has taken its words of the current one.
     uint8_t* ktile = smem + C::kStageOffset + warp * 2 * C::kTileBytes;
     uint8_t* vtile = ktile + C::kTileBytes;
     // this lane's half word of its first code word in the K tile and in the V tile; word m is 64 m / 16 m bytes
     // away in the XOR sense (the tiles are 128-byte aligned)
-    const uint8_t* my_ktile = ktile + (r >> 1) * 256 + 8 * (r & 1) + 2 * koff0;
-    const uint8_t* my_vtile = vtile + (r >> 1) * 256 + 8 * (r & 1) + 16 * (8 * pu + vx);
-    uint64_t* tbar = &ctl->bar[warp];
-    uint32_t tphase = 0u;
+    const uint32_t my_ktile = (uint32_t)(C::kStageOffset + warp * 2 * C::kTileBytes + (r >> 1) * 256 + 8 * (r & 1)) + 2u * koff0;
+    const uint32_t my_vtile = (uint32_t)(C::kStageOffset + warp * 2 * C::kTileBytes + C::kTileBytes + (r >> 1) * 256 + 8 * (r & 1)) +
+                              16u * (8 * pu + vx);
+    uint64_t* kbar = &ctl->bar[warp][0];
+    uint64_t* vbar = &ctl->bar[warp][1];
+    uint32_t kphase = 0u, vphase = 0u;
     bool bulk = true;                       // false after a wait that gave up: plain loads from then on
-    bool t_out = false;                     // copies into the tiles have been requested and not yet awaited
+    bool k_out = false, v_out = false;      // a copy into the tile has been requested and not yet awaited
     const int n_blocks_cta = (n_tok + kTokenBlock - 1) / kTokenBlock;   // blocks holding a valid token
     // bytes of this warp's tile of iteration `it` (per tensor)
     auto tile_bytes = [&](int it) -> uint32_t {
@@ -399,46 +402,64 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
         nb = nb < 0 ? 0 : (nb > C::kBlocksPerIter ? C::kBlocksPerIter : nb);
         return (uint32_t)nb * 256u;
     };
-    auto request_tiles = [&](int it) {      // lane 0 only
-        const uint32_t bytes = tile_bytes(it);
-        if (bytes == 0u) return;
+    auto request_tile = [&](uint8_t* tile, uint64_t* bar, const uint8_t* base, int it, uint32_t bytes) {      // lane 0 only
         const int64_t off = (int64_t)(it * C::kWarps + warp) * (C::kBlocksPerIter * 256);
         fence_async_smem();
-        mbar_expect_tx(tbar, 2u * bytes);
-        bulk_copy_g2s(ktile, kbase + off, bytes, tbar);
-        bulk_copy_g2s(vtile, vbase + off, bytes, tbar);
+        mbar_expect_tx(bar, bytes);
+        bulk_copy_g2s(tile, base + off, bytes, bar);
     };
     uint2 kw[4], vw[8];
-    // the words of tile `it` into registers; then the tiles are free for iteration it + 1
-    auto take_tiles = [&](int it) {
+    // the K words of tile `it` into registers; then the tile is free for iteration it + 1
+    auto take_k = [&](int it) {
         bool have = false;
         const uint32_t bytes = tile_bytes(it);
         if (bulk && bytes != 0u) {
-            have = mbar_wait(tbar, tphase);
+            have = mbar_wait(kbar, kphase);
             have = __all_sync(0xffffffffu, have);
-            if (have) { tphase ^= 1u; t_out = false; } else bulk = false;
+            if (have) { kphase ^= 1u; k_out = false; } else bulk = false;
         }
         if (have || bytes == 0u) {
 #pragma unroll
-            for (int m = 0; m < 4; ++m)
-                kw[m] = *reinterpret_cast<const uint2*>(smem + ((uint32_t)(my_ktile - smem) ^ (64u * m)));
-#pragma unroll
-            for (int m = 0; m < 8; ++m)
-                vw[m] = *reinterpret_cast<const uint2*>(smem + ((uint32_t)(my_vtile - smem) ^ (16u * m)));
+            for (int m = 0; m < 4; ++m) kw[m] = *reinterpret_cast<const uint2*>(smem + (my_ktile ^ (64u * m)));
         } else {
-            const int64_t off = (int64_t)((it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1)) * 256 + 8 * (r & 1);
-            const bool in = ((it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1)) < n_blocks_cta;
+            const int blk = (it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1);
+            const int64_t off = (int64_t)blk * 256 + 8 * (r & 1);
 #pragma unroll
             for (int m = 0; m < 4; ++m)
-                kw[m] = in ? __ldg(reinterpret_cast<const uint2*>(kbase + off + 2u * (koff0 ^ (32u * m)))) : make_uint2(0u, 0u);
-#pragma unroll
-            for (int m = 0; m < 8; ++m)
-                vw[m] = in ? __ldg(reinterpret_cast<const uint2*>(vbase + off + 16u * (8 * pu + (vx ^ m)))) : make_uint2(0u, 0u);
+                kw[m] = blk < n_blocks_cta ? __ldg(reinterpret_cast<const uint2*>(kbase + off + 2u * (koff0 ^ (32u * m))))
+                                           : make_uint2(0u, 0u);
         }
         __syncwarp();
-        if (bulk && it + 1 < n_iters && tile_bytes(it + 1) != 0u) {
-            t_out = true;
-            if (lane == 0) request_tiles(it + 1);
+        const uint32_t next = it + 1 < n_iters ? tile_bytes(it + 1) : 0u;
+        if (bulk && next != 0u) {
+            k_out = true;
+            if (lane == 0) request_tile(ktile, kbar, kbase, it + 1, next);
+        }
+    };
+    auto take_v = [&](int it) {
+        bool have = false;
+        const uint32_t bytes = tile_bytes(it);
+        if (bulk && bytes != 0u) {
+            have = mbar_wait(vbar, vphase);
+            have = __all_sync(0xffffffffu, have);
+            if (have) { vphase ^= 1u; v_out = false; } else bulk = false;
+        }
+        if (have || bytes == 0u) {
+#pragma unroll
+            for (int m = 0; m < 8; ++m) vw[m] = *reinterpret_cast<const uint2*>(smem + (my_vtile ^ (16u * m)));
+        } else {
+            const int blk = (it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1);
+            const int64_t off = (int64_t)blk * 256 + 8 * (r & 1);
+#pragma unroll
+            for (int m = 0; m < 8; ++m)
+                vw[m] = blk < n_blocks_cta ? __ldg(reinterpret_cast<const uint2*>(vbase + off + 16u * (8 * pu + (vx ^ m))))
+                                           : make_uint2(0u, 0u);
+        }
+        __syncwarp();
+        const uint32_t next = it + 1 < n_iters ? tile_bytes(it + 1) : 0u;
+        if (bulk && next != 0u) {
+            v_out = true;
+            if (lane == 0) request_tile(vtile, vbar, vbase, it + 1, next);
         }
     };
 
@@ -453,15 +474,21 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     }
     if (threadIdx.x == 4) ctl->want = 0;
     if (threadIdx.x == 5) {
-        for (int w = 0; w < C::kWarps; ++w) mbar_init(&ctl->bar[w], 1);
+        for (int w = 0; w < C::kWarps; ++w) {
+            mbar_init(&ctl->bar[w][0], 1);
+            mbar_init(&ctl->bar[w][1], 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
         qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)head_group * R) * 128 + i]) * scale_log2e;
     __syncthreads();
     // the first code tiles travel during the table build
-    t_out = tile_bytes(0) != 0u;
-    if (lane == 0) request_tiles(0);
+    k_out = v_out = tile_bytes(0) != 0u;
+    if (lane == 0 && k_out) {
+        request_tile(ktile, kbar, kbase, 0, tile_bytes(0));
+        request_tile(vtile, vbar, vbase, 0, tile_bytes(0));
+    }
 
     // Table build, first pass: fp32 entries into the staging area (the later bins), entry (h, g, j)
     // at word (h*16 + g)*256 + (j ^ (16*(h/2) + g)): a warp writing 32 consecutive j of one (h, g)
@@ -556,48 +583,45 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     }
     const uint32_t head_rec = smem_addr(&ctl->head[hb]);                // record of head hb; head 2 + hb is 32 bytes on
 
+    // K side of one token: four 64-bit lookups (one per code word, both head pairs), then one MMA chain:
+    // fragment row r takes the words of pair 0, row r + 8 the words of pair 1 (the two halves of a lookup
+    // are neighbours in the A fragment), two code words per MMA.  The scores of the lane's two heads come
+    // out as exact integers held in floats.
+    float sc[2][8];
+    auto k_lookup = [&](uint2 (&dst)[4], int k) {
+#pragma unroll
+        for (int m = 0; m < 4; ++m)
+            dst[m] = *reinterpret_cast<const uint2*>(smem + k_row_index(kw[m], k, koff0 ^ (32u * m)));
+    };
+    auto k_score = [&](const uint2 (&src)[4], int k) {
+        int d[4];
+        // columns start at 2^23 as float bits (low sums) and 0 (high sums): low + 256 * high < 2^21, so the
+        // float with these bits, minus 2^23, is the integer score, exactly
+        mma_bytesum_first(d, src[0].x, src[0].y, src[1].x, src[1].y, bsel, 0x4b000000);
+        mma_bytesum_acc(d, src[2].x, src[2].y, src[3].x, src[3].y, bsel);
+        sc[0][k] = __int_as_float(d[0] + (d[1] << 8)) - 8388608.f;
+        sc[1][k] = __int_as_float(d[2] + (d[3] << 8)) - 8388608.f;
+    };
+
+    // The loop is software-pipelined: the K side of iteration it + 1 is interleaved, token by token, with the
+    // V side of iteration it, so that the lookups' and the MMAs' latencies pass behind the bin updates.
+    uint2 a[2][4];
+    take_k(0);
+    static_for<8>([&](auto kc_) {
+        constexpr int k = decltype(kc_)::value;
+        k_lookup(a[k & 1], k);
+        if (k >= 1) k_score(a[(k - 1) & 1], k - 1);
+    });
+    k_score(a[1], 7);
+    take_v(0);
+
     for (int it = 0; it < n_iters; ++it) {
-        take_tiles(it);
-        // the heads' control records as they stand now (used after the K side)
+        // the heads' control records as they stand now
         int4 seen[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u)
             asm volatile("ld.volatile.shared.v4.s32 {%0,%1,%2,%3}, [%4];"
                          : "=r"(seen[u].x), "=r"(seen[u].y), "=r"(seen[u].z), "=r"(seen[u].w) : "r"(head_rec + 32u * u));
-
-        // K side: the scores of this quad's eight tokens for the lane's two heads, as exact integers
-        // held in floats.  One 64-bit lookup per (token, code word) serves both head pairs.
-        float sc[2][8];
-        uint2 a[2][2][4];                        // [buffer][token][code word]
-        auto lookups = [&](uint2 (&dst)[2][4], int k0) {
-#pragma unroll
-            for (int kk = 0; kk < 2; ++kk)
-#pragma unroll
-                for (int m = 0; m < 4; ++m)
-                    dst[kk][m] = *reinterpret_cast<const uint2*>(smem + k_row_index(kw[m], k0 + kk, koff0 ^ (32u * m)));
-        };
-        // One MMA chain per token: fragment row r takes the words of pair 0, row r + 8 the words of pair 1
-        // (the two halves of a 64-bit lookup are neighbours in the A fragment), two code words per MMA.
-        auto scores = [&](const uint2 (&src)[2][4], int k0) {
-#pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {
-                int d[4];
-                // columns start at 2^23 as float bits (low sums) and 0 (high sums): low + 256 * high < 2^21, so
-                // the float with these bits, minus 2^23, is the integer score, exactly
-                mma_bytesum_first(d, src[kk][0].x, src[kk][0].y, src[kk][1].x, src[kk][1].y, bsel, 0x4b000000);
-                mma_bytesum_acc(d, src[kk][2].x, src[kk][2].y, src[kk][3].x, src[kk][3].y, bsel);
-                sc[0][k0 + kk] = __int_as_float(d[0] + (d[1] << 8)) - 8388608.f;
-                sc[1][k0 + kk] = __int_as_float(d[2] + (d[3] << 8)) - 8388608.f;
-            }
-        };
-        lookups(a[0], 0);
-        lookups(a[1], 2);
-        scores(a[0], 0);
-        lookups(a[0], 4);
-        scores(a[1], 2);
-        lookups(a[1], 6);
-        scores(a[0], 4);
-        scores(a[1], 6);
 
         // tokens past the end of the context (only the warp that holds the ragged end pays)
         const int tok0 = ((it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1)) * kTokenBlock + 8 * (r & 1);
@@ -607,11 +631,11 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             for (int k = 0; k < 8; ++k)
                 if (tok0 + k >= n_tok) sc[0][k] = sc[1][k] = -1.f;
         }
-        // Per head, from this lane's own eight tokens: reference exponent ref = ceil(largest score),
-        // weights 2^(score - ref) <= 1 and their sum.  Usual case, decided from the records read at the
-        // top of the iteration: no request pending, the scores fit the unit, the sum is small and the
-        // total far from its limit -> the sum goes to the total without waiting for the old value.  (No
-        // event can have happened since the records were read: an event needs this warp.)
+        // Per head, from this lane's own eight tokens: reference exponent ref >= largest score, weights
+        // 2^(score - ref) <= 1 and their sum.  Usual case, decided from the records just read: no request
+        // pending, the scores fit the unit, the sum is small and the total far from its limit -> the sum
+        // goes to the total without waiting for the old value.  (No event can happen between the read of the
+        // records and this warp's bin updates: an event needs this warp.)
         int ref[2], eu[2];
         float y[2][8], zlane[2];
         unsigned int ci[2];
@@ -622,8 +646,10 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
 #pragma unroll
             for (int k = 0; k < 8; ++k) mx = fmaxf(mx, sc[u][k]);
             have = mx >= 0.f;                                           // this lane holds a token of the context
-            ref[u] = have ? (int)ceilf(mx * delta[u]) : kUnset;
-            const float fref = have ? (float)ref[u] : 0.f;
+            // ref = round(mx * delta) + 1, formed with the 1.5 * 2^23 trick (no conversion instruction)
+            const float t = fmaf(mx, delta[u], 12582912.f);
+            const float fref = have ? (t - 12582912.f) + 1.f : 0.f;
+            ref[u] = have ? (__float_as_int(t) - 0x4b400000) + 1 : kUnset;
             float z = 0.f;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
@@ -643,11 +669,11 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             ci[u] = 0u;
             bool f = seen[u].z == 0 && eu[u] != kUnset;
             if (f && have) {
-                f = ref[u] - eu[u] <= kMaxWeightBits;
                 // this lane's weights in the current unit, rounded up, in units of 256
                 const float cw = (z * pow2i(ref[u] - eu[u]) * 1.00002f + 8.f) * (1.f / 256.f) + 1.f;
                 ci[u] = (unsigned int)fminf(cw, 6.7e7f);
-                f = f && ci[u] < kFastLane256 && (unsigned int)seen[u].y + 8u * kFastLane256 + kFastSlack256 < kBinLimit256;
+                f = ref[u] - eu[u] <= kMaxWeightBits && cw < (float)kFastLane256 &&
+                    (unsigned int)seen[u].y + 8u * kFastLane256 + kFastSlack256 < kBinLimit256;
             }
             fast = fast && f;
         }
@@ -661,12 +687,16 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             eu[0] = e2.x;
             eu[1] = e2.y;
         }
-        if (!have) continue;
 
-        // V side: this lane's integer weights into the bins of its two heads, for its eight groups
-        const float f0 = pow2i(ref[0] - eu[0]), f1 = pow2i(ref[1] - eu[1]);   // powers of two <= 2^kMaxWeightBits
+        // V side of this iteration (the lane's integer weights into the bins of its two heads, for its
+        // eight groups; a lane without tokens adds zeros) interleaved with the K side of the next one
+        // (past the last iteration it runs on whatever the tile holds; nothing uses those scores).
+        const float f0 = have ? pow2i(ref[0] - eu[0]) : 0.f;            // powers of two <= 2^kMaxWeightBits
+        const float f1 = have ? pow2i(ref[1] - eu[1]) : 0.f;
+        if (it + 1 < n_iters) take_k(it + 1);
         static_for<8>([&](auto kc_) {
             constexpr int k = decltype(kc_)::value;
+            k_lookup(a[k & 1], k);
             const uint32_t w0 = __float2uint_rn(y[0][k] * f0), w1 = __float2uint_rn(y[1][k] * f1);
             static_for<8>([&](auto mc_) {
                 constexpr int m = decltype(mc_)::value;
@@ -674,10 +704,16 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 atomicAdd(bin, w0);
                 atomicAdd(bin + 32, w1);
             });
+            if (k >= 1) k_score(a[(k - 1) & 1], k - 1);
         });
+        k_score(a[1], 7);
+        if (it + 1 < n_iters) take_v(it + 1);
     }
     // (after a wait that gave up, a requested copy may still be on its way: it must land before the CTA ends)
-    if (!bulk && t_out) mbar_wait(tbar, tphase);
+    if (!bulk) {
+        if (k_out) mbar_wait(kbar, kphase);
+        if (v_out) mbar_wait(vbar, vphase);
+    }
     // Warps that are done keep joining coarsening events until every warp is done.
     for (int guard = 0; guard < 4096; ++guard) {
         event_barrier(C::kThreads);

@@ -474,7 +474,7 @@ cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offs
     const int64_t n_vec = sh.n_seq * n_tokens;
     const int64_t tiles = (n_vec + kTileVecs - 1) / kTileVecs;
     // split the groups over CTAs while the grid would leave SMs idle
-    int64_t n_gsplit = (2 * 148 + tiles * sh.n_kv_heads - 1) / (tiles * sh.n_kv_heads);
+    int64_t n_gsplit = (2 * (int64_t)device_sm_count() + tiles * sh.n_kv_heads - 1) / (tiles * sh.n_kv_heads);
     if (n_gsplit > C::G) n_gsplit = C::G;
     if (n_gsplit < 1) n_gsplit = 1;
     const int groups_per_cta = (int)((C::G + n_gsplit - 1) / n_gsplit);
@@ -482,7 +482,9 @@ cudaError_t launch_enc(const __half* x, const float* cb, const int32_t* seq_offs
     const int64_t grid = tiles * sh.n_kv_heads * n_gsplit;
     if (grid > 0x7fffffff) return cudaErrorInvalidConfiguration;
     const size_t smem = (size_t)2 * C::kBufWords * 4 + sizeof(EncCtl);
-    cudaError_t e = cudaFuncSetAttribute(encode_tuned_kernel<kC, kMT, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // call-site slots of ensure_dynamic_smem: 16 ... 27, one per template instance
+    constexpr int kSlot = 16 + 4 * (kC == 2 ? 0 : kC == 4 ? 1 : 2) + 2 * (kMT == 1 ? 0 : 1) + (kWide ? 1 : 0);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(encode_tuned_kernel<kC, kMT, kWide>), (int)smem, kSlot);
     if (e != cudaSuccess) return e;
     encode_tuned_kernel<kC, kMT, kWide><<<dim3((unsigned)grid, x2 ? 2u : 1u), kEncThreads, smem, st>>>(
         x, cb, seq_offsets, sh, n_tokens, token_offset, codes, groups_per_cta, x2, cb2, codes2);
@@ -503,7 +505,7 @@ cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t*
 {
     const int64_t n_vec = sh.n_seq * n_tokens;
     if (n_vec == 0) return cudaSuccess;
-    const bool few = n_vec * sh.n_kv_heads < (int64_t)148 * 512 * 2;    // not enough vectors for 64 per warp
+    const bool few = n_vec * sh.n_kv_heads < (int64_t)device_sm_count() * 512 * 2;    // not enough vectors for 64 per warp
     if (sh.b > 8) {
         switch (sh.c) {
             case 2: return few ? launch_enc<2, 1, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)

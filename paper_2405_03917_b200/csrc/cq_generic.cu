@@ -64,7 +64,8 @@ cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_
     if (total == 0) return cudaSuccess;
     const int threads = 256;
     const int64_t blocks = (total + threads - 1) / threads;
-    const int grid = (int)(blocks < 148 * 64 ? blocks : 148 * 64);
+    const int64_t cap = (int64_t)device_sm_count() * 64;
+    const int grid = (int)(blocks < cap ? blocks : cap);
     encode_generic_kernel<<<grid, threads, 0, st>>>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes);
     return cudaGetLastError();
 }
@@ -236,7 +237,8 @@ static int words_grid(const Shape& sh)
 {
     const int64_t words = sh.n_seq * sh.n_kv_heads * sh.n_blocks * sh.G;
     const int64_t blocks = (words + 255) / 256;
-    return (int)(blocks < 148 * 32 ? (blocks > 0 ? blocks : 1) : 148 * 32);
+    const int64_t cap = (int64_t)device_sm_count() * 32;
+    return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
 }
 
 cudaError_t launch_to_rowmajor(const uint8_t* codes, const Shape& sh, uint8_t* rowmajor, cudaStream_t st)
@@ -555,9 +557,9 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
 
 int decode_generic_splits(const Shape& sh)
 {
-    // enough CTAs for a few waves of 148 SMs, at least 256 tokens per split
+    // enough CTAs for a few waves of the SMs, at least 256 tokens per split
     const int64_t items = sh.n_seq * sh.n_q_heads;
-    int64_t want = (148 * 8 + items - 1) / (items > 0 ? items : 1);
+    int64_t want = ((int64_t)device_sm_count() * 8 + items - 1) / (items > 0 ? items : 1);
     const int64_t cap = (sh.max_tokens + 255) / 256;
     if (want > cap) want = cap;
     if (want < 1) want = 1;
@@ -607,7 +609,7 @@ cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint
 {
     int n_splits = decode_generic_splits(sh);
     const size_t smem = (size_t)2 * sh.G * sh.K * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(decode_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_generic_kernel), (int)smem, 32);
     if (e != cudaSuccess) return e;
     // tables of more than a third of an SM's shared memory: fewer, larger CTAs keep the SM's warps busy
     const int threads = smem > 72 * 1024 ? (smem > 110 * 1024 ? kGenericThreadsMax : 512) : kGenericThreads;
@@ -615,7 +617,7 @@ cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint
         // one CTA per SM, each paying a table build over the whole codebook: split the contexts only as far
         // as two CTAs per SM need it (never into more partial slots than the workspace holds)
         const int64_t items = sh.n_seq * sh.n_q_heads;
-        int64_t want = (2 * 148 + items - 1) / items;
+        int64_t want = (2 * (int64_t)device_sm_count() + items - 1) / items;
         const int64_t cap = (sh.max_tokens + threads - 1) / threads;
         if (want > cap) want = cap;
         if (want < 1) want = 1;
@@ -638,7 +640,7 @@ cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t
     int n_splits = decode_generic_splits(sh);
     {
         const int64_t items = sh.n_seq * sh.n_q_heads;
-        int64_t want = (2 * 148 + items - 1) / items;
+        int64_t want = (2 * (int64_t)device_sm_count() + items - 1) / items;
         const int64_t cap = (sh.max_tokens + kRopeThreads - 1) / kRopeThreads;
         if (want > cap) want = cap;
         if (want < 1) want = 1;
@@ -650,7 +652,7 @@ cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t
     const int stage = (sh.G * sh.K + sh.head_dim) % 4 == 0 && (sh.G * sh.K * sh.c) % 4 == 0 &&
                       smem + book <= (size_t)220 * 1024;
     if (stage) smem += book;
-    cudaError_t e = cudaFuncSetAttribute(decode_rope_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_rope_kernel), (int)smem, 33);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(n_splits * sh.n_q_heads * sh.n_seq);
     decode_rope_kernel<<<grid, kRopeThreads, smem, st>>>(q, kc, vc, kcb, vcb, seq_lens, rope_cos, rope_sin, pairing,

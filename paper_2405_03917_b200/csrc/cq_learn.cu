@@ -174,7 +174,8 @@ cudaError_t launch_kmeanspp_init(const __half* x, const float* weights, const do
     double* dist = reinterpret_cast<double*>(static_cast<char*>(workspace) + l.codes);
     const int n_prob = sh.n_kv_heads * sh.G;
     const int64_t pairs = n_vec * n_prob;
-    const int dist_grid = (int)((pairs + 255) / 256 < 148 * 16 ? (pairs + 255) / 256 : 148 * 16);
+    const int64_t dist_cap = (int64_t)device_sm_count() * 16;
+    const int dist_grid = (int)((pairs + 255) / 256 < dist_cap ? (pairs + 255) / 256 : dist_cap);
     double* contrib = reinterpret_cast<double*>(static_cast<char*>(workspace) + l.codes + l.dist);
     for (int k = 0; k < sh.K; ++k) {
         pp_pick_kernel<<<n_prob, kPickThreads, 0, st>>>(x, uniforms, contrib, n_vec, n_prob, sh.c, sh.K, k, codebooks);
@@ -197,7 +198,7 @@ cudaError_t launch_lloyd_step(const __half* x, const float* weights, const float
                                                : launch_encode_generic(x, cb_in, nullptr, es, n_vec, 0, codes, st);
     if (e != cudaSuccess) return e;
     const size_t smem = (size_t)(2 * sh.K * sh.c + sh.K) * sizeof(float);
-    e = cudaFuncSetAttribute(lloyd_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(lloyd_update_kernel), (int)smem, 34);
     if (e != cudaSuccess) return e;
     lloyd_update_kernel<<<sh.n_kv_heads * sh.G, kUpdThreads, smem, st>>>(x, weights, codes, cb_in, es, n_vec, cb_out,
                                                                          objective);
