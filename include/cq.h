@@ -236,7 +236,10 @@ int cq_decode_attn_rope(const void *q_fp16, const void *k_codes, const void *v_c
 /*
  * Same operation with an explicit kernel choice, for tests and benchmarks:
  * variant 0 = automatic (what cq_decode_attn uses), 1 = generic kernel,
- * 2 = tuned kernel (CQ_ERR_UNSUPPORTED when the shape has none).
+ * 2 = tuned kernel (CQ_ERR_UNSUPPORTED when the shape has none), 3 = tuned kernel
+ * with one table word per query head, also for the shapes (CQ-8c8b with a multiple
+ * of four query heads per KV head) where 2 takes the kernel that shares table words
+ * between query heads; the same as 2 for every other shape.
  */
 int cq_decode_attn_variant(const void *q_fp16, const void *k_codes, const void *v_codes,
                            const float *k_cb, const float *v_cb, const int32_t *seq_lens, float scale,

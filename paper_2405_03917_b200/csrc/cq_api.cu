@@ -243,21 +243,21 @@ int cq_decode_attn_variant(const void* q_fp16, const void* k_codes, const void* 
     Shape sh;
     int st = make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
     if (st != CQ_OK) return st;
-    if (variant < 0 || variant > 2) return CQ_ERR_SHAPE;
+    if (variant < 0 || variant > 3) return CQ_ERR_SHAPE;
     if (!aligned16(k_codes) || !aligned16(v_codes) || !aligned16(workspace) || !aligned16(k_cb) || !aligned16(v_cb) ||
         (reinterpret_cast<uintptr_t>(q_fp16) & 1u) || (reinterpret_cast<uintptr_t>(out) & 3u))
         return CQ_ERR_ALIGN;
     if (workspace_bytes < round_up(partial_bytes(sh), 256)) return CQ_ERR_WORKSPACE;
     const bool tuned_ok = decode_tuned_supported(sh);
-    if (variant == 2 && !tuned_ok) return CQ_ERR_UNSUPPORTED;
-    const bool use_tuned = variant == 2 || (variant == 0 && tuned_ok);
+    if ((variant == 2 || variant == 3) && !tuned_ok) return CQ_ERR_UNSUPPORTED;
+    const bool use_tuned = variant == 2 || variant == 3 || (variant == 0 && tuned_ok);
     if (!use_tuned && (int64_t)sh.G * sh.K > kGenericMaxTableEntries) return CQ_ERR_UNSUPPORTED;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const __half* q = static_cast<const __half*>(q_fp16);
     const uint8_t* kc = static_cast<const uint8_t*>(k_codes);
     const uint8_t* vc = static_cast<const uint8_t*>(v_codes);
     float* partials = static_cast<float*>(workspace);
-    cudaError_t e = use_tuned ? launch_decode_tuned(q, kc, vc, k_cb, v_cb, seq_lens, scale, sh, out, partials, cs)
+    cudaError_t e = use_tuned ? launch_decode_tuned(q, kc, vc, k_cb, v_cb, seq_lens, scale, sh, out, partials, cs, variant == 3)
                               : launch_decode_generic(q, kc, vc, k_cb, v_cb, seq_lens, scale, sh, out, partials, cs);
     return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
 }

@@ -106,9 +106,11 @@ cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t
                                int pairing, float scale, const Shape& sh, float* out, float* partials, cudaStream_t st);
 bool decode_tuned_supported(const Shape& sh);
 int decode_tuned_parts(const Shape& sh);      // partial slots per (sequence, query head)
+// per_head_tables: keep to decode_tuned_kernel (one table word per query head) also where the kernel
+// with shared table words (cq_decode_pair.cu) would be picked.
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
-                                float* out, float* partials, cudaStream_t st);
+                                float* out, float* partials, cudaStream_t st, bool per_head_tables = false);
 
 // CQ-8c8b with a multiple of four query heads per KV head: two query heads per table word (cq_decode_pair.cu).
 bool decode_pair_supported(const Shape& sh);

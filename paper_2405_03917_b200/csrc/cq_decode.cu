@@ -1237,15 +1237,18 @@ bool decode_tuned_supported(const Shape& sh)
 
 int decode_tuned_parts(const Shape& sh)
 {
-    if (decode_pair_supported(sh)) return decode_pair_plan(sh).n_parts;
-    return plan_dispatch(sh).n_parts;
+    // (either kernel may be asked for: the workspace holds the larger of the two plans)
+    const int own = plan_dispatch(sh).n_parts;
+    if (!decode_pair_supported(sh)) return own;
+    const int pair = decode_pair_plan(sh).n_parts;
+    return pair > own ? pair : own;
 }
 
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh, float* out,
-                                float* partials, cudaStream_t st)
+                                float* partials, cudaStream_t st, bool per_head_tables)
 {
-    if (decode_pair_supported(sh)) {
+    if (!per_head_tables && decode_pair_supported(sh)) {
         const DecodePlan pp = decode_pair_plan(sh);
         const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st);
         if (ep != cudaSuccess) return ep;

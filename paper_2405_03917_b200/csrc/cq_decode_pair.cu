@@ -332,6 +332,10 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     const int hkv = head_group / kv_share;
     const int64_t s = item / n_head_groups;
 
+    // (the query travels while the context length is looked up)
+    const __half* qrow = q + (s * sh.n_q_heads + (int64_t)head_group * R) * 128;
+    const __half q_lo = qrow[threadIdx.x], q_hi = qrow[C::kThreads + threadIdx.x];
+    static_assert(R * 128 == 2 * C::kThreads, "two query elements per thread");
     int64_t n = seq_lens[s];
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
     const int64_t t_begin = (int64_t)part * chunk_tokens;
@@ -480,8 +484,8 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = threadIdx.x; i < R * 128; i += C::kThreads)
-        qs[i] = __half2float(q[(s * sh.n_q_heads + (int64_t)head_group * R) * 128 + i]) * scale_log2e;
+    qs[threadIdx.x] = __half2float(q_lo) * scale_log2e;
+    qs[C::kThreads + threadIdx.x] = __half2float(q_hi) * scale_log2e;
     __syncthreads();
     // the first code tiles travel during the table build
     k_out = v_out = tile_bytes(0) != 0u;
@@ -556,10 +560,12 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
 #pragma unroll 8
         for (int i = 0; i < kRows / C::kWarps; ++i) {
             const int j = warp * (kRows / C::kWarps) + i;
-            const float u0 = fminf(rintf((s0[j ^ lane] - m0) * inv0), 65535.f);
-            const float u1 = fminf(rintf((s1[j ^ lane] - m1) * inv1), 65535.f);
+            // round to nearest by adding 1.5 * 2^23: the integer is then in the low mantissa bits (no
+            // conversion instruction; non-finite inputs end up clamped like everything else)
+            const float u0 = fminf(fmaxf((s0[j ^ lane] - m0) * inv0, 0.f), 65535.f) + 12582912.f;
+            const float u1 = fminf(fmaxf((s1[j ^ lane] - m1) * inv1, 0.f), 65535.f) + 12582912.f;
             *reinterpret_cast<uint32_t*>(smem + j * C::kKRowBytes + (2 * g + hp) * 4) =
-                (uint32_t)fmaxf(u0, 0.f) | ((uint32_t)fmaxf(u1, 0.f) << 16);
+                ((uint32_t)__float_as_int(u0) & 0xffffu) | ((uint32_t)__float_as_int(u1) << 16);
         }
         if (threadIdx.x < R) {
             float o = 0.f;
@@ -734,12 +740,12 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
         const float* cg = vcb + (((int64_t)hkv * 16 + g) * kRows + warp * (kRows / C::kWarps)) * 8;
         const uint8_t* brow = smem + C::kVOffset + warp * (kRows / C::kWarps) * C::kVRowBytes + lane * 4;
 #pragma unroll 1
-        for (int i0 = 0; i0 < kRows / C::kWarps; i0 += 4) {
-            float cv[4][8];
+        for (int i0 = 0; i0 < kRows / C::kWarps; i0 += 8) {
+            float cv[8][8];                       // eight centroids in flight per lane (the loop's registers are free now)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) load_centroid<8>(cg + (i0 + i) * 8, cv[i], cb_aligned32 != 0);
+            for (int i = 0; i < 8; ++i) load_centroid<8>(cg + (i0 + i) * 8, cv[i], cb_aligned32 != 0);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 const float b0 = (float)*reinterpret_cast<const uint32_t*>(brow + (i0 + i) * C::kVRowBytes);
                 const float b1 = (float)*reinterpret_cast<const uint32_t*>(brow + (i0 + i) * C::kVRowBytes + 128);
                 l0 += b0;
@@ -790,8 +796,8 @@ bool decode_pair_supported(const Shape& sh)
 
 // Launch plan.  Two CTAs share an SM.  The table build and the bins x centroids product are paid
 // once per CTA, so a CTA takes its whole context (up to 65536 tokens) unless the grid would leave
-// CTA slots idle.  When every context fits one CTA, the items beyond the last full wave of CTAs are
-// spread over k <= 4 CTAs each, k chosen so that this last wave ends as early as possible.
+// CTA slots idle.  When every context fits one CTA, the items beyond the last full wave of CTAs may be
+// spread over k <= 4 CTAs each (see below).
 DecodePlan decode_pair_plan(const Shape& sh)
 {
     using C = PairCfg;
@@ -801,19 +807,28 @@ DecodePlan decode_pair_plan(const Shape& sh)
     const int64_t round = C::kRoundTokens;
     int64_t chunk = (sh.max_tokens + round - 1) / round * round;
     if (chunk > 65536) chunk = 65536;
-    while (chunk > 2048 && 2 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
+    // (split only until every SM has one and a half CTAs: a CTA that has an SM to itself still runs at
+    // more than half of the SM's rate, and every split pays another table build)
+    while (chunk > 2048 && 4 * items * ((sh.max_tokens + chunk - 1) / chunk) < 3 * slots)
         chunk = (chunk / 2 + round - 1) / round * round;
     pl.chunk = (int)chunk;
     pl.n_parts = (int)((sh.max_tokens + chunk - 1) / chunk);
     pl.tail_first = -1;
     pl.grid = (unsigned)(items * pl.n_parts);
+    // Last wave.  Splitting an item over k CTAs shortens it, but every CTA pays the table build and
+    // the bins x centroids product, which cost about as much as seven loop iterations (measured), and
+    // a CTA that has an SM to itself runs at about 1 / 0.62 of the rate of two that share one.  Take
+    // the k <= 4 with the smallest estimated duration of the wave.
     const int64_t rest = items % slots;
     if (pl.n_parts == 1 && items > slots && rest > 0) {
+        const double iters = (double)chunk / (double)round, fixed = 7.4;
         int best_k = 1;
-        double best = 1.0;
-        for (int k = 2; k <= 4; ++k) {
-            if (chunk / k < 2048) break;
-            const double cost = (double)((rest * k + slots - 1) / slots) / k + 0.02 * (k - 1);
+        double best = 1e30;
+        for (int k = 1; k <= 4; ++k) {
+            if (k > 1 && chunk / k < 2048) break;
+            const int64_t ctas = rest * k;
+            const double waves = (double)((ctas + slots - 1) / slots);
+            const double cost = waves * (fixed + iters / k) / (fixed + iters) * (2 * ctas <= slots ? 0.62 : 1.0);
             if (cost < best - 1e-9) { best = cost; best_k = k; }
         }
         if (best_k > 1) {
