@@ -36,7 +36,8 @@
 // Lane roles: lane = (r, p) = (lane / 4, lane % 4).  Quad r owns the tokens 8 (r % 2) ... + 7 of
 // block r / 2 of the warp's four 16-token blocks.  With hb = p % 2 and pu = p / 2:
 //   K row j (128 bytes): bytes 8 g ... 8 g + 7 = (pair 0 word, pair 1 word) of group g.  The
-//     lane's m-th K code word: group 4 ((r ^ m) % 4) + p  (16 lanes, 16 groups: distinct banks).
+//     lane's m-th K code word: group 4 ((r' ^ m) % 4) + p with r' = r with its two low bits swapped
+//     (16 lanes, 16 groups: distinct banks).
 //   bins row j (256 bytes): word 32 (h / 2) + 16 (h % 2) + g.  The lane serves heads hb and
 //     2 + hb; its m-th V code word: group 8 pu + ((r + 4 pu) % 8 ^ m), so that for every m the 32
 //     lanes touch 32 distinct banks (and the 64-bit reads of the staging tile do not collide).
@@ -376,7 +377,9 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     load_unit(cva, kcb, 0);
 
     // table offsets of this lane's code words (bytes inside a K row / inside plane 0 of a bins row)
-    const uint32_t koff0 = 8u * (4 * (r & 3) + p);                     // m-th K code word: koff0 ^ (32 m)
+    // m-th K code word: koff0 ^ (32 m).  (The two low bits of r are swapped so that the quads of a half warp,
+    // which read the two 8-byte halves of code words in two blocks, also spread over the staging tile's banks.)
+    const uint32_t koff0 = 8u * (4 * (((r >> 1) & 1) | ((r & 1) << 1)) + p);
     const int vx = (r + 4 * pu) & 7;
     uint32_t voffs[2] = {0u, 0u};                                        // m-th V code word: byte m % 4 of voffs[m / 4]
 #pragma unroll
@@ -684,9 +687,18 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             fast = fast && f;
         }
         if (__all_sync(0xffffffffu, fast)) {
-            if (have && pu == 0) {                   // (the lanes p and p + 2 of a quad hold the same tokens)
-                atomicAdd(&ctl->head[hb].total, ci[0]);
-                atomicAdd(&ctl->head[2 + hb].total, ci[1]);
+            // one add per head for the warp: the lanes' sums in steps of 16 (rounded up, below 2^12 each), the two
+            // heads with hb = 0 / 1 in the two halves of a word, summed over the warp; lanes 0 ... 3 add one head each
+            // (the lanes p and p + 2 of a quad hold the same tokens: only p < 2 counts)
+            uint32_t packed[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const uint32_t c16 = (have && pu == 0) ? (ci[u] + 15u) >> 4 : 0u;
+                packed[u] = __reduce_add_sync(0xffffffffu, c16 << (16 * hb));
+            }
+            if (lane < 4) {
+                const uint32_t pk = (lane & 2) ? packed[1] : packed[0];                 // head 2 (lane / 2) + lane % 2
+                atomicAdd(&ctl->head[lane].total, ((lane & 1) ? pk >> 16 : pk & 0xffffu) << 4);
             }
         } else {
             const int2 e2 = reserve_slow(smem, ctl, ref[0], ref[1], zlane[0], zlane[1]);
