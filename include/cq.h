@@ -13,6 +13,7 @@
  *
  * and, around them: cq_encode_kv (key and value of the same tokens in one launch),
  * cq_decode_attn_rope (key codes taken before the rotary embedding, Section 3.2),
+ * cq_prefill_attn (causal attention of a run of new tokens over the coded cache),
  * cq_decode_attn_static (no caller workspace), cq_decode_step_host (one decode
  * step from host buffers) and the centroid learning of Section 3.2.1
  * (cq_kmeanspp_init, cq_lloyd_step, cq_learn_centroids).
@@ -232,6 +233,41 @@ int cq_decode_attn_rope(const void *q_fp16, const void *k_codes, const void *v_c
                         int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
                         int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
                         void *stream);
+
+/*
+ * Causal attention of a run of new tokens over the CQ-coded cache: a prompt, or a chunk of
+ * one.  Section 2.1 of the paper: Eq. 1 gives the output of the current token from the keys
+ * and values of all tokens up to and including it; this call applies it to each of the
+ * n_q_tokens newest cached tokens of every sequence, K and V being the CQ reconstructions
+ * (Section 3.2).  The codes of the new tokens must already be in the cache (cq_encode /
+ * cq_encode_kv with token_offset = old length): seq_lens[s] counts them.  Query i of
+ * sequence s sits at position seq_lens[s] - n_q_tokens + i and attends the cached tokens
+ * 0 ... that position:
+ *
+ *   s_t = scale * <q_i, Khat_t>,  p = softmax(s_0 .. s_pos),  out_i = sum_t p_t Vhat_t
+ *
+ *   q_fp16  device, fp16 [n_seq][n_q_tokens][n_q_heads][head_dim], 16-byte aligned
+ *   out     device, fp32 [n_seq][n_q_tokens][n_q_heads][head_dim], 16-byte aligned
+ *   codes, codebooks, seq_lens, scale, the head mapping: as for cq_decode_attn
+ *
+ * A query whose position is negative (seq_lens[s] < n_q_tokens) has nothing to attend and
+ * gets a zero row.  No workspace.  head_dim 128 with one byte per code and c = 2, 4 or 8
+ * (and a number of query heads per KV head that divides 64) runs on tensor cores: the
+ * codes are turned back into fp16 vectors tile by tile, so results carry fp16 rounding of
+ * the centroids and of the softmax weights (within the library's attention tolerance);
+ * every other supported shape runs on a plain kernel.  CQ_ERR_SHAPE for n_q_tokens < 1 or
+ * > max_tokens.
+ */
+int cq_prefill_attn(const void *q_fp16, const void *k_codes, const void *v_codes,
+                    const float *k_cb, const float *v_cb, const int32_t *seq_lens, float scale,
+                    int n_seq, int n_q_tokens, int n_q_heads, int n_kv_heads, int head_dim,
+                    int c, int b, int64_t max_tokens, float *out, void *stream);
+/* The same with an explicit kernel choice (tests, benchmarks): 0 = automatic, 1 = plain
+ * kernel, 2 = tensor-core kernel (CQ_ERR_UNSUPPORTED when the shape has none). */
+int cq_prefill_attn_variant(const void *q_fp16, const void *k_codes, const void *v_codes,
+                            const float *k_cb, const float *v_cb, const int32_t *seq_lens, float scale,
+                            int n_seq, int n_q_tokens, int n_q_heads, int n_kv_heads, int head_dim,
+                            int c, int b, int64_t max_tokens, float *out, int variant, void *stream);
 
 /*
  * Same operation with an explicit kernel choice, for tests and benchmarks:

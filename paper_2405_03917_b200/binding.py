@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 # Every symbol include/cq.h declares.
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant", "cq_encode_kv",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
-           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
+           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
            "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
 
 
@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.cq_decode_attn_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
         L.cq_decode_attn.restype = i32
         L.cq_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp, sz, vp]
+        for f in (L.cq_prefill_attn, L.cq_prefill_attn_variant):
+            f.restype = i32
+        L.cq_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i32, i64, vp, vp]
+        L.cq_prefill_attn_variant.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i32, i64, vp, i32, vp]
         L.cq_decode_attn_variant.restype = i32
         L.cq_decode_attn_variant.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp,
                                              sz, i32, vp]
@@ -215,6 +219,32 @@ def cq_decode_attn(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor
                                       _dev(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
                                       workspace.numel(), variant, _stream())
     _check(st, "cq_decode_attn")
+    return out
+
+
+def cq_prefill_attn(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor,
+                    v_cb: torch.Tensor, seq_lens: torch.Tensor, scale: float, c: int, b: int, max_tokens: int,
+                    out: Optional[torch.Tensor] = None, variant: int = 0) -> torch.Tensor:
+    """Causal attention of the n_q newest cached tokens.  q fp16 (n_seq, n_q, Hq, head_dim); seq_lens counts
+    the cached tokens including the new ones.  Returns out fp32 (n_seq, n_q, Hq, head_dim)."""
+    n_seq, n_q, n_q_heads, head_dim = q.shape
+    n_kv_heads = k_cb.shape[0]
+    for nm, cb in (("k_cb", k_cb), ("v_cb", v_cb)):
+        if tuple(cb.shape) != (n_kv_heads, head_dim // max(c, 1), 1 << b, c):
+            raise ValueError(f"{nm} shape {tuple(cb.shape)} does not match heads/groups/centroids")
+    need_codes = cq_codes_bytes(n_seq, max_tokens, n_kv_heads, head_dim, c, b)
+    if need_codes and (k_codes.numel() < need_codes or v_codes.numel() < need_codes):
+        raise ValueError(f"code buffers must hold {need_codes} bytes")
+    if seq_lens.numel() != n_seq:
+        raise ValueError("seq_lens must have n_seq entries")
+    if out is None:
+        out = torch.empty(n_seq, n_q, n_q_heads, head_dim, dtype=torch.float32, device=q.device)
+    st = lib().cq_prefill_attn_variant(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+                                       _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
+                                       _dev(v_cb, torch.float32, "v_cb"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                       float(scale), n_seq, n_q, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
+                                       _dev(out, torch.float32, "out"), variant, _stream())
+    _check(st, "cq_prefill_attn")
     return out
 
 

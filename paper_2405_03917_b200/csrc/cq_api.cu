@@ -297,6 +297,37 @@ int cq_decode_attn_rope(const void* q_fp16, const void* k_codes, const void* v_c
     return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
 }
 
+int cq_prefill_attn_variant(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
+                            const float* v_cb, const int32_t* seq_lens, float scale, int n_seq, int n_q_tokens,
+                            int n_q_heads, int n_kv_heads, int head_dim, int c, int b, int64_t max_tokens, float* out,
+                            int variant, void* stream)
+{
+    if (!q_fp16 || !k_codes || !v_codes || !k_cb || !v_cb || !seq_lens || !out) return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (n_q_tokens <= 0 || n_q_tokens > max_tokens) return CQ_ERR_SHAPE;
+    if (variant < 0 || variant > 2) return CQ_ERR_SHAPE;
+    if ((int64_t)n_seq * n_q_tokens * n_q_heads > (int64_t)1 << 30) return CQ_ERR_UNSUPPORTED;
+    if (!aligned16(k_codes) || !aligned16(v_codes) || !aligned16(k_cb) || !aligned16(v_cb) || !aligned16(q_fp16) ||
+        !aligned16(out))
+        return CQ_ERR_ALIGN;
+    const bool mma_ok = prefill_mma_supported(sh);
+    if (variant == 2 && !mma_ok) return CQ_ERR_UNSUPPORTED;
+    cudaError_t e = launch_prefill(static_cast<const __half*>(q_fp16), static_cast<const uint8_t*>(k_codes),
+                                   static_cast<const uint8_t*>(v_codes), k_cb, v_cb, seq_lens, scale, sh, n_q_tokens, out,
+                                   variant == 1, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_prefill_attn(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb, const float* v_cb,
+                    const int32_t* seq_lens, float scale, int n_seq, int n_q_tokens, int n_q_heads, int n_kv_heads,
+                    int head_dim, int c, int b, int64_t max_tokens, float* out, void* stream)
+{
+    return cq_prefill_attn_variant(q_fp16, k_codes, v_codes, k_cb, v_cb, seq_lens, scale, n_seq, n_q_tokens, n_q_heads,
+                                   n_kv_heads, head_dim, c, b, max_tokens, out, 0, stream);
+}
+
 // ---------------------------------------------------------------------------------------------
 // cq_decode_attn_static: the split-K partials live in this array instead of a caller workspace.
 // In host code the name `g_static_workspace` is only a handle for the runtime, not a device

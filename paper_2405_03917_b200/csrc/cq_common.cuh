@@ -119,6 +119,12 @@ cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t
                                const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
                                float* partials, cudaStream_t st);
 
+// Causal attention of the n_q newest cached tokens of every sequence (cq_prefill.cu); `generic` forces the plain kernel.
+bool prefill_mma_supported(const Shape& sh);
+cudaError_t launch_prefill(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
+                           const int32_t* seq_lens, float scale, const Shape& sh, int n_q, float* out, bool generic,
+                           cudaStream_t st);
+
 // dst[i] = src[i] + 1 for i < n (context length after one appended token).
 cudaError_t launch_add_one(const int32_t* src, int32_t* dst, int n, cudaStream_t st);
 
