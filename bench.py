@@ -10,10 +10,10 @@ head attends over the coded cache (cq_decode_attn).  Inputs are seeded and synth
                     [--workload cfg2|cfg1|cfg4|cfg0] [--extras none|default|decode|all]
 
 Prints ONE JSON line (rank 0).  `value` is KV tokens/s with everything resident in HBM;
-`e2e` is the same metric through cq_decode_step_host with host buffers; `roofline` is the
-decode-attention kernel against the measured HBM copy bandwidth (`shared_memory` beside it
-gives the same launch against the SM's shared-memory pipe, the unit that actually limits
-it); `cpu_baseline` is the fp64 CPU oracle on a bounded sample.  With --impl reference the oracle itself is the timed arm.
+`e2e` is the same metric through cq_decode_step_host with host buffers; `roofline` describes
+the decode-attention call against the two ceilings it has - the measured HBM copy bandwidth
+and the SMs' shared-memory pipe - names the lower one as the bound and carries both
+fractions; `cpu_baseline` is the fp64 CPU oracle on a bounded sample.  With --impl reference the oracle itself is the timed arm.
 Under torchrun every rank runs its own replica of the batch (weak scaling, no collective
 on the data path).
 """
@@ -54,10 +54,10 @@ def measured_peaks():
 
 
 def kernel_source_hash():
-    """sha256 over the decode kernel's source files (the kernel the roofline object describes)."""
+    """sha256 over the decode kernels' source files (the kernels the roofline object describes)."""
     import hashlib
     h = hashlib.sha256()
-    for f in ("cq_decode.cu", "cq_common.cuh"):
+    for f in ("cq_decode.cu", "cq_decode_pair.cu", "cq_decode_util.cuh", "cq_bulk_copy.cuh", "cq_common.cuh"):
         h.update(open(os.path.join(ROOT, "paper_2405_03917_b200", "csrc", f), "rb").read())
     return h.hexdigest()
 
@@ -206,6 +206,44 @@ class DecodeState:
             ev[1].record()
 
 
+def shared_word_kernel(w) -> bool:
+    """Shapes served by the kernel that keeps two query heads in one table word (cq_decode_pair.cu)."""
+    return w.head_dim == 128 and w.b == 8 and w.c == 8 and (w.n_q_heads // w.n_kv_heads) % 4 == 0
+
+
+def decode_roofline(w, st, ms, dev, sm_mhz=None):
+    """The two ceilings of one decode-attention call that took `ms`:
+    hbm   - the bytes the call must read (codes addressed by seq_lens, both codebooks once per KV head,
+            queries, output) against the measured copy bandwidth;
+    smem  - the 4-byte shared-memory lane operations the formulation needs per (token, KV head): one bin
+            add per (group, query head) plus the table lookups (one per (group, query head); one per
+            (group, two query heads) where a table word holds two heads), against 32 lanes per clock
+            and SM at the sampled SM clock.
+    `bound` names the ceiling that allows less (the larger minimum time)."""
+    hbm, which = measured_peaks()
+    props = torch.cuda.get_device_properties(dev)
+    n_sm = props.multi_processor_count
+    mhz = float(sm_mhz) if sm_mhz else props.clock_rate / 1e3
+    R = w.n_q_heads // w.n_kv_heads
+    per_tok = w.G * R + (w.G * R // 2 if shared_word_kernel(w) else w.G * R)
+    lane_ops = float(per_tok) * st.kv_tokens() * w.n_kv_heads
+    smem_peak = n_sm * 32 * mhz * 1e6
+    nbytes = st.algorithmic_bytes()
+    t_hbm, t_smem = nbytes / (hbm * 1e9), lane_ops / smem_peak
+    a_hbm, a_smem = nbytes / (ms * 1e-3) / 1e9, lane_ops / (ms * 1e-3)
+    o = {"kernel": ("decode_pair_kernel" if shared_word_kernel(w) else
+                    "decode_wide_kernel" if w.b == 10 else "decode_tuned_kernel") + " + merge_kernel (one cq_decode_attn call)",
+         "launch_ms": ms, "algorithmic_bytes_per_launch": nbytes, "traffic": None,
+         "hbm": {"achieved": a_hbm, "peak": hbm, "unit": "GB/s", "frac": a_hbm / hbm, "frac_of_8tbs_nominal": a_hbm / 8000.0,
+                 "peak_source": which + " copy bandwidth", "min_ms": t_hbm * 1e3},
+         "smem": {"achieved": a_smem, "peak": smem_peak, "unit": "lane-ops/s", "frac": a_smem / smem_peak,
+                  "lane_ops_per_kv_head_token": per_tok, "min_ms": t_smem * 1e3,
+                  "peak_source": f"32 lanes/clk/SM x {n_sm} SMs x {mhz:.0f} MHz (sampled SM clock)"}}
+    lower = "hbm" if t_hbm >= t_smem else "smem"
+    o.update(bound=lower, achieved=o[lower]["achieved"], peak=o[lower]["peak"], unit=o[lower]["unit"], frac=o[lower]["frac"])
+    return o
+
+
 def time_steps(fn, steps, warmup, world, dev):
     for _ in range(warmup):
         fn(None)
@@ -322,10 +360,12 @@ def extra_encode_cfg3(cq, dev, reps=5):
     # ALU-pipe operations per score (two index packs and one 3-input min per two scores) on a pipe of
     # 64 lanes per clock and SM (148 SMs, nominal 1965 MHz).
     pairs = vectors * w.G * (1 << w.b)
-    alu_peak = 148 * 64 * 1965e6
+    props = torch.cuda.get_device_properties(dev)
+    n_sm, mhz = props.multi_processor_count, props.clock_rate / 1e3
+    alu_peak = n_sm * 64 * mhz * 1e6
     res["roofline"] = {"bound": "alu", "achieved": 1.5 * pairs / (ms * 1e-3), "peak": alu_peak, "unit": "lane-ops/s",
                        "frac": 1.5 * pairs / (ms * 1e-3) / alu_peak, "traffic": None,
-                       "peak_source": "64 ALU lanes/clk/SM x 148 SMs x 1965 MHz"}
+                       "peak_source": f"64 ALU lanes/clk/SM x {n_sm} SMs x {mhz:.0f} MHz (device maximum)"}
     return res
 
 
@@ -387,10 +427,43 @@ def extra_decode(cq, dev, w, reps=20):
         st.step(cq, e)
     torch.cuda.synchronize()
     ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
-    hbm, _ = measured_peaks()
-    gbs = st.algorithmic_bytes() / (ms * 1e-3) / 1e9
     return {"workload": w.name, "decode_ms": ms, "kv_tokens_per_s": st.kv_tokens() / (ms * 1e-3),
-            "query_heads_per_s": w.n_seq * w.n_q_heads / (ms * 1e-3), "gbs": gbs, "frac_of_measured_hbm": gbs / hbm}
+            "query_heads_per_s": w.n_seq * w.n_q_heads / (ms * 1e-3), "roofline": decode_roofline(w, st, ms, dev)}
+
+
+def extra_prefill(cq, dev, reps=5):
+    """cq_prefill_attn on a Mistral-7B-shaped GQA layer (CQ-8c8b): 4 sequences whose caches hold 8192 tokens,
+    the newest 2048 of which are the chunk being prefilled (causal)."""
+    w0 = synth.WORKLOADS[2]
+    n_seq, cap, n_q = 4, 8192, 2048
+    w = synth.Workload("prefill_mistral_7b_gqa_8c8b_chunk2048_of_8192", 8, w0.c, w0.b, 1, n_seq, w0.n_q_heads, w0.n_kv_heads, cap)
+    st = DecodeState(w, 0, dev, cq)
+    g = torch.Generator(device="cpu").manual_seed(88)
+    q = torch.randn(n_seq, n_q, w.n_q_heads, w.head_dim, generator=g).to(torch.float16).to(dev)
+    out = torch.empty(n_seq, n_q, w.n_q_heads, w.head_dim, dtype=torch.float32, device=dev)
+    run = lambda: cq.cq_prefill_attn(q, st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.seq_lens, st.scale, w.c, w.b, cap, out=out)
+    for _ in range(2):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    # useful contraction work: every (query, head) against the tokens up to its position, QK^T and PV
+    keys = sum(cap - n_q + i + 1 for i in range(n_q))
+    flops = 4.0 * n_seq * w.n_q_heads * keys * w.head_dim
+    peak = None
+    try:
+        peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+    except Exception:
+        peak = 1590.0
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"workload": w.name, "ms": ms, "query_tokens_per_s": n_seq * n_q / (ms * 1e-3),
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
+                         "peak_source": "measured bf16 GEMM burst (fp16 has the same nominal rate); mma.sync path"}}
 
 
 def extra_decode_rope(cq, dev, w, reps=5):
@@ -512,32 +585,19 @@ def main():
             dist.destroy_process_group()
         return 0
 
-    hbm, which = measured_peaks()
     last = states[-1]
     dec_ms = statistics.mean(inner_ms)
-    achieved = last.algorithmic_bytes() / (dec_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_tuned_kernel + merge_kernel (one cq_decode_attn call, one layer)",
-                "achieved": achieved, "peak": hbm, "peak_source": which + " copy bandwidth", "unit": "GB/s",
-                "frac": achieved / hbm, "frac_of_8tbs_nominal": achieved / 8000.0, "traffic": None,
-                "algorithmic_bytes_per_launch": last.algorithmic_bytes(), "launch_ms": dec_ms}
+    roofline = decode_roofline(w, last, dec_ms, dev, (clocks or {}).get("sm_mhz"))
     tr = os.path.join(ROOT, "profiles", "decode_traffic.json")
     if os.path.exists(tr):
         try:
             t = json.load(open(tr)).get(w.name)
-            # the counters describe one build of the kernel: any later edit of its source voids them
+            # the counters describe one build of the kernels: any later edit of their source voids them
             if t and t.get("kernel_source_sha256") == kernel_source_hash():
                 roofline["traffic"] = t["dram_bytes_per_launch"]
                 roofline["traffic_source"] = t.get("source")
         except Exception:
             pass
-    # The unit that limits the kernel: one 4-byte shared-memory lookup and one 4-byte shared-memory
-    # add per (token, KV head, group, query head of the KV head), 32 lanes per clock and SM.
-    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
-    lane_ops = 2.0 * last.kv_tokens() * w.n_kv_heads * w.G * (w.n_q_heads // w.n_kv_heads)
-    smem_peak = 148 * 32 * sm_mhz * 1e6
-    shared = {"bound": "shared-memory pipe (32 lanes/clk/SM x 148 SMs x sampled SM clock)",
-              "achieved": lane_ops / (dec_ms * 1e-3), "peak": smem_peak, "unit": "lane-ops/s",
-              "frac": lane_ops / (dec_ms * 1e-3) / smem_peak}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -547,18 +607,22 @@ def main():
             "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": args.steps * 3 * len(states),      # per layer: append-encode (K and V), attention, merge
-            "roofline": roofline, "shared_memory": shared}
+            "roofline": roofline}
 
     if args.extras != "none" and world == 1:
         extras = {}
         try:
+            del st, states, last
+            torch.cuda.empty_cache()
             if args.extras != "decode":
                 extras["encode"] = extra_encode_cfg3(cq, dev)
+            # the other decode workloads, each with its own roofline object (one layer each)
+            extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
+            extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
+            extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
+            extras["decode_cfg6_2c8b"] = extra_decode(cq, dev, synth.WORKLOADS[6])
+            extras["prefill"] = extra_prefill(cq, dev)
             if args.extras in ("decode", "all"):
-                extras["decode_cfg1"] = extra_decode(cq, dev, synth.WORKLOADS[1])
-                extras["decode_cfg4_layer0"] = extra_decode(cq, dev, synth.WORKLOADS[4])
-                extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
-                extras["decode_cfg6_2c8b"] = extra_decode(cq, dev, synth.WORKLOADS[6])
                 extras["decode_rope_cfg1"] = extra_decode_rope(cq, dev, synth.WORKLOADS[1])
                 extras["encode_cfg5_8c10b"] = extra_encode_wide(cq, dev, synth.WORKLOADS[5])
             if args.extras == "all":
@@ -567,7 +631,7 @@ def main():
             extras["error"] = repr(e)
         line["extras"] = extras
     if not args.no_cpu_baseline and world == 1:
-        del st, states, last
+        st = states = last = None
         torch.cuda.empty_cache()
         r = time_oracle(w, 10, 1, target_s=12.0)
         line["cpu_baseline"] = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
