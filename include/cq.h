@@ -195,7 +195,10 @@ int cq_decode_attn(const void *q_fp16, const void *k_codes, const void *v_codes,
  *     nothing is launched; use cq_decode_attn with your own workspace for those.
  *   - The first call on each device looks up the device address of the array (the device
  *     must be current, as for every call); make that first call before any stream capture
- *     begins.  A failure of the look-up is reported as CQ_ERR_CUDA.
+ *     begins.  A failure of the look-up is reported as CQ_ERR_CUDA.  The address is kept
+ *     for the life of the process: after cudaDeviceReset (or any other teardown of the
+ *     device's primary context) it is stale, so do not call this entry point again in a
+ *     process that has reset the device.
  *   - All calls on a device share the one array.  It keeps what the last call left in it;
  *     that is harmless, because every call overwrites each partial it later reads and
  *     nothing has to start at zero.  Two calls that overlap on the GPU (different streams,

@@ -292,6 +292,15 @@ def cq_decode_attn_static(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch
     GPU share the array and must be ordered by the caller."""
     n_seq, n_q_heads, head_dim = q.shape
     n_kv_heads = k_cb.shape[0]
+    # the same shape checks as cq_decode_attn (they allocate nothing)
+    for nm, cb in (("k_cb", k_cb), ("v_cb", v_cb)):
+        if tuple(cb.shape) != (n_kv_heads, head_dim // max(c, 1), 1 << b, c):
+            raise ValueError(f"{nm} shape {tuple(cb.shape)} does not match heads/groups/centroids")
+    need_codes = cq_codes_bytes(n_seq, max_tokens, n_kv_heads, head_dim, c, b)
+    if need_codes and (k_codes.numel() < need_codes or v_codes.numel() < need_codes):
+        raise ValueError(f"code buffers must hold {need_codes} bytes")
+    if seq_lens.numel() != n_seq:
+        raise ValueError("seq_lens must have n_seq entries")
     st = lib().cq_decode_attn_static(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
                                      _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
                                      _dev(v_cb, torch.float32, "v_cb"), _dev(seq_lens, torch.int32, "seq_lens"),

@@ -422,10 +422,12 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     for (int d = threadIdx.x; d < sh.head_dim; d += blockDim.x) qsm[d] = __half2float(qv[d]);
     for (int e = threadIdx.x; e < GK; e += blockDim.x) bins[e] = 0.f;
     const float* kcb_h = kcb + (int64_t)hkv * GK * sh.c;
+    bool staged_late = false;                  // the staged copy did not arrive in time
     if (stage_codebook) {
         // Centroid gathers then come from shared memory.  One thread hands the copy to the bulk-copy
-        // engine in pieces of 32 KiB; if the barrier does not complete within its poll limit, the
-        // threads copy the codebook themselves (the same bytes, so a late bulk copy does no harm).
+        // engine in pieces of 32 KiB.  If the barrier does not complete within its poll limit, the CTA
+        // leaves the staging area alone and gathers from global memory instead (the copy may still be
+        // writing there), and waits once more before it ends, so that no copy outlives the CTA.
         const uint32_t book_bytes = (uint32_t)GK * sh.c * sizeof(float);
         if (threadIdx.x == 0) {
             mbar_init(&book_bar, 1);
@@ -439,12 +441,8 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 bulk_copy_g2s(reinterpret_cast<char*>(kcb_s) + off, reinterpret_cast<const char*>(kcb_h) + off, piece, &book_bar);
             }
         }
-        if (__syncthreads_or(mbar_wait(&book_bar, 0) ? 0 : 1)) {      // same decision in every thread
-            const float4* src = reinterpret_cast<const float4*>(kcb_h);
-            float4* dst = reinterpret_cast<float4*>(kcb_s);
-            for (int e = threadIdx.x; e < GK * sh.c / 4; e += blockDim.x) dst[e] = src[e];
-        }
-        kcb_h = kcb_s;
+        staged_late = __syncthreads_or(mbar_wait(&book_bar, 0) ? 0 : 1) != 0;      // same decision in every thread
+        if (!staged_late) kcb_h = kcb_s;
     }
     __syncthreads();
 
@@ -553,6 +551,8 @@ decode_rope_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
         for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
         if ((threadIdx.x & 31) == 0) part[2 + d] = a;
     }
+    // a staged copy that was late must have landed before the CTA's shared memory is given up
+    if (staged_late) mbar_wait(&book_bar, 0);
 }
 
 int decode_generic_splits(const Shape& sh)

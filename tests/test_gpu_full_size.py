@@ -94,7 +94,7 @@ def seeded_items(w, n_items, seed, must=()):
 def test_config1_llama2_7b_4c8b_decode_full_size():
     w = synth.WORKLOADS[1]
     st = bench.DecodeState(w, 0, torch.device(DEV), cq)
-    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 16, 101))       # 16 items = 16 query heads x 4096 tokens
+    ties, total, a, r = check_items(w, 0, st, seeded_items(w, 64, 101))       # 64 items = 64 query heads x 4096 tokens
     assert ties <= total // 500
     print(f"config 1: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
 

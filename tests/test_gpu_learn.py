@@ -58,10 +58,24 @@ def test_one_iteration_from_common_state(c, b, n_heads, n_vec, weighted):
     want, codes, obj = oracle.lloyd_step(x.numpy(), None if w is None else w.numpy(), cb0, c, b)
     got, gobj = cq.cq_lloyd_step(x.to(DEV), None if w is None else w.to(DEV), torch.from_numpy(cb0).to(DEV), c, b)
     got, gobj = got.cpu().numpy(), gobj.cpu().numpy()
-    # fp32 accumulation of up to n_vec terms per centroid; a near-tie may move one member
+    # The assignment is cq_encode: inside the near-tie band it may give a vector to another centroid than
+    # the oracle does.  Those vectors are named (the GPU's own assignment against the oracle's) and the
+    # centroids that gain or lose one of them are set aside; every other centroid has the same members on
+    # both sides and must agree within fp32 accumulation of up to n_vec terms.
+    buf = torch.zeros(cq.cq_codes_bytes(1, n_vec, n_heads, 128, c, b), dtype=torch.uint8, device=DEV)
+    cq.cq_encode(x.view(1, n_vec, n_heads, 128).to(DEV), torch.from_numpy(cb0).to(DEV), c, b, buf, n_vec)
+    gcodes = cq.cq_codes_to_rowmajor(buf, 1, n_vec, n_heads, 128, c, b).cpu().numpy().astype(np.int64)[0]
+    moved = gcodes != codes                                              # (n_vec, n_heads, G)
+    H.check_codes(x.numpy(), cb0, gcodes, c, b)                          # ... and every move is a near-tie
+    touched = np.zeros(want.shape[:3], dtype=bool)                       # (n_heads, G, 2^b)
+    v, h, g = np.nonzero(moved)
+    touched[h, g, gcodes[v, h, g]] = True
+    touched[h, g, codes[v, h, g]] = True
+    assert moved.sum() <= max(2, moved.size // 2000), f"{moved.sum()} of {moved.size} vectors moved"
     scale = np.abs(want).max()
     close = np.abs(got - want) <= 2e-5 * scale + 2e-5 * np.abs(want)
-    assert close.mean() > 0.999, f"{(~close).sum()} of {close.size} centroid components differ"
+    bad = ~close & ~touched[..., None]
+    assert not bad.any(), f"{bad.sum()} centroid components differ although their members are the same"
     np.testing.assert_allclose(gobj, obj, rtol=1e-5)
 
 

@@ -403,3 +403,44 @@ def test_library_is_loaded_from_the_tree():
     assert os.path.samefile(os.path.dirname(cq.library_path()), os.path.dirname(cq.__file__))
     maps = open("/proc/self/maps").read()
     assert "libcq.so" in maps
+
+
+@pytest.mark.parametrize("c,n_q,n_kv", [(8, 8, 2), (8, 2, 2), (4, 2, 1), (2, 1, 1)])
+def test_repeated_calls_agree(c, n_q, n_kv):
+    # Coarsening events depend on the order in which warps arrive, so the integer weight unit - and with it the
+    # last bits of the output - may differ from run to run.  Twenty calls on the same inputs: the spread of
+    # every output element is reported and bounded (2e-6 absolute is a thousandth of the max-abs tolerance).
+    lens = [5000, 1234, 4096, 77]
+    cap = 5000
+    w = H.small_workload("repeat", 0, c, 8, len(lens), n_q, n_kv, cap)
+    xk = synth.layer_activations(w, 0, False, len(lens), cap)
+    xv = synth.layer_activations(w, 0, True, len(lens), cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False).to(DEV), synth.layer_codebooks(w, 0, True).to(DEV)
+    kb = torch.zeros(cq.cq_codes_bytes(len(lens), cap, n_kv, 128, c, 8), dtype=torch.uint8, device=DEV)
+    vb = torch.zeros_like(kb)
+    cq.cq_encode_kv(xk.to(DEV), xv.to(DEV), kcb, vcb, c, 8, kb, vb, cap)
+    q = synth.queries(0, 0, len(lens), n_q).to(DEV)
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    outs = torch.stack([cq.cq_decode_attn(q, kb, vb, kcb, vcb, sl, 128 ** -0.5, c, 8, cap).clone() for _ in range(20)])
+    spread = float((outs.max(dim=0).values - outs.min(dim=0).values).max().item())
+    print(f"c={c} R={n_q // n_kv}: largest spread over 20 calls {spread:.3e}")
+    assert spread <= 2e-6
+
+
+@pytest.mark.parametrize("n_q,n_kv", [(4, 1), (8, 1), (16, 2)])
+def test_both_tuned_kernels_for_four_heads_per_kv_head(n_q, n_kv):
+    # CQ-8c8b with a multiple of four query heads per KV head has two tuned kernels: the one with two query heads
+    # per table word (variant 2, what variant 0 picks) and the one with a table word per query head (variant 3).
+    lens = [3000, 17, 2049, 0, 512]
+    cap = 3000
+    w = H.small_workload("two_kernels", 0, 8, 8, len(lens), n_q, n_kv, cap)
+    xk = synth.layer_activations(w, 0, False, len(lens), cap)
+    xv = synth.layer_activations(w, 0, True, len(lens), cap)
+    kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
+    kc_rm, _ = H.oracle_encode_rowmajor(xk, kcb, 8, 8)
+    vc_rm, _ = H.oracle_encode_rowmajor(xv, vcb, 8, 8)
+    q = synth.queries(0, 0, len(lens), n_q)
+    for variant in (2, 3):
+        got, ref = attn_both(q, kc_rm, vc_rm, kcb, vcb, lens, 128 ** -0.5, 8, 8, variant)
+        for s_ in range(len(lens)):
+            H.check_attn(got[s_], ref[s_], f"variant {variant} seq {s_}")
