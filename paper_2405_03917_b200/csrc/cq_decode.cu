@@ -221,7 +221,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     }
     const int head_group = item % n_head_groups;      // query heads head_group * R ... + R - 1
     const int hkv = kShared ? head_group / kv_share : head_group;
-    const int64_t s = item / n_head_groups;
+    const int64_t s = seq_by_rank(seq_lens, (int)sh.n_seq, sh.max_tokens, item / n_head_groups);
 
     int64_t n = seq_lens[s];
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
@@ -781,7 +781,7 @@ decode_wide_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
         part = whole ? 0 : (blockIdx.x - tail_first) % n_parts;
     }
     const int hq = item % sh.n_q_heads;
-    const int64_t s = item / sh.n_q_heads;
+    const int64_t s = seq_by_rank(seq_lens, (int)sh.n_seq, sh.max_tokens, item / sh.n_q_heads);
     const int hkv = hq / sh.R;
 
     int64_t n = seq_lens[s];

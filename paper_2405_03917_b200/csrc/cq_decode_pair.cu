@@ -331,7 +331,7 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     }
     const int head_group = item % n_head_groups;
     const int hkv = head_group / kv_share;
-    const int64_t s = item / n_head_groups;
+    const int64_t s = seq_by_rank(seq_lens, (int)sh.n_seq, sh.max_tokens, item / n_head_groups);
 
     // (the query travels while the context length is looked up)
     const __half* qrow = q + (s * sh.n_q_heads + (int64_t)head_group * R) * 128;

@@ -84,6 +84,27 @@ __device__ __forceinline__ void load_centroid(const float* p, float (&cv)[kC], b
     }
 }
 
+// Work items are handed out longest context first: with contexts of different lengths the CTAs that start
+// last are then the short ones, and the launch ends more evenly.  Returns the sequence whose context is the
+// `rank`-th longest (ties: lower index first).  Every warp finds it by itself - lane j holds the length of
+// sequence j and counts, by shuffles, the sequences that come before its own - so no barrier and no shared
+// memory are needed.  Batches of more than 32 sequences keep their own order (the search would cost more
+// than it gains).  Entered by whole warps.
+__device__ __forceinline__ int seq_by_rank(const int32_t* __restrict__ seq_lens, int n_seq, int64_t max_tokens, int rank)
+{
+    if (n_seq > 32 || n_seq < 2) return rank;
+    const int lane = threadIdx.x & 31;
+    int mine = lane < n_seq ? seq_lens[lane] : -1;
+    mine = mine < 0 ? (lane < n_seq ? 0 : -1) : (mine > max_tokens ? (int)max_tokens : mine);
+    int before = 0;
+    for (int k = 0; k < n_seq; ++k) {
+        const int other = __shfl_sync(0xffffffffu, mine, k);
+        before += (other > mine || (other == mine && k < lane)) ? 1 : 0;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, lane < n_seq && before == rank);
+    return hit ? __ffs(hit) - 1 : rank;
+}
+
 // byte `k` (0..15) of a 16-byte code word
 __device__ __forceinline__ uint32_t word32(const uint4& w, int k)
 {
