@@ -557,7 +557,18 @@ def main():
     D = w.head_dim
     ws_h = torch.empty(cq.cq_decode_step_host_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, w.c, w.b, st.cap),
                        dtype=torch.uint8, device=dev)
-    host = [(x.q.cpu().pin_memory(), x.k_new.cpu().pin_memory(), x.v_new.cpu().pin_memory()) for x in states]
+    def pinned_block(x):
+        # query, key and value of a step back to back in one pinned block: they travel in one copy
+        parts = (x.q, x.k_new, x.v_new)
+        block = torch.empty(sum(p.numel() for p in parts), dtype=torch.float16).pin_memory()
+        views, at = [], 0
+        for p in parts:
+            v = block[at:at + p.numel()].view(p.shape)
+            v.copy_(p.cpu())
+            views.append(v)
+            at += p.numel()
+        return tuple(views)
+    host = [pinned_block(x) for x in states]
     lens_h = (st.lens_cpu - 1).contiguous()
     out_h = torch.empty(w.n_seq, w.n_q_heads, D, dtype=torch.float32).pin_memory()
 

@@ -339,6 +339,8 @@ int cq_learn_centroids(const void *x_fp16, const float *weights, const double *u
  *
  *   q_host       [n_seq][n_q_heads][head_dim] fp16   (pinned memory recommended)
  *   k_new_host, v_new_host   [n_seq][n_kv_heads][head_dim] fp16
+ *                (when q_host, k_new_host and v_new_host lie back to back in host memory, in
+ *                this order, the three travel in one copy instead of three)
  *   seq_lens_host [n_seq] int32: tokens already cached, each < max_tokens
  *   k_codes, v_codes, k_cb, v_cb   device, as in cq_decode_attn (codes are updated)
  *   out_host     [n_seq][n_q_heads][head_dim] fp32

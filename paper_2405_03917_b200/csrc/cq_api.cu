@@ -496,14 +496,37 @@ int cq_decode_step_host(const void* q_host, const void* k_new_host, const void* 
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     // The new token is appended at position seq_lens[s]; the attention then reads seq_lens[s] + 1 tokens.
-    if (cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
-    if (cudaMemcpyAsync(d_k, k_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
-    if (cudaMemcpyAsync(d_v, v_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
-    if (cudaMemcpyAsync(d_sl, seq_lens_host, slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    // Few, large copies: query, key and value travel in one copy when the caller keeps them back to back
+    // in host memory (the staging areas are then packed the same way); both length arrays travel in one
+    // copy from a small array on the stack (pageable source: the call returns once it has been read).
+    const bool packed = static_cast<const char*>(k_new_host) == static_cast<const char*>(q_host) + qb &&
+                        static_cast<const char*>(v_new_host) == static_cast<const char*>(k_new_host) + kvb &&
+                        qb % 16 == 0 && kvb % 16 == 0;
+    if (packed) {
+        d_k = d_q + qb;
+        d_v = d_k + kvb;            // (fits: the three areas were sized with their paddings)
+        if (cudaMemcpyAsync(d_q, q_host, qb + 2 * kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    } else {
+        if (cudaMemcpyAsync(d_q, q_host, qb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+        if (cudaMemcpyAsync(d_k, k_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+        if (cudaMemcpyAsync(d_v, v_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    }
+    constexpr int kStackSeqs = 1024;
+    if (n_seq <= kStackSeqs) {
+        int32_t both[2 * kStackSeqs];
+        for (int s = 0; s < n_seq; ++s) {
+            both[s] = seq_lens_host[s];
+            both[n_seq + s] = seq_lens_host[s] + 1;
+        }
+        d_sl1 = d_sl + n_seq;       // (fits: two padded areas were reserved)
+        if (cudaMemcpyAsync(d_sl, both, 2 * slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    } else {
+        if (cudaMemcpyAsync(d_sl, seq_lens_host, slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+        if (launch_add_one(d_sl, d_sl1, n_seq, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    }
     int st = cq_encode_kv(d_k, d_v, k_cb, v_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, k_codes, v_codes,
                           stream);
     if (st != CQ_OK) return st;
-    if (launch_add_one(d_sl, d_sl1, n_seq, cs) != cudaSuccess) return CQ_ERR_CUDA;
     st = cq_decode_attn(d_q, k_codes, v_codes, k_cb, v_cb, d_sl1, scale, n_seq, n_q_heads, n_kv_heads, head_dim, c, b,
                         max_tokens, d_out, attn_ws, attn_bytes, stream);
     if (st != CQ_OK) return st;

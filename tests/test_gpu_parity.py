@@ -366,7 +366,9 @@ def test_token_permutation_and_seq_len_padding_invariance():
     np.testing.assert_allclose(out, base, rtol=0, atol=2e-5)
 
 
-def test_decode_step_from_host_buffers():
+@pytest.mark.parametrize("packed", [False, True])
+def test_decode_step_from_host_buffers(packed):
+    # packed: query, key and value back to back in one pinned block (they then travel in one copy)
     c, b, D, cap, n_seq, n_q, n_kv = 8, 8, 128, 200, 3, 4, 2
     w = H.small_workload("t", 66, c, b, n_seq, n_q, n_kv, cap)
     xk = synth.layer_activations(w, 0, False, n_seq, cap)
@@ -381,7 +383,15 @@ def test_decode_step_from_host_buffers():
     ws = torch.empty(cq.cq_decode_step_host_workspace_bytes(n_seq, n_q, n_kv, D, c, b, cap), dtype=torch.uint8,
                      device=DEV)
     out_host = torch.empty(n_seq, n_q, D, dtype=torch.float32).pin_memory()
-    cq.cq_decode_step_host(q.pin_memory(), k_new.pin_memory(), v_new.pin_memory(),
+    if packed:
+        block = torch.empty(q.numel() + k_new.numel() + v_new.numel(), dtype=torch.float16).pin_memory()
+        hq = block[:q.numel()].view(q.shape)
+        hk = block[q.numel():q.numel() + k_new.numel()].view(k_new.shape)
+        hv = block[q.numel() + k_new.numel():].view(v_new.shape)
+        hq.copy_(q); hk.copy_(k_new); hv.copy_(v_new)
+    else:
+        hq, hk, hv = q.pin_memory(), k_new.pin_memory(), v_new.pin_memory()
+    cq.cq_decode_step_host(hq, hk, hv,
                            torch.tensor(lens, dtype=torch.int32), kbuf, vbuf, kcb.to(DEV), vcb.to(DEV),
                            D ** -0.5, c, b, cap, out_host, ws)
     # oracle: same cache with the new token written at position lens[s], context lens[s] + 1
