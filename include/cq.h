@@ -286,11 +286,15 @@ int cq_decode_attn_variant(const void *q_fp16, const void *k_codes, const void *
                            int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
                            int variant, void *stream);
 
-/* cq_encode with an explicit kernel choice (same variant numbers, and 3 = the
- * few-vector kernel: one warp per (vector, group) with the group's codebook in
- * shared memory, which variant 0 picks for appends of up to 128 vectors per head
- * when the shape has no tuned kernel;
- * CQ_ERR_UNSUPPORTED when 2^b * c * 4 bytes exceed 48 KiB). */
+/* cq_encode with an explicit kernel choice: 0 = automatic, 1 = generic kernel,
+ * 2 = the tuned kernels built on warp-level tensor-core instructions
+ * (CQ_ERR_UNSUPPORTED when the shape has none), 3 = the few-vector kernel: one
+ * warp per (vector, group) with the group's codebook in shared memory, which
+ * variant 0 picks for appends of up to 128 vectors per head when the shape has no
+ * tuned kernel (CQ_ERR_UNSUPPORTED when 2^b * c * 4 bytes exceed 48 KiB),
+ * 4 = the bulk kernel with accumulators in tensor memory (head_dim 128, b = 8,
+ * c in {2, 4, 8}, else CQ_ERR_UNSUPPORTED), which variant 0 picks for these shapes
+ * once the input fills the device.  Every variant returns the same codes. */
 int cq_encode_variant(const void *x_fp16, const float *codebooks, const int32_t *seq_offsets,
                       int64_t n_seq, int64_t n_tokens, int64_t token_offset, int64_t max_tokens,
                       int n_heads, int head_dim, int c, int b, void *codes_out, int variant,

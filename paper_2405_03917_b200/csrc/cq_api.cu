@@ -140,10 +140,11 @@ int cq_encode_variant(const void* x_fp16, const float* codebooks, const int32_t*
     if (n_tokens < 0 || token_offset < 0) return CQ_ERR_SHAPE;
     if (!seq_offsets && token_offset + n_tokens > max_tokens) return CQ_ERR_SHAPE;
     if (!aligned16(x_fp16) || !aligned16(codebooks) || !aligned16(codes_out)) return CQ_ERR_ALIGN;
-    if (variant < 0 || variant > 3) return CQ_ERR_SHAPE;
+    if (variant < 0 || variant > 4) return CQ_ERR_SHAPE;
     if (n_tokens == 0) return CQ_OK;
     const bool tuned_ok = encode_tuned_supported(sh);
     if (variant == 2 && !tuned_ok) return CQ_ERR_UNSUPPORTED;
+    if (variant == 4 && !encode_tc_supported(sh)) return CQ_ERR_UNSUPPORTED;
     const bool small_ok = encode_small_supported(sh);
     if (variant == 3 && !small_ok) return CQ_ERR_UNSUPPORTED;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
@@ -155,10 +156,16 @@ int cq_encode_variant(const void* x_fp16, const float* codebooks, const int32_t*
                                              token_offset, static_cast<uint8_t*>(codes_out), cs);
         return es == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
     }
+    if (variant == 4) {
+        cudaError_t et = launch_encode_tc(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh, n_tokens, token_offset,
+                                          static_cast<uint8_t*>(codes_out), cs, nullptr, nullptr, nullptr);
+        return et == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    }
     const bool use_tuned = variant == 2 || (variant == 0 && tuned_ok);
     cudaError_t e = use_tuned
                         ? launch_encode_tuned(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh, n_tokens,
-                                              token_offset, static_cast<uint8_t*>(codes_out), cs)
+                                              token_offset, static_cast<uint8_t*>(codes_out), cs, nullptr, nullptr, nullptr,
+                                              variant == 0)
                         : launch_encode_generic(static_cast<const __half*>(x_fp16), codebooks, seq_offsets, sh,
                                                 n_tokens, token_offset, static_cast<uint8_t*>(codes_out), cs);
     return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;

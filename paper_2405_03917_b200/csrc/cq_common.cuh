@@ -86,11 +86,18 @@ cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_
 bool encode_small_supported(const Shape& sh);       // few-vector kernel: the group's codebook fits 48 KiB
 cudaError_t launch_encode_small(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                 int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
+// tcgen05 / tensor-memory encode kernel (head_dim 128, b = 8, c in {2, 4, 8}); same arguments as launch_encode_tuned
+bool encode_tc_supported(const Shape& sh);
+cudaError_t launch_encode_tc(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh, int64_t n_tokens,
+                             int64_t token_offset, uint8_t* codes, cudaStream_t st, const __half* x2, const float* cb2,
+                             uint8_t* codes2);
 bool encode_tuned_supported(const Shape& sh);
 // (x2, cb2, codes2): an optional second tensor of the same shape, encoded by the same launch.
+// allow_tc: bulk inputs of byte codes go to the tensor-memory kernel (false: always the mma.sync kernels).
 cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                 int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st,
-                                const __half* x2 = nullptr, const float* cb2 = nullptr, uint8_t* codes2 = nullptr);
+                                const __half* x2 = nullptr, const float* cb2 = nullptr, uint8_t* codes2 = nullptr,
+                                bool allow_tc = true);
 
 cudaError_t launch_to_rowmajor(const uint8_t* codes, const Shape& sh, uint8_t* rowmajor, cudaStream_t st);
 cudaError_t launch_from_rowmajor(const uint8_t* rowmajor, const Shape& sh, uint8_t* codes, cudaStream_t st);

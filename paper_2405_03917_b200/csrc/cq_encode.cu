@@ -67,6 +67,13 @@ __device__ __forceinline__ float min3f(float a, float b, float c)
     return d;
 }
 
+// D = A * B (no accumulator to clear beforehand)
+__device__ __forceinline__ void mma_f16_first(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
 __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
     asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -336,9 +343,10 @@ encode_tuned_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1
                 const uint32_t i0 = nt * 8, i1 = nt * 8 + 1;      // centroid index without the lane's 2p
 #pragma unroll
                 for (int mt = 0; mt < kMT; ++mt) {
-                    float d[4] = {0.f, 0.f, 0.f, 0.f};
+                    float d[4];
+                    mma_f16_first(d, a[mt][0], b[0].x, b[0].y);
 #pragma unroll
-                    for (int st = 0; st < C::kSteps; ++st) mma_f16(d, a[mt][st], b[st].x, b[st].y);
+                    for (int st = 1; st < C::kSteps; ++st) mma_f16(d, a[mt][st], b[st].x, b[st].y);
                     const float v0p = __uint_as_float((__float_as_uint(d[0]) & keep) | i0);
                     const float v1p = __uint_as_float((__float_as_uint(d[1]) & keep) | i1);
                     const float v2p = __uint_as_float((__float_as_uint(d[2]) & keep) | i0);
@@ -501,11 +509,13 @@ bool encode_tuned_supported(const Shape& sh)
 
 cudaError_t launch_encode_tuned(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                 int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st,
-                                const __half* x2, const float* cb2, uint8_t* codes2)
+                                const __half* x2, const float* cb2, uint8_t* codes2, bool allow_tc)
 {
     const int64_t n_vec = sh.n_seq * n_tokens;
     if (n_vec == 0) return cudaSuccess;
     const bool few = n_vec * sh.n_kv_heads < (int64_t)device_sm_count() * 512 * 2;    // not enough vectors for 64 per warp
+    if (allow_tc && !few && encode_tc_supported(sh))
+        return launch_encode_tc(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2);
     if (sh.b > 8) {
         switch (sh.c) {
             case 2: return few ? launch_enc<2, 1, true>(x, cb, seq_offsets, sh, n_tokens, token_offset, codes, st, x2, cb2, codes2)

@@ -46,7 +46,7 @@ def test_encode_shapes_and_ragged_tails(c, b, head_dim, n_heads, n_tokens):
     xk, xv, kcb, vcb, _ = H.generic_case(11 * c + b, 2, n_tokens, n_heads, n_heads, head_dim, c, b)
     tuned = head_dim == 128 and b == 8 and c in (2, 4, 8)
     for x, cb in ((xk, kcb), (xv, vcb)):
-        for variant in (1, 0, 3) + ((2,) if tuned else ()):       # generic, automatic, few-vector, tuned
+        for variant in (1, 0, 3) + ((2, 4) if tuned else ()):     # generic, automatic, few-vector, tuned, tensor-memory
             _, rm = encode_both(x, cb, c, b, n_tokens, variant)
             H.check_codes(x.numpy().reshape(-1, n_heads, head_dim), cb.numpy(),
                           rm.reshape(-1, n_heads, head_dim // c), c, b)
@@ -62,10 +62,65 @@ def test_encode_codebook_contains_inputs_and_exact_ties():
     hh = torch.arange(H_)[None, :, None]
     gg = torch.arange(D // c)[None, None, :]
     x = cb[hh, gg, pick[0]].reshape(1, 64, H_, D)        # group g of token t = centroid pick[t, h, g]
-    for variant in (1, 0, 2, 3):
+    for variant in (1, 0, 2, 3, 4):
         _, rm = encode_both(x.to(torch.float16), cb, c, b, 64, variant)
         want = torch.where(pick == 200, torch.tensor(7), pick).numpy()
         assert np.array_equal(rm.astype(np.int64), want)
+
+
+@pytest.mark.parametrize("c,n_seq,n_tokens,n_heads", [(8, 2, 700, 3), (2, 1, 1300, 2), (4, 3, 257, 2), (8, 1, 9, 1)])
+def test_tensor_memory_encode_kernel(c, n_seq, n_tokens, n_heads):
+    # several 256-vector tiles with a ragged last one, groups split over CTAs, sequences that end inside a tile
+    xk, xv, kcb, vcb, _ = H.generic_case(900 + c + n_tokens, n_seq, n_tokens, n_heads, n_heads, 128, c, 8)
+    for x, cb in ((xk, kcb), (xv, vcb)):
+        _, rm = encode_both(x, cb, c, 8, n_tokens, 4)
+        H.check_codes(x.numpy().reshape(-1, n_heads, 128), cb.numpy(), rm.reshape(-1, n_heads, 128 // c), c, 8)
+    # the key and the value in one launch, appended behind per-sequence offsets
+    cap = n_tokens + 40
+    nbytes = cq.cq_codes_bytes(n_seq, cap, n_heads, 128, c, 8)
+    want_k, want_v, got_k, got_v = (torch.zeros(nbytes, dtype=torch.uint8, device=DEV) for _ in range(4))
+    offs = torch.arange(n_seq, dtype=torch.int32, device=DEV) * 13
+    cq.cq_encode(xk.to(DEV), kcb.to(DEV), c, 8, want_k, cap, seq_offsets=offs, variant=1)
+    cq.cq_encode(xv.to(DEV), vcb.to(DEV), c, 8, want_v, cap, seq_offsets=offs, variant=1)
+    cq.cq_encode(xk.to(DEV), kcb.to(DEV), c, 8, got_k, cap, seq_offsets=offs, variant=4)
+    cq.cq_encode(xv.to(DEV), vcb.to(DEV), c, 8, got_v, cap, seq_offsets=offs, variant=4)
+    assert torch.equal(got_k, want_k) and torch.equal(got_v, want_v)
+
+
+def test_tensor_memory_encode_codebooks_fp16_cannot_carry():
+    # centroids beyond the fp16 range in one group, huge norms in another: those groups are encoded the exact way
+    c, n_heads, n_tokens = 8, 2, 300
+    xk, _, kcb, _, _ = H.generic_case(77, 1, n_tokens, n_heads, n_heads, 128, c, 8)
+    kcb = kcb.clone()
+    kcb[0, 3] *= 30000.0
+    kcb[1, 5, 17] = 250.0
+    kcb[1, 9] *= 1e-6
+    for variant in (4, 2):
+        _, rm = encode_both(xk, kcb, c, 8, n_tokens, variant)
+        H.check_codes(xk.numpy().reshape(-1, n_heads, 128), kcb.numpy(), rm.reshape(-1, n_heads, 128 // c), c, 8)
+
+
+def test_bulk_encode_takes_the_same_codes_on_every_path():
+    # enough vectors that the automatic choice is the bulk kernel (key and value in one launch as well)
+    c, n_heads, n_tokens = 8, 32, 4800
+    g = torch.Generator().manual_seed(31)
+    xk = torch.randn(1, n_tokens, n_heads, 128, generator=g).to(torch.float16)
+    xv = (torch.randn(1, n_tokens, n_heads, 128, generator=g) * 0.3).to(torch.float16)
+    kcb = torch.randn(n_heads, 16, 256, c, generator=g)
+    vcb = torch.randn(n_heads, 16, 256, c, generator=g) * 0.3
+    nbytes = cq.cq_codes_bytes(1, n_tokens, n_heads, 128, c, 8)
+    bufs = {}
+    for variant in (0, 2, 4):
+        bufs[variant], _ = encode_both(xk, kcb, c, 8, n_tokens, variant)
+    assert torch.equal(bufs[0], bufs[2]) and torch.equal(bufs[0], bufs[4])
+    got_k, got_v = (torch.zeros(nbytes, dtype=torch.uint8, device=DEV) for _ in range(2))
+    cq.cq_encode_kv(xk.to(DEV), xv.to(DEV), kcb.to(DEV), vcb.to(DEV), c, 8, got_k, got_v, n_tokens)
+    want_v, _ = encode_both(xv, vcb, c, 8, n_tokens, 2)
+    assert torch.equal(got_k, bufs[2]) and torch.equal(got_v, want_v)
+    # a sample of the tokens against the oracle
+    idx = np.random.default_rng(3).integers(0, n_tokens, size=64)
+    rm = cq.cq_codes_to_rowmajor(got_k, 1, n_tokens, n_heads, 128, c, 8).cpu().numpy()[0, idx]
+    H.check_codes(xk[0, idx].numpy(), kcb.numpy(), rm, c, 8)
 
 
 def test_append_positions_and_untouched_bytes():
