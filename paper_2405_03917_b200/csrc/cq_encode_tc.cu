@@ -19,17 +19,21 @@
 // lane i, and a thread reads the 256 scores of ITS row with tcgen05.ld: no accumulator registers
 // to clear, no B fragments to fetch in the selecting warps, no quad to merge, and - because the
 // winner is found by exact re-evaluation anyway - no index packed into every score.  A thread
-// keeps the minimum of each of 32 subsets of the centroids (index mod 32), one 3-input min per
-// two scores; the subset with the smallest minimum is evaluated exactly (8 centroids, direct form
+// keeps the minimum of each of 16 subsets of the centroids (index mod 16), one 3-input min per
+// two scores; the subset with the smallest minimum is evaluated exactly (16 centroids, direct form
 // sum (x - C)^2 in fp32, lowest index on ties) and the second smallest subset minimum bounds
 // every other centroid from below.  The exact winner is accepted if that bound is farther away
 // than a bound on the evaluation error; otherwise (near-ties, ties across subsets, codebooks
 // fp16 cannot carry) the warp recomputes that row over all 256 centroids exactly.
 //
 // A CTA of 8 warps holds two tiles of 128 vectors (warps 0-3 and 4-7; a warp reaches the tensor
-// memory lanes 32 (warp % 4) ... + 31) of one head, which share the prepared centroids, and walks
-// the groups: operands of group k + 1 are prepared and its MMAs run while group k's rows are
-// finished.  Tensor memory: 2 x 256 columns, all that an SM has, so one CTA per SM.
+// memory lanes 32 (warp % 4) ... + 31) of one head, which share the prepared centroids.  Two CTAs
+// live on an SM, each with 256 of its 512 tensor-memory columns, so a tile's accumulator is
+// 128 x 128: the scores of a step arrive in two halves (centroids 0-127, then 128-255) through the
+// same columns.  While one half is scanned the tensor core has nothing of this CTA to do; the
+// other CTA, and the operand preparation and row finishing placed behind each MMA issue, fill
+// the time.  A CTA takes up to four pairs of row tiles through every group before it moves to
+// the next group, so a group's centroids are prepared once per up to 1024 vectors.
 #include "cq_common.cuh"
 
 namespace cq {
@@ -51,19 +55,21 @@ struct TcCfg {
     static constexpr int kCbf = 256 * kC * 4;                     // the group's centroids as fp32
     static constexpr int kAOff = 0;                               // [2 buffers]
     static constexpr int kBOff = kAOff + 2 * kABuf;               // [2 buffers]
-    static constexpr int kCbfOff = kBOff + 2 * kBBuf;             // [3 slots]
-    static constexpr int kCtlOff = kCbfOff + 3 * kCbf;
+    static constexpr int kCbfOff = kBOff + 2 * kBBuf;             // [2 slots]
+    static constexpr int kCtlOff = kCbfOff + 2 * kCbf;
     static constexpr int kUsedBytes = kCtlOff + 256;
-    static constexpr int kSmemBytes = 120 * 1024;                 // more than half an SM: one CTA per SM (it takes all tensor memory)
+    static constexpr int kSmemBytes = 100 * 1024;                 // two CTAs per SM and never three (each holds half the tensor memory)
     static_assert(kUsedBytes <= kSmemBytes, "shared memory");
 };
 
+constexpr int kTcColumns = 256;            // tensor-memory columns of a CTA: 128 per row tile
+
 struct TcCtl {
-    int range_flag[3][8];      // per warp, non-zero: its centroids of the prepared group hold values fp16 cannot carry
-    float nmax[3][8];          // per warp, the largest ||C_j||^2 among its centroids of the prepared group
+    int range_flag[2][8];      // per warp, non-zero: its centroids of the prepared group hold values fp16 cannot carry
+    float nmax[2][8];          // per warp, the largest ||C_j||^2 among its centroids of the prepared group
     uint32_t tmem_base;
-    int wait_failed;           // a wait on the MMA barrier gave up
-    uint64_t bar;              // completion of the MMAs of one group
+    int wait_failed;           // a wait on an MMA barrier gave up
+    uint64_t bar[2];           // completion of the MMAs of the low / high half of a step
 };
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -102,28 +108,32 @@ __device__ __forceinline__ uint64_t tc_desc(uint32_t saddr, uint32_t chunk_strid
     return d;
 }
 
-// D[128 x 256] (+)= A[128 x 16] * B[256 x 16]^T, fp16 operands from shared memory, fp32 accumulator in tensor memory
+// D[128 x 128] (+)= A[128 x 16] * B[128 x 16]^T, fp16 operands from shared memory, fp32 accumulator in tensor memory
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate)
 {
-    // instruction descriptor: D fp32, A and B fp16, both K-major, N = 256, M = 128
-    const uint32_t idesc = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+    // instruction descriptor: D fp32, A and B fp16, both K-major, N = 128, M = 128
+    const uint32_t idesc = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0) : "memory");
 }
 
-// 64 consecutive accumulator columns of this thread's row, complete on return (the loads and the wait for them are one
-// statement, so that nothing that uses the values can be scheduled ahead of the wait)
-__device__ __forceinline__ void tc_ld64(float (&lo)[32], float (&hi)[32], uint32_t taddr)
+// Starts the load of 32 consecutive accumulator columns of this thread's row; the values are there after tc_ld_wait.
+__device__ __forceinline__ void tc_ld32_issue(float (&v)[32], uint32_t taddr)
 {
-    uint32_t* u = reinterpret_cast<uint32_t*>(lo);
-    uint32_t* w = reinterpret_cast<uint32_t*>(hi);
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%64];\n\t"
-                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%65];\n\t"
-                 "tcgen05.wait::ld.sync.aligned;"
-                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31]),
-                   "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]), "=r"(w[8]), "=r"(w[9]), "=r"(w[10]), "=r"(w[11]), "=r"(w[12]), "=r"(w[13]), "=r"(w[14]), "=r"(w[15]), "=r"(w[16]), "=r"(w[17]), "=r"(w[18]), "=r"(w[19]), "=r"(w[20]), "=r"(w[21]), "=r"(w[22]), "=r"(w[23]), "=r"(w[24]), "=r"(w[25]), "=r"(w[26]), "=r"(w[27]), "=r"(w[28]), "=r"(w[29]), "=r"(w[30]), "=r"(w[31])
-                 : "r"(taddr), "r"(taddr + 32u) : "memory");
+    uint32_t* u = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+                 : "r"(taddr) : "memory");
+}
+// Waits for the loads issued so far.  The registers pass through the statement, so that nothing that uses them is
+// scheduled ahead of the wait.
+__device__ __forceinline__ void tc_ld_wait(float (&v)[32])
+{
+    uint32_t* u = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]), "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]), "+r"(u[16]), "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]), "+r"(u[23]), "+r"(u[24]), "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]), "+r"(u[30]), "+r"(u[31])
+                 :: "memory");
 }
 
 // Waits for the phase with the given parity; gives up after a bounded number of polls (returns false).
@@ -166,27 +176,38 @@ __device__ __forceinline__ int tc_exact_code(const float (&xg)[kC], const float*
     return arg;
 }
 
-// B operand of one group: thread j prepares centroid j (K slots as in the header comment), keeps the fp32 centroid
-// for the exact evaluations, and every warp leaves its largest squared norm and its range flag in the control block.
+
+// Centroid j = threadIdx.x of a group, from global memory into registers.
 template <int kC>
-__device__ __forceinline__ void tc_prepare_b(const float* __restrict__ cb_g, unsigned char* bbuf, float* cbf, TcCtl* ctl, int slot)
+__device__ __forceinline__ void tc_fetch_centroid(const float* __restrict__ cb_g, float (&cv)[kC])
 {
-    using C = TcCfg<kC>;
     const int j = threadIdx.x;
-    float cv[kC];
     if (kC == 2) {
         const float2 a = *reinterpret_cast<const float2*>(cb_g + j * 2);
         cv[0] = a.x; cv[1] = a.y;
-        *reinterpret_cast<float2*>(cbf + j * 2) = a;
     } else {
         const float4 a = *reinterpret_cast<const float4*>(cb_g + j * kC);
         cv[0] = a.x; cv[1] = a.y; cv[2 % kC] = a.z; cv[3 % kC] = a.w;
-        *reinterpret_cast<float4*>(cbf + j * kC) = a;
         if (kC == 8) {
             const float4 b = *reinterpret_cast<const float4*>(cb_g + j * kC + 4);
             cv[4 % kC] = b.x; cv[5 % kC] = b.y; cv[6 % kC] = b.z; cv[7 % kC] = b.w;
-            *reinterpret_cast<float4*>(cbf + j * kC + (kC == 8 ? 4 : 0)) = b;
         }
+    }
+}
+
+// B operand of one group: thread j prepares centroid j (K slots as in the header comment), keeps the fp32 centroid
+// for the exact evaluations, and every warp leaves its largest squared norm and its range flag in the control block.
+template <int kC>
+__device__ __forceinline__ void tc_prepare_b(const float (&cv)[kC], unsigned char* bbuf, float* cbf, TcCtl* ctl, int slot)
+{
+    using C = TcCfg<kC>;
+    const int j = threadIdx.x;
+    if (kC == 2) {
+        *reinterpret_cast<float2*>(cbf + j * 2) = make_float2(cv[0], cv[1]);
+    } else {
+#pragma unroll
+        for (int w = 0; w < kC; w += 4)
+            *reinterpret_cast<float4*>(cbf + j * kC + w) = make_float4(cv[w], cv[w + 1], cv[(w + 2) % kC], cv[(w + 3) % kC]);
     }
     float nrm = 0.f, amax = 0.f;
     float t0[kC], t1[kC], t2[kC];
@@ -200,10 +221,10 @@ __device__ __forceinline__ void tc_prepare_b(const float* __restrict__ cb_g, uns
     tc_split3(nrm, n0, n1, n2);
     const bool bad = !(amax < 16000.f) || !(nrm < 60000.f);
     const unsigned any_bad = __ballot_sync(0xffffffffu, bad);
-    const float wmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(nrm)));   // nrm >= 0: bits order as values
+    const float wmax = __uint_as_float(__reduce_max_sync(0xffffffffu, bad ? 0u : __float_as_uint(nrm)));   // nrm >= 0: bits order as values
     if ((threadIdx.x & 31) == 0) {
         ctl->range_flag[slot][threadIdx.x >> 5] = any_bad != 0;
-        ctl->nmax[slot][threadIdx.x >> 5] = bad ? 0.f : wmax;
+        ctl->nmax[slot][threadIdx.x >> 5] = wmax;
     }
     const uint32_t ones = 0x3c003c00u;               // half2(1, 1)
     uint32_t pr[C::kSteps][8];
@@ -246,8 +267,22 @@ __device__ __forceinline__ void tc_prepare_b(const float* __restrict__ cb_g, uns
     }
 }
 
-// A operand row of one vector for one group.  xw: the group's kC / 2 words (two fp16 channels each), X its squared
-// norm; atile: the row tile's first K step.
+// The kC / 2 words (two fp16 channels each) of one group of one vector, from global memory.
+template <int kC>
+__device__ __forceinline__ void tc_fetch_x(const __half* gp, uint32_t (&xw)[kC / 2])
+{
+    if (kC == 2) {
+        xw[0] = *reinterpret_cast<const uint32_t*>(gp);
+    } else if (kC == 4) {
+        const uint2 t = *reinterpret_cast<const uint2*>(gp);
+        xw[0] = t.x; xw[1 % (kC / 2)] = t.y;
+    } else {
+        const uint4 t = *reinterpret_cast<const uint4*>(gp);
+        xw[0] = t.x; xw[1 % (kC / 2)] = t.y; xw[2 % (kC / 2)] = t.z; xw[3 % (kC / 2)] = t.w;
+    }
+}
+
+// A operand row of one vector for one group.  xw: the group's words, X its squared norm; atile: the row tile's first K step.
 template <int kC>
 __device__ __forceinline__ void tc_build_a(const uint32_t (&xw)[kC / 2], float X, unsigned char* atile, int row)
 {
@@ -280,10 +315,12 @@ __device__ __forceinline__ void tc_build_a(const uint32_t (&xw)[kC / 2], float X
 
 static_assert(sizeof(TcCtl) <= 256, "control block");
 
+// One step = one pair of row tiles (256 vectors) against one group.  A CTA takes 2^log_rt pairs of row tiles through
+// its groups; blockIdx.x = (block of row-tile pairs, head, group split).
 template <int kC>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, const int32_t* __restrict__ seq_offsets,
-                 Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes1, int groups_per_cta,
+                 Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes1, int groups_per_cta, int log_rt,
                  const __half* __restrict__ x2, const float* __restrict__ cb2, uint8_t* __restrict__ codes2)
 {
     const __half* x = blockIdx.y ? x2 : x1;
@@ -303,22 +340,20 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
     const int n_gsplit = (G + groups_per_cta - 1) / groups_per_cta;
     const int gs = blockIdx.x % n_gsplit;
     const int h = (blockIdx.x / n_gsplit) % n_heads;
-    const int64_t tile = blockIdx.x / (n_gsplit * n_heads);
+    const int64_t tile_block = blockIdx.x / (n_gsplit * n_heads);
     const int g_begin = gs * groups_per_cta;
     const int g_end = g_begin + groups_per_cta < G ? g_begin + groups_per_cta : G;
-    const int n_steps = g_end - g_begin;
+    const int rt_mask = (1 << log_rt) - 1;
+    const int n_steps = (g_end - g_begin) << log_rt;     // step st: group g_begin + (st >> log_rt), row-tile pair st & rt_mask
 
-    const int64_t v = tile * kTcTileVecs + tile_id * 128 + row;
-    const bool live = v < n_vec;
-    const __half* xrow = x + ((live ? v : 0) * n_heads + h) * 128;
-
-    // tensor memory (warp 0 allocates all 512 columns and frees them at the end), the MMA barrier
+    // tensor memory (warp 0 allocates the CTA's columns and frees them at the end), the MMA barriers
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(tc_smem_u32(&ctl->tmem_base)) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&ctl->tmem_base)), "n"(kTcColumns) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (threadIdx.x == 32) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(&ctl->bar)) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(&ctl->bar[0])) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(tc_smem_u32(&ctl->bar[1])) : "memory");
         ctl->wait_failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -326,99 +361,124 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctl->tmem_base);
-    const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)tile_id * 256u;
+    const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)tile_id * 128u;
 
-    auto group_ptr = [&](int st) { return cb + ((int64_t)h * G + g_begin + st) * 256 * kC; };
     auto a_buf = [&](int buf) { return tc_smem + C::kAOff + buf * C::kABuf; };
     auto b_buf = [&](int buf) { return tc_smem + C::kBOff + buf * C::kBBuf; };
     auto cbf_slot = [&](int slot) { return reinterpret_cast<float*>(tc_smem + C::kCbfOff + slot * C::kCbf); };
+    auto vec_of = [&](int st) { return (tile_block * (rt_mask + 1) + (st & rt_mask)) * kTcTileVecs + tile_id * 128 + row; };
 
-    // operands of step st into buffer st % 2 (centroids and control words into slot st % 3); returns the row's words
-    uint32_t xw_next[kC / 2];
-    float X_next;
-    auto prepare = [&](int st) {
-        tc_prepare_b<kC>(group_ptr(st), b_buf(st & 1), cbf_slot(st % 3), ctl, st % 3);
-        X_next = 0.f;
+    // Operands of a step travel global memory -> registers (fetch, half a step ahead) -> shared memory (build).
+    uint32_t xw_pf[kC / 2];
+    float cv_pf[kC];
+    auto fetch = [&](int st) {
+        const int64_t v = vec_of(st);
 #pragma unroll
-        for (int w = 0; w < kC / 2; ++w) xw_next[w] = 0u;
-        if (live) {
-            const __half* gp = xrow + (g_begin + st) * kC;
-            if (kC == 2) {
-                xw_next[0] = *reinterpret_cast<const uint32_t*>(gp);
-            } else if (kC == 4) {
-                const uint2 t = *reinterpret_cast<const uint2*>(gp);
-                xw_next[0] = t.x; xw_next[1 % (kC / 2)] = t.y;
-            } else {
-                const uint4 t = *reinterpret_cast<const uint4*>(gp);
-                xw_next[0] = t.x; xw_next[1 % (kC / 2)] = t.y; xw_next[2 % (kC / 2)] = t.z; xw_next[3 % (kC / 2)] = t.w;
-            }
-#pragma unroll
-            for (int w = 0; w < kC / 2; ++w) {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&xw_next[w]));
-                X_next = fmaf(f.x, f.x, X_next);
-                X_next = fmaf(f.y, f.y, X_next);
-            }
-        }
-        tc_build_a<kC>(xw_next, X_next, a_buf(st & 1) + tile_id * C::kSteps * C::kATile, row);
+        for (int w = 0; w < kC / 2; ++w) xw_pf[w] = 0u;
+        if (v < n_vec) tc_fetch_x<kC>(x + (v * n_heads + h) * 128 + (g_begin + (st >> log_rt)) * kC, xw_pf);
+        if ((st & rt_mask) == 0) tc_fetch_centroid<kC>(cb + ((int64_t)h * G + g_begin + (st >> log_rt)) * 256 * kC, cv_pf);
     };
-    // the MMAs of step st (both row tiles), then the commit that arrives on the barrier when they are done
-    auto issue = [&](int st) {
-        const uint32_t a0 = tc_smem_u32(a_buf(st & 1)), b0 = tc_smem_u32(b_buf(st & 1));
+    uint32_t xw_nxt[kC / 2];
+    float X_nxt;
+    auto build = [&](int st) {
+        const int gslot = (st >> log_rt) & 1;
+        if ((st & rt_mask) == 0) tc_prepare_b<kC>(cv_pf, b_buf(gslot), cbf_slot(gslot), ctl, gslot);
+        X_nxt = 0.f;
+#pragma unroll
+        for (int w = 0; w < kC / 2; ++w) {
+            xw_nxt[w] = xw_pf[w];
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&xw_pf[w]));
+            X_nxt = fmaf(f.x, f.x, X_nxt);
+            X_nxt = fmaf(f.y, f.y, X_nxt);
+        }
+        tc_build_a<kC>(xw_pf, X_nxt, a_buf(st & 1) + tile_id * C::kSteps * C::kATile, row);
+    };
+    // the MMAs of one half of step st (both row tiles; half 1 = centroids 128 ... 255), then the commit that arrives
+    // on that half's barrier when they are done
+    auto issue = [&](int st, int half) {
+        const uint32_t a0 = tc_smem_u32(a_buf(st & 1)), b0 = tc_smem_u32(b_buf((st >> log_rt) & 1)) + half * (128 * 16);
 #pragma unroll
         for (int t = 0; t < 2; ++t)
 #pragma unroll
             for (int s = 0; s < C::kSteps; ++s)
-                tc_mma(tmem_base + t * 256, tc_desc(a0 + (t * C::kSteps + s) * C::kATile, 128 * 16),
+                tc_mma(tmem_base + t * 128, tc_desc(a0 + (t * C::kSteps + s) * C::kATile, 128 * 16),
                        tc_desc(b0 + s * C::kBTile, 256 * 16), s > 0 ? 1u : 0u);
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&ctl->bar)) : "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&ctl->bar[half])) : "memory");
+    };
+    // minima of the 16 subsets (centroid index mod 16) over the 128 scores of the half that is in tensor memory
+    auto scan_half = [&](float (&sb)[16]) {
+        float va[32], vb[32];
+        auto consume = [&](const float (&v)[32]) {
+#pragma unroll
+            for (int q = 0; q < 16; ++q) sb[q] = tc_min3(sb[q], v[q], v[q + 16]);
+        };
+        tc_ld32_issue(va, taddr);
+        tc_ld_wait(va);
+        tc_ld32_issue(vb, taddr + 32);
+        consume(va);
+        tc_ld_wait(vb);
+        tc_ld32_issue(va, taddr + 64);
+        consume(vb);
+        tc_ld_wait(va);
+        tc_ld32_issue(vb, taddr + 96);
+        consume(va);
+        tc_ld_wait(vb);
+        consume(vb);
     };
 
-    prepare(0);
+    fetch(0);
+    build(0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        issue(0);
+        issue(0, 0);
     }
 
     for (int st = 0; st < n_steps; ++st) {
-        const int g = g_begin + st, slot = st % 3;
+        const int g = g_begin + (st >> log_rt), slot = (st >> log_rt) & 1;
         uint32_t xw[kC / 2];
 #pragma unroll
-        for (int w = 0; w < kC / 2; ++w) xw[w] = xw_next[w];
-        const float X = X_next;
-        if (st + 1 < n_steps) prepare(st + 1);           // while the MMAs of step st run
+        for (int w = 0; w < kC / 2; ++w) xw[w] = xw_nxt[w];
+        const float X = X_nxt;
+        if (st + 1 < n_steps) fetch(st + 1);
 
         bool scores_valid = *reinterpret_cast<volatile int*>(&ctl->wait_failed) == 0;
-        if (scores_valid && !tc_wait(&ctl->bar, (uint32_t)(st & 1))) {
+        if (scores_valid && !tc_wait(&ctl->bar[0], (uint32_t)(st & 1))) {
             ctl->wait_failed = 1;                        // never expected: every row of this CTA goes the exact way from here on
             scores_valid = false;
         }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-
-        // subset minima of the row's 256 scores: subset q = centroid index mod 32
-        float sb[32];
+        float sb[16];
 #pragma unroll
-        for (int q = 0; q < 32; ++q) sb[q] = kTcInf;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float s0[32], s1[32];
-            tc_ld64(s0, s1, taddr + 64 * i);
-#pragma unroll
-            for (int q = 0; q < 32; ++q) sb[q] = tc_min3(sb[q], s0[q], s1[q]);
+        for (int q = 0; q < 16; ++q) sb[q] = kTcInf;
+        scan_half(sb);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();                                 // the low half has been read: its columns take the high half
+        if (threadIdx.x == 0 && *reinterpret_cast<volatile int*>(&ctl->wait_failed) == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            issue(st, 1);
         }
+        if (st + 1 < n_steps) build(st + 1);             // while the MMAs of the high half run
+
+        if (scores_valid && !tc_wait(&ctl->bar[1], (uint32_t)(st & 1))) {
+            ctl->wait_failed = 1;
+            scores_valid = false;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        scan_half(sb);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();                                 // tensor memory is free again; the operands of step st + 1 are complete
         if (threadIdx.x == 0 && st + 1 < n_steps && *reinterpret_cast<volatile int*>(&ctl->wait_failed) == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            issue(st + 1);
+            issue(st + 1, 0);
         }
 
-        // control words of this step
-        bool out_of_range = false;
-        float nmax = 0.f;
+        // control words of this step's group
+        bool out_of_range;
+        float nmax;
         {
             const int4 f0 = *reinterpret_cast<const int4*>(&ctl->range_flag[slot][0]);
             const int4 f1 = *reinterpret_cast<const int4*>(&ctl->range_flag[slot][4]);
@@ -429,25 +489,30 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
         }
         const float* cbf = cbf_slot(slot);
 
-        // smallest and second smallest subset minimum; the subset number rides in the low five mantissa bits
+        // smallest and second smallest subset minimum (a tournament of (smallest, second) pairs); the subset number
+        // rides in the low four mantissa bits, which also makes the 16 values differ
         float m1v, s2;
         {
-            float t[32];
+            float lo[8], hi[8];
 #pragma unroll
-            for (int q = 0; q < 32; ++q) t[q] = __uint_as_float((__float_as_uint(sb[q]) & ~31u) | (uint32_t)q);
-            float a[11];
+            for (int i = 0; i < 8; ++i) {
+                const float ta = __uint_as_float((__float_as_uint(sb[2 * i]) & ~15u) | (uint32_t)(2 * i));
+                const float tb = __uint_as_float((__float_as_uint(sb[2 * i + 1]) & ~15u) | (uint32_t)(2 * i + 1));
+                lo[i] = fminf(ta, tb);
+                hi[i] = fmaxf(ta, tb);
+            }
 #pragma unroll
-            for (int q = 0; q < 10; ++q) a[q] = tc_min3(t[3 * q], t[3 * q + 1], t[3 * q + 2]);
-            a[10] = fminf(t[30], t[31]);
-            m1v = fminf(tc_min3(tc_min3(a[0], a[1], a[2]), tc_min3(a[3], a[4], a[5]), tc_min3(a[6], a[7], a[8])), fminf(a[9], a[10]));
+            for (int n = 4; n >= 1; n >>= 1)
 #pragma unroll
-            for (int q = 0; q < 32; ++q) t[q] = t[q] > m1v ? t[q] : kTcInf;          // all t differ: only the smallest drops out
-#pragma unroll
-            for (int q = 0; q < 10; ++q) a[q] = tc_min3(t[3 * q], t[3 * q + 1], t[3 * q + 2]);
-            a[10] = fminf(t[30], t[31]);
-            s2 = fminf(tc_min3(tc_min3(a[0], a[1], a[2]), tc_min3(a[3], a[4], a[5]), tc_min3(a[6], a[7], a[8])), fminf(a[9], a[10]));
+                for (int i = 0; i < n; ++i) {
+                    const float m = fminf(lo[i], lo[i + n]);
+                    hi[i] = tc_min3(fmaxf(lo[i], lo[i + n]), hi[i], hi[i + n]);
+                    lo[i] = m;
+                }
+            m1v = lo[0];
+            s2 = hi[0];
         }
-        const int qw = (int)(__float_as_uint(m1v) & 31u);
+        const int qw = (int)(__float_as_uint(m1v) & 15u);
         float xg[kC];
 #pragma unroll
         for (int w = 0; w < kC / 2; ++w) {
@@ -455,12 +520,12 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
             xg[2 * w] = f.x;
             xg[2 * w + 1] = f.y;
         }
-        // the winner's subset, exactly: centroids qw, qw + 32, ..., qw + 224 in ascending order
+        // the winner's subset, exactly: centroids qw, qw + 16, ..., qw + 240 in ascending order
         float dbest = kTcInf;
         int code = 0;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int j = qw + 32 * k;
+        for (int k = 0; k < 16; ++k) {
+            const int j = qw + 16 * k;
             float cc[kC];
             if (kC == 2) {
                 const float2 t2 = *reinterpret_cast<const float2*>(cbf + j * 2);
@@ -481,10 +546,12 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
             if (dd < dbest) { dbest = dd; code = j; }            // ascending j: strict < keeps the lowest
         }
         // Evaluation error of a score: fp32 accumulation of up to ~20 terms bounded by 2 (X + N) in magnitude, plus
-        // the five mantissa bits given to the subset number.  dbest is exact.
-        const float ss = __uint_as_float(__float_as_uint(s2) & ~31u);
-        const float tau = 1.6e-5f * (X + nmax) + 8e-6f * fabsf(ss);
+        // the four mantissa bits given to the subset number.  dbest is exact.
+        const float ss = __uint_as_float(__float_as_uint(s2) & ~15u);
+        const float tau = 1.6e-5f * (X + nmax) + 4e-6f * fabsf(ss);
         const bool certain = scores_valid && !out_of_range && (ss - dbest > tau);
+        const int64_t v = vec_of(st);
+        const bool live = v < n_vec;
         // exact recomputation of the uncertain rows, one row at a time by the whole warp
         unsigned pending = __ballot_sync(0xffffffffu, !certain && live);
         while (pending) {
@@ -515,7 +582,7 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
     __syncthreads();
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTcColumns) : "memory");
     }
 }
 
@@ -525,20 +592,25 @@ cudaError_t launch_enc_tc(const __half* x, const float* cb, const int32_t* seq_o
 {
     using C = TcCfg<kC>;
     const int64_t n_vec = sh.n_seq * n_tokens;
-    const int64_t tiles = (n_vec + kTcTileVecs - 1) / kTcTileVecs;
+    const int64_t tile_pairs = (n_vec + kTcTileVecs - 1) / kTcTileVecs;
+    const int64_t slots = 2 * (int64_t)device_sm_count();          // CTAs in flight
+    // row-tile pairs per CTA: as many as leave four waves of CTAs
+    int log_rt = 2;
+    while (log_rt > 0 && ((tile_pairs + (1 << log_rt) - 1) >> log_rt) * sh.n_kv_heads < 4 * slots) --log_rt;
+    const int64_t blocks = (tile_pairs + (1 << log_rt) - 1) >> log_rt;
     // split the groups over CTAs while the grid would leave SMs idle
-    int64_t n_gsplit = ((int64_t)device_sm_count() + tiles * sh.n_kv_heads - 1) / (tiles * sh.n_kv_heads);
+    int64_t n_gsplit = (slots + blocks * sh.n_kv_heads - 1) / (blocks * sh.n_kv_heads);
     if (n_gsplit > C::G) n_gsplit = C::G;
     if (n_gsplit < 1) n_gsplit = 1;
     const int groups_per_cta = (int)((C::G + n_gsplit - 1) / n_gsplit);
     n_gsplit = (C::G + groups_per_cta - 1) / groups_per_cta;
-    const int64_t grid = tiles * sh.n_kv_heads * n_gsplit;
+    const int64_t grid = blocks * sh.n_kv_heads * n_gsplit;
     if (grid > 0x7fffffff) return cudaErrorInvalidConfiguration;
     constexpr int kSlot = 44 + (kC == 2 ? 0 : kC == 4 ? 1 : 2);       // call-site slots 44 ... 46 of ensure_dynamic_smem
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(encode_tc_kernel<kC>), C::kSmemBytes, kSlot);
     if (e != cudaSuccess) return e;
     encode_tc_kernel<kC><<<dim3((unsigned)grid, x2 ? 2u : 1u), kTcThreads, C::kSmemBytes, st>>>(
-        x, cb, seq_offsets, sh, n_tokens, token_offset, codes, groups_per_cta, x2, cb2, codes2);
+        x, cb, seq_offsets, sh, n_tokens, token_offset, codes, groups_per_cta, log_rt, x2, cb2, codes2);
     return cudaGetLastError();
 }
 
