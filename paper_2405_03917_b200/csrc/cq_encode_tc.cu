@@ -26,22 +26,21 @@
 // than a bound on the evaluation error; otherwise (near-ties, ties across subsets, codebooks
 // fp16 cannot carry) the warp recomputes that row over all 256 centroids exactly.
 //
-// A CTA of 8 warps holds two tiles of 128 vectors (warps 0-3 and 4-7; a warp reaches the tensor
-// memory lanes 32 (warp % 4) ... + 31) of one head, which share the prepared centroids.  Two CTAs
-// live on an SM, each with 256 of its 512 tensor-memory columns, so a tile's accumulator is
-// 128 x 128: the scores of a step arrive in two halves (centroids 0-127, then 128-255) through the
-// same columns.  While one half is scanned the tensor core has nothing of this CTA to do; the
-// other CTA, and the operand preparation and row finishing placed behind each MMA issue, fill
-// the time.  A CTA takes up to four pairs of row tiles through every group before it moves to
-// the next group, so a group's centroids are prepared once per up to 1024 vectors.
+// A CTA is one tile of 128 vectors of one head: 4 warps, warp w owning the tensor memory lanes
+// 32 w ... 32 w + 31, and 128 tensor-memory columns, so that four CTAs (three for c = 8, whose
+// operands take more shared memory) live on an SM and fill each other's waits.  The accumulator is
+// therefore 128 x 128: the scores of a step arrive in two halves (centroids 0-127, then 128-255)
+// through the same columns, and the operand preparation and the row finishing are placed behind
+// the MMA issues.  A CTA takes up to eight row tiles through every group before it moves to the
+// next group, so a group's centroids are prepared once per up to 1024 vectors.
 #include "cq_common.cuh"
 
 namespace cq {
 
 namespace {
 
-constexpr int kTcThreads = 256;
-constexpr int kTcTileVecs = 256;          // vectors per CTA: two tiles of 128
+constexpr int kTcThreads = 128;
+constexpr int kTcTileVecs = 128;          // vectors of a row tile
 constexpr float kTcInf = __builtin_huge_valf();
 
 template <int kC>
@@ -50,26 +49,39 @@ struct TcCfg {
     static constexpr int kSteps = (kC == 8) ? 2 : 1;              // K steps (16 fp16 slots each)
     static constexpr int kATile = 128 * 32;                       // bytes of one A tile of one K step
     static constexpr int kBTile = 256 * 32;
-    static constexpr int kABuf = 2 * kSteps * kATile;             // both row tiles
+    static constexpr int kABuf = kSteps * kATile;
     static constexpr int kBBuf = kSteps * kBTile;
     static constexpr int kCbf = 256 * kC * 4;                     // the group's centroids as fp32
+    static constexpr int kMaxLogRt = (kC == 8) ? 2 : 3;           // up to 2^kMaxLogRt row tiles per CTA
+    static constexpr int kCtasPerSm = (kC == 8) ? 3 : 4;
     static constexpr int kAOff = 0;                               // [2 buffers]
     static constexpr int kBOff = kAOff + 2 * kABuf;               // [2 buffers]
     static constexpr int kCbfOff = kBOff + 2 * kBBuf;             // [2 slots]
-    static constexpr int kCtlOff = kCbfOff + 2 * kCbf;
+    static constexpr int kRowOff = kCbfOff + 2 * kCbf;            // [row tiles][128 threads] row records
+    static constexpr int kCtlOff = kRowOff + (1 << kMaxLogRt) * kTcThreads * 16;
     static constexpr int kUsedBytes = kCtlOff + 256;
-    static constexpr int kSmemBytes = 100 * 1024;                 // two CTAs per SM and never three (each holds half the tensor memory)
-    static_assert(kUsedBytes <= kSmemBytes, "shared memory");
+    // at least 46 KiB, so that a fifth CTA (for which no tensor memory would be left) never fits an SM
+    static constexpr int kSmemBytes = kUsedBytes > 46 * 1024 ? kUsedBytes : 46 * 1024;
+    static_assert(kCtasPerSm * (kSmemBytes + 1024) <= 228 * 1024, "shared memory of an SM");
+    static_assert((kCtasPerSm + 1) * (kSmemBytes + 1024) > 228 * 1024, "one CTA too many would fit");
 };
 
-constexpr int kTcColumns = 256;            // tensor-memory columns of a CTA: 128 per row tile
+constexpr int kTcColumns = 128;            // tensor-memory columns of a CTA
+
+// What a thread needs of one of its rows, worked out once: where the vector's head slice starts and where its code of
+// group 0 goes (the code of group g follows kTokenBlock * g bytes on).
+struct TcRow {
+    const __half* x;           // null: no such vector
+    int64_t code_offset;       // negative: the token has no position in the cache
+};
+static_assert(sizeof(TcRow) == 16, "row record");
 
 struct TcCtl {
-    int range_flag[2][8];      // per warp, non-zero: its centroids of the prepared group hold values fp16 cannot carry
-    float nmax[2][8];          // per warp, the largest ||C_j||^2 among its centroids of the prepared group
+    int range_flag[2][8];      // per warp and pass, non-zero: those centroids of the prepared group hold values fp16 cannot carry
+    float nmax[2][8];          // per warp and pass, the largest ||C_j||^2 among those centroids
     uint32_t tmem_base;
     int wait_failed;           // a wait on an MMA barrier gave up
-    uint64_t bar[2];           // completion of the MMAs of the low / high half of a step
+    uint64_t bar[2];           // completion of the MMA of the low / high half of a step
 };
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -177,11 +189,10 @@ __device__ __forceinline__ int tc_exact_code(const float (&xg)[kC], const float*
 }
 
 
-// Centroid j = threadIdx.x of a group, from global memory into registers.
+// Centroid j of a group, from global memory into registers.
 template <int kC>
-__device__ __forceinline__ void tc_fetch_centroid(const float* __restrict__ cb_g, float (&cv)[kC])
+__device__ __forceinline__ void tc_fetch_centroid(const float* __restrict__ cb_g, int j, float (&cv)[kC])
 {
-    const int j = threadIdx.x;
     if (kC == 2) {
         const float2 a = *reinterpret_cast<const float2*>(cb_g + j * 2);
         cv[0] = a.x; cv[1] = a.y;
@@ -195,13 +206,12 @@ __device__ __forceinline__ void tc_fetch_centroid(const float* __restrict__ cb_g
     }
 }
 
-// B operand of one group: thread j prepares centroid j (K slots as in the header comment), keeps the fp32 centroid
-// for the exact evaluations, and every warp leaves its largest squared norm and its range flag in the control block.
+// B operand of one group, one centroid: K slots as in the header comment; keeps the fp32 centroid for the exact
+// evaluations; every warp leaves its largest squared norm and its range flag of this pass in the control block.
 template <int kC>
-__device__ __forceinline__ void tc_prepare_b(const float (&cv)[kC], unsigned char* bbuf, float* cbf, TcCtl* ctl, int slot)
+__device__ __forceinline__ void tc_prepare_b(const float (&cv)[kC], int j, unsigned char* bbuf, float* cbf, TcCtl* ctl, int slot, int pass)
 {
     using C = TcCfg<kC>;
-    const int j = threadIdx.x;
     if (kC == 2) {
         *reinterpret_cast<float2*>(cbf + j * 2) = make_float2(cv[0], cv[1]);
     } else {
@@ -223,8 +233,8 @@ __device__ __forceinline__ void tc_prepare_b(const float (&cv)[kC], unsigned cha
     const unsigned any_bad = __ballot_sync(0xffffffffu, bad);
     const float wmax = __uint_as_float(__reduce_max_sync(0xffffffffu, bad ? 0u : __float_as_uint(nrm)));   // nrm >= 0: bits order as values
     if ((threadIdx.x & 31) == 0) {
-        ctl->range_flag[slot][threadIdx.x >> 5] = any_bad != 0;
-        ctl->nmax[slot][threadIdx.x >> 5] = wmax;
+        ctl->range_flag[slot][pass * 4 + (threadIdx.x >> 5)] = any_bad != 0;
+        ctl->nmax[slot][pass * 4 + (threadIdx.x >> 5)] = wmax;
     }
     const uint32_t ones = 0x3c003c00u;               // half2(1, 1)
     uint32_t pr[C::kSteps][8];
@@ -315,10 +325,10 @@ __device__ __forceinline__ void tc_build_a(const uint32_t (&xw)[kC / 2], float X
 
 static_assert(sizeof(TcCtl) <= 256, "control block");
 
-// One step = one pair of row tiles (256 vectors) against one group.  A CTA takes 2^log_rt pairs of row tiles through
-// its groups; blockIdx.x = (block of row-tile pairs, head, group split).
+// One step = one row tile (128 vectors) against one group.  A CTA takes 2^log_rt row tiles through its groups;
+// blockIdx.x = (block of row tiles, head, group split).
 template <int kC>
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, TcCfg<kC>::kCtasPerSm)
 encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, const int32_t* __restrict__ seq_offsets,
                  Shape sh, int64_t n_tokens, int64_t token_offset, uint8_t* __restrict__ codes1, int groups_per_cta, int log_rt,
                  const __half* __restrict__ x2, const float* __restrict__ cb2, uint8_t* __restrict__ codes2)
@@ -332,8 +342,7 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
     TcCtl* ctl = reinterpret_cast<TcCtl*>(tc_smem + C::kCtlOff);
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int tile_id = warp >> 2;                       // row tile of this warp
-    const int row = (warp & 3) * 32 + lane;              // row within the tile = tensor memory lane
+    const int row = threadIdx.x;                         // row within the tile = tensor memory lane
     const int n_heads = sh.n_kv_heads;
     const int64_t n_vec = sh.n_seq * n_tokens;
 
@@ -344,7 +353,7 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
     const int g_begin = gs * groups_per_cta;
     const int g_end = g_begin + groups_per_cta < G ? g_begin + groups_per_cta : G;
     const int rt_mask = (1 << log_rt) - 1;
-    const int n_steps = (g_end - g_begin) << log_rt;     // step st: group g_begin + (st >> log_rt), row-tile pair st & rt_mask
+    const int n_steps = (g_end - g_begin) << log_rt;     // step st: group g_begin + (st >> log_rt), row tile st & rt_mask
 
     // tensor memory (warp 0 allocates the CTA's columns and frees them at the end), the MMA barriers
     if (warp == 0) {
@@ -361,28 +370,46 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctl->tmem_base);
-    const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)tile_id * 128u;
+    const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
 
     auto a_buf = [&](int buf) { return tc_smem + C::kAOff + buf * C::kABuf; };
     auto b_buf = [&](int buf) { return tc_smem + C::kBOff + buf * C::kBBuf; };
     auto cbf_slot = [&](int slot) { return reinterpret_cast<float*>(tc_smem + C::kCbfOff + slot * C::kCbf); };
-    auto vec_of = [&](int st) { return (tile_block * (rt_mask + 1) + (st & rt_mask)) * kTcTileVecs + tile_id * 128 + row; };
+    TcRow* rows = reinterpret_cast<TcRow*>(tc_smem + C::kRowOff) + threadIdx.x;      // record of row tile r: rows[r * kTcThreads]
+    for (int r = 0; r <= rt_mask; ++r) {
+        const int64_t v = (tile_block * (rt_mask + 1) + r) * kTcTileVecs + row;
+        TcRow rec;
+        rec.x = nullptr;
+        rec.code_offset = -1;
+        if (v < n_vec) {
+            rec.x = x + (v * n_heads + h) * 128;
+            const int64_t s = v / n_tokens, i = v % n_tokens;
+            const int64_t pos = token_offset + (seq_offsets ? seq_offsets[s] : 0) + i;
+            if (pos >= 0 && pos < sh.max_tokens) rec.code_offset = code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, 0) + pos % kTokenBlock;
+        }
+        rows[r * kTcThreads] = rec;                      // read back by this thread only
+    }
 
-    // Operands of a step travel global memory -> registers (fetch, half a step ahead) -> shared memory (build).
+    // The vector's words travel global memory -> registers (fetch, half a step ahead) -> shared memory (build).
     uint32_t xw_pf[kC / 2];
-    float cv_pf[kC];
     auto fetch = [&](int st) {
-        const int64_t v = vec_of(st);
+        const __half* xr = rows[(st & rt_mask) * kTcThreads].x;
 #pragma unroll
         for (int w = 0; w < kC / 2; ++w) xw_pf[w] = 0u;
-        if (v < n_vec) tc_fetch_x<kC>(x + (v * n_heads + h) * 128 + (g_begin + (st >> log_rt)) * kC, xw_pf);
-        if ((st & rt_mask) == 0) tc_fetch_centroid<kC>(cb + ((int64_t)h * G + g_begin + (st >> log_rt)) * 256 * kC, cv_pf);
+        if (xr) tc_fetch_x<kC>(xr + (g_begin + (st >> log_rt)) * kC, xw_pf);
     };
     uint32_t xw_nxt[kC / 2];
     float X_nxt;
     auto build = [&](int st) {
         const int gslot = (st >> log_rt) & 1;
-        if ((st & rt_mask) == 0) tc_prepare_b<kC>(cv_pf, b_buf(gslot), cbf_slot(gslot), ctl, gslot);
+        if ((st & rt_mask) == 0) {                       // a new group: centroids threadIdx.x and threadIdx.x + 128
+            const float* cb_g = cb + ((int64_t)h * G + g_begin + (st >> log_rt)) * 256 * kC;
+            float cv[2][kC];
+            tc_fetch_centroid<kC>(cb_g, threadIdx.x, cv[0]);
+            tc_fetch_centroid<kC>(cb_g, threadIdx.x + 128, cv[1]);
+            tc_prepare_b<kC>(cv[0], threadIdx.x, b_buf(gslot), cbf_slot(gslot), ctl, gslot, 0);
+            tc_prepare_b<kC>(cv[1], threadIdx.x + 128, b_buf(gslot), cbf_slot(gslot), ctl, gslot, 1);
+        }
         X_nxt = 0.f;
 #pragma unroll
         for (int w = 0; w < kC / 2; ++w) {
@@ -391,18 +418,15 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
             X_nxt = fmaf(f.x, f.x, X_nxt);
             X_nxt = fmaf(f.y, f.y, X_nxt);
         }
-        tc_build_a<kC>(xw_pf, X_nxt, a_buf(st & 1) + tile_id * C::kSteps * C::kATile, row);
+        tc_build_a<kC>(xw_pf, X_nxt, a_buf(st & 1), row);
     };
-    // the MMAs of one half of step st (both row tiles; half 1 = centroids 128 ... 255), then the commit that arrives
-    // on that half's barrier when they are done
+    // the MMA of one half of step st (half 1 = centroids 128 ... 255), then the commit that arrives on that half's
+    // barrier when it is done
     auto issue = [&](int st, int half) {
         const uint32_t a0 = tc_smem_u32(a_buf(st & 1)), b0 = tc_smem_u32(b_buf((st >> log_rt) & 1)) + half * (128 * 16);
 #pragma unroll
-        for (int t = 0; t < 2; ++t)
-#pragma unroll
-            for (int s = 0; s < C::kSteps; ++s)
-                tc_mma(tmem_base + t * 128, tc_desc(a0 + (t * C::kSteps + s) * C::kATile, 128 * 16),
-                       tc_desc(b0 + s * C::kBTile, 256 * 16), s > 0 ? 1u : 0u);
+        for (int s = 0; s < C::kSteps; ++s)
+            tc_mma(tmem_base, tc_desc(a0 + s * C::kATile, 128 * 16), tc_desc(b0 + s * C::kBTile, 256 * 16), s > 0 ? 1u : 0u);
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(tc_smem_u32(&ctl->bar[half])) : "memory");
     };
     // minima of the 16 subsets (centroid index mod 16) over the 128 scores of the half that is in tensor memory
@@ -460,7 +484,7 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             issue(st, 1);
         }
-        if (st + 1 < n_steps) build(st + 1);             // while the MMAs of the high half run
+        if (st + 1 < n_steps) build(st + 1);             // while the MMA of the high half runs
 
         if (scores_valid && !tc_wait(&ctl->bar[1], (uint32_t)(st & 1))) {
             ctl->wait_failed = 1;
@@ -520,9 +544,9 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
             xg[2 * w] = f.x;
             xg[2 * w + 1] = f.y;
         }
-        // the winner's subset, exactly: centroids qw, qw + 16, ..., qw + 240 in ascending order
-        float dbest = kTcInf;
-        int code = 0;
+        // the winner's subset, exactly: centroids qw, qw + 16, ..., qw + 240; the smallest distance by a tournament in
+        // which the lower index wins ties
+        float dk[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const int j = qw + 16 * k;
@@ -543,15 +567,32 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
                 const float diff = xg[i] - cc[i];
                 dd = fmaf(diff, diff, dd);
             }
-            if (dd < dbest) { dbest = dd; code = j; }            // ascending j: strict < keeps the lowest
+            dk[k] = dd;
         }
+        int ik[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool right = dk[2 * i + 1] < dk[2 * i];        // strict: the lower index keeps a tie
+            ik[i] = right ? 2 * i + 1 : 2 * i;
+            dk[i] = right ? dk[2 * i + 1] : dk[2 * i];
+        }
+#pragma unroll
+        for (int n = 4; n >= 1; n >>= 1)
+#pragma unroll
+            for (int i = 0; i < n; ++i) {
+                const bool right = dk[2 * i + 1] < dk[2 * i];
+                ik[i] = right ? ik[2 * i + 1] : ik[2 * i];
+                dk[i] = right ? dk[2 * i + 1] : dk[2 * i];
+            }
+        float dbest = dk[0];
+        int code = qw + 16 * ik[0];
         // Evaluation error of a score: fp32 accumulation of up to ~20 terms bounded by 2 (X + N) in magnitude, plus
         // the four mantissa bits given to the subset number.  dbest is exact.
         const float ss = __uint_as_float(__float_as_uint(s2) & ~15u);
         const float tau = 1.6e-5f * (X + nmax) + 4e-6f * fabsf(ss);
         const bool certain = scores_valid && !out_of_range && (ss - dbest > tau);
-        const int64_t v = vec_of(st);
-        const bool live = v < n_vec;
+        const TcRow rec = rows[(st & rt_mask) * kTcThreads];
+        const bool live = rec.x != nullptr;
         // exact recomputation of the uncertain rows, one row at a time by the whole warp
         unsigned pending = __ballot_sync(0xffffffffu, !certain && live);
         while (pending) {
@@ -569,12 +610,7 @@ encode_tc_kernel(const __half* __restrict__ x1, const float* __restrict__ cb1, c
             const int ec = tc_exact_code<kC>(xs, cbf, lane, &ed);
             if (lane == src) { code = ec; dbest = ed; }
         }
-        if (live) {
-            const int64_t s = v / n_tokens, i = v % n_tokens;
-            const int64_t pos = token_offset + (seq_offsets ? seq_offsets[s] : 0) + i;
-            if (pos >= 0 && pos < sh.max_tokens)
-                codes[code_word_offset(sh, n_heads, s, h, pos / kTokenBlock, g) + (int)(pos % kTokenBlock)] = (uint8_t)code;
-        }
+        if (rec.code_offset >= 0) codes[rec.code_offset + g * kTokenBlock] = (uint8_t)code;
     }
 
     // every MMA that was issued has been waited for (or the wait gave up); hand the tensor memory back
@@ -592,12 +628,12 @@ cudaError_t launch_enc_tc(const __half* x, const float* cb, const int32_t* seq_o
 {
     using C = TcCfg<kC>;
     const int64_t n_vec = sh.n_seq * n_tokens;
-    const int64_t tile_pairs = (n_vec + kTcTileVecs - 1) / kTcTileVecs;
-    const int64_t slots = 2 * (int64_t)device_sm_count();          // CTAs in flight
-    // row-tile pairs per CTA: as many as leave four waves of CTAs
-    int log_rt = 2;
-    while (log_rt > 0 && ((tile_pairs + (1 << log_rt) - 1) >> log_rt) * sh.n_kv_heads < 4 * slots) --log_rt;
-    const int64_t blocks = (tile_pairs + (1 << log_rt) - 1) >> log_rt;
+    const int64_t tiles = (n_vec + kTcTileVecs - 1) / kTcTileVecs;
+    const int64_t slots = C::kCtasPerSm * (int64_t)device_sm_count();          // CTAs in flight
+    // row tiles per CTA: as many as leave four waves of CTAs
+    int log_rt = C::kMaxLogRt;
+    while (log_rt > 0 && ((tiles + (1 << log_rt) - 1) >> log_rt) * sh.n_kv_heads < 4 * slots) --log_rt;
+    const int64_t blocks = (tiles + (1 << log_rt) - 1) >> log_rt;
     // split the groups over CTAs while the grid would leave SMs idle
     int64_t n_gsplit = (slots + blocks * sh.n_kv_heads - 1) / (blocks * sh.n_kv_heads);
     if (n_gsplit > C::G) n_gsplit = C::G;
