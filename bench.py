@@ -175,7 +175,7 @@ class DecodeState:
         self.seq_lens = self.lens_cpu.to(dev)
         self.append_pos = (self.lens_cpu - 1).to(dev)
         self.out = torch.empty(w.n_seq, w.n_q_heads, D, dtype=torch.float32, device=dev)
-        self.ws = torch.empty(max(256, cq.cq_decode_attn_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, c, b,
+        self.ws = torch.empty(max(256, cq.cq_decode_step_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, c, b,
                                                                         self.cap)), dtype=torch.uint8, device=dev)
         self.scale = D ** -0.5
 
@@ -193,8 +193,17 @@ class DecodeState:
         return codes + books + qo
 
     def step(self, cq, ev=None):
-        """Append-encode the new token (K, V) at the last position, then attend."""
+        """Append-encode the new token (K, V) at the last position, then attend: one cq_decode_step call where the
+        kernel appends inside the attention launch, else cq_encode_kv followed by cq_decode_attn."""
         w = self.w
+        if shared_word_kernel(w):
+            if ev is not None:
+                ev[0].record()
+            cq.cq_decode_step(self.q, self.k_new, self.v_new, self.append_pos, self.k_codes, self.v_codes, self.k_cb,
+                              self.v_cb, self.scale, w.c, w.b, self.cap, out=self.out, workspace=self.ws)
+            if ev is not None:
+                ev[1].record()
+            return
         cq.cq_encode_kv(self.k_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim),
                         self.v_new.view(w.n_seq, 1, w.n_kv_heads, w.head_dim), self.k_cb, self.v_cb, w.c, w.b,
                         self.k_codes, self.v_codes, self.cap, seq_offsets=self.append_pos)
@@ -232,7 +241,7 @@ def decode_roofline(w, st, ms, dev, sm_mhz=None):
     t_hbm, t_smem = nbytes / (hbm * 1e9), lane_ops / smem_peak
     a_hbm, a_smem = nbytes / (ms * 1e-3) / 1e9, lane_ops / (ms * 1e-3)
     o = {"kernel": ("decode_pair_kernel" if shared_word_kernel(w) else
-                    "decode_wide_kernel" if w.b == 10 else "decode_tuned_kernel") + " + merge_kernel (one cq_decode_attn call)",
+                    "decode_wide_kernel" if w.b == 10 else "decode_tuned_kernel") + " + merge_kernel (one attention call)",
          "launch_ms": ms, "algorithmic_bytes_per_launch": nbytes, "traffic": None,
          "hbm": {"achieved": a_hbm, "peak": hbm, "unit": "GB/s", "frac": a_hbm / hbm, "frac_of_8tbs_nominal": a_hbm / 8000.0,
                  "peak_source": which + " copy bandwidth", "min_ms": t_hbm * 1e3},
@@ -618,7 +627,8 @@ def main():
             "clocks": clocks,
             "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": args.steps * 3 * len(states),      # per layer: append-encode (K and V), attention, merge
+            # per layer: attention (which appends the new token where the kernel can) and merge, else also the append-encode
+            "gpu_launches": args.steps * (2 if shared_word_kernel(w) else 3) * len(states),
             "roofline": roofline}
 
     if args.extras != "none" and world == 1:

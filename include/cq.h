@@ -335,10 +335,40 @@ int cq_learn_centroids(const void *x_fp16, const float *weights, const double *u
                        double *objective_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * One decode step of one layer on DEVICE buffers: the new token's key and value
+ * vectors are encoded (CQ encode, Section 3.2, as cq_encode does) and appended at
+ * position seq_lens[s] of every sequence, and the step's query attends over
+ * seq_lens[s] + 1 tokens (Eq. 1, as cq_decode_attn does).  For CQ-8c8b with
+ * head_dim 128 and a multiple of four query heads per KV head the append happens
+ * INSIDE the attention launch: the CTAs whose part of the context holds the new
+ * position work the codes out, use them, and one of them writes them to the
+ * cache; the step is then one attention launch plus the merge.  Every other shape
+ * runs cq_encode_kv and cq_decode_attn one after the other.
+ *
+ *   q_fp16       [n_seq][n_q_heads][head_dim] fp16, device
+ *   k_new_fp16, v_new_fp16   [n_seq][n_kv_heads][head_dim] fp16, device, 16-byte aligned
+ *   seq_lens     [n_seq] int32, device: tokens cached BEFORE the step; not modified (the caller
+ *                adds one to its own copy).  A sequence already at max_tokens gets no new token
+ *                and attends over its max_tokens cached ones.
+ *   k_codes, v_codes   device, layout of cq_encode; one byte per group is written per sequence
+ *                and KV head.  Must not alias each other.
+ *   out          [n_seq][n_q_heads][head_dim] fp32, device
+ *   workspace    device, 16-byte aligned, at least cq_decode_step_workspace_bytes(...) bytes
+ * Errors: as cq_decode_attn.  Asynchronous on `stream`.
+ */
+size_t cq_decode_step_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim,
+                                      int c, int b, int64_t max_tokens);
+int cq_decode_step(const void *q_fp16, const void *k_new_fp16, const void *v_new_fp16,
+                   const int32_t *seq_lens, void *k_codes, void *v_codes, const float *k_cb,
+                   const float *v_cb, float scale, int n_seq, int n_q_heads, int n_kv_heads,
+                   int head_dim, int c, int b, int64_t max_tokens, float *out, void *workspace,
+                   size_t workspace_bytes, void *stream);
+
+/*
  * One decode step of one layer driven from HOST buffers (the end-to-end path):
  * copies the step's query and the new token's key and value vectors to the
- * device, appends the new token's codes at position seq_lens_host[s] of every
- * sequence (cq_encode), attends over seq_lens_host[s] + 1 tokens (cq_decode_attn)
+ * device, runs cq_decode_step (the new token's codes appended at position
+ * seq_lens_host[s] of every sequence, attention over seq_lens_host[s] + 1 tokens)
  * and copies the result back.  Synchronises `stream` before returning.
  *
  *   q_host       [n_seq][n_q_heads][head_dim] fp16   (pinned memory recommended)

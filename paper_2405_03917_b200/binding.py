@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 # Every symbol include/cq.h declares.
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant", "cq_encode_kv",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
-           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_host_workspace_bytes",
+           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_workspace_bytes", "cq_decode_step", "cq_decode_step_host_workspace_bytes",
            "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
 
 
@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.cq_lloyd_step.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.cq_learn_centroids.restype = i32
         L.cq_learn_centroids.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.cq_decode_step_workspace_bytes.restype = sz
+        L.cq_decode_step_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
+        L.cq_decode_step.restype = i32
+        L.cq_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp, sz, vp]
         L.cq_decode_step_host_workspace_bytes.restype = sz
         L.cq_decode_step_host_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
         L.cq_decode_step_host.restype = i32
@@ -307,6 +311,42 @@ def cq_decode_attn_static(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch
                                      float(scale), n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
                                      _dev(out, torch.float32, "out"), _stream())
     _check(st, "cq_decode_attn_static")
+    return out
+
+
+def cq_decode_step_workspace_bytes(n_seq: int, n_q_heads: int, n_kv_heads: int, head_dim: int, c: int, b: int,
+                                   max_tokens: int) -> int:
+    return int(lib().cq_decode_step_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens))
+
+
+def cq_decode_step(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, seq_lens: torch.Tensor,
+                   k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor, v_cb: torch.Tensor, scale: float,
+                   c: int, b: int, max_tokens: int, out: Optional[torch.Tensor] = None,
+                   workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """One decode step on device buffers: q fp16 (n_seq, n_q_heads, D), k_new / v_new fp16 (n_seq, n_kv_heads, D),
+    seq_lens int32 (n_seq,) = tokens cached before the step.  The caches take the new token's codes; returns the
+    attention output fp32 (n_seq, n_q_heads, D) over seq_lens + 1 tokens."""
+    n_seq, n_q_heads, head_dim = q.shape
+    n_kv_heads = k_cb.shape[0]
+    if tuple(k_new.shape) != (n_seq, n_kv_heads, head_dim) or tuple(v_new.shape) != (n_seq, n_kv_heads, head_dim):
+        raise ValueError("k_new and v_new must be (n_seq, n_kv_heads, head_dim)")
+    if seq_lens.numel() != n_seq:
+        raise ValueError("seq_lens must have n_seq entries")
+    need_codes = cq_codes_bytes(n_seq, max_tokens, n_kv_heads, head_dim, c, b)
+    if need_codes and (k_codes.numel() < need_codes or v_codes.numel() < need_codes):
+        raise ValueError(f"code buffers hold {k_codes.numel()} / {v_codes.numel()} bytes, {need_codes} needed")
+    need = cq_decode_step_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    if out is None:
+        out = torch.empty(n_seq, n_q_heads, head_dim, dtype=torch.float32, device=q.device)
+    st = lib().cq_decode_step(_dev(q, torch.float16, "q"), _dev(k_new, torch.float16, "k_new"), _dev(v_new, torch.float16, "v_new"),
+                              _dev(seq_lens, torch.int32, "seq_lens"), _dev(k_codes, torch.uint8, "k_codes"),
+                              _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
+                              _dev(v_cb, torch.float32, "v_cb"), float(scale), n_seq, n_q_heads, n_kv_heads, head_dim, c, b,
+                              max_tokens, _dev(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
+                              workspace.numel(), _stream())
+    _check(st, "cq_decode_step")
     return out
 
 

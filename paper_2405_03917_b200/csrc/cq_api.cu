@@ -456,6 +456,52 @@ int cq_learn_centroids(const void* x_fp16, const float* weights, const double* u
 
 // Staging area of cq_decode_step_host inside the caller's workspace (all 256-byte aligned):
 //   [q fp16][k_new fp16][v_new fp16][seq_lens int32][seq_lens+1 int32][out fp32][attention workspace]
+size_t cq_decode_step_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                                      int64_t max_tokens)
+{
+    const size_t attn = cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens);
+    if (attn == 0) return 0;
+    return attn + round_up((size_t)n_seq * 4, 256);          // the lengths after the append, where they are needed
+}
+
+int cq_decode_step(const void* q_fp16, const void* k_new_fp16, const void* v_new_fp16, const int32_t* seq_lens,
+                   void* k_codes, void* v_codes, const float* k_cb, const float* v_cb, float scale, int n_seq,
+                   int n_q_heads, int n_kv_heads, int head_dim, int c, int b, int64_t max_tokens, float* out,
+                   void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!q_fp16 || !k_new_fp16 || !v_new_fp16 || !seq_lens || !k_codes || !v_codes || !k_cb || !v_cb || !out || !workspace)
+        return CQ_ERR_NULL;
+    Shape sh;
+    int st = make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh);
+    if (st != CQ_OK) return st;
+    if (!aligned16(k_codes) || !aligned16(v_codes) || !aligned16(workspace) || !aligned16(k_cb) || !aligned16(v_cb) ||
+        !aligned16(k_new_fp16) || !aligned16(v_new_fp16) || (reinterpret_cast<uintptr_t>(q_fp16) & 1u) ||
+        (reinterpret_cast<uintptr_t>(out) & 3u))
+        return CQ_ERR_ALIGN;
+    if (k_codes == v_codes) return CQ_ERR_SHAPE;
+    const size_t attn_bytes = round_up(partial_bytes(sh), 256);
+    if (workspace_bytes < attn_bytes + round_up((size_t)n_seq * 4, 256)) return CQ_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (decode_tuned_supported(sh) && decode_fused_append_supported(sh)) {
+        AppendArgs app;
+        app.k_new = static_cast<const __half*>(k_new_fp16);
+        app.v_new = static_cast<const __half*>(v_new_fp16);
+        app.kc_w = static_cast<uint8_t*>(k_codes);
+        app.vc_w = static_cast<uint8_t*>(v_codes);
+        cudaError_t e = launch_decode_step_fused(static_cast<const __half*>(q_fp16), app.kc_w, app.vc_w, k_cb, v_cb, seq_lens,
+                                                 scale, sh, out, static_cast<float*>(workspace), app, cs);
+        return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    }
+    // every other shape: the append is a launch of its own, the attention reads the lengths plus one
+    int32_t* sl1 = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + attn_bytes);
+    if (launch_add_one(seq_lens, sl1, n_seq, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    st = cq_encode_kv(k_new_fp16, v_new_fp16, k_cb, v_cb, seq_lens, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b,
+                      k_codes, v_codes, stream);
+    if (st != CQ_OK) return st;
+    return cq_decode_attn(q_fp16, k_codes, v_codes, k_cb, v_cb, sl1, scale, n_seq, n_q_heads, n_kv_heads, head_dim, c, b,
+                          max_tokens, out, workspace, attn_bytes, stream);
+}
+
 size_t cq_decode_step_host_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
                                            int64_t max_tokens)
 {
@@ -496,16 +542,13 @@ int cq_decode_step_host(const void* q_host, const void* k_new_host, const void* 
     char* d_k = w;                 w += round_up(kvb, 256);
     char* d_v = w;                 w += round_up(kvb, 256);
     int32_t* d_sl = reinterpret_cast<int32_t*>(w);   w += round_up(slb, 256);
-    int32_t* d_sl1 = reinterpret_cast<int32_t*>(w);  w += round_up(slb, 256);
     float* d_out = reinterpret_cast<float*>(w);      w += round_up(ob, 256);
-    void* attn_ws = w;
-    const size_t attn_bytes = workspace_bytes - (size_t)(w - static_cast<char*>(workspace));
+    void* step_ws = w;              // attention partials, and the lengths plus one for the shapes that need them
+    const size_t step_bytes = workspace_bytes - (size_t)(w - static_cast<char*>(workspace));
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    // The new token is appended at position seq_lens[s]; the attention then reads seq_lens[s] + 1 tokens.
     // Few, large copies: query, key and value travel in one copy when the caller keeps them back to back
-    // in host memory (the staging areas are then packed the same way); both length arrays travel in one
-    // copy from a small array on the stack (pageable source: the call returns once it has been read).
+    // in host memory (the staging areas are then packed the same way).
     const bool packed = static_cast<const char*>(k_new_host) == static_cast<const char*>(q_host) + qb &&
                         static_cast<const char*>(v_new_host) == static_cast<const char*>(k_new_host) + kvb &&
                         qb % 16 == 0 && kvb % 16 == 0;
@@ -518,24 +561,10 @@ int cq_decode_step_host(const void* q_host, const void* k_new_host, const void* 
         if (cudaMemcpyAsync(d_k, k_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
         if (cudaMemcpyAsync(d_v, v_new_host, kvb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
     }
-    constexpr int kStackSeqs = 1024;
-    if (n_seq <= kStackSeqs) {
-        int32_t both[2 * kStackSeqs];
-        for (int s = 0; s < n_seq; ++s) {
-            both[s] = seq_lens_host[s];
-            both[n_seq + s] = seq_lens_host[s] + 1;
-        }
-        d_sl1 = d_sl + n_seq;       // (fits: two padded areas were reserved)
-        if (cudaMemcpyAsync(d_sl, both, 2 * slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
-    } else {
-        if (cudaMemcpyAsync(d_sl, seq_lens_host, slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
-        if (launch_add_one(d_sl, d_sl1, n_seq, cs) != cudaSuccess) return CQ_ERR_CUDA;
-    }
-    int st = cq_encode_kv(d_k, d_v, k_cb, v_cb, d_sl, n_seq, 1, 0, max_tokens, n_kv_heads, head_dim, c, b, k_codes, v_codes,
-                          stream);
-    if (st != CQ_OK) return st;
-    st = cq_decode_attn(d_q, k_codes, v_codes, k_cb, v_cb, d_sl1, scale, n_seq, n_q_heads, n_kv_heads, head_dim, c, b,
-                        max_tokens, d_out, attn_ws, attn_bytes, stream);
+    if (cudaMemcpyAsync(d_sl, seq_lens_host, slb, cudaMemcpyHostToDevice, cs) != cudaSuccess) return CQ_ERR_CUDA;
+    // The new token is appended at position seq_lens[s]; the attention then reads seq_lens[s] + 1 tokens.
+    const int st = cq_decode_step(d_q, d_k, d_v, d_sl, k_codes, v_codes, k_cb, v_cb, scale, n_seq, n_q_heads, n_kv_heads,
+                                  head_dim, c, b, max_tokens, d_out, step_ws, step_bytes, stream);
     if (st != CQ_OK) return st;
     if (cudaMemcpyAsync(out_host, d_out, ob, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return CQ_ERR_CUDA;
     if (cudaStreamSynchronize(cs) != cudaSuccess) return CQ_ERR_CUDA;

@@ -80,6 +80,15 @@ struct DecodePlan {
     unsigned grid;
 };
 
+// The token that a decode step appends before it attends (all null: none).  k_new, v_new: fp16
+// (n_seq, n_kv_heads, head_dim); kc_w, vc_w: the caches, which take the token's codes at position seq_lens[s].
+struct AppendArgs {
+    const __half* k_new = nullptr;
+    const __half* v_new = nullptr;
+    uint8_t* kc_w = nullptr;
+    uint8_t* vc_w = nullptr;
+};
+
 // ---- launchers implemented in the .cu files (return cudaGetLastError()) ----
 cudaError_t launch_encode_generic(const __half* x, const float* cb, const int32_t* seq_offsets, const Shape& sh,
                                   int64_t n_tokens, int64_t token_offset, uint8_t* codes, cudaStream_t st);
@@ -118,13 +127,20 @@ int decode_tuned_parts(const Shape& sh);      // partial slots per (sequence, qu
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
                                 float* out, float* partials, cudaStream_t st, bool per_head_tables = false);
+// True when launch_decode_tuned would take a kernel that can append a token inside the attention launch.
+bool decode_fused_append_supported(const Shape& sh);
+// One decode step: the token (app) is encoded and appended at position seq_lens[s] and the attention covers
+// seq_lens[s] + 1 tokens, in one attention launch (plus the merge).  Only where decode_fused_append_supported.
+cudaError_t launch_decode_step_fused(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
+                                     const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
+                                     float* out, float* partials, const AppendArgs& app, cudaStream_t st);
 
 // CQ-8c8b with a multiple of four query heads per KV head: two query heads per table word (cq_decode_pair.cu).
 bool decode_pair_supported(const Shape& sh);
 DecodePlan decode_pair_plan(const Shape& sh);
 cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
                                const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
-                               float* partials, cudaStream_t st);
+                               float* partials, cudaStream_t st, const AppendArgs& app = AppendArgs());
 
 // Causal attention of the n_q newest cached tokens of every sequence (cq_prefill.cu); `generic` forces the plain kernel.
 bool prefill_mma_supported(const Shape& sh);

@@ -1244,6 +1244,19 @@ int decode_tuned_parts(const Shape& sh)
     return pair > own ? pair : own;
 }
 
+bool decode_fused_append_supported(const Shape& sh) { return decode_pair_supported(sh); }
+
+cudaError_t launch_decode_step_fused(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
+                                     const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
+                                     float* out, float* partials, const AppendArgs& app, cudaStream_t st)
+{
+    if (!decode_pair_supported(sh)) return cudaErrorNotSupported;
+    const DecodePlan pp = decode_pair_plan(sh);
+    const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, app);
+    if (ep != cudaSuccess) return ep;
+    return launch_merge(partials, pp.n_parts, sh, out, st);
+}
+
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh, float* out,
                                 float* partials, cudaStream_t st, bool per_head_tables)

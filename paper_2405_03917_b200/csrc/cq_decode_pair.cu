@@ -94,6 +94,7 @@ struct PairCtl {
     float offset[4];           // per head: sum over groups of the entry taken out of each group
     float mins[4][16];         // per (head, group): smallest table entry
     uint64_t bar[PairCfg::kWarps][2];   // per warp: arrival of its K tile and of its V tile
+    uint8_t newcode[2][16];    // codes of the token this launch appends (key, value), when its position is in the CTA's range
 };
 static_assert(sizeof(PairCtl) <= PairCfg::kCtlBytes, "control block");
 
@@ -298,11 +299,71 @@ __device__ __noinline__ int2 reserve_slow(uint8_t* smem, PairCtl* ctl, int ref_l
     return make_int2(eu[0], eu[1]);
 }
 
+// The value codes of the token that the launch appends (CQ encode, Section 3.2), by the whole CTA: warp w takes
+// groups 2 w and 2 w + 1, its lanes walk the centroids; d_j = sum_i (x_i - C_ji)^2 in fp32 in the order of the
+// encode kernels, lowest index on ties.  The codes go to the control block and, from the CTA that `writer` names,
+// to position `pos` of the cache.  (The key codes come out of the table build, which reads the key centroids anyway.)
+__device__ __noinline__ void encode_new_value(PairCtl* ctl, AppendArgs app, const float* __restrict__ vcb, Shape sh,
+                                              int64_t s, int hkv, int64_t pos, bool writer, bool aligned32)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll 1
+    for (int e = 0; e < 2; ++e) {
+        const int g = warp * 2 + e;
+        const __half* xp = app.v_new + (s * sh.n_kv_heads + hkv) * 128 + g * 8;
+        const float* cg = vcb + ((int64_t)hkv * 16 + g) * kRows * 8;
+        float xg[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) xg[i] = __half2float(xp[i]);
+        float best = INFINITY;
+        int arg = 0;
+        float cv[kRows / 32][8];                      // all loads in flight at once
+#pragma unroll
+        for (int t = 0; t < kRows / 32; ++t) load_centroid<8>(cg + (int64_t)(t * 32 + lane) * 8, cv[t], aligned32);
+#pragma unroll
+        for (int t = 0; t < kRows / 32; ++t) {
+            const int j = t * 32 + lane;
+            float d = 0.f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float diff = xg[i] - cv[t][i];
+                d = fmaf(diff, diff, d);
+            }
+            if (d < best) { best = d; arg = j; }        // j increases with t: strict < keeps the lowest index
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+            if (ob < best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+        }
+        if (lane == 0) {
+            ctl->newcode[1][g] = (uint8_t)arg;
+            if (writer) app.vc_w[code_word_offset(sh, sh.n_kv_heads, s, hkv, pos / kTokenBlock, g) + pos % kTokenBlock] = (uint8_t)arg;
+        }
+    }
+}
+
+// Puts the new token's codes into a 64-bit code word that was loaded straight from global memory: word_off is the
+// word's byte offset inside its warp's tile, new_off + 16 g that of the new token's code of group g.
+__device__ __noinline__ uint2 patch_word(uint2 w, uint32_t word_off, uint32_t new_off, const uint8_t* newcode)
+{
+#pragma unroll 1
+    for (int g = 0; g < 16; ++g) {
+        const uint32_t d = new_off + 16u * g - word_off;
+        if (d < 4u)
+            w.x = (w.x & ~(0xffu << (8 * d))) | ((uint32_t)newcode[g] << (8 * d));
+        else if (d < 8u)
+            w.y = (w.y & ~(0xffu << (8 * (d - 4)))) | ((uint32_t)newcode[g] << (8 * (d - 4)));
+    }
+    return w;
+}
+
 __global__ void __launch_bounds__(PairCfg::kThreads, 2)
 decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                    const float* __restrict__ kcb, const float* __restrict__ vcb,
                    const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                   int tail_first, int cb_aligned32, float* __restrict__ partials)
+                   int tail_first, int cb_aligned32, float* __restrict__ partials, AppendArgs app)
 {
     using C = PairCfg;
     constexpr int R = C::kHeads;
@@ -339,6 +400,10 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     static_assert(R * 128 == 2 * C::kThreads, "two query elements per thread");
     int64_t n = seq_lens[s];
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
+    // With an append, seq_lens counts the tokens cached before this launch: the new token takes position n and
+    // the attention covers n + 1 tokens (a sequence at capacity gets no new token).
+    const bool has_new = app.k_new != nullptr && n < sh.max_tokens;
+    if (has_new) ++n;
     const int64_t t_begin = (int64_t)part * chunk_tokens;
     const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
     const int stride = partial_stride(128);
@@ -359,6 +424,13 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
 
     const int64_t blk0 = t_begin / kTokenBlock;
     const int n_tok = (int)(t_end - blk0 * kTokenBlock);                   // tokens of this CTA, counted from its first block
+    // The new token, when its position is in this CTA's range: which warp's tile of which iteration holds its block.
+    // The CTA works its codes out itself (so do the CTAs of the other query heads that share the KV head) and puts
+    // them into the staged tile; the CTA of the KV head's first four query heads also writes them to the cache.
+    const bool new_here = has_new && t_begin <= n - 1 && n - 1 < t_end;
+    const int new_blk = new_here ? (int)((n - 1) / kTokenBlock - blk0) : 0;
+    const int new_it = new_blk / (C::kWarps * C::kBlocksPerIter), new_warp = (new_blk / C::kBlocksPerIter) % C::kWarps;
+    const uint32_t new_off = (uint32_t)(new_blk % C::kBlocksPerIter) * 256u + (uint32_t)((n - 1) % kTokenBlock);   // + 16 g: byte in the tile
     const int n_iters = (n_tok + C::kRoundTokens - 1) / C::kRoundTokens;
     const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, blk0, 0);
     const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, blk0, 0);
@@ -425,16 +497,23 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             have = __all_sync(0xffffffffu, have);
             if (have) { kphase ^= 1u; k_out = false; } else bulk = false;
         }
+        const bool patch = new_here && it == new_it && warp == new_warp;
         if (have || bytes == 0u) {
+            if (patch) {
+                if (lane < 16) ktile[new_off + 16u * lane] = ctl->newcode[0][lane];
+                __syncwarp();
+            }
 #pragma unroll
             for (int m = 0; m < 4; ++m) kw[m] = *reinterpret_cast<const uint2*>(smem + (my_ktile ^ (64u * m)));
         } else {
             const int blk = (it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1);
             const int64_t off = (int64_t)blk * 256 + 8 * (r & 1);
 #pragma unroll
-            for (int m = 0; m < 4; ++m)
+            for (int m = 0; m < 4; ++m) {
                 kw[m] = blk < n_blocks_cta ? __ldg(reinterpret_cast<const uint2*>(kbase + off + 2u * (koff0 ^ (32u * m))))
                                            : make_uint2(0u, 0u);
+                if (patch) kw[m] = patch_word(kw[m], (uint32_t)((r >> 1) * 256 + 8 * (r & 1)) + 2u * (koff0 ^ (32u * m)), new_off, ctl->newcode[0]);
+            }
         }
         __syncwarp();
         const uint32_t next = it + 1 < n_iters ? tile_bytes(it + 1) : 0u;
@@ -451,16 +530,23 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             have = __all_sync(0xffffffffu, have);
             if (have) { vphase ^= 1u; v_out = false; } else bulk = false;
         }
+        const bool patch = new_here && it == new_it && warp == new_warp;
         if (have || bytes == 0u) {
+            if (patch) {
+                if (lane < 16) vtile[new_off + 16u * lane] = ctl->newcode[1][lane];
+                __syncwarp();
+            }
 #pragma unroll
             for (int m = 0; m < 8; ++m) vw[m] = *reinterpret_cast<const uint2*>(smem + (my_vtile ^ (16u * m)));
         } else {
             const int blk = (it * C::kWarps + warp) * C::kBlocksPerIter + (r >> 1);
             const int64_t off = (int64_t)blk * 256 + 8 * (r & 1);
 #pragma unroll
-            for (int m = 0; m < 8; ++m)
+            for (int m = 0; m < 8; ++m) {
                 vw[m] = blk < n_blocks_cta ? __ldg(reinterpret_cast<const uint2*>(vbase + off + 16u * (8 * pu + (vx ^ m))))
                                            : make_uint2(0u, 0u);
+                if (patch) vw[m] = patch_word(vw[m], (uint32_t)((r >> 1) * 256 + 8 * (r & 1)) + 16u * (8 * pu + (vx ^ m)), new_off, ctl->newcode[1]);
+            }
         }
         __syncwarp();
         const uint32_t next = it + 1 < n_iters ? tile_bytes(it + 1) : 0u;
@@ -489,6 +575,7 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     }
     qs[threadIdx.x] = __half2float(q_lo) * scale_log2e;
     qs[C::kThreads + threadIdx.x] = __half2float(q_hi) * scale_log2e;
+    if (new_here) encode_new_value(ctl, app, vcb, sh, s, hkv, n - 1, head_group % kv_share == 0, cb_aligned32 != 0);
     __syncthreads();
     // the first code tiles travel during the table build
     k_out = v_out = tile_bytes(0) != 0u;
@@ -504,8 +591,19 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     {
         float qreg[R][8];
         float vmin[R], vmax[R];
+        // the new token's key, when this CTA appends it: its code of group g is the centroid nearest to it, found on
+        // the way (d_j = sum_i (x_i - C_ji)^2 in fp32 in the order of the encode kernels, lowest index on ties)
+        float xnew[8], dnew = INFINITY;
+        int jnew = 0;
         auto build_unit = [&](const float (&cv)[kJb][8], int u) {
             const int g = warp * 2 + (u >> 1);
+            if ((u & 1) == 0 && new_here) {
+                const __half* xp = app.k_new + (s * sh.n_kv_heads + hkv) * 128 + g * 8;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) xnew[i] = __half2float(xp[i]);
+                dnew = INFINITY;
+                jnew = 0;
+            }
             if ((u & 1) == 0) {
 #pragma unroll
                 for (int h = 0; h < R; ++h) {
@@ -526,6 +624,28 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                     vmin[h] = fminf(vmin[h], dot);
                     vmax[h] = fmaxf(vmax[h], dot);
                     stage[(h * 16 + g) * kRows + (j ^ (16 * (h >> 1) + g))] = dot;
+                }
+                if (new_here) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float diff = xnew[i] - cv[jb][i];
+                        d = fmaf(diff, diff, d);
+                    }
+                    if (d < dnew) { dnew = d; jnew = j; }        // a lane's j ascend: strict < keeps the lowest index
+                }
+            }
+            if ((u & 1) == 1 && new_here) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ob = __shfl_xor_sync(0xffffffffu, dnew, o);
+                    const int oa = __shfl_xor_sync(0xffffffffu, jnew, o);
+                    if (ob < dnew || (ob == dnew && oa < jnew)) { dnew = ob; jnew = oa; }
+                }
+                if (lane == 0) {
+                    ctl->newcode[0][g] = (uint8_t)jnew;
+                    if (head_group % kv_share == 0)
+                        app.kc_w[code_word_offset(sh, sh.n_kv_heads, s, hkv, (n - 1) / kTokenBlock, g) + (n - 1) % kTokenBlock] = (uint8_t)jnew;
                 }
             }
             if ((u & 1) == 1) {
@@ -856,14 +976,14 @@ DecodePlan decode_pair_plan(const Shape& sh)
 
 cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
                                const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
-                               float* partials, cudaStream_t st)
+                               float* partials, cudaStream_t st, const AppendArgs& app)
 {
     using C = PairCfg;
     const cudaError_t attr = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_pair_kernel), C::kSmemBytes, 0);
     if (attr != cudaSuccess) return attr;
     const int aligned = ((reinterpret_cast<uintptr_t>(kcb) | reinterpret_cast<uintptr_t>(vcb)) & 31u) == 0 ? 1 : 0;
     decode_pair_kernel<<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk,
-                                                                    pl.n_parts, pl.tail_first, aligned, partials);
+                                                                    pl.n_parts, pl.tail_first, aligned, partials, app);
     return cudaGetLastError();
 }
 
