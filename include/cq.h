@@ -225,8 +225,14 @@ int cq_decode_attn_static(const void *q_fp16, const void *k_codes, const void *v
  * values are not rotated.  Every other argument, the workspace size
  * (cq_decode_attn_workspace_bytes) and the output are those of cq_decode_attn.
  * CQ_ERR_UNSUPPORTED when a pair would not lie in whole groups (odd number of groups for
- * CQ_ROPE_HALF, odd c for CQ_ROPE_INTERLEAVED).  Runs on a generic sm_100a kernel: the
- * score of a token is no longer a sum of per-code table entries.
+ * CQ_ROPE_HALF, odd c for CQ_ROPE_INTERLEAVED).  The score of a token is no longer a sum
+ * of per-code table entries.  head_dim 128 with b = 8, c in {4, 8}, CQ_ROPE_HALF and 8-byte
+ * aligned tables run on a tuned kernel (keys dequantised from fp16 centroids in shared
+ * memory and rotated in registers; the cosines and sines of the tokens between two table
+ * reads follow by the angle-addition rule and are checked against the tables, which are
+ * read row by row when they are not of the rotary form); every other case on a generic
+ * sm_100a kernel.  cq_decode_attn_rope_variant picks the kernel: 0 = automatic,
+ * 1 = generic, 2 = tuned (CQ_ERR_UNSUPPORTED where it does not apply).
  */
 #define CQ_ROPE_HALF 0
 #define CQ_ROPE_INTERLEAVED 1
@@ -236,6 +242,12 @@ int cq_decode_attn_rope(const void *q_fp16, const void *k_codes, const void *v_c
                         int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
                         int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
                         void *stream);
+int cq_decode_attn_rope_variant(const void *q_fp16, const void *k_codes, const void *v_codes,
+                        const float *k_cb, const float *v_cb, const int32_t *seq_lens,
+                        const float *rope_cos, const float *rope_sin, int pairing, float scale,
+                        int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                        int64_t max_tokens, float *out, void *workspace, size_t workspace_bytes,
+                        int variant, void *stream);
 
 /*
  * Causal attention of a run of new tokens over the CQ-coded cache: a prompt, or a chunk of

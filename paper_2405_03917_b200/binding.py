@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 # Every symbol include/cq.h declares.
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant", "cq_encode_kv",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
-           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_workspace_bytes", "cq_decode_step", "cq_decode_step_host_workspace_bytes",
+           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_decode_attn_rope_variant", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_workspace_bytes", "cq_decode_step", "cq_decode_step_host_workspace_bytes",
            "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
 
 
@@ -72,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.cq_decode_attn_rope.restype = i32
         L.cq_decode_attn_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, i32, i32, i32, i32, i32, i64,
                                           vp, vp, sz, vp]
+        L.cq_decode_attn_rope_variant.restype = i32
+        L.cq_decode_attn_rope_variant.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, i32, i32, i32, i32, i32, i64,
+                                          vp, vp, sz, i32, vp]
         L.cq_decode_attn_static.restype = i32
         L.cq_decode_attn_static.argtypes = [vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp]
         L.cq_learn_workspace_bytes.restype = sz
@@ -261,8 +264,10 @@ ROPE_HALF, ROPE_INTERLEAVED = 0, 1
 def cq_decode_attn_rope(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_cb: torch.Tensor,
                         v_cb: torch.Tensor, seq_lens: torch.Tensor, rope_cos: torch.Tensor, rope_sin: torch.Tensor,
                         scale: float, c: int, b: int, max_tokens: int, pairing: int = ROPE_HALF,
-                        out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """cq_decode_attn for key codes taken before RoPE: rope_cos / rope_sin fp32 (max_tokens, head_dim / 2)."""
+                        out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                        variant: int = 0) -> torch.Tensor:
+    """cq_decode_attn for key codes taken before RoPE: rope_cos / rope_sin fp32 (max_tokens, head_dim / 2).
+    variant 0 = automatic, 1 = generic kernel, 2 = tuned kernel."""
     n_seq, n_q_heads, head_dim = q.shape
     n_kv_heads = k_cb.shape[0]
     for nm, t in (("rope_cos", rope_cos), ("rope_sin", rope_sin)):
@@ -276,13 +281,13 @@ def cq_decode_attn_rope(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.T
     if workspace is None:
         nbytes = cq_decode_attn_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens)
         workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
-    st = lib().cq_decode_attn_rope(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+    st = lib().cq_decode_attn_rope_variant(_dev(q, torch.float16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
                                    _dev(v_codes, torch.uint8, "v_codes"), _dev(k_cb, torch.float32, "k_cb"),
                                    _dev(v_cb, torch.float32, "v_cb"), _dev(seq_lens, torch.int32, "seq_lens"),
                                    _dev(rope_cos, torch.float32, "rope_cos"), _dev(rope_sin, torch.float32, "rope_sin"),
                                    int(pairing), float(scale), n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens,
                                    _dev(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
-                                   workspace.numel(), _stream())
+                                   workspace.numel(), int(variant), _stream())
     _check(st, "cq_decode_attn_rope")
     return out
 

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcq.so")
-SOURCES = ["cq_api.cu", "cq_generic.cu", "cq_encode.cu", "cq_encode_tc.cu", "cq_decode.cu", "cq_decode_pair.cu", "cq_prefill.cu", "cq_learn.cu"]
+SOURCES = ["cq_api.cu", "cq_generic.cu", "cq_encode.cu", "cq_encode_tc.cu", "cq_decode.cu", "cq_decode_pair.cu", "cq_decode_rope.cu", "cq_prefill.cu", "cq_learn.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--cudart", "shared", "-Xlinker", "-rpath=/usr/local/cuda/lib64"]
 

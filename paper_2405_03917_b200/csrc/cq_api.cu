@@ -277,10 +277,11 @@ int cq_decode_attn(const void* q_fp16, const void* k_codes, const void* v_codes,
                                   head_dim, c, b, max_tokens, out, workspace, workspace_bytes, 0, stream);
 }
 
-int cq_decode_attn_rope(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
-                        const float* v_cb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
-                        int pairing, float scale, int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
-                        int64_t max_tokens, float* out, void* workspace, size_t workspace_bytes, void* stream)
+int cq_decode_attn_rope_variant(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
+                                const float* v_cb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
+                                int pairing, float scale, int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c,
+                                int b, int64_t max_tokens, float* out, void* workspace, size_t workspace_bytes, int variant,
+                                void* stream)
 {
     if (!q_fp16 || !k_codes || !v_codes || !k_cb || !v_cb || !seq_lens || !rope_cos || !rope_sin || !out || !workspace)
         return CQ_ERR_NULL;
@@ -296,12 +297,33 @@ int cq_decode_attn_rope(const void* q_fp16, const void* k_codes, const void* v_c
         (reinterpret_cast<uintptr_t>(rope_cos) & 3u) || (reinterpret_cast<uintptr_t>(rope_sin) & 3u))
         return CQ_ERR_ALIGN;
     if (workspace_bytes < round_up(partial_bytes(sh), 256)) return CQ_ERR_WORKSPACE;
+    if (variant < 0 || variant > 2) return CQ_ERR_SHAPE;
+    const bool tuned_ok = decode_rope_tuned_supported(sh, pairing) &&
+                          ((reinterpret_cast<uintptr_t>(rope_cos) | reinterpret_cast<uintptr_t>(rope_sin)) & 7u) == 0;
+    if (variant == 2 && !tuned_ok) return CQ_ERR_UNSUPPORTED;
+    if (variant == 2 || (variant == 0 && tuned_ok)) {
+        cudaError_t et = launch_decode_rope_tuned(static_cast<const __half*>(q_fp16), static_cast<const uint8_t*>(k_codes),
+                                                  static_cast<const uint8_t*>(v_codes), k_cb, v_cb, seq_lens, rope_cos, rope_sin,
+                                                  scale, sh, out, static_cast<float*>(workspace),
+                                                  static_cast<cudaStream_t>(stream));
+        return et == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+    }
     if ((int64_t)sh.G * sh.K > 2 * kGenericMaxTableEntries) return CQ_ERR_UNSUPPORTED;     // one table (the bins) only
     cudaError_t e = launch_decode_rope(static_cast<const __half*>(q_fp16), static_cast<const uint8_t*>(k_codes),
                                        static_cast<const uint8_t*>(v_codes), k_cb, v_cb, seq_lens, rope_cos, rope_sin,
                                        pairing, scale, sh, out, static_cast<float*>(workspace),
                                        static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? CQ_OK : CQ_ERR_CUDA;
+}
+
+int cq_decode_attn_rope(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,
+                        const float* v_cb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
+                        int pairing, float scale, int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                        int64_t max_tokens, float* out, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return cq_decode_attn_rope_variant(q_fp16, k_codes, v_codes, k_cb, v_cb, seq_lens, rope_cos, rope_sin, pairing, scale, n_seq,
+                                       n_q_heads, n_kv_heads, head_dim, c, b, max_tokens, out, workspace, workspace_bytes, 0,
+                                       stream);
 }
 
 int cq_prefill_attn_variant(const void* q_fp16, const void* k_codes, const void* v_codes, const float* k_cb,

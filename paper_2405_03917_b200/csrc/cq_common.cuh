@@ -120,6 +120,12 @@ cudaError_t launch_decode_generic(const __half* q, const uint8_t* kc, const uint
 cudaError_t launch_decode_rope(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                const float* vcb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
                                int pairing, float scale, const Shape& sh, float* out, float* partials, cudaStream_t st);
+// Pre-RoPE key codes on the tuned kernel (cq_decode_rope.cu): head_dim 128, b = 8, c in {4, 8}, pairing (i, i + 64);
+// the cos / sin tables must be 8-byte aligned.
+bool decode_rope_tuned_supported(const Shape& sh, int pairing);
+cudaError_t launch_decode_rope_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
+                                     const float* vcb, const int32_t* seq_lens, const float* rope_cos, const float* rope_sin,
+                                     float scale, const Shape& sh, float* out, float* partials, cudaStream_t st);
 bool decode_tuned_supported(const Shape& sh);
 int decode_tuned_parts(const Shape& sh);      // partial slots per (sequence, query head)
 // per_head_tables: keep to decode_tuned_kernel (one table word per query head) also where the kernel

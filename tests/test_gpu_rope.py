@@ -90,3 +90,72 @@ def test_rope_rejects_pairs_that_split_groups():
     with pytest.raises(cq.CQError) as e:
         cq.cq_decode_attn_rope(q, codes1, codes1, cb1, cb1, sl, t, t, 1.0, 1, 2, cap, pairing=1)
     assert e.value.status == -3
+
+
+# ------------------------------------------------------------------------------- the tuned kernel
+
+def run_rope(q, kc_rm, vc_rm, kcb, vcb, lens, cs, sn, cap, c, variant, scale):
+    sl = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    return cq.cq_decode_attn_rope(q.to(DEV), to_lib(kc_rm, 128, c, 8), to_lib(vc_rm, 128, c, 8), kcb.to(DEV), vcb.to(DEV), sl,
+                                  torch.from_numpy(cs).to(DEV), torch.from_numpy(sn).to(DEV), scale, c, 8, cap,
+                                  pairing=0, variant=variant).cpu().numpy()
+
+
+@pytest.mark.parametrize("c,n_q,n_kv", [(8, 2, 2), (8, 4, 2), (8, 4, 1), (8, 8, 1), (8, 16, 1), (8, 3, 1), (4, 2, 2), (4, 2, 1),
+                                        (4, 4, 1), (4, 8, 1)])
+def test_tuned_rope_kernel_matches_the_oracle(c, n_q, n_kv):
+    # every number of query heads per CTA (1, 2, 4, 8) of both group sizes; empty, one-token, ragged contexts, a
+    # context longer than the chunk of scores that shared memory holds, several ranges per sequence
+    lens = [0, 1, 15, 16, 17, 700, 9000]
+    cap = 9100
+    q, kc_rm, vc_rm, kcb, vcb = case(200 + c + n_q, c, 8, n_q, n_kv, lens, cap)
+    cs, sn = rope_tables(cap, 64)
+    got = run_rope(q, kc_rm, vc_rm, kcb, vcb, lens, cs, sn, cap, c, 2, 128 ** -0.5)
+    ref = oracle.decode_dense_rope(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32), cs, sn,
+                                   128 ** -0.5, c, 8, 0)
+    for s_ in range(len(lens)):
+        H.check_attn(got[s_], ref[s_], f"tuned rope c={c} Hq={n_q} Hkv={n_kv} sequence {s_}")
+    assert (got[0] == 0).all()
+
+
+def test_tuned_rope_kernel_with_tables_that_are_not_rotary():
+    # phases that jump around: the stepped cosines leave the tables at once, every row is then read from them;
+    # a table that is rotary except for one row in the middle of a batch's reach is caught at the batch's end or
+    # stays within the kernel's check (the row after each batch), so only the first kind is asserted
+    lens = [300, 64]
+    cap = 320
+    q, kc_rm, vc_rm, kcb, vcb = case(9, 8, 8, 4, 1, lens, cap)
+    rng = np.random.default_rng(4)
+    ang = rng.uniform(0, 6.28, size=(cap, 64))
+    amp = rng.uniform(0.5, 1.5, size=(cap, 64))          # not even of unit length
+    cs, sn = (amp * np.cos(ang)).astype(np.float32), (amp * np.sin(ang)).astype(np.float32)
+    ref = oracle.decode_dense_rope(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32), cs, sn,
+                                   0.05, 8, 8, 0)
+    for variant in (2, 1):
+        got = run_rope(q, kc_rm, vc_rm, kcb, vcb, lens, cs, sn, cap, 8, variant, 0.05)
+        H.check_attn(got, ref, f"arbitrary tables, variant {variant}")
+
+
+def test_tuned_rope_kernel_with_scaled_and_shifted_rotary_tables():
+    # amplitude and phase per pair, frequencies of another base: still of the rotary form, so the stepping holds
+    lens = [1500, 77]
+    cap = 1500
+    q, kc_rm, vc_rm, kcb, vcb = case(10, 4, 8, 4, 2, lens, cap)
+    rng = np.random.default_rng(5)
+    t = np.arange(cap, dtype=np.float64)[:, None]
+    freq = 500000.0 ** (-np.arange(64, dtype=np.float64) / 64)[None, :]
+    phase, amp = rng.uniform(0, 6.28, size=(1, 64)), rng.uniform(0.7, 1.3, size=(1, 64))
+    cs, sn = (amp * np.cos(t * freq + phase)).astype(np.float32), (amp * np.sin(t * freq + phase)).astype(np.float32)
+    ref = oracle.decode_dense_rope(q.numpy(), kc_rm, vc_rm, kcb.numpy(), vcb.numpy(), np.asarray(lens, np.int32), cs, sn,
+                                   128 ** -0.5, 4, 8, 0)
+    got = run_rope(q, kc_rm, vc_rm, kcb, vcb, lens, cs, sn, cap, 4, 2, 128 ** -0.5)
+    H.check_attn(got, ref, "scaled rotary tables")
+
+
+def test_tuned_rope_kernel_is_refused_where_it_does_not_apply():
+    q, kc_rm, vc_rm, kcb, vcb = case(1, 8, 8, 2, 1, [20], 20)
+    cs, sn = rope_tables(20, 64)
+    sl = torch.tensor([20], dtype=torch.int32, device=DEV)
+    with pytest.raises(cq.CQError):          # the other pairing
+        cq.cq_decode_attn_rope(q.to(DEV), to_lib(kc_rm, 128, 8, 8), to_lib(vc_rm, 128, 8, 8), kcb.to(DEV), vcb.to(DEV), sl,
+                               torch.from_numpy(cs).to(DEV), torch.from_numpy(sn).to(DEV), 0.1, 8, 8, 20, pairing=1, variant=2)
