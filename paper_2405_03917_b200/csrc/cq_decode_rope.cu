@@ -6,7 +6,9 @@
 // the query with a dequantised, rotated key: there is no table of per-code score terms.  What the
 // kernel does instead:
 //   - A CTA serves up to 8 query heads of one KV head (what the bins leave room for) over a range of
-//     the context; the KV head's key centroids sit in shared memory as fp16 (64 KiB).
+//     the context; the KV head's key centroids sit in shared memory as fp16 (64 KiB), code-major
+//     ([code][group][channel]), so that the 32 lanes of a gather - each in its own group's columns -
+//     touch 32 different banks whatever the codes are.  The bins are code-major for the same reason.
 //   - Lane l of a warp owns the pairs i = 2l, 2l + 1.  For a batch of 32 / heads consecutive tokens it
 //     gathers the two half2 words of its channels per token, rotates them and multiplies by its slice
 //     of every head's query: 32 partial scores per lane, which a five-stage exchange between the
@@ -46,8 +48,8 @@ struct RtCfg {
     static constexpr int G = 128 / kC;
     static constexpr int kT = 32 / kHeads;                        // tokens of a warp's batch
     static constexpr int kChunk = kRtScoreBytes / 4 / kHeads;     // tokens whose scores are kept at a time
-    static constexpr int kBookOff = 0;                            // fp16 [G][256][kC]
-    static constexpr int kBinsOff = 128 * 256 * 2;                // fp32 [kHeads][G][256]
+    static constexpr int kBookOff = 0;                            // fp16 [256][G][kC]
+    static constexpr int kBinsOff = 128 * 256 * 2;                // fp32 [kHeads][256][G]
     static constexpr int kScoreOff = kBinsOff + kHeads * G * 256 * 4;      // fp32 [kHeads][kChunk]
     static constexpr int kCtlOff = kScoreOff + kRtScoreBytes;
     static constexpr int kSmemBytes = kCtlOff + 2048;
@@ -82,7 +84,7 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
     const int n_hgroups = sh.n_q_heads / kHeads;
     const int split = blockIdx.x % n_splits;
     const int hg = (blockIdx.x / n_splits) % n_hgroups;
-    const int64_t s = blockIdx.x / (n_splits * n_hgroups);
+    const int64_t s = seq_by_rank(seq_lens, (int)sh.n_seq, sh.max_tokens, (int)(blockIdx.x / (n_splits * n_hgroups)));   // longest first
     const int hq0 = hg * kHeads, hkv = hq0 / sh.R;
     const int stride = partial_stride(128);
 
@@ -105,9 +107,11 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
         const float4* src = reinterpret_cast<const float4*>(kcb + (int64_t)hkv * 128 * 256);
         uint2* dst = reinterpret_cast<uint2*>(rt_smem + C::kBookOff);
         for (int i = threadIdx.x; i < 128 * 256 / 4; i += kRtThreads) {
+            // four channels of centroid (g, j): piece i of the global [g][j][c] order goes to the [j][g][c] order
+            const int per = kC / 4, g = i / (256 * per), j = (i / per) % 256, w4 = i % per;
             const float4 v = ldg_f4(reinterpret_cast<const float*>(src + i));
             const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
-            dst[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+            dst[(j * G + g) * per + w4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
         }
         for (int i = threadIdx.x; i < kHeads * G * 256 / 4; i += kRtThreads)
             reinterpret_cast<float4*>(bins)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -139,8 +143,9 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
     }
     // words of the lane's two channels inside a centroid, and its two groups
     const int gA = (2 * lane) / kC, gB = gA + G / 2;
-    const uint32_t wsel = (uint32_t)((2 * lane) % kC) / 2u;
-    const uint32_t rowA = (uint32_t)gA * 256u, rowB = (uint32_t)gB * 256u;
+    // word of the lane's channels a in the centroid row of a code: code * (64 words) + colA; channels b: + 32 words
+    const uint32_t colA = (uint32_t)(gA * kC + (2 * lane) % kC) / 2u, colB = colA + 32u;
+    static_assert(128 / 2 == 64, "64 words of fp16 pairs per code");
     const uint8_t* kseq = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
     const uint8_t* vseq = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
     float l_thr[kHeads];
@@ -153,60 +158,84 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
 
         // -------------------------------------------------------------- scores of the chunk
         float lane_max = -INFINITY;                  // over the scores of this lane's head
+        // a batch's key codes of the lane's two groups and the table rows of its first token
+        auto load_batch = [&](int64_t t0, uint32_t (&ca)[kWords], uint32_t (&cbw)[kWords], float2& cs0, float2& sn0) {
+            const uint8_t* pa = kseq + (t0 / kTokenBlock) * sh.block_bytes + (t0 % kTokenBlock);
+            if (kT == 32) {
+                const bool two = t0 + 16 < t_end;
+                const uint4 a0 = *reinterpret_cast<const uint4*>(pa + gA * kTokenBlock), b0w = *reinterpret_cast<const uint4*>(pa + gB * kTokenBlock);
+                const uint4 a1 = two ? *reinterpret_cast<const uint4*>(pa + sh.block_bytes + gA * kTokenBlock) : make_uint4(0u, 0u, 0u, 0u);
+                const uint4 b1 = two ? *reinterpret_cast<const uint4*>(pa + sh.block_bytes + gB * kTokenBlock) : make_uint4(0u, 0u, 0u, 0u);
+                ca[0] = a0.x; ca[1 % kWords] = a0.y; ca[2 % kWords] = a0.z; ca[3 % kWords] = a0.w;
+                ca[4 % kWords] = a1.x; ca[5 % kWords] = a1.y; ca[6 % kWords] = a1.z; ca[7 % kWords] = a1.w;
+                cbw[0] = b0w.x; cbw[1 % kWords] = b0w.y; cbw[2 % kWords] = b0w.z; cbw[3 % kWords] = b0w.w;
+                cbw[4 % kWords] = b1.x; cbw[5 % kWords] = b1.y; cbw[6 % kWords] = b1.z; cbw[7 % kWords] = b1.w;
+            } else if (kT == 16) {
+                const uint4 a0 = *reinterpret_cast<const uint4*>(pa + gA * kTokenBlock), b0w = *reinterpret_cast<const uint4*>(pa + gB * kTokenBlock);
+                ca[0] = a0.x; ca[1 % kWords] = a0.y; ca[2 % kWords] = a0.z; ca[3 % kWords] = a0.w;
+                cbw[0] = b0w.x; cbw[1 % kWords] = b0w.y; cbw[2 % kWords] = b0w.z; cbw[3 % kWords] = b0w.w;
+            } else if (kT == 8) {
+                const uint2 a0 = *reinterpret_cast<const uint2*>(pa + gA * kTokenBlock), b0w = *reinterpret_cast<const uint2*>(pa + gB * kTokenBlock);
+                ca[0] = a0.x; ca[1 % kWords] = a0.y;
+                cbw[0] = b0w.x; cbw[1 % kWords] = b0w.y;
+            } else {
+                ca[0] = *reinterpret_cast<const uint32_t*>(pa + gA * kTokenBlock);
+                cbw[0] = *reinterpret_cast<const uint32_t*>(pa + gB * kTokenBlock);
+            }
+            cs0 = *reinterpret_cast<const float2*>(rope_cos + t0 * 64 + 2 * lane);
+            sn0 = *reinterpret_cast<const float2*>(rope_sin + t0 * 64 + 2 * lane);
+        };
+        uint32_t ca[kWords], cbw[kWords];
+        float2 cs0 = make_float2(1.f, 1.f), sn0 = make_float2(0.f, 0.f);
+        if (warp * kT < chunk_len) load_batch(chunk_begin + warp * kT, ca, cbw, cs0, sn0);
         for (int b0 = warp * kT; b0 < chunk_len; b0 += kRtWarps * kT) {
             const int64_t t0 = chunk_begin + b0;
-            // the batch's key codes of the lane's two groups
-            uint32_t ca[kWords], cbw[kWords];
-            {
-                const uint8_t* pa = kseq + (t0 / kTokenBlock) * sh.block_bytes + (t0 % kTokenBlock);
-                if (kT == 32) {
-                    const bool two = t0 + 16 < t_end;
-                    const uint4 a0 = *reinterpret_cast<const uint4*>(pa + gA * kTokenBlock), b0w = *reinterpret_cast<const uint4*>(pa + gB * kTokenBlock);
-                    const uint4 a1 = two ? *reinterpret_cast<const uint4*>(pa + sh.block_bytes + gA * kTokenBlock) : make_uint4(0u, 0u, 0u, 0u);
-                    const uint4 b1 = two ? *reinterpret_cast<const uint4*>(pa + sh.block_bytes + gB * kTokenBlock) : make_uint4(0u, 0u, 0u, 0u);
-                    ca[0] = a0.x; ca[1 % kWords] = a0.y; ca[2 % kWords] = a0.z; ca[3 % kWords] = a0.w;
-                    ca[4 % kWords] = a1.x; ca[5 % kWords] = a1.y; ca[6 % kWords] = a1.z; ca[7 % kWords] = a1.w;
-                    cbw[0] = b0w.x; cbw[1 % kWords] = b0w.y; cbw[2 % kWords] = b0w.z; cbw[3 % kWords] = b0w.w;
-                    cbw[4 % kWords] = b1.x; cbw[5 % kWords] = b1.y; cbw[6 % kWords] = b1.z; cbw[7 % kWords] = b1.w;
-                } else if (kT == 16) {
-                    const uint4 a0 = *reinterpret_cast<const uint4*>(pa + gA * kTokenBlock), b0w = *reinterpret_cast<const uint4*>(pa + gB * kTokenBlock);
-                    ca[0] = a0.x; ca[1 % kWords] = a0.y; ca[2 % kWords] = a0.z; ca[3 % kWords] = a0.w;
-                    cbw[0] = b0w.x; cbw[1 % kWords] = b0w.y; cbw[2 % kWords] = b0w.z; cbw[3 % kWords] = b0w.w;
-                } else if (kT == 8) {
-                    const uint2 a0 = *reinterpret_cast<const uint2*>(pa + gA * kTokenBlock), b0w = *reinterpret_cast<const uint2*>(pa + gB * kTokenBlock);
-                    ca[0] = a0.x; ca[1 % kWords] = a0.y;
-                    cbw[0] = b0w.x; cbw[1 % kWords] = b0w.y;
-                } else {
-                    ca[0] = *reinterpret_cast<const uint32_t*>(pa + gA * kTokenBlock);
-                    cbw[0] = *reinterpret_cast<const uint32_t*>(pa + gB * kTokenBlock);
-                }
-            }
             float p[32];
-            // the partial scores of the batch; from_tables: every token's row is read from the tables, else the rows
+            // The partial scores of the batch; from_tables: every token's row is read from the tables, else the rows
             // after the first follow by the step rotation.  Returns false when the stepped rows leave the tables.
+            // With one head per CTA the query is rotated instead of the key (by the opposite angle): the rotated
+            // query u = q_a cos + q_b sin, v = q_b cos - q_a sin steps like the angle does, and the score term of a
+            // pair is k_a u + k_b v.
             auto batch = [&](auto from_tables) -> bool {
                 constexpr bool kFromTables = decltype(from_tables)::value;
-                float2 cs = *reinterpret_cast<const float2*>(rope_cos + t0 * 64 + 2 * lane);
-                float2 sn = *reinterpret_cast<const float2*>(rope_sin + t0 * 64 + 2 * lane);
+                float2 cs = cs0, sn = sn0;
+                float2 u = make_float2(0.f, 0.f), v = make_float2(0.f, 0.f);
+                if (kHeads == 1) {
+                    u = make_float2(fmaf(qa[0][0], cs.x, qb[0][0] * sn.x), fmaf(qa[0][1], cs.y, qb[0][1] * sn.y));
+                    v = make_float2(fmaf(qb[0][0], cs.x, -qa[0][0] * sn.x), fmaf(qb[0][1], cs.y, -qa[0][1] * sn.y));
+                }
 #pragma unroll
                 for (int j = 0; j < kT; ++j) {
-                    const uint32_t wa = book[((rowA + rt_code<kWords>(ca, j)) * kC) / 2 + wsel];
-                    const uint32_t wb = book[((rowB + rt_code<kWords>(cbw, j)) * kC) / 2 + wsel];
+                    const uint32_t wa = book[rt_code<kWords>(ca, j) * 64u + colA];
+                    const uint32_t wb = book[rt_code<kWords>(cbw, j) * 64u + colB];
                     const float2 ka = __half22float2(*reinterpret_cast<const __half2*>(&wa));
                     const float2 kb = __half22float2(*reinterpret_cast<const __half2*>(&wb));
-                    // the rotated key of the lane's four channels
-                    const float ra0 = ka.x * cs.x - kb.x * sn.x, rb0 = kb.x * cs.x + ka.x * sn.x;
-                    const float ra1 = ka.y * cs.y - kb.y * sn.y, rb1 = kb.y * cs.y + ka.y * sn.y;
+                    if (kHeads == 1) {
+                        p[j] = fmaf(ka.x, u.x, fmaf(kb.x, v.x, fmaf(ka.y, u.y, kb.y * v.y)));
+                    } else {
+                        // the rotated key of the lane's four channels
+                        const float ra0 = ka.x * cs.x - kb.x * sn.x, rb0 = kb.x * cs.x + ka.x * sn.x;
+                        const float ra1 = ka.y * cs.y - kb.y * sn.y, rb1 = kb.y * cs.y + ka.y * sn.y;
 #pragma unroll
-                    for (int h = 0; h < kHeads; ++h)
-                        p[h * kT + j] = fmaf(qa[h][0], ra0, fmaf(qb[h][0], rb0, fmaf(qa[h][1], ra1, qb[h][1] * rb1)));
-                    // cosine and sine of the next position
+                        for (int h = 0; h < kHeads; ++h)
+                            p[h * kT + j] = fmaf(qa[h][0], ra0, fmaf(qb[h][0], rb0, fmaf(qa[h][1], ra1, qb[h][1] * rb1)));
+                    }
+                    // the next position
                     if (kFromTables) {
                         if (j + 1 < kT) {
                             const int64_t tn = t0 + j + 1 < sh.max_tokens ? t0 + j + 1 : t0 + j;
                             cs = *reinterpret_cast<const float2*>(rope_cos + tn * 64 + 2 * lane);
                             sn = *reinterpret_cast<const float2*>(rope_sin + tn * 64 + 2 * lane);
+                            if (kHeads == 1) {
+                                u = make_float2(fmaf(qa[0][0], cs.x, qb[0][0] * sn.x), fmaf(qa[0][1], cs.y, qb[0][1] * sn.y));
+                                v = make_float2(fmaf(qb[0][0], cs.x, -qa[0][0] * sn.x), fmaf(qb[0][1], cs.y, -qa[0][1] * sn.y));
+                            }
                         }
+                    } else if (kHeads == 1) {
+                        const float ux = fmaf(u.x, st_re.x, v.x * st_im.x), vx = fmaf(v.x, st_re.x, -u.x * st_im.x);
+                        const float uy = fmaf(u.y, st_re.y, v.y * st_im.y), vy = fmaf(v.y, st_re.y, -u.y * st_im.y);
+                        u = make_float2(ux, uy);
+                        v = make_float2(vx, vy);
                     } else {
                         const float cx = cs.x * st_re.x - sn.x * st_im.x, sx = sn.x * st_re.x + cs.x * st_im.x;
                         const float cy = cs.y * st_re.y - sn.y * st_im.y, sy = sn.y * st_re.y + cs.y * st_im.y;
@@ -215,20 +244,33 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
                     }
                 }
                 if (kFromTables) return true;
-                // (cs, sn) is now the prediction for position t0 + kT: it must be what the tables hold there
+                // what was stepped to is the prediction for position t0 + kT: it must be what the tables hold there
                 bool off = false;
                 if (t0 + kT < sh.max_tokens) {
                     const float2 ct = *reinterpret_cast<const float2*>(rope_cos + (t0 + kT) * 64 + 2 * lane);
                     const float2 stt = *reinterpret_cast<const float2*>(rope_sin + (t0 + kT) * 64 + 2 * lane);
                     const float tol = 2e-5f;
-                    off = !(fabsf(ct.x - cs.x) <= tol * (1.f + fabsf(ct.x))) || !(fabsf(ct.y - cs.y) <= tol * (1.f + fabsf(ct.y))) ||
-                          !(fabsf(stt.x - sn.x) <= tol * (1.f + fabsf(stt.x))) || !(fabsf(stt.y - sn.y) <= tol * (1.f + fabsf(stt.y)));
+                    if (kHeads == 1) {
+                        const float ux = fmaf(qa[0][0], ct.x, qb[0][0] * stt.x), uy = fmaf(qa[0][1], ct.y, qb[0][1] * stt.y);
+                        const float vx = fmaf(qb[0][0], ct.x, -qa[0][0] * stt.x), vy = fmaf(qb[0][1], ct.y, -qa[0][1] * stt.y);
+                        const float bx = tol * (fabsf(qa[0][0]) + fabsf(qb[0][0])) * (1.f + fabsf(ct.x) + fabsf(stt.x));
+                        const float by = tol * (fabsf(qa[0][1]) + fabsf(qb[0][1])) * (1.f + fabsf(ct.y) + fabsf(stt.y));
+                        off = !(fabsf(ux - u.x) <= bx) || !(fabsf(vx - v.x) <= bx) || !(fabsf(uy - u.y) <= by) || !(fabsf(vy - v.y) <= by);
+                    } else {
+                        off = !(fabsf(ct.x - cs.x) <= tol * (1.f + fabsf(ct.x))) || !(fabsf(ct.y - cs.y) <= tol * (1.f + fabsf(ct.y))) ||
+                              !(fabsf(stt.x - sn.x) <= tol * (1.f + fabsf(stt.x))) || !(fabsf(stt.y - sn.y) <= tol * (1.f + fabsf(stt.y)));
+                    }
                 }
                 return !__any_sync(0xffffffffu, off);
             };
             if (exact || !batch(std::false_type())) {
                 exact = true;                            // this batch, and every later one of the warp, from the tables
                 batch(std::true_type());
+            }
+            // the next batch's words travel during the exchange
+            {
+                const int nb = b0 + kRtWarps * kT;
+                if (nb < chunk_len) load_batch(chunk_begin + nb, ca, cbw, cs0, sn0);
             }
             // Sum over the lanes: after the stage with offset o a lane keeps the half of its slots whose index has
             // bit o like its own lane number; after five stages lane L holds slot L = (head L / kT, token L % kT).
@@ -296,13 +338,11 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
 #pragma unroll
                 for (int k = 0; k < kRun; ++k) {
                     const int tl = blk * kTokenBlock + run * kRun + k;
-                    if (tl < chunk_len) {
-                        const uint32_t code = rt_code<kRun / 4>(cw, k);
+                    const uint32_t code = rt_code<kRun / 4>(cw, k);
 #pragma unroll
-                        for (int h = 0; h < kHeads; ++h) {
-                            const float w = scores[h * C::kChunk + tl];
-                            if (w != 0.f) atomicAdd(&bins[(h * G + g) * 256 + code], w);
-                        }
+                    for (int h = 0; h < kHeads; ++h) {
+                        const float w = tl < chunk_len ? scores[h * C::kChunk + tl] : 0.f;      // (adding zero changes nothing)
+                        atomicAdd(&bins[(h * 256 + code) * G + g], w);
                     }
                 }
             }
@@ -325,29 +365,42 @@ decode_rope_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict
         part0[(int64_t)threadIdx.x * n_splits * stride + 0] = ctl->m_run[threadIdx.x];
         part0[(int64_t)threadIdx.x * n_splits * stride + 1] = l;
     }
-    for (int o = warp; o < kHeads * G; o += kRtWarps) {
-        const int h = o / G, g = o % G;
-        const float* cg = vcb + ((int64_t)hkv * G + g) * 256 * kC;
-        float acc[kC];
+    // bins x value centroids: lane = group (two lanes per group for c = 8, one for the even and one for the odd codes),
+    // a warp per 16 codes, the warps' sums added through shared memory (the score area is free now)
+    {
+        constexpr int kLanesPerGroup = 32 / G;
+        const int g = lane % G, sub = lane / G;
+        float* red = scores;                                     // [warps][128]
+#pragma unroll 1
+        for (int h = 0; h < kHeads; ++h) {
+            float acc[kC];
 #pragma unroll
-        for (int k = 0; k < kC; ++k) acc[k] = 0.f;
-#pragma unroll 2
-        for (int jj = 0; jj < 256 / 32; ++jj) {
-            const int j = jj * 32 + lane;
-            const float w = bins[(h * G + g) * 256 + j];
-            float cv[kC];
-            load_centroid<kC>(cg + (int64_t)j * kC, cv, false);
+            for (int k = 0; k < kC; ++k) acc[k] = 0.f;
+#pragma unroll 4
+            for (int i = 0; i < 16 / kLanesPerGroup; ++i) {
+                const int j = warp * 16 + kLanesPerGroup * i + sub;
+                const float w = bins[(h * 256 + j) * G + g];
+                float cv[kC];
+                load_centroid<kC>(vcb + (((int64_t)hkv * G + g) * 256 + j) * kC, cv, false);
 #pragma unroll
-            for (int k = 0; k < kC; ++k) acc[k] = fmaf(w, cv[k], acc[k]);
-        }
+                for (int k = 0; k < kC; ++k) acc[k] = fmaf(w, cv[k], acc[k]);
+            }
+            if (kLanesPerGroup == 2) {
 #pragma unroll
-        for (int k = 0; k < kC; ++k) {
+                for (int k = 0; k < kC; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], 16);
+            }
+            if (sub == 0) {
 #pragma unroll
-            for (int of = 16; of > 0; of >>= 1) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], of);
-        }
-        if (lane == 0) {
+                for (int k = 0; k < kC; ++k) red[warp * 128 + g * kC + k] = acc[k];
+            }
+            __syncthreads();
+            if (threadIdx.x < 128) {
+                float v = 0.f;
 #pragma unroll
-            for (int k = 0; k < kC; ++k) part0[(int64_t)h * n_splits * stride + 2 + g * kC + k] = acc[k];
+                for (int w = 0; w < kRtWarps; ++w) v += red[w * 128 + threadIdx.x];
+                part0[(int64_t)h * n_splits * stride + 2 + threadIdx.x] = v;
+            }
+            __syncthreads();
         }
     }
 }
