@@ -477,7 +477,8 @@ def extra_prefill(cq, dev, reps=5):
 
 
 def extra_decode_rope(cq, dev, w, reps=5):
-    """Attention over codes of pre-RoPE keys (generic kernel) on the shape of a decode workload."""
+    """Attention over codes of pre-RoPE keys (cq_decode_attn_rope: the tuned kernel where the shape has one) on the
+    shape of a decode workload."""
     st = DecodeState(w, 0, dev, cq)
     P = w.head_dim // 2
     ang = torch.arange(st.cap, dtype=torch.float64, device=dev)[:, None] * \
@@ -644,8 +645,8 @@ def main():
             extras["decode_cfg5_8c10b"] = extra_decode(cq, dev, synth.WORKLOADS[5], reps=5)
             extras["decode_cfg6_2c8b"] = extra_decode(cq, dev, synth.WORKLOADS[6])
             extras["prefill"] = extra_prefill(cq, dev)
+            extras["decode_rope_cfg1"] = extra_decode_rope(cq, dev, synth.WORKLOADS[1])
             if args.extras in ("decode", "all"):
-                extras["decode_rope_cfg1"] = extra_decode_rope(cq, dev, synth.WORKLOADS[1])
                 extras["encode_cfg5_8c10b"] = extra_encode_wide(cq, dev, synth.WORKLOADS[5])
             if args.extras == "all":
                 extras["learn"] = extra_learn(cq, dev)
