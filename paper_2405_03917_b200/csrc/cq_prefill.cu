@@ -99,8 +99,8 @@ prefill_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__
 // tensor-core kernel
 // ------------------------------------------------------------------------------------------
 struct PfCfg {
-    static constexpr int kWarps = 4, kThreads = kWarps * 32;
-    static constexpr int kRows = 64;              // (query, head) rows per CTA: 16 per warp
+    static constexpr int kWarps = 8, kThreads = kWarps * 32;
+    static constexpr int kRows = 128;             // (query, head) rows per CTA: 16 per warp
     static constexpr int kTile = 64;              // cached tokens per step
     static constexpr int kRowBytes = 256;         // 128 fp16 channels
     static constexpr int kCbBytes = 128 * 256 * 2;                     // one codebook as fp16: [G][256][c]
@@ -108,7 +108,7 @@ struct PfCfg {
     static constexpr int kQOffset = 2 * kCbBytes;
     static constexpr int kKtOffset = kQOffset + kRows * kRowBytes;
     static constexpr int kVtOffset = kKtOffset + kTile * kRowBytes;
-    static constexpr int kSmemBytes = kVtOffset + kTile * kRowBytes;   // 176 KiB
+    static constexpr int kSmemBytes = kVtOffset + kTile * kRowBytes;   // 192 KiB
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -329,7 +329,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
 
 bool prefill_mma_supported(const Shape& sh)
 {
-    return sh.head_dim == 128 && sh.b == 8 && (sh.c == 2 || sh.c == 4 || sh.c == 8) && sh.R <= 64 && 64 % sh.R == 0;
+    return sh.head_dim == 128 && sh.b == 8 && (sh.c == 2 || sh.c == 4 || sh.c == 8) && sh.R <= 64 && PfCfg::kRows % sh.R == 0;
 }
 
 cudaError_t launch_prefill(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
