@@ -106,9 +106,10 @@ struct PfCfg {
     static constexpr int kCbBytes = 128 * 256 * 2;                     // one codebook as fp16: [G][256][c]
     static constexpr int kKcbOffset = 0, kVcbOffset = kCbBytes;
     static constexpr int kQOffset = 2 * kCbBytes;
-    static constexpr int kKtOffset = kQOffset + kRows * kRowBytes;
-    static constexpr int kVtOffset = kKtOffset + kTile * kRowBytes;
-    static constexpr int kSmemBytes = kVtOffset + kTile * kRowBytes;   // 192 KiB
+    static constexpr int kKtOffset = kQOffset + kRows * kRowBytes;     // K tiles, two buffers
+    static constexpr int kVtOffset = kKtOffset + 2 * kTile * kRowBytes; // V tiles, two buffers
+    static constexpr int kTileBytes = kTile * kRowBytes;
+    static constexpr int kSmemBytes = kVtOffset + 2 * kTile * kRowBytes;   // 224 KiB
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -197,9 +198,8 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
     const uint32_t q_s = smem_u32(smem + C::kQOffset), kt_s = smem_u32(smem + C::kKtOffset), vt_s = smem_u32(smem + C::kVtOffset);
 
-    for (int64_t jt = 0; jt < n_tiles; ++jt) {
-        const int64_t j0 = jt * C::kTile;
-        // ---- codes -> fp16 tiles: a work item is (8 tokens, one group)
+    // codes -> fp16 tiles of the 64 tokens from j0 on, into buffer `buf`: a work item is (8 tokens, one group)
+    auto dequantise = [&](int64_t j0, int buf) {
         for (int item = threadIdx.x; item < 8 * G; item += C::kThreads) {
             const int g = item % G, oct = item / G;                      // tokens 8 oct .. 8 oct + 7 of the tile
             const int64_t blk = j0 / kTokenBlock + (oct >> 1);
@@ -215,18 +215,26 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 const int tok = 8 * oct + k;
                 const uint32_t dst = tile_off(tok, (g * kC) >> 3) + (uint32_t)((g * kC) & 7) * 2u;
                 if (kC == 8) {
-                    *reinterpret_cast<uint4*>(smem + C::kKtOffset + dst) = *reinterpret_cast<const uint4*>(smem + C::kKcbOffset + (g * 256 + kcode) * 16);
-                    *reinterpret_cast<uint4*>(smem + C::kVtOffset + dst) = *reinterpret_cast<const uint4*>(smem + C::kVcbOffset + (g * 256 + vcode) * 16);
+                    *reinterpret_cast<uint4*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint4*>(smem + C::kKcbOffset + (g * 256 + kcode) * 16);
+                    *reinterpret_cast<uint4*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint4*>(smem + C::kVcbOffset + (g * 256 + vcode) * 16);
                 } else if (kC == 4) {
-                    *reinterpret_cast<uint2*>(smem + C::kKtOffset + dst) = *reinterpret_cast<const uint2*>(smem + C::kKcbOffset + (g * 256 + kcode) * 8);
-                    *reinterpret_cast<uint2*>(smem + C::kVtOffset + dst) = *reinterpret_cast<const uint2*>(smem + C::kVcbOffset + (g * 256 + vcode) * 8);
+                    *reinterpret_cast<uint2*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint2*>(smem + C::kKcbOffset + (g * 256 + kcode) * 8);
+                    *reinterpret_cast<uint2*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint2*>(smem + C::kVcbOffset + (g * 256 + vcode) * 8);
                 } else {
-                    *reinterpret_cast<uint32_t*>(smem + C::kKtOffset + dst) = *reinterpret_cast<const uint32_t*>(smem + C::kKcbOffset + (g * 256 + kcode) * 4);
-                    *reinterpret_cast<uint32_t*>(smem + C::kVtOffset + dst) = *reinterpret_cast<const uint32_t*>(smem + C::kVcbOffset + (g * 256 + vcode) * 4);
+                    *reinterpret_cast<uint32_t*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint32_t*>(smem + C::kKcbOffset + (g * 256 + kcode) * 4);
+                    *reinterpret_cast<uint32_t*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint32_t*>(smem + C::kVcbOffset + (g * 256 + vcode) * 4);
                 }
             }
         }
-        __syncthreads();
+    };
+    if (n_tiles > 0) dequantise(0, 0);
+    __syncthreads();
+
+    for (int64_t jt = 0; jt < n_tiles; ++jt) {
+        const int64_t j0 = jt * C::kTile;
+        const int buf = (int)(jt & 1);
+        // the next tile is dequantised into the other buffer (last read before the barrier that ended the step before)
+        if (jt + 1 < n_tiles) dequantise(j0 + C::kTile, buf ^ 1);
 
         // ---- S = Q Khat^T for the warp's 16 rows and the tile's 64 tokens
         float sc[8][4];
@@ -245,7 +253,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             for (int ntp = 0; ntp < 4; ++ntp) {
                 uint32_t b[4];
                 const int mi = lane >> 3;
-                ldmatrix_x4(b, kt_s + tile_off(16 * ntp + (lane & 7) + 8 * (mi >> 1), 2 * ks + (mi & 1)));
+                ldmatrix_x4(b, kt_s + buf * C::kTileBytes + tile_off(16 * ntp + (lane & 7) + 8 * (mi >> 1), 2 * ks + (mi & 1)));
                 mma_f16(sc[2 * ntp], a, b[0], b[1]);
                 mma_f16(sc[2 * ntp + 1], a, b[2], b[3]);
             }
@@ -299,11 +307,11 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             for (int ntp = 0; ntp < 8; ++ntp) {
                 uint32_t b[4];
                 const int mi = lane >> 3;
-                ldmatrix_x4_trans(b, vt_s + tile_off(16 * ks + (lane & 7) + 8 * (mi & 1), 2 * ntp + (mi >> 1)));
+                ldmatrix_x4_trans(b, vt_s + buf * C::kTileBytes + tile_off(16 * ks + (lane & 7) + 8 * (mi & 1), 2 * ntp + (mi >> 1)));
                 mma_f16(o[2 * ntp], pa[ks], b[0], b[1]);
                 mma_f16(o[2 * ntp + 1], pa[ks], b[2], b[3]);
             }
-        __syncthreads();                                                 // the tiles are rewritten next
+        __syncthreads();                                                 // the next tile is complete; this one may be rewritten
     }
 
     // ---- normalise and write (l is spread over the quad)
