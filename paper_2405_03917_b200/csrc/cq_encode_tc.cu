@@ -5,8 +5,8 @@
 // channels of a vector is replaced by the index of its nearest centroid in L2 distance, lowest
 // index on exact ties.
 //
-// Arithmetic: that of encode_tuned_kernel.  For 128 vectors x 256 centroids of one group ONE
-// tcgen05.mma (M = 128, N = 256, K = 16; two of them, accumulating, for c = 8) evaluates
+// Arithmetic: that of encode_tuned_kernel.  For 128 vectors x 128 centroids of one group ONE
+// tcgen05.mma (M = 128, N = 128, K = 16; two of them, accumulating, for c = 8) evaluates
 //     d_j ~ ||x_g||^2 - 2 <x_g, C_j> + ||C_j||^2
 // with the fp32 centroids and norms carried as sums of three fp16 terms, so that every product is
 // exact and only the fp32 accumulation rounds.  K slots, in pairs:
