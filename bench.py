@@ -215,6 +215,21 @@ class DecodeState:
             ev[1].record()
 
 
+def attach_traffic(roofline, workload_name):
+    """DRAM bytes of one launch from the committed ncu counters, when the kernels have not changed since."""
+    tr = os.path.join(ROOT, "profiles", "decode_traffic.json")
+    if not os.path.exists(tr):
+        return
+    try:
+        t = json.load(open(tr)).get(workload_name)
+        # the counters describe one build of the kernels: any later edit of their source voids them
+        if t and t.get("kernel_source_sha256") == kernel_source_hash():
+            roofline["traffic"] = t["dram_bytes_per_launch"]
+            roofline["traffic_source"] = t.get("source")
+    except Exception:
+        pass
+
+
 def shared_word_kernel(w) -> bool:
     """Shapes served by the kernel that keeps two query heads in one table word (cq_decode_pair.cu)."""
     return w.head_dim == 128 and w.b == 8 and w.c == 8 and (w.n_q_heads // w.n_kv_heads) % 4 == 0
@@ -437,8 +452,10 @@ def extra_decode(cq, dev, w, reps=20):
         st.step(cq, e)
     torch.cuda.synchronize()
     ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
-    return {"workload": w.name, "decode_ms": ms, "kv_tokens_per_s": st.kv_tokens() / (ms * 1e-3),
-            "query_heads_per_s": w.n_seq * w.n_q_heads / (ms * 1e-3), "roofline": decode_roofline(w, st, ms, dev)}
+    res = {"workload": w.name, "decode_ms": ms, "kv_tokens_per_s": st.kv_tokens() / (ms * 1e-3),
+           "query_heads_per_s": w.n_seq * w.n_q_heads / (ms * 1e-3), "roofline": decode_roofline(w, st, ms, dev)}
+    attach_traffic(res["roofline"], w.name)
+    return res
 
 
 def extra_prefill(cq, dev, reps=5):
@@ -610,16 +627,7 @@ def main():
     last = states[-1]
     dec_ms = statistics.mean(inner_ms)
     roofline = decode_roofline(w, last, dec_ms, dev, (clocks or {}).get("sm_mhz"))
-    tr = os.path.join(ROOT, "profiles", "decode_traffic.json")
-    if os.path.exists(tr):
-        try:
-            t = json.load(open(tr)).get(w.name)
-            # the counters describe one build of the kernels: any later edit of their source voids them
-            if t and t.get("kernel_source_sha256") == kernel_source_hash():
-                roofline["traffic"] = t["dram_bytes_per_launch"]
-                roofline["traffic_source"] = t.get("source")
-        except Exception:
-            pass
+    attach_traffic(roofline, w.name)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
