@@ -637,7 +637,9 @@ def main():
             "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             # per layer: attention (which appends the new token where the kernel can) and merge, else also the append-encode
-            "gpu_launches": args.steps * (2 if shared_word_kernel(w) else 3) * len(states),
+            "gpu_launches": args.steps * len(states) * (cq.cq_decode_step_launches(w.n_seq, w.n_q_heads, w.n_kv_heads, w.head_dim,
+                                                                                   w.c, w.b, st.cap)
+                                                         if shared_word_kernel(w) else 3),
             "roofline": roofline}
 
     if args.extras != "none" and world == 1:

@@ -370,6 +370,11 @@ int cq_learn_centroids(const void *x_fp16, const float *weights, const double *u
  */
 size_t cq_decode_step_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, int head_dim,
                                       int c, int b, int64_t max_tokens);
+/* Kernel launches of one cq_decode_step call on this shape (1: the attention kernel appends the
+ * token and, with one part of the context per CTA, also writes the output; 2: plus the merge of
+ * the partials; 4: lengths plus one, append, attention, merge); 0 for an unsupported shape. */
+int cq_decode_step_launches(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b,
+                            int64_t max_tokens);
 int cq_decode_step(const void *q_fp16, const void *k_new_fp16, const void *v_new_fp16,
                    const int32_t *seq_lens, void *k_codes, void *v_codes, const float *k_cb,
                    const float *v_cb, float scale, int n_seq, int n_q_heads, int n_kv_heads,

@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(_HERE, "libcq.so")
 # Every symbol include/cq.h declares.
 EXPORTS = ["cq_layout_version", "cq_status_string", "cq_codes_bytes", "cq_encode", "cq_encode_variant", "cq_encode_kv",
            "cq_codes_to_rowmajor", "cq_codes_from_rowmajor", "cq_decode_attn_workspace_bytes", "cq_decode_attn",
-           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_decode_attn_rope_variant", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_workspace_bytes", "cq_decode_step", "cq_decode_step_host_workspace_bytes",
+           "cq_decode_attn_variant", "cq_decode_attn_rope", "cq_decode_attn_rope_variant", "cq_prefill_attn", "cq_prefill_attn_variant", "cq_decode_attn_static", "cq_decode_step_workspace_bytes", "cq_decode_step_launches", "cq_decode_step", "cq_decode_step_host_workspace_bytes",
            "cq_decode_step_host", "cq_learn_workspace_bytes", "cq_kmeanspp_init", "cq_lloyd_step", "cq_learn_centroids"]
 
 
@@ -87,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.cq_learn_centroids.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.cq_decode_step_workspace_bytes.restype = sz
         L.cq_decode_step_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i64]
+        L.cq_decode_step_launches.restype = i32
+        L.cq_decode_step_launches.argtypes = [i32, i32, i32, i32, i32, i32, i64]
         L.cq_decode_step.restype = i32
         L.cq_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, f32, i32, i32, i32, i32, i32, i32, i64, vp, vp, sz, vp]
         L.cq_decode_step_host_workspace_bytes.restype = sz
@@ -322,6 +324,11 @@ def cq_decode_attn_static(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch
 def cq_decode_step_workspace_bytes(n_seq: int, n_q_heads: int, n_kv_heads: int, head_dim: int, c: int, b: int,
                                    max_tokens: int) -> int:
     return int(lib().cq_decode_step_workspace_bytes(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens))
+
+
+def cq_decode_step_launches(n_seq: int, n_q_heads: int, n_kv_heads: int, head_dim: int, c: int, b: int, max_tokens: int) -> int:
+    """Kernel launches of one cq_decode_step call on this shape."""
+    return int(lib().cq_decode_step_launches(n_seq, n_q_heads, n_kv_heads, head_dim, c, b, max_tokens))
 
 
 def cq_decode_step(q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, seq_lens: torch.Tensor,

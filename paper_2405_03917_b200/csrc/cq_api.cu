@@ -486,6 +486,15 @@ size_t cq_decode_step_workspace_bytes(int n_seq, int n_q_heads, int n_kv_heads, 
     return attn + round_up((size_t)n_seq * 4, 256);          // the lengths after the append, where they are needed
 }
 
+int cq_decode_step_launches(int n_seq, int n_q_heads, int n_kv_heads, int head_dim, int c, int b, int64_t max_tokens)
+{
+    Shape sh;
+    if (make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh) != CQ_OK) return 0;
+    if (decode_tuned_supported(sh) && decode_fused_append_supported(sh))
+        return decode_pair_plan(sh).n_parts == 1 ? 1 : 2;        // attention (with the append inside) [+ merge]
+    return 4;                                                      // lengths plus one, append, attention, merge
+}
+
 int cq_decode_step(const void* q_fp16, const void* k_new_fp16, const void* v_new_fp16, const int32_t* seq_lens,
                    void* k_codes, void* v_codes, const float* k_cb, const float* v_cb, float scale, int n_seq,
                    int n_q_heads, int n_kv_heads, int head_dim, int c, int b, int64_t max_tokens, float* out,

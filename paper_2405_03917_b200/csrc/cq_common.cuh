@@ -146,7 +146,9 @@ bool decode_pair_supported(const Shape& sh);
 DecodePlan decode_pair_plan(const Shape& sh);
 cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
                                const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
-                               float* partials, cudaStream_t st, const AppendArgs& app = AppendArgs());
+                               float* partials, cudaStream_t st, const AppendArgs& app = AppendArgs(), float* out = nullptr);
+// (out: where the attention output goes; with one part per item (pl.n_parts == 1) the kernel writes it itself and
+// no merge is needed, otherwise out is left alone and the caller merges the partials)
 
 // Causal attention of the n_q newest cached tokens of every sequence (cq_prefill.cu); `generic` forces the plain kernel.
 bool prefill_mma_supported(const Shape& sh);

@@ -1252,8 +1252,8 @@ cudaError_t launch_decode_step_fused(const __half* q, const uint8_t* kc, const u
 {
     if (!decode_pair_supported(sh)) return cudaErrorNotSupported;
     const DecodePlan pp = decode_pair_plan(sh);
-    const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, app);
-    if (ep != cudaSuccess) return ep;
+    const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, app, out);
+    if (ep != cudaSuccess || pp.n_parts == 1) return ep;
     return launch_merge(partials, pp.n_parts, sh, out, st);
 }
 
@@ -1263,8 +1263,8 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
 {
     if (!per_head_tables && decode_pair_supported(sh)) {
         const DecodePlan pp = decode_pair_plan(sh);
-        const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st);
-        if (ep != cudaSuccess) return ep;
+        const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, AppendArgs(), out);
+        if (ep != cudaSuccess || pp.n_parts == 1) return ep;      // one part per item: the kernel wrote the output itself
         return launch_merge(partials, pp.n_parts, sh, out, st);
     }
     const Plan pl = plan_dispatch(sh);

@@ -363,7 +363,7 @@ __global__ void __launch_bounds__(PairCfg::kThreads, 2)
 decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                    const float* __restrict__ kcb, const float* __restrict__ vcb,
                    const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                   int tail_first, int cb_aligned32, float* __restrict__ partials, AppendArgs app)
+                   int tail_first, int cb_aligned32, float* __restrict__ partials, AppendArgs app, float* __restrict__ out)
 {
     using C = PairCfg;
     constexpr int R = C::kHeads;
@@ -419,6 +419,8 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             const int h = i / stride, d = i % stride;
             part_base[(int64_t)h * n_parts * stride + d] = d == 0 ? -INFINITY : 0.f;
         }
+        if (out)            // one part per item and nothing to attend: the zero row of the merge
+            for (int i = threadIdx.x; i < R * 128; i += C::kThreads) out[(s * sh.n_q_heads + (int64_t)head_group * R) * 128 + i] = 0.f;
         return;
     }
 
@@ -915,6 +917,17 @@ decode_pair_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 part_base[(int64_t)h * n_parts * stride + 1] = v;                                            // normaliser, in the same unit
             }
         }
+        // One part per item (out != null only then): the partial is the whole sum, so the CTA normalises it itself
+        // and no merge launch follows.
+        if (out) {
+            __syncthreads();
+            for (int i = threadIdx.x; i < R * 128; i += C::kThreads) {
+                const int h = i >> 7, d = i & 127;
+                const float* ph = part_base + (int64_t)h * n_parts * stride;
+                const float l = ph[1];
+                out[(s * sh.n_q_heads + (int64_t)head_group * R + h) * 128 + d] = l > 0.f ? ph[2 + d] / l : 0.f;
+            }
+        }
     }
 }
 
@@ -976,14 +989,15 @@ DecodePlan decode_pair_plan(const Shape& sh)
 
 cudaError_t launch_decode_pair(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
                                const int32_t* seq_lens, float scale, const Shape& sh, const DecodePlan& pl,
-                               float* partials, cudaStream_t st, const AppendArgs& app)
+                               float* partials, cudaStream_t st, const AppendArgs& app, float* out)
 {
     using C = PairCfg;
     const cudaError_t attr = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_pair_kernel), C::kSmemBytes, 0);
     if (attr != cudaSuccess) return attr;
     const int aligned = ((reinterpret_cast<uintptr_t>(kcb) | reinterpret_cast<uintptr_t>(vcb)) & 31u) == 0 ? 1 : 0;
     decode_pair_kernel<<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk,
-                                                                    pl.n_parts, pl.tail_first, aligned, partials, app);
+                                                                    pl.n_parts, pl.tail_first, aligned, partials, app,
+                                                                    pl.n_parts == 1 ? out : nullptr);
     return cudaGetLastError();
 }
 
