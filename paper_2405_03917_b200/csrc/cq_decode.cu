@@ -191,8 +191,9 @@ __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
                     const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                    int tail_first, int cb_aligned32, int kv_share, float* __restrict__ partials)
+                    int tail_first, int cb_aligned32, int kv_share, float* __restrict__ partials, float* __restrict__ out)
 {
+    // out: non-null only when every item is one part; the CTA then normalises its partial itself (no merge launch).
     // R is the number of query heads one CTA serves.  A KV head with more query heads than that
     // (kv_share groups of R; kShared) is served by kv_share CTAs, which read the same codes and codebooks.
     using C = Cfg<G, R>;
@@ -240,6 +241,8 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
             const int h = i / stride, d = i % stride;
             part_base[(int64_t)h * n_parts * stride + d] = d == 0 ? -INFINITY : 0.f;
         }
+        if (out)            // nothing to attend: the zero row of the merge
+            for (int i = threadIdx.x; i < R * 128; i += C::kThreads) out[(s * sh.n_q_heads + (int64_t)head_group * R) * 128 + i] = 0.f;
         return;
     }
 
@@ -708,6 +711,15 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
         use_unit(cva, u);
         if (u + 2 < kUnits) load_unit(cva, vcb, u + 2);
         use_unit(cvb, u + 1);
+    }
+    if (out) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < R * 128; i += C::kThreads) {
+            const int h = i >> 7, d = i & 127;
+            const float* ph = part_base + (int64_t)h * n_parts * stride;
+            const float l = ph[1];
+            out[(s * sh.n_q_heads + (int64_t)head_group * R + h) * 128 + d] = l > 0.f ? ph[2 + d] / l : 0.f;
+        }
     }
 }
 
@@ -1181,7 +1193,7 @@ Plan plan_for(const Shape& sh)
 template <int G, int R>
 cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
                        const int32_t* seq_lens, float scale, const Shape& sh, const Plan& pl, float* partials,
-                       cudaStream_t st)
+                       cudaStream_t st, float* out)
 {
     using C = Cfg<G, R>;
     const int kv_share = sh.R / R;
@@ -1193,11 +1205,11 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
     if (kv_share > 1)
         decode_tuned_kernel<G, R, true><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
             q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
-            kv_share, partials);
+            kv_share, partials, pl.n_parts == 1 ? out : nullptr);
     else
         decode_tuned_kernel<G, R, false><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
             q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
-            kv_share, partials);
+            kv_share, partials, pl.n_parts == 1 ? out : nullptr);
     return cudaGetLastError();
 }
 
@@ -1278,13 +1290,14 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
             partials);
         e = cudaGetLastError();
     }
-    else if (sh.G == 16 && heads_per_cta(sh) == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 16 && heads_per_cta(sh) == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 16 && heads_per_cta(sh) == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 32 && heads_per_cta(sh) == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 32 && heads_per_cta(sh) == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
-    else if (sh.G == 64) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st);
+    else if (sh.G == 16 && heads_per_cta(sh) == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
+    else if (sh.G == 16 && heads_per_cta(sh) == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
+    else if (sh.G == 16 && heads_per_cta(sh) == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
+    else if (sh.G == 32 && heads_per_cta(sh) == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
+    else if (sh.G == 32 && heads_per_cta(sh) == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
+    else if (sh.G == 64) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
     if (e != cudaSuccess) return e;
+    if (pl.n_parts == 1 && !wide_shape(sh)) return e;           // one part per item: the kernel wrote the output itself
     return launch_merge(partials, pl.n_parts, sh, out, st);
 }
 
