@@ -178,6 +178,8 @@ class DecodeState:
         self.ws = torch.empty(max(256, cq.cq_decode_step_workspace_bytes(w.n_seq, w.n_q_heads, w.n_kv_heads, D, c, b,
                                                                         self.cap)), dtype=torch.uint8, device=dev)
         self.scale = D ** -0.5
+        # launches of one cq_decode_step call: 1 or 2 where the attention kernel appends the token itself
+        self.fused_launches = cq.cq_decode_step_launches(w.n_seq, w.n_q_heads, w.n_kv_heads, D, c, b, self.cap)
 
     def kv_tokens(self) -> int:
         return int(self.lens_cpu.sum().item())
@@ -196,7 +198,7 @@ class DecodeState:
         """Append-encode the new token (K, V) at the last position, then attend: one cq_decode_step call where the
         kernel appends inside the attention launch, else cq_encode_kv followed by cq_decode_attn."""
         w = self.w
-        if shared_word_kernel(w):
+        if self.fused_launches <= 2:
             if ev is not None:
                 ev[0].record()
             cq.cq_decode_step(self.q, self.k_new, self.v_new, self.append_pos, self.k_codes, self.v_codes, self.k_cb,
@@ -637,9 +639,7 @@ def main():
             "e2e": {"value": kv_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             # per layer: attention (which appends the new token where the kernel can) and merge, else also the append-encode
-            "gpu_launches": args.steps * len(states) * (cq.cq_decode_step_launches(w.n_seq, w.n_q_heads, w.n_kv_heads, w.head_dim,
-                                                                                   w.c, w.b, st.cap)
-                                                         if shared_word_kernel(w) else 3),
+            "gpu_launches": args.steps * len(states) * (st.fused_launches if st.fused_launches <= 2 else 3),
             "roofline": roofline}
 
     if args.extras != "none" and world == 1:

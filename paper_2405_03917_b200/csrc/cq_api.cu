@@ -491,7 +491,7 @@ int cq_decode_step_launches(int n_seq, int n_q_heads, int n_kv_heads, int head_d
     Shape sh;
     if (make_shape(n_seq, max_tokens, n_q_heads, n_kv_heads, head_dim, c, b, &sh) != CQ_OK) return 0;
     if (decode_tuned_supported(sh) && decode_fused_append_supported(sh))
-        return decode_pair_plan(sh).n_parts == 1 ? 1 : 2;        // attention (with the append inside) [+ merge]
+        return decode_step_fused_launches(sh);                   // attention (with the append inside) [+ merge]
     return 4;                                                      // lengths plus one, append, attention, merge
 }
 

@@ -132,9 +132,11 @@ int decode_tuned_parts(const Shape& sh);      // partial slots per (sequence, qu
 // with shared table words (cq_decode_pair.cu) would be picked.
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
-                                float* out, float* partials, cudaStream_t st, bool per_head_tables = false);
+                                float* out, float* partials, cudaStream_t st, bool per_head_tables = false,
+                                const AppendArgs& app = AppendArgs());
 // True when launch_decode_tuned would take a kernel that can append a token inside the attention launch.
 bool decode_fused_append_supported(const Shape& sh);
+int decode_step_fused_launches(const Shape& sh);      // 1: the attention kernel also writes the output; 2: plus the merge
 // One decode step: the token (app) is encoded and appended at position seq_lens[s] and the attention covers
 // seq_lens[s] + 1 tokens, in one attention launch (plus the merge).  Only where decode_fused_append_supported.
 cudaError_t launch_decode_step_fused(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,

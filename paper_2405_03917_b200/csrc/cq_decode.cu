@@ -60,7 +60,8 @@ struct Cfg {
     // One plane: K and V planes share a row (K at +0, V at +128).  Two planes: separate tables.
     static constexpr int kVOffset = (kPlanes == 1) ? 128 : kRows * kRowBytes;
     static constexpr int kTableBytes = (kPlanes == 1) ? kRows * kRowBytes : 2 * kRows * kRowBytes;
-    static constexpr int kCtlBytes = 128 + R * 128 * 4;                  // control words + scaled query
+    static constexpr int kNewOffset = 128 + R * 128 * 4;                 // codes of an appended token: [key | value][64 groups]
+    static constexpr int kCtlBytes = kNewOffset + 128;                   // control words + scaled query + those codes
     static constexpr int kSmemBytes = kTableBytes + kCtlBytes;
 
     // word inside a plane that lane (r, p) uses for its m-th code word
@@ -186,12 +187,70 @@ __device__ __forceinline__ float fold_channels(const float (&a)[kC], int lane)
 }
 
 
+// byte k (0..15) of a 16-byte code word replaced
+__device__ __forceinline__ void put_code(uint4& w, int k, uint32_t code)
+{
+    const uint32_t keep = ~(0xffu << (8 * (k & 3))), put = code << (8 * (k & 3));
+    if ((k >> 2) == 0) w.x = (w.x & keep) | put;
+    else if ((k >> 2) == 1) w.y = (w.y & keep) | put;
+    else if ((k >> 2) == 2) w.z = (w.z & keep) | put;
+    else w.w = (w.w & keep) | put;
+}
+
+// The value codes of the token that the launch appends (CQ encode, Section 3.2), by the whole CTA: a warp takes
+// the groups it owns, its lanes walk the centroids; d_j = sum_i (x_i - C_ji)^2 in fp32 in the order of the encode
+// kernels, lowest index on ties.  The codes go to newcode[g] and, from the CTA that `writer` names, to position
+// `pos` of the cache.  (The key codes come out of the table build, which reads the key centroids anyway.)
+template <int kC, int kGroupsPerWarp>
+__device__ __noinline__ void encode_new_value_tuned(uint8_t* newcode, const __half* __restrict__ v_new, uint8_t* vc_w,
+                                                    const float* __restrict__ vcb, Shape sh, int64_t s, int hkv, int64_t pos,
+                                                    bool writer)
+{
+    constexpr int G = 128 / kC;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll 1
+    for (int e = 0; e < kGroupsPerWarp; ++e) {
+        const int g = warp * kGroupsPerWarp + e;
+        const __half* xp = v_new + (s * sh.n_kv_heads + hkv) * 128 + g * kC;
+        const float* cg = vcb + ((int64_t)hkv * G + g) * kRows * kC;
+        float xg[kC];
+#pragma unroll
+        for (int i = 0; i < kC; ++i) xg[i] = __half2float(xp[i]);
+        float cv[kRows / 32][kC];                     // all loads in flight at once
+#pragma unroll
+        for (int t = 0; t < kRows / 32; ++t) load_centroid<kC>(cg + (int64_t)(t * 32 + lane) * kC, cv[t], false);
+        float best = INFINITY;
+        int arg = 0;
+#pragma unroll
+        for (int t = 0; t < kRows / 32; ++t) {
+            float d = 0.f;
+#pragma unroll
+            for (int i = 0; i < kC; ++i) {
+                const float diff = xg[i] - cv[t][i];
+                d = fmaf(diff, diff, d);
+            }
+            if (d < best) { best = d; arg = t * 32 + lane; }        // ascending: strict < keeps the lowest index
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+            if (ob < best || (ob == best && oa < arg)) { best = ob; arg = oa; }
+        }
+        if (lane == 0) {
+            newcode[g] = (uint8_t)arg;
+            if (writer) vc_w[code_word_offset(sh, sh.n_kv_heads, s, hkv, pos / kTokenBlock, g) + pos % kTokenBlock] = (uint8_t)arg;
+        }
+    }
+}
+
 template <int G, int R, bool kShared>
 __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
                     const int32_t* __restrict__ seq_lens, float scale_log2e, Shape sh, int chunk_tokens, int n_parts,
-                    int tail_first, int cb_aligned32, int kv_share, float* __restrict__ partials, float* __restrict__ out)
+                    int tail_first, int cb_aligned32, int kv_share, float* __restrict__ partials, float* __restrict__ out,
+                    AppendArgs app)
 {
     // out: non-null only when every item is one part; the CTA then normalises its partial itself (no merge launch).
     // R is the number of query heads one CTA serves.  A KV head with more query heads than that
@@ -226,6 +285,10 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 
     int64_t n = seq_lens[s];
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
+    // With an append, seq_lens counts the tokens cached before this launch: the new token takes position n and
+    // the attention covers n + 1 tokens (a sequence at capacity gets no new token).
+    const bool has_new = app.k_new != nullptr && n < sh.max_tokens;
+    if (has_new) ++n;
     const int64_t t_begin = (int64_t)part * chunk_tokens;
     const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
     const int stride = partial_stride(128);
@@ -251,6 +314,14 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     const int64_t blk_lim = (t_end + kTokenBlock - 1) / kTokenBlock;       // blocks holding a valid token
     const int n_iters = (int)((t_end - t_begin + C::kRoundTokens - 1) / C::kRoundTokens);
     const int qb = (C::kBlocksPerIter == 8) ? r : (r & 3);                 // block of this quad inside the warp's iteration
+    // The new token, when its position is in this CTA's range: the CTA works its codes out itself (so do the CTAs of
+    // the other query heads that share the KV head) and puts them into the code words it loads of that block; one
+    // CTA per KV head also writes them to the cache.
+    const bool new_here = has_new && t_begin <= n - 1 && n - 1 < t_end;
+    const int64_t new_blk = (n - 1) / kTokenBlock;
+    const int new_tok = (int)((n - 1) % kTokenBlock);
+    const bool new_writer = !kShared || head_group % kv_share == 0;
+    uint8_t* newcode = smem + C::kTableBytes + C::kNewOffset;               // [key | value][64]
     uint32_t lane_off[C::kSlots];      // byte offset of this lane's word inside a plane, per code word
 #pragma unroll
     for (int m = 0; m < C::kSlots; ++m) lane_off[m] = 4u * C::word(r, p, m) + C::lane_plane_bytes(r);
@@ -265,6 +336,11 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 #pragma unroll
             for (int m = 0; m < C::kSlots; ++m)
                 dst[m] = ldg_codes(reinterpret_cast<const uint4*>(bp + C::group_of(lane_off[m] >> 2) * kTokenBlock));
+            if (new_here && blk == new_blk) {
+                const uint8_t* nc = newcode + (base == vbase ? 64 : 0);
+#pragma unroll
+                for (int m = 0; m < C::kSlots; ++m) put_code(dst[m], new_tok, nc[C::group_of(lane_off[m] >> 2)]);
+            }
         } else {
 #pragma unroll
             for (int m = 0; m < C::kSlots; ++m) dst[m] = make_uint4(0u, 0u, 0u, 0u);
@@ -307,12 +383,26 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     // rows) would fall into one bank, so the build writes row j rotated by j words and a second
     // pass un-rotates every row.  Entries are half2 (hi, lo) of LUT * 2^-kexp; kexp = 0 unless an
     // entry reaches 2^15 (then the build is repeated once with the exponent that fits).
+    if (new_here)
+        encode_new_value_tuned<kC, C::kGroupsPerWarp>(newcode + 64, app.v_new, app.vc_w, vcb, sh, s, hkv, n - 1, new_writer);
+    // the new token's key, when this CTA appends it: its code of group g is the centroid nearest to it, found on the
+    // way (d_j = sum_i (x_i - C_ji)^2 in fp32 in the order of the encode kernels, lowest index on ties)
+    float xnew[kC], dnew = INFINITY;
+    int jnew = 0;
     float lut_scale = 1.f;           // scores in table units * lut_scale = log2-domain scores
     for (int attempt = 0; attempt < 2; ++attempt) {
         const float inv = 1.f / lut_scale;
         float absmax = 0.f;
+        const bool find_key = new_here && attempt == 0;
         auto build_unit = [&](const float (&cv)[kJb][kC], int u) {
             const int g = warp * C::kGroupsPerWarp + u / kUnitsPerGroup;
+            if (find_key && u % kUnitsPerGroup == 0) {
+                const __half* xp = app.k_new + (s * sh.n_kv_heads + hkv) * 128 + g * kC;
+#pragma unroll
+                for (int i = 0; i < kC; ++i) xnew[i] = __half2float(xp[i]);
+                dnew = INFINITY;
+                jnew = 0;
+            }
             float qreg[R][kC];
 #pragma unroll
             for (int h = 0; h < R; ++h)
@@ -331,6 +421,28 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     uint8_t* row = smem + j * kRowBytes + C::plane_of(g, h) * 128;
                     *reinterpret_cast<uint32_t*>(row + ((C::word_of(g, h) + j) & 31) * 4) = e;
                     if (C::kReplica) *reinterpret_cast<uint32_t*>(row + ((16 + g + j) & 31) * 4) = e;
+                }
+                if (find_key) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int i = 0; i < kC; ++i) {
+                        const float diff = xnew[i] - cv[jb][i];
+                        d = fmaf(diff, diff, d);
+                    }
+                    if (d < dnew) { dnew = d; jnew = j; }        // a lane's j ascend: strict < keeps the lowest index
+                }
+            }
+            if (find_key && u % kUnitsPerGroup == kUnitsPerGroup - 1) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float ob = __shfl_xor_sync(0xffffffffu, dnew, o);
+                    const int oa = __shfl_xor_sync(0xffffffffu, jnew, o);
+                    if (ob < dnew || (ob == dnew && oa < jnew)) { dnew = ob; jnew = oa; }
+                }
+                if (lane == 0) {
+                    newcode[g] = (uint8_t)jnew;
+                    if (new_writer)
+                        app.kc_w[code_word_offset(sh, sh.n_kv_heads, s, hkv, (n - 1) / kTokenBlock, g) + (n - 1) % kTokenBlock] = (uint8_t)jnew;
                 }
             }
         };
@@ -1193,7 +1305,7 @@ Plan plan_for(const Shape& sh)
 template <int G, int R>
 cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb, const float* vcb,
                        const int32_t* seq_lens, float scale, const Shape& sh, const Plan& pl, float* partials,
-                       cudaStream_t st, float* out)
+                       cudaStream_t st, float* out, const AppendArgs& app)
 {
     using C = Cfg<G, R>;
     const int kv_share = sh.R / R;
@@ -1205,11 +1317,11 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
     if (kv_share > 1)
         decode_tuned_kernel<G, R, true><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
             q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
-            kv_share, partials, pl.n_parts == 1 ? out : nullptr);
+            kv_share, partials, pl.n_parts == 1 ? out : nullptr, app);
     else
         decode_tuned_kernel<G, R, false><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
             q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
-            kv_share, partials, pl.n_parts == 1 ? out : nullptr);
+            kv_share, partials, pl.n_parts == 1 ? out : nullptr, app);
     return cudaGetLastError();
 }
 
@@ -1256,26 +1368,29 @@ int decode_tuned_parts(const Shape& sh)
     return pair > own ? pair : own;
 }
 
-bool decode_fused_append_supported(const Shape& sh) { return decode_pair_supported(sh); }
+bool decode_fused_append_supported(const Shape& sh) { return decode_tuned_supported(sh) && !wide_shape(sh); }
+
+int decode_step_fused_launches(const Shape& sh)
+{
+    if (decode_pair_supported(sh)) return decode_pair_plan(sh).n_parts == 1 ? 1 : 2;
+    return plan_dispatch(sh).n_parts == 1 ? 1 : 2;
+}
 
 cudaError_t launch_decode_step_fused(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                      const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh,
                                      float* out, float* partials, const AppendArgs& app, cudaStream_t st)
 {
-    if (!decode_pair_supported(sh)) return cudaErrorNotSupported;
-    const DecodePlan pp = decode_pair_plan(sh);
-    const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, app, out);
-    if (ep != cudaSuccess || pp.n_parts == 1) return ep;
-    return launch_merge(partials, pp.n_parts, sh, out, st);
+    if (!decode_fused_append_supported(sh)) return cudaErrorNotSupported;
+    return launch_decode_tuned(q, kc, vc, kcb, vcb, seq_lens, scale, sh, out, partials, st, false, app);
 }
 
 cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_t* vc, const float* kcb,
                                 const float* vcb, const int32_t* seq_lens, float scale, const Shape& sh, float* out,
-                                float* partials, cudaStream_t st, bool per_head_tables)
+                                float* partials, cudaStream_t st, bool per_head_tables, const AppendArgs& app)
 {
     if (!per_head_tables && decode_pair_supported(sh)) {
         const DecodePlan pp = decode_pair_plan(sh);
-        const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, AppendArgs(), out);
+        const cudaError_t ep = launch_decode_pair(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pp, partials, st, app, out);
         if (ep != cudaSuccess || pp.n_parts == 1) return ep;      // one part per item: the kernel wrote the output itself
         return launch_merge(partials, pp.n_parts, sh, out, st);
     }
@@ -1283,6 +1398,7 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
     if (pl.chunk <= 0) return cudaErrorNotSupported;
     cudaError_t e = cudaErrorNotSupported;
     if (wide_shape(sh)) {
+        if (app.k_new) return cudaErrorNotSupported;          // this kernel does not append
         e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_wide_kernel), WideCfg::kSmemBytes, 1);
         if (e != cudaSuccess) return e;
         decode_wide_kernel<<<pl.grid, WideCfg::kThreads, WideCfg::kSmemBytes, st>>>(
@@ -1290,12 +1406,12 @@ cudaError_t launch_decode_tuned(const __half* q, const uint8_t* kc, const uint8_
             partials);
         e = cudaGetLastError();
     }
-    else if (sh.G == 16 && heads_per_cta(sh) == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
-    else if (sh.G == 16 && heads_per_cta(sh) == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
-    else if (sh.G == 16 && heads_per_cta(sh) == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
-    else if (sh.G == 32 && heads_per_cta(sh) == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
-    else if (sh.G == 32 && heads_per_cta(sh) == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
-    else if (sh.G == 64) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out);
+    else if (sh.G == 16 && heads_per_cta(sh) == 1) e = launch_cfg<16, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out, app);
+    else if (sh.G == 16 && heads_per_cta(sh) == 2) e = launch_cfg<16, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out, app);
+    else if (sh.G == 16 && heads_per_cta(sh) == 4) e = launch_cfg<16, 4>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out, app);
+    else if (sh.G == 32 && heads_per_cta(sh) == 1) e = launch_cfg<32, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out, app);
+    else if (sh.G == 32 && heads_per_cta(sh) == 2) e = launch_cfg<32, 2>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out, app);
+    else if (sh.G == 64) e = launch_cfg<64, 1>(q, kc, vc, kcb, vcb, seq_lens, scale, sh, pl, partials, st, out, app);
     if (e != cudaSuccess) return e;
     if (pl.n_parts == 1 && !wide_shape(sh)) return e;           // one part per item: the kernel wrote the output itself
     return launch_merge(partials, pl.n_parts, sh, out, st);
