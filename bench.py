@@ -194,6 +194,16 @@ class DecodeState:
         qo = w.n_seq * w.n_q_heads * w.head_dim * (2 + 4)
         return codes + books + qo
 
+    def attend(self, cq, ev=None):
+        """Decode attention alone (cq_decode_attn) over the cache as it stands."""
+        w = self.w
+        if ev is not None:
+            ev[0].record()
+        cq.cq_decode_attn(self.q, self.k_codes, self.v_codes, self.k_cb, self.v_cb, self.seq_lens, self.scale,
+                          w.c, w.b, self.cap, out=self.out, workspace=self.ws)
+        if ev is not None:
+            ev[1].record()
+
     def step(self, cq, ev=None):
         """Append-encode the new token (K, V) at the last position, then attend: one cq_decode_step call where the
         kernel appends inside the attention launch, else cq_encode_kv followed by cq_decode_attn."""
@@ -445,13 +455,15 @@ def extra_encode_wide(cq, dev, w, reps=3):
 
 
 def extra_decode(cq, dev, w, reps=20):
+    """One decode-attention call (cq_decode_attn, no append) of another workload, with its roofline."""
     st = DecodeState(w, 0, dev, cq)
     for _ in range(3):
         st.step(cq)
+        st.attend(cq)
     torch.cuda.synchronize()
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
     for e in evs:
-        st.step(cq, e)
+        st.attend(cq, e)
     torch.cuda.synchronize()
     ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
     res = {"workload": w.name, "decode_ms": ms, "kv_tokens_per_s": st.kv_tokens() / (ms * 1e-3),

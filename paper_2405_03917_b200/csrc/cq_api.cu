@@ -11,7 +11,7 @@ namespace {
 constexpr int kDeviceSlots = 64;
 std::mutex g_device_mutex;
 int g_sm_count[kDeviceSlots] = {};                   // 0: not queried yet
-int g_smem_set[kDeviceSlots][64] = {};               // per device and call site: dynamic shared memory size already set
+int g_smem_set[kDeviceSlots][96] = {};               // per device and call site: dynamic shared memory size already set
 }  // namespace
 
 int device_sm_count()
@@ -38,7 +38,7 @@ cudaError_t ensure_dynamic_smem(const void* func, int bytes, int slot)
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kDeviceSlots || slot < 0 || slot >= 64)
+    if (dev < 0 || dev >= kDeviceSlots || slot < 0 || slot >= 96)
         return cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     std::lock_guard<std::mutex> lock(g_device_mutex);
     if (g_smem_set[dev][slot] >= bytes && bytes > 0) return cudaSuccess;

@@ -244,7 +244,9 @@ __device__ __noinline__ void encode_new_value_tuned(uint8_t* newcode, const __ha
     }
 }
 
-template <int G, int R, bool kShared>
+// kAppend: the launch also encodes and appends one token per sequence (a second instance, so that the plain attention
+// carries none of that code)
+template <int G, int R, bool kShared, bool kAppend>
 __global__ void __launch_bounds__(Cfg<G, R>::kThreads, Cfg<G, R>::kMinBlocks)
 decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
                     const float* __restrict__ kcb, const float* __restrict__ vcb,
@@ -287,7 +289,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     n = n < 0 ? 0 : (n > sh.max_tokens ? sh.max_tokens : n);
     // With an append, seq_lens counts the tokens cached before this launch: the new token takes position n and
     // the attention covers n + 1 tokens (a sequence at capacity gets no new token).
-    const bool has_new = app.k_new != nullptr && n < sh.max_tokens;
+    const bool has_new = kAppend && app.k_new != nullptr && n < sh.max_tokens;
     if (has_new) ++n;
     const int64_t t_begin = (int64_t)part * chunk_tokens;
     const int64_t t_end = (whole || t_begin + chunk_tokens >= n) ? n : t_begin + chunk_tokens;
@@ -317,7 +319,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     // The new token, when its position is in this CTA's range: the CTA works its codes out itself (so do the CTAs of
     // the other query heads that share the KV head) and puts them into the code words it loads of that block; one
     // CTA per KV head also writes them to the cache.
-    const bool new_here = has_new && t_begin <= n - 1 && n - 1 < t_end;
+    const bool new_here = kAppend && has_new && t_begin <= n - 1 && n - 1 < t_end;
     const int64_t new_blk = (n - 1) / kTokenBlock;
     const int new_tok = (int)((n - 1) % kTokenBlock);
     const bool new_writer = !kShared || head_group % kv_share == 0;
@@ -336,7 +338,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
 #pragma unroll
             for (int m = 0; m < C::kSlots; ++m)
                 dst[m] = ldg_codes(reinterpret_cast<const uint4*>(bp + C::group_of(lane_off[m] >> 2) * kTokenBlock));
-            if (new_here && blk == new_blk) {
+            if (kAppend && new_here && blk == new_blk) {
                 const uint8_t* nc = newcode + (base == vbase ? 64 : 0);
 #pragma unroll
                 for (int m = 0; m < C::kSlots; ++m) put_code(dst[m], new_tok, nc[C::group_of(lane_off[m] >> 2)]);
@@ -383,7 +385,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     // rows) would fall into one bank, so the build writes row j rotated by j words and a second
     // pass un-rotates every row.  Entries are half2 (hi, lo) of LUT * 2^-kexp; kexp = 0 unless an
     // entry reaches 2^15 (then the build is repeated once with the exponent that fits).
-    if (new_here)
+    if (kAppend && new_here)
         encode_new_value_tuned<kC, C::kGroupsPerWarp>(newcode + 64, app.v_new, app.vc_w, vcb, sh, s, hkv, n - 1, new_writer);
     // the new token's key, when this CTA appends it: its code of group g is the centroid nearest to it, found on the
     // way (d_j = sum_i (x_i - C_ji)^2 in fp32 in the order of the encode kernels, lowest index on ties)
@@ -393,10 +395,10 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
     for (int attempt = 0; attempt < 2; ++attempt) {
         const float inv = 1.f / lut_scale;
         float absmax = 0.f;
-        const bool find_key = new_here && attempt == 0;
+        const bool find_key = kAppend && new_here && attempt == 0;
         auto build_unit = [&](const float (&cv)[kJb][kC], int u) {
             const int g = warp * C::kGroupsPerWarp + u / kUnitsPerGroup;
-            if (find_key && u % kUnitsPerGroup == 0) {
+            if (kAppend && find_key && u % kUnitsPerGroup == 0) {
                 const __half* xp = app.k_new + (s * sh.n_kv_heads + hkv) * 128 + g * kC;
 #pragma unroll
                 for (int i = 0; i < kC; ++i) xnew[i] = __half2float(xp[i]);
@@ -422,7 +424,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     *reinterpret_cast<uint32_t*>(row + ((C::word_of(g, h) + j) & 31) * 4) = e;
                     if (C::kReplica) *reinterpret_cast<uint32_t*>(row + ((16 + g + j) & 31) * 4) = e;
                 }
-                if (find_key) {
+                if (kAppend && find_key) {
                     float d = 0.f;
 #pragma unroll
                     for (int i = 0; i < kC; ++i) {
@@ -432,7 +434,7 @@ decode_tuned_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc
                     if (d < dnew) { dnew = d; jnew = j; }        // a lane's j ascend: strict < keeps the lowest index
                 }
             }
-            if (find_key && u % kUnitsPerGroup == kUnitsPerGroup - 1) {
+            if (kAppend && find_key && u % kUnitsPerGroup == kUnitsPerGroup - 1) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) {
                     const float ob = __shfl_xor_sync(0xffffffffu, dnew, o);
@@ -1311,17 +1313,25 @@ cudaError_t launch_cfg(const __half* q, const uint8_t* kc, const uint8_t* vc, co
     const int kv_share = sh.R / R;
     // call-site slots of ensure_dynamic_smem: 1 is the wide kernel, 2 ... 13 the template instances
     constexpr int kSlot = 2 + 2 * ((G == 16 ? 0 : G == 32 ? 3 : 5) + (R == 1 ? 0 : R == 2 ? 1 : 2));
-    cudaError_t e = kv_share > 1 ? ensure_dynamic_smem(reinterpret_cast<const void*>(decode_tuned_kernel<G, R, true>), C::kSmemBytes, kSlot)
-                                 : ensure_dynamic_smem(reinterpret_cast<const void*>(decode_tuned_kernel<G, R, false>), C::kSmemBytes, kSlot + 1);
-    if (e != cudaSuccess) return e;
-    if (kv_share > 1)
-        decode_tuned_kernel<G, R, true><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
-            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
-            kv_share, partials, pl.n_parts == 1 ? out : nullptr, app);
-    else
-        decode_tuned_kernel<G, R, false><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(
-            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),
-            kv_share, partials, pl.n_parts == 1 ? out : nullptr, app);
+    const bool append = app.k_new != nullptr;
+    // one launch per (shared KV head or not, appending or not) instance; smem call-site slots kSlot, kSlot + 1 and 64 + those
+#define CQ_LAUNCH_TUNED(SHARED, APPEND, SLOT)                                                                                   \
+    do {                                                                                                                        \
+        cudaError_t e_ = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_tuned_kernel<G, R, SHARED, APPEND>),           \
+                                             C::kSmemBytes, SLOT);                                                              \
+        if (e_ != cudaSuccess) return e_;                                                                                       \
+        decode_tuned_kernel<G, R, SHARED, APPEND><<<pl.grid, C::kThreads, C::kSmemBytes, st>>>(                                  \
+            q, kc, vc, kcb, vcb, seq_lens, scale * kLog2e, sh, pl.chunk, pl.n_parts, pl.tail_first, aligned32(kcb, vcb),         \
+            kv_share, partials, pl.n_parts == 1 ? out : nullptr, app);                                                          \
+    } while (0)
+    if (kv_share > 1) {
+        if (append) CQ_LAUNCH_TUNED(true, true, 62 + kSlot);
+        else CQ_LAUNCH_TUNED(true, false, kSlot);
+    } else {
+        if (append) CQ_LAUNCH_TUNED(false, true, 62 + kSlot + 1);
+        else CQ_LAUNCH_TUNED(false, false, kSlot + 1);
+    }
+#undef CQ_LAUNCH_TUNED
     return cudaGetLastError();
 }
 
