@@ -121,3 +121,60 @@ def test_argument_validation_happens_on_the_host(L):
     assert rope(c=1, b=2, pairing=1) == -3     # an interleaved pair would span two groups
     assert rope(cos=p + 2) == -4
     assert rope(ws_bytes=16) == -5
+
+
+def test_new_entry_points_validate_on_the_host(L):
+    p = 0x10000
+    f32 = ctypes.c_float
+    # cq_decode_step: null pointers, shapes, alignment of the new key / value, aliasing caches, workspace size
+    step = lambda **kw: L.cq_decode_step(*[kw.get(k, d) for k, d in [
+        ("q", p), ("k", p), ("v", p), ("sl", p), ("kc", p), ("vc", p + 4096), ("kcb", p), ("vcb", p), ("scale", f32(0.1)),
+        ("n_seq", 2), ("hq", 8), ("hkv", 2), ("D", 128), ("c", 8), ("b", 8), ("cap", 64), ("out", p), ("ws", p),
+        ("ws_bytes", 1 << 30), ("stream", None)]])
+    assert step(k=None) == -1
+    assert step(sl=None) == -1
+    assert step(hkv=3) == -2
+    assert step(vc=p) == -2                    # the two caches must be different buffers
+    assert step(b=11) == -3
+    assert step(k=p + 2) == -4
+    assert step(ws_bytes=64) == -5
+    # launches of a step: the attention kernel appends and writes the output (1), plus a merge for split contexts (2),
+    # or lengths + append + attention + merge (4) where no kernel appends; 0 for a shape the library refuses
+    assert cq.cq_decode_step_launches(64, 32, 8, 128, 8, 8, 16384) in (1, 2)
+    assert cq.cq_decode_step_launches(16, 32, 32, 128, 4, 8, 4096) in (1, 2)
+    assert cq.cq_decode_step_launches(2, 8, 2, 128, 8, 8, 1 << 20) == 2          # few long contexts: split, so a merge follows
+    assert cq.cq_decode_step_launches(16, 32, 32, 128, 8, 10, 8192) == 4         # CQ-8c10b: no appending kernel
+    assert cq.cq_decode_step_launches(2, 4, 2, 64, 4, 5, 100) == 4
+    assert cq.cq_decode_step_launches(2, 4, 3, 64, 4, 5, 100) == 0
+    assert cq.cq_decode_step_workspace_bytes(4, 8, 2, 128, 8, 8, 100) > cq.cq_decode_attn_workspace_bytes(4, 8, 2, 128, 8, 8, 100)
+
+    # cq_prefill_attn: more queries than the cache holds, bad variant, null pointers
+    pre = lambda **kw: L.cq_prefill_attn_variant(*[kw.get(k, d) for k, d in [
+        ("q", p), ("kc", p), ("vc", p), ("kcb", p), ("vcb", p), ("sl", p), ("scale", f32(0.1)), ("n_seq", 1), ("n_q", 4),
+        ("hq", 4), ("hkv", 2), ("D", 128), ("c", 8), ("b", 8), ("cap", 64), ("out", p), ("variant", 0), ("stream", None)]])
+    assert pre(q=None) == -1
+    assert pre(n_q=65) == -2
+    assert pre(variant=7) == -2
+    assert pre(hkv=3) == -2
+    assert pre(b=10, variant=2) == -3          # the tensor-core kernel takes byte codes only
+
+    # cq_decode_attn_rope_variant: pairing, groups that a pair would split, the tuned kernel's shapes
+    rope = lambda **kw: L.cq_decode_attn_rope_variant(*[kw.get(k, d) for k, d in [
+        ("q", p), ("kc", p), ("vc", p), ("kcb", p), ("vcb", p), ("sl", p), ("cos", p), ("sin", p), ("pairing", 0),
+        ("scale", f32(0.1)), ("n_seq", 1), ("hq", 4), ("hkv", 2), ("D", 128), ("c", 8), ("b", 8), ("cap", 64),
+        ("out", p), ("ws", p), ("ws_bytes", 1 << 30), ("variant", 0), ("stream", None)]])
+    assert rope(cos=None) == -1
+    assert rope(pairing=2) == -2
+    assert rope(variant=3) == -2
+    assert rope(pairing=1, variant=2) == -3    # the tuned kernel pairs (i, i + 64) only
+    assert rope(c=2, variant=2) == -3
+    assert rope(cos=p + 4, variant=2) == -3    # tables must be 8-byte aligned for it
+    assert rope(cos=p + 2) == -4
+
+    # cq_encode_variant 4: the tensor-memory kernel takes byte codes of head_dim 128 only
+    encv = lambda **kw: L.cq_encode_variant(*[kw.get(k, d) for k, d in [
+        ("x", p), ("cb", p), ("so", None), ("n_seq", 1), ("n_tok", 4), ("off", 0), ("cap", 16),
+        ("heads", 1), ("D", 128), ("c", 8), ("b", 8), ("out", p), ("variant", 4), ("stream", None)]])
+    assert encv(b=10) == -3
+    assert encv(D=64) == -3
+    assert encv(variant=5) == -2
