@@ -53,11 +53,11 @@ def measured_peaks():
     return HBM_FALLBACK_GBS, "fallback"
 
 
-def kernel_source_hash():
-    """sha256 over the decode kernels' source files (the kernels the roofline object describes)."""
+def kernel_source_hash(files=("cq_decode.cu", "cq_decode_pair.cu", "cq_decode_util.cuh", "cq_bulk_copy.cuh", "cq_common.cuh")):
+    """sha256 over the source files of a decode kernel (the kernel a roofline object describes)."""
     import hashlib
     h = hashlib.sha256()
-    for f in ("cq_decode.cu", "cq_decode_pair.cu", "cq_decode_util.cuh", "cq_bulk_copy.cuh", "cq_common.cuh"):
+    for f in files:
         h.update(open(os.path.join(ROOT, "paper_2405_03917_b200", "csrc", f), "rb").read())
     return h.hexdigest()
 
@@ -235,7 +235,7 @@ def attach_traffic(roofline, workload_name):
     try:
         t = json.load(open(tr)).get(workload_name)
         # the counters describe one build of the kernels: any later edit of their source voids them
-        if t and t.get("kernel_source_sha256") == kernel_source_hash():
+        if t and t.get("kernel_source_sha256") == kernel_source_hash(tuple(t["files"])):
             roofline["traffic"] = t["dram_bytes_per_launch"]
             roofline["traffic_source"] = t.get("source")
     except Exception:
