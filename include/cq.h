@@ -350,12 +350,13 @@ int cq_learn_centroids(const void *x_fp16, const float *weights, const double *u
  * One decode step of one layer on DEVICE buffers: the new token's key and value
  * vectors are encoded (CQ encode, Section 3.2, as cq_encode does) and appended at
  * position seq_lens[s] of every sequence, and the step's query attends over
- * seq_lens[s] + 1 tokens (Eq. 1, as cq_decode_attn does).  For CQ-8c8b with
- * head_dim 128 and a multiple of four query heads per KV head the append happens
- * INSIDE the attention launch: the CTAs whose part of the context holds the new
- * position work the codes out, use them, and one of them writes them to the
- * cache; the step is then one attention launch plus the merge.  Every other shape
- * runs cq_encode_kv and cq_decode_attn one after the other.
+ * seq_lens[s] + 1 tokens (Eq. 1, as cq_decode_attn does).  For head_dim 128 with
+ * b = 8 and c in {2, 4, 8} (the shapes with tuned decode kernels) the append
+ * happens INSIDE the attention launch: the CTAs whose part of the context holds
+ * the new position work the codes out, use them, and one of them writes them to
+ * the cache; the step is then one attention launch, plus the merge of the partials
+ * where contexts are split over CTAs (cq_decode_step_launches tells).  Every other
+ * shape runs cq_encode_kv and cq_decode_attn one after the other.
  *
  *   q_fp16       [n_seq][n_q_heads][head_dim] fp16, device
  *   k_new_fp16, v_new_fp16   [n_seq][n_kv_heads][head_dim] fp16, device, 16-byte aligned
