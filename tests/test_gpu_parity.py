@@ -421,16 +421,16 @@ def test_token_permutation_and_seq_len_padding_invariance():
     np.testing.assert_allclose(out, base, rtol=0, atol=2e-5)
 
 
-@pytest.mark.parametrize("packed", [False, True])
-def test_decode_step_from_host_buffers(packed):
+@pytest.mark.parametrize("packed,n_seq", [(False, 3), (True, 3), (True, 9), (False, 8)])
+def test_decode_step_from_host_buffers(packed, n_seq):
     # packed: query, key and value back to back in one pinned block (they then travel in one copy)
-    c, b, D, cap, n_seq, n_q, n_kv = 8, 8, 128, 200, 3, 4, 2
+    c, b, D, cap, n_q, n_kv = 8, 8, 128, 200, 4, 2
     w = H.small_workload("t", 66, c, b, n_seq, n_q, n_kv, cap)
     xk = synth.layer_activations(w, 0, False, n_seq, cap)
     xv = synth.layer_activations(w, 0, True, n_seq, cap)
     kcb, vcb = synth.layer_codebooks(w, 0, False), synth.layer_codebooks(w, 0, True)
     q = synth.queries(66, 0, n_seq, n_q)
-    lens = [150, 0, 199]                       # tokens already cached; the step appends one more
+    lens = ([150, 0, 199] * 3)[:n_seq]         # tokens already cached; the step appends one more
     kbuf, _ = encode_both(xk, kcb, c, b, cap)
     vbuf, _ = encode_both(xv, vcb, c, b, cap)
     k_new = torch.stack([xk[s, 7] for s in range(n_seq)]).contiguous()      # (n_seq, n_kv, D)
