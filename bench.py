@@ -267,8 +267,10 @@ def decode_roofline(w, st, ms, dev, sm_mhz=None):
     nbytes = st.algorithmic_bytes()
     t_hbm, t_smem = nbytes / (hbm * 1e9), lane_ops / smem_peak
     a_hbm, a_smem = nbytes / (ms * 1e-3) / 1e9, lane_ops / (ms * 1e-3)
+    merged = w.b == 10 or st.fused_launches != 1         # a merge launch follows unless the kernel writes the output itself
     o = {"kernel": ("decode_pair_kernel" if shared_word_kernel(w) else
-                    "decode_wide_kernel" if w.b == 10 else "decode_tuned_kernel") + " + merge_kernel (one attention call)",
+                    "decode_wide_kernel" if w.b == 10 else "decode_tuned_kernel") +
+                   (" + merge_kernel (one attention call)" if merged else " (one attention call; the kernel writes the output itself)"),
          "launch_ms": ms, "algorithmic_bytes_per_launch": nbytes, "traffic": None,
          "hbm": {"achieved": a_hbm, "peak": hbm, "unit": "GB/s", "frac": a_hbm / hbm, "frac_of_8tbs_nominal": a_hbm / 8000.0,
                  "peak_source": which + " copy bandwidth", "min_ms": t_hbm * 1e3},
