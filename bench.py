@@ -3,8 +3,9 @@
 
 One "step" is one decode step over every layer of the workload (default: CQ-8c8b on a
 Mistral-7B-shaped GQA layer, batch 64, context 16384, one layer): per layer the new token's
-key and value vectors are CQ-encoded and appended (cq_encode, K and V), then every query
-head attends over the coded cache (cq_decode_attn).  Inputs are seeded and synthetic.
+key and value vectors are CQ-encoded and appended and every query head attends over the coded
+cache (cq_decode_step: one launch where the attention kernel appends the token itself, else
+cq_encode_kv followed by cq_decode_attn).  Inputs are seeded and synthetic.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload cfg2|cfg1|cfg4|cfg0] [--extras none|default|decode|all]
