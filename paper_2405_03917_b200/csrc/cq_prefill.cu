@@ -155,7 +155,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     const int R = sh.R;
     const int q_per_tile = C::kRows / R;                                 // query tokens of one row tile
 
-    const int tile = blockIdx.x % row_tiles;
+    const int tile = row_tiles - 1 - blockIdx.x % row_tiles;               // later queries attend more tokens: they start first
     const int hkv = (blockIdx.x / row_tiles) % sh.n_kv_heads;
     const int64_t s = blockIdx.x / ((int64_t)row_tiles * sh.n_kv_heads);
     int64_t n = seq_lens[s];
