@@ -199,8 +199,11 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     const uint32_t q_s = smem_u32(smem + C::kQOffset), kt_s = smem_u32(smem + C::kKtOffset), vt_s = smem_u32(smem + C::kVtOffset);
 
     // codes -> fp16 tiles of the 64 tokens from j0 on, into buffer `buf`: a work item is (8 tokens, one group)
+    // (with fewer items than threads the warps that take them alternate from tile to tile, so that every warp
+    // dequantises every other tile and goes straight on to the MMAs on the tiles between)
     auto dequantise = [&](int64_t j0, int buf) {
-        for (int item = threadIdx.x; item < 8 * G; item += C::kThreads) {
+        const int first = (threadIdx.x + ((j0 / C::kTile) & 1) * (C::kThreads / 2)) % C::kThreads;
+        for (int item = first; item < 8 * G; item += C::kThreads) {
             const int g = item % G, oct = item / G;                      // tokens 8 oct .. 8 oct + 7 of the tile
             const int64_t blk = j0 / kTokenBlock + (oct >> 1);
             uint2 kw = make_uint2(0u, 0u), vw = make_uint2(0u, 0u);
