@@ -99,7 +99,9 @@ prefill_generic_kernel(const __half* __restrict__ q, const uint8_t* __restrict__
 // tensor-core kernel
 // ------------------------------------------------------------------------------------------
 struct PfCfg {
-    static constexpr int kWarps = 8, kThreads = kWarps * 32;
+    static constexpr int kWarps = 8;                                    // warps that multiply (16 rows each)
+    static constexpr int kProducerWarps = 4;                            // warps that dequantise the tiles
+    static constexpr int kThreads = (kWarps + kProducerWarps) * 32;
     static constexpr int kRows = 128;             // (query, head) rows per CTA: 16 per warp
     static constexpr int kTile = 64;              // cached tokens per step
     static constexpr int kRowBytes = 256;         // 128 fp16 channels
@@ -202,8 +204,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     // (with fewer items than threads the warps that take them alternate from tile to tile, so that every warp
     // dequantises every other tile and goes straight on to the MMAs on the tiles between)
     auto dequantise = [&](int64_t j0, int buf) {
-        const int first = (threadIdx.x + ((j0 / C::kTile) & 1) * (C::kThreads / 2)) % C::kThreads;
-        for (int item = first; item < 8 * G; item += C::kThreads) {
+        for (int item = threadIdx.x - C::kWarps * 32; item < 8 * G; item += C::kProducerWarps * 32) {
             const int g = item % G, oct = item / G;                      // tokens 8 oct .. 8 oct + 7 of the tile
             const int64_t blk = j0 / kTokenBlock + (oct >> 1);
             uint2 kw = make_uint2(0u, 0u), vw = make_uint2(0u, 0u);
@@ -230,14 +231,26 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             }
         }
     };
-    if (n_tiles > 0) dequantise(0, 0);
-    __syncthreads();
+    // Producer warps fill the two tile buffers, the other warps multiply; named barriers 1 + buf ("buffer free") and
+    // 3 + buf ("buffer full") hand a buffer back and forth, registers move from the producers to the multipliers.
+    constexpr int kAll = C::kThreads;
+    if (warp >= C::kWarps) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        for (int64_t jt = 0; jt < n_tiles; ++jt) {
+            const int buf = (int)(jt & 1);
+            if (jt >= 2) asm volatile("bar.sync %0, %1;" ::"r"(1 + buf), "n"(kAll) : "memory");
+            dequantise(jt * C::kTile, buf);
+            __threadfence_block();
+            asm volatile("bar.arrive %0, %1;" ::"r"(3 + buf), "n"(kAll) : "memory");
+        }
+        return;
+    }
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
 
     for (int64_t jt = 0; jt < n_tiles; ++jt) {
         const int64_t j0 = jt * C::kTile;
         const int buf = (int)(jt & 1);
-        // the next tile is dequantised into the other buffer (last read before the barrier that ended the step before)
-        if (jt + 1 < n_tiles) dequantise(j0 + C::kTile, buf ^ 1);
+        asm volatile("bar.sync %0, %1;" ::"r"(3 + buf), "n"(kAll) : "memory");
 
         // ---- S = Q Khat^T for the warp's 16 rows and the tile's 64 tokens
         float sc[8][4];
@@ -314,7 +327,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 mma_f16(o[2 * ntp], pa[ks], b[0], b[1]);
                 mma_f16(o[2 * ntp + 1], pa[ks], b[2], b[3]);
             }
-        __syncthreads();                                                 // the next tile is complete; this one may be rewritten
+        if (jt + 2 < n_tiles) asm volatile("bar.arrive %0, %1;" ::"r"(1 + buf), "n"(kAll) : "memory");   // the buffer is free again
     }
 
     // ---- normalise and write (l is spread over the quad)
