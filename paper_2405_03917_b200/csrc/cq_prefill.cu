@@ -248,6 +248,13 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
         return;
     }
     asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+    // the warp's query rows as A fragments, kept in registers for the whole context
+    uint32_t qf[8][4];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        const int mi = lane >> 3;
+        ldmatrix_x4(qf[ks], q_s + tile_off(warp * 16 + (lane & 7) + 8 * (mi & 1), 2 * ks + (mi >> 1)));
+    }
 
     for (int64_t jt = 0; jt < n_tiles; ++jt) {
         const int64_t j0 = jt * C::kTile;
@@ -262,11 +269,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             for (int j = 0; j < 4; ++j) sc[nt][j] = 0.f;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            uint32_t a[4];
-            {
-                const int mi = lane >> 3;
-                ldmatrix_x4(a, q_s + tile_off(warp * 16 + (lane & 7) + 8 * (mi & 1), 2 * ks + (mi >> 1)));
-            }
+            const uint32_t (&a)[4] = qf[ks];
 #pragma unroll
             for (int ntp = 0; ntp < 4; ++ntp) {
                 uint32_t b[4];
