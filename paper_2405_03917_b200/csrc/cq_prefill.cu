@@ -144,6 +144,14 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// 2^x by the special-function unit (two units in the last place; P is rounded to fp16 afterwards)
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int kC>
 __global__ void __launch_bounds__(PfCfg::kThreads, 1)
 prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc, const uint8_t* __restrict__ vc,
@@ -196,6 +204,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     // positions of this thread's two rows
     const int rho_a = warp * 16 + r, rho_b = rho_a + 8;
     const int64_t pos_a = pos0 + rho_a / R, pos_b = pos0 + rho_b / R;
+    const int64_t pos_warp = pos0 + (warp * 16) / R;                      // smallest position among the warp's rows
 
     const int64_t n_tiles = pos_last < 0 ? 0 : pos_last / C::kTile + 1;
     const uint8_t* kbase = kc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
@@ -279,47 +288,78 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 mma_f16(sc[2 * ntp + 1], a, b[2], b[3]);
             }
         }
-        // ---- mask, running maximum, P
-        float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int64_t tok = j0 + 8 * nt + 2 * p + (j & 1);
-                const int64_t pos = (j < 2) ? pos_a : pos_b;
-                const float v = tok <= pos ? sc[nt][j] * scale_log2e : -INFINITY;
-                sc[nt][j] = v;
-                mx[j >> 1] = fmaxf(mx[j >> 1], v);
-            }
+        // ---- running maximum and P.  A tile that lies wholly below every row's causal limit needs no mask: the
+        // maximum is taken over the raw scores and the scale folded into the exponent's multiply-add.
         float corr[2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
-            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-            const float m_new = fmaxf(m_run[h], mx[h]);
-            corr[h] = m_new == -INFINITY ? 1.f : exp2f(m_run[h] - m_new);
-            m_run[h] = m_new;
-            l_run[h] *= corr[h];
-        }
         uint32_t pa[4][4];                                               // P as A fragments: one per 16 tokens
+        if (j0 + C::kTile - 1 <= pos_warp && scale_log2e > 0.f) {
+            float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            float pv[4];
+            for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float mrow = m_run[j >> 1];
-                pv[j] = mrow == -INFINITY ? 0.f : exp2f(sc[nt][j] - mrow);
-                l_run[j >> 1] += pv[j];
+                for (int j = 0; j < 4; ++j) mx[j >> 1] = fmaxf(mx[j >> 1], sc[nt][j]);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+                const float m_new = fmaxf(m_run[h], mx[h] * scale_log2e);      // finite: the tile has no masked score
+                corr[h] = exp2f(m_run[h] - m_new);
+                m_run[h] = m_new;
+                l_run[h] *= corr[h];
             }
-            pa[nt >> 1][(nt & 1) * 2 + 0] = pack_half2(pv[0], pv[1]);
-            pa[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(pv[2], pv[3]);
-        }
 #pragma unroll
-        for (int nt = 0; nt < 16; ++nt) {
-            o[nt][0] *= corr[0];
-            o[nt][1] *= corr[0];
-            o[nt][2] *= corr[1];
-            o[nt][3] *= corr[1];
+            for (int nt = 0; nt < 8; ++nt) {
+                float pv[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    pv[j] = ex2_approx(fmaf(sc[nt][j], scale_log2e, -m_run[j >> 1]));
+                    l_run[j >> 1] += pv[j];
+                }
+                pa[nt >> 1][(nt & 1) * 2 + 0] = pack_half2(pv[0], pv[1]);
+                pa[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(pv[2], pv[3]);
+            }
+        } else {
+            float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t tok = j0 + 8 * nt + 2 * p + (j & 1);
+                    const int64_t pos = (j < 2) ? pos_a : pos_b;
+                    const float v = tok <= pos ? sc[nt][j] * scale_log2e : -INFINITY;
+                    sc[nt][j] = v;
+                    mx[j >> 1] = fmaxf(mx[j >> 1], v);
+                }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+                mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+                const float m_new = fmaxf(m_run[h], mx[h]);
+                corr[h] = m_new == -INFINITY ? 1.f : exp2f(m_run[h] - m_new);
+                m_run[h] = m_new;
+                l_run[h] *= corr[h];
+            }
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                float pv[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float mrow = m_run[j >> 1];
+                    pv[j] = mrow == -INFINITY ? 0.f : exp2f(sc[nt][j] - mrow);
+                    l_run[j >> 1] += pv[j];
+                }
+                pa[nt >> 1][(nt & 1) * 2 + 0] = pack_half2(pv[0], pv[1]);
+                pa[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(pv[2], pv[3]);
+            }
+        }
+        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {   // most tiles leave every maximum as it was
+#pragma unroll
+            for (int nt = 0; nt < 16; ++nt) {
+                o[nt][0] *= corr[0];
+                o[nt][1] *= corr[0];
+                o[nt][2] *= corr[1];
+                o[nt][3] *= corr[1];
+            }
         }
         // ---- O += P Vhat
 #pragma unroll
