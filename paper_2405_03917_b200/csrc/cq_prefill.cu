@@ -15,6 +15,8 @@
 //     softmax is the usual running-maximum form in the log2 domain.  Four producer warps do the
 //     gathering into two tile buffers while eight warps (16 rows each) multiply; named barriers
 //     hand a buffer back and forth, and the producers give most of their registers to the others.
+//     The multiplying warps hold their query fragments in registers; a tile wholly below the
+//     causal limit of a warp's rows skips the mask and folds the scale into the exponent.
 //   prefill_generic_kernel: any supported shape, one CTA per (sequence, query, head), plain loops.
 #include "cq_common.cuh"
 
