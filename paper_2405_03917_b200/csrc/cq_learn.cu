@@ -17,46 +17,83 @@ namespace {
 // problem p = h * G + g; vector i.  dist[p][i]: squared distance of vector i to its nearest centre
 // so far; contrib[p][i] = w_i * dist[p][i], the term of the k-means++ draw.
 
-// One CTA per problem.  The CTA stages tiles of contributions in shared memory (coalesced loads);
-// thread 0 adds them up in index order, so the fp64 running sum is the sequential one.
+// One CTA per problem.  The CTA stages tiles of contributions in shared memory (coalesced loads, the next
+// tile while the current one is summed); thread 0 adds them up in index order, so the fp64 running sum is
+// the sequential one.  The running sum at the end of every tile is kept: it never decreases (the
+// contributions are not negative), so the walk that looks for the drawn vector starts at the first tile
+// whose end reaches the target, from the sum before that tile - the same additions in the same order as a
+// walk from the first vector, without repeating them.
 constexpr int kPickThreads = 128;
 constexpr int kPickTile = 2048;
+constexpr int kPickPrefixes = 1024;              // tile ends that are kept (later tiles are walked one by one)
+
+// sum += v[0] + ... in order, sixteen loads in flight ahead of the chain of additions
+__device__ __forceinline__ double pick_sum_tile(const double* tile, int m, double sum)
+{
+    int e = 0;
+    for (; e + 16 <= m; e += 16) {
+        double v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = tile[e + j];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) sum = __dadd_rn(sum, v[j]);
+    }
+    for (; e < m; ++e) sum = __dadd_rn(sum, tile[e]);
+    return sum;
+}
+
 __global__ void __launch_bounds__(kPickThreads)
 pp_pick_kernel(const __half* __restrict__ x, const double* __restrict__ uniforms, const double* __restrict__ contrib,
                int64_t n_vec, int n_prob, int c, int K, int k, float* __restrict__ codebooks)
 {
-    __shared__ double tile[kPickTile];
+    __shared__ double tile[2][kPickTile];
+    __shared__ double s_prefix[kPickPrefixes];
     __shared__ double s_total;
     __shared__ long long s_pick;
     const int p = blockIdx.x;
     const double u = uniforms[(int64_t)p * K + k];
     const double* cp = contrib + (int64_t)p * n_vec;
+    const int64_t n_tiles = (n_vec + kPickTile - 1) / kPickTile;
+    auto stage = [&](int64_t t, int buf) {
+        const int64_t t0 = t * kPickTile;
+        const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
+        for (int e = threadIdx.x; e < m; e += kPickThreads) tile[buf][e] = cp[t0 + e];
+    };
     if (threadIdx.x == 0) s_pick = -1;
     if (k > 0) {
         double total = 0.0;
-        for (int64_t t0 = 0; t0 < n_vec; t0 += kPickTile) {
-            const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
-            __syncthreads();
-            for (int e = threadIdx.x; e < m; e += kPickThreads) tile[e] = cp[t0 + e];
-            __syncthreads();
-            if (threadIdx.x == 0)
-                for (int e = 0; e < m; ++e) total = __dadd_rn(total, tile[e]);
+        stage(0, 0);
+        for (int64_t t = 0; t < n_tiles; ++t) {
+            __syncthreads();                                  // tile t is staged, the other buffer is free
+            if (t + 1 < n_tiles) stage(t + 1, (int)((t + 1) & 1));
+            if (threadIdx.x == 0) {
+                const int64_t t0 = t * kPickTile;
+                const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
+                total = pick_sum_tile(tile[t & 1], m, total);
+                if (t < kPickPrefixes) s_prefix[t] = total;
+            }
         }
         if (threadIdx.x == 0) s_total = total;
         __syncthreads();
         if (s_total > 0.0) {
             const double target = __dmul_rn(u, s_total);
-            double run = 0.0;
-            for (int64_t t0 = 0; t0 < n_vec; t0 += kPickTile) {
+            // first tile whose end reaches the target (every thread takes the same decision)
+            int64_t first = 0;
+            const int64_t kept = n_tiles < kPickPrefixes ? n_tiles : kPickPrefixes;
+            while (first < kept && !(s_prefix[first] >= target)) ++first;
+            if (first == n_tiles) first = n_tiles - 1;      // rounding put the target past the total: the last tile decides
+            double run = first > 0 ? s_prefix[first - 1] : 0.0;
+            for (int64_t t = first; t < n_tiles; ++t) {
+                const int64_t t0 = t * kPickTile;
                 const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
                 __syncthreads();
                 if (s_pick >= 0) break;                     // same value in every thread: read after the barrier
-                for (int e = threadIdx.x; e < m; e += kPickThreads) tile[e] = cp[t0 + e];
+                for (int e = threadIdx.x; e < m; e += kPickThreads) tile[0][e] = cp[t0 + e];
                 __syncthreads();
                 if (threadIdx.x == 0)
                     for (int e = 0; e < m; ++e) {
-                        run = __dadd_rn(run, tile[e]);
-                        if (run >= target && tile[e] > 0.0) { s_pick = t0 + e; break; }
+                        run = __dadd_rn(run, tile[0][e]);
+                        if (run >= target && tile[0][e] > 0.0) { s_pick = t0 + e; break; }
                     }
             }
             __syncthreads();
