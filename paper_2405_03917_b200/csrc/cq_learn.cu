@@ -57,7 +57,8 @@ pp_pick_kernel(const __half* __restrict__ x, const double* __restrict__ uniforms
     auto stage = [&](int64_t t, int buf) {
         const int64_t t0 = t * kPickTile;
         const int m = (int)(n_vec - t0 < kPickTile ? n_vec - t0 : kPickTile);
-        for (int e = threadIdx.x; e < m; e += kPickThreads) tile[buf][e] = cp[t0 + e];
+        // warp 0 does not stage: its first thread is busy with the chain of additions
+        for (int e = (int)threadIdx.x - 32; e >= 0 && e < m; e += kPickThreads - 32) tile[buf][e] = cp[t0 + e];
     };
     if (threadIdx.x == 0) s_pick = -1;
     if (k > 0) {
@@ -112,25 +113,54 @@ pp_pick_kernel(const __half* __restrict__ x, const double* __restrict__ uniforms
     }
 }
 
-__global__ void pp_dist_kernel(const __half* __restrict__ x, const float* __restrict__ weights,
-                               const float* __restrict__ codebooks, int64_t n_vec, int n_prob, int c, int K, int k,
-                               double* __restrict__ dist, double* __restrict__ contrib)
+// Distances to the nearest chosen centre and the contributions w * D, for tiles of 32 vectors x 32 problems.
+// x and the weights are vector-major, the distances and contributions problem-major (a draw reads one
+// problem's run): the tile is turned in shared memory so that every global access runs along the
+// contiguous index.  Thread (tx, ty): tx is the vector when the problem-major arrays are touched and the
+// problem when x is read.
+constexpr int kDistTile = 32;
+__global__ void __launch_bounds__(256)
+pp_dist_kernel(const __half* __restrict__ x, const float* __restrict__ weights, const float* __restrict__ codebooks,
+               int64_t n_vec, int n_prob, int c, int K, int k, double* __restrict__ dist, double* __restrict__ contrib)
 {
-    const int64_t total = n_vec * n_prob;
-    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-        const int p = (int)(idx / n_vec);
-        const int64_t i = idx % n_vec;
-        const __half* xv = x + (i * n_prob + p) * c;
-        const float* cb = codebooks + ((int64_t)p * K + k) * c;
-        double d = 0.0;
-        for (int q = 0; q < c; ++q) {
-            const double diff = __dsub_rn((double)__half2float(xv[q]), (double)cb[q]);
-            d = __dadd_rn(d, __dmul_rn(diff, diff));
+    __shared__ double d_s[kDistTile][kDistTile + 1];          // [problem][vector]
+    __shared__ double c_s[kDistTile][kDistTile + 1];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int64_t tiles_i = (n_vec + kDistTile - 1) / kDistTile;
+    const int64_t tiles_p = (n_prob + kDistTile - 1) / kDistTile;
+    for (int64_t tile = blockIdx.x; tile < tiles_i * tiles_p; tile += gridDim.x) {
+        const int64_t i0 = (tile % tiles_i) * kDistTile;
+        const int p0 = (int)(tile / tiles_i) * kDistTile;
+        if (k > 0) {
+            for (int pp = ty; pp < kDistTile; pp += 8)
+                if (p0 + pp < n_prob && i0 + tx < n_vec) d_s[pp][tx] = dist[(int64_t)(p0 + pp) * n_vec + i0 + tx];
         }
-        if (k > 0 && !(d < dist[idx])) d = dist[idx];
-        dist[idx] = d;
-        const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
-        contrib[idx] = __dmul_rn(w, d);
+        __syncthreads();
+        for (int ii = ty; ii < kDistTile; ii += 8) {
+            const int64_t i = i0 + ii;
+            const int p = p0 + tx;
+            if (i < n_vec && p < n_prob) {
+                const __half* xv = x + (i * n_prob + p) * c;
+                const float* cb = codebooks + ((int64_t)p * K + k) * c;
+                double d = 0.0;
+                for (int q = 0; q < c; ++q) {
+                    const double diff = __dsub_rn((double)__half2float(xv[q]), (double)cb[q]);
+                    d = __dadd_rn(d, __dmul_rn(diff, diff));
+                }
+                if (k > 0 && !(d < d_s[tx][ii])) d = d_s[tx][ii];
+                const double w = weights ? (double)weights[i * n_prob + p] : 1.0;
+                d_s[tx][ii] = d;
+                c_s[tx][ii] = __dmul_rn(w, d);
+            }
+        }
+        __syncthreads();
+        for (int pp = ty; pp < kDistTile; pp += 8)
+            if (p0 + pp < n_prob && i0 + tx < n_vec) {
+                const int64_t idx = (int64_t)(p0 + pp) * n_vec + i0 + tx;
+                dist[idx] = d_s[pp][tx];
+                contrib[idx] = c_s[pp][tx];
+            }
+        __syncthreads();
     }
 }
 
@@ -210,9 +240,9 @@ cudaError_t launch_kmeanspp_init(const __half* x, const float* weights, const do
     const LearnLayout l = learn_layout(sh, n_vec);
     double* dist = reinterpret_cast<double*>(static_cast<char*>(workspace) + l.codes);
     const int n_prob = sh.n_kv_heads * sh.G;
-    const int64_t pairs = n_vec * n_prob;
-    const int64_t dist_cap = (int64_t)device_sm_count() * 16;
-    const int dist_grid = (int)((pairs + 255) / 256 < dist_cap ? (pairs + 255) / 256 : dist_cap);
+    const int64_t dist_tiles = ((n_vec + kDistTile - 1) / kDistTile) * ((n_prob + kDistTile - 1) / kDistTile);
+    const int64_t dist_cap = (int64_t)device_sm_count() * 64;
+    const int dist_grid = (int)(dist_tiles < dist_cap ? dist_tiles : dist_cap);
     double* contrib = reinterpret_cast<double*>(static_cast<char*>(workspace) + l.codes + l.dist);
     for (int k = 0; k < sh.K; ++k) {
         pp_pick_kernel<<<n_prob, kPickThreads, 0, st>>>(x, uniforms, contrib, n_vec, n_prob, sh.c, sh.K, k, codebooks);
