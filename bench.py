@@ -406,6 +406,7 @@ def extra_encode_cfg3(cq, dev, reps=5):
                        "unit": "lane-ops/s", "frac": 0.5 * pairs / (ms * 1e-3) / alu_peak, "traffic": None,
                        "lane_ops_per_score": 0.5,
                        "peak_source": f"64 ALU lanes/clk/SM x {n_sm} SMs x {mhz:.0f} MHz (device maximum)"}
+    attach_traffic(res["roofline"], w.name)
     return res
 
 
@@ -505,9 +506,11 @@ def extra_prefill(cq, dev, reps=5):
     except Exception:
         peak = 1590.0
     tf = flops / (ms * 1e-3) / 1e12
-    return {"workload": w.name, "ms": ms, "query_tokens_per_s": n_seq * n_q / (ms * 1e-3),
-            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
-                         "peak_source": "measured bf16 GEMM burst (fp16 has the same nominal rate); mma.sync path"}}
+    res = {"workload": w.name, "ms": ms, "query_tokens_per_s": n_seq * n_q / (ms * 1e-3),
+           "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
+                        "peak_source": "measured bf16 GEMM burst (fp16 has the same nominal rate); mma.sync path"}}
+    attach_traffic(res["roofline"], w.name)
+    return res
 
 
 def extra_decode_rope(cq, dev, w, reps=5):
