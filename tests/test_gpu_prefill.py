@@ -66,6 +66,17 @@ def test_queries_without_a_position_give_zero_rows(variant):
     H.check_attn(got, ref, "short caches")
 
 
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("scale", [-0.07, 0.0])
+def test_scales_that_are_not_positive(variant, scale):
+    # a negative scale turns the order of the scores around (the kernel's shortcut for tiles below the causal limit
+    # takes the maximum of the raw scores and must not be used), a zero scale gives the plain mean of the values
+    lens = [400, 130]
+    q, kc_rm, vc_rm, kcb, vcb = random_case(11, 8, 8, 12, 4, 1, lens, 400)
+    got, ref = run_both(q, kc_rm, vc_rm, kcb, vcb, lens, scale, 8, 8, variant)
+    H.check_attn(got, ref, f"scale {scale}")
+
+
 def test_generic_kernel_covers_other_shapes():
     # head_dim 64 with 5-bit codes, and codes wider than a byte: no tensor-core kernel, the plain one serves
     for (D, c, b, Hq, Hkv) in [(64, 4, 5, 4, 2), (128, 8, 10, 2, 1), (32, 1, 3, 3, 3)]:
