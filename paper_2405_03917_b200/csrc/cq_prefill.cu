@@ -106,6 +106,12 @@ struct PfCfg {
     static constexpr int kWarps = 8;                                    // warps that multiply (16 rows each)
     static constexpr int kProducerWarps = 4;                            // warps that dequantise the tiles
     static constexpr int kThreads = (kWarps + kProducerWarps) * 32;
+    // Registers: the CTA is launched with 168 per thread (the most 384 threads can have); the producers go down to
+    // 40, the multiplying warps up to 232.  The registers the producers give back must cover what the others ask
+    // for, or the increase waits for ever (48 for the producers does: 4 x 120 < 8 x 64).
+    static constexpr int kLaunchRegs = 168, kProducerRegs = 40, kMultiplierRegs = 232;
+    static_assert((kLaunchRegs - kProducerRegs) * kProducerWarps >= (kMultiplierRegs - kLaunchRegs) * kWarps,
+                  "setmaxnreg: the producers must release what the multiplying warps take");
     static constexpr int kRows = 128;             // (query, head) rows per CTA: 16 per warp
     static constexpr int kTile = 64;              // cached tokens per step
     static constexpr int kRowBytes = 256;         // 128 fp16 channels
