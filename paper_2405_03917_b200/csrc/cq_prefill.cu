@@ -222,7 +222,7 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     // codes -> fp16 tiles of the 64 tokens from j0 on, into buffer `buf`: a work item is (8 tokens, one group)
     // (with fewer items than threads the warps that take them alternate from tile to tile, so that every warp
     // dequantises every other tile and goes straight on to the MMAs on the tiles between)
-    auto dequantise = [&](int64_t j0, int buf) {
+    auto dequantise_groups = [&](int64_t j0, int buf) {
         for (int item = threadIdx.x - C::kWarps * 32; item < 8 * G; item += C::kProducerWarps * 32) {
             const int g = item % G, oct = item / G;                      // tokens 8 oct .. 8 oct + 7 of the tile
             const int64_t blk = j0 / kTokenBlock + (oct >> 1);
@@ -249,6 +249,59 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 }
             }
         }
+    };
+    // The same with work items of (8 tokens, one 16-byte chunk of the row = 8 channels = 8 / c groups): 128 items,
+    // one per producer thread, which gathers the chunk's centroids per token and stores the 16 bytes at once.
+    // Measured on the prefill shape of the benchmark: c = 2 5.24 -> 3.91 ms, but c = 4 3.55 -> 3.66 and c = 8
+    // 3.32 -> 3.56 ms, so only c = 2 takes this form.
+    auto dequantise_chunks = [&](int64_t j0, int buf) {
+        constexpr int kGpi = 8 / kC;                                     // groups per item
+        const int item = threadIdx.x - C::kWarps * 32;
+        const int chunk = item & 15, oct = item >> 4;                    // tokens 8 oct .. 8 oct + 7 of the tile
+        const int64_t blk = j0 / kTokenBlock + (oct >> 1);
+        uint2 kw[kGpi], vw[kGpi];
+#pragma unroll
+        for (int i = 0; i < kGpi; ++i) {
+            kw[i] = make_uint2(0u, 0u);
+            vw[i] = make_uint2(0u, 0u);
+            if (blk < sh.n_blocks) {
+                const int64_t off = blk * (G * kTokenBlock) + (chunk * kGpi + i) * kTokenBlock + 8 * (oct & 1);
+                kw[i] = *reinterpret_cast<const uint2*>(kbase + off);
+                vw[i] = *reinterpret_cast<const uint2*>(vbase + off);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t kv[4], vv[4];
+#pragma unroll
+            for (int i = 0; i < kGpi; ++i) {
+                const uint32_t kcode = ((k < 4 ? kw[i].x : kw[i].y) >> (8 * (k & 3))) & 0xffu;
+                const uint32_t vcode = ((k < 4 ? vw[i].x : vw[i].y) >> (8 * (k & 3))) & 0xffu;
+                const uint32_t krow = ((chunk * kGpi + i) * 256 + kcode) * (2 * kC);
+                const uint32_t vrow = ((chunk * kGpi + i) * 256 + vcode) * (2 * kC);
+                if (kC == 8) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(smem + C::kKcbOffset + krow);
+                    const uint4 b2 = *reinterpret_cast<const uint4*>(smem + C::kVcbOffset + vrow);
+                    kv[0] = a.x; kv[1] = a.y; kv[2] = a.z; kv[3] = a.w;
+                    vv[0] = b2.x; vv[1] = b2.y; vv[2] = b2.z; vv[3] = b2.w;
+                } else if (kC == 4) {
+                    const uint2 a = *reinterpret_cast<const uint2*>(smem + C::kKcbOffset + krow);
+                    const uint2 b2 = *reinterpret_cast<const uint2*>(smem + C::kVcbOffset + vrow);
+                    kv[(2 * i) & 3] = a.x; kv[(2 * i + 1) & 3] = a.y;
+                    vv[(2 * i) & 3] = b2.x; vv[(2 * i + 1) & 3] = b2.y;
+                } else {
+                    kv[i & 3] = *reinterpret_cast<const uint32_t*>(smem + C::kKcbOffset + krow);
+                    vv[i & 3] = *reinterpret_cast<const uint32_t*>(smem + C::kVcbOffset + vrow);
+                }
+            }
+            const uint32_t dst = tile_off(8 * oct + k, chunk);
+            *reinterpret_cast<uint4*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = make_uint4(kv[0], kv[1], kv[2], kv[3]);
+            *reinterpret_cast<uint4*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = make_uint4(vv[0], vv[1], vv[2], vv[3]);
+        }
+    };
+    auto dequantise = [&](int64_t j0, int buf) {
+        if (kC == 2) dequantise_chunks(j0, buf);
+        else dequantise_groups(j0, buf);
     };
     // Producer warps fill the two tile buffers, the other warps multiply; named barriers 1 + buf ("buffer free") and
     // 3 + buf ("buffer full") hand a buffer back and forth, registers move from the producers to the multipliers.
