@@ -191,8 +191,16 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     for (int i = threadIdx.x; i < 128 * 256 / 2; i += C::kThreads) {
         const float2 a = *reinterpret_cast<const float2*>(kcb + (int64_t)hkv * 128 * 256 + 2 * i);
         const float2 b = *reinterpret_cast<const float2*>(vcb + (int64_t)hkv * 128 * 256 + 2 * i);
-        *reinterpret_cast<uint32_t*>(smem + C::kKcbOffset + 4 * i) = pack_half2(a.x, a.y);
-        *reinterpret_cast<uint32_t*>(smem + C::kVcbOffset + 4 * i) = pack_half2(b.x, b.y);
+        // code-major ([code][group][channel]): the lanes of a gather take different groups, so they meet in no bank
+        // whatever the codes are.  For c = 2 (one word per centroid, a lane gathers the groups 4 chunk + i) group g
+        // sits in column 16 (g mod 4) + g / 4, so that the 16 chunks of one gather fall into 16 different banks.
+        int w;
+        {
+            const int g = (2 * i) / (256 * kC), code = ((2 * i) / kC) % 256, ch = (2 * i) % kC;
+            w = kC == 2 ? code * G + 16 * (g & 3) + (g >> 2) : ((code * G + g) * kC + ch) / 2;
+        }
+        *reinterpret_cast<uint32_t*>(smem + C::kKcbOffset + 4 * w) = pack_half2(a.x, a.y);
+        *reinterpret_cast<uint32_t*>(smem + C::kVcbOffset + 4 * w) = pack_half2(b.x, b.y);
     }
     for (int i = threadIdx.x; i < C::kRows * 16; i += C::kThreads) {
         const int rho = i >> 4, chunk = i & 15;
@@ -238,11 +246,11 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
                 const int tok = 8 * oct + k;
                 const uint32_t dst = tile_off(tok, (g * kC) >> 3) + (uint32_t)((g * kC) & 7) * 2u;
                 if (kC == 8) {
-                    *reinterpret_cast<uint4*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint4*>(smem + C::kKcbOffset + (g * 256 + kcode) * 16);
-                    *reinterpret_cast<uint4*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint4*>(smem + C::kVcbOffset + (g * 256 + vcode) * 16);
+                    *reinterpret_cast<uint4*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint4*>(smem + C::kKcbOffset + (kcode * G + g) * 16);
+                    *reinterpret_cast<uint4*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint4*>(smem + C::kVcbOffset + (vcode * G + g) * 16);
                 } else if (kC == 4) {
-                    *reinterpret_cast<uint2*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint2*>(smem + C::kKcbOffset + (g * 256 + kcode) * 8);
-                    *reinterpret_cast<uint2*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint2*>(smem + C::kVcbOffset + (g * 256 + vcode) * 8);
+                    *reinterpret_cast<uint2*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint2*>(smem + C::kKcbOffset + (kcode * G + g) * 8);
+                    *reinterpret_cast<uint2*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint2*>(smem + C::kVcbOffset + (vcode * G + g) * 8);
                 } else {
                     *reinterpret_cast<uint32_t*>(smem + C::kKtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint32_t*>(smem + C::kKcbOffset + (g * 256 + kcode) * 4);
                     *reinterpret_cast<uint32_t*>(smem + C::kVtOffset + buf * C::kTileBytes + dst) = *reinterpret_cast<const uint32_t*>(smem + C::kVcbOffset + (g * 256 + vcode) * 4);
@@ -277,8 +285,9 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
             for (int i = 0; i < kGpi; ++i) {
                 const uint32_t kcode = ((k < 4 ? kw[i].x : kw[i].y) >> (8 * (k & 3))) & 0xffu;
                 const uint32_t vcode = ((k < 4 ? vw[i].x : vw[i].y) >> (8 * (k & 3))) & 0xffu;
-                const uint32_t krow = ((chunk * kGpi + i) * 256 + kcode) * (2 * kC);
-                const uint32_t vrow = ((chunk * kGpi + i) * 256 + vcode) * (2 * kC);
+                // (the c = 2 placement of the codebooks; the other sizes do not take this form)
+                const uint32_t krow = (kcode * G + 16 * i + chunk) * 4;
+                const uint32_t vrow = (vcode * G + 16 * i + chunk) * 4;
                 if (kC == 8) {
                     const uint4 a = *reinterpret_cast<const uint4*>(smem + C::kKcbOffset + krow);
                     const uint4 b2 = *reinterpret_cast<const uint4*>(smem + C::kVcbOffset + vrow);
