@@ -10,7 +10,8 @@
 // contractions run on the tensor cores:
 //   prefill_mma_kernel (head_dim 128, one byte per code, c = 2, 4 or 8): one CTA per (sequence,
 //     KV head, tile of 128 (query, head of the KV head's group) rows).  Both codebooks are kept
-//     in shared memory as fp16; per tile of 64 cached tokens the K and V codes are gathered into
+//     in shared memory as fp16, code-major, so that the lanes of a gather (one group each) meet
+//     in no bank whatever the codes are; per tile of 64 cached tokens the K and V codes are gathered into
 //     fp16 tiles, S = Q Khat^T and O += P Vhat are m16n8k16 MMAs with fp32 accumulators, and the
 //     softmax is the usual running-maximum form in the log2 domain.  Four producer warps do the
 //     gathering into two tile buffers while eight warps (16 rows each) multiply; named barriers
