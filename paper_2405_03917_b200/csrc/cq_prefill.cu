@@ -228,9 +228,8 @@ prefill_mma_kernel(const __half* __restrict__ q, const uint8_t* __restrict__ kc,
     const uint8_t* vbase = vc + code_word_offset(sh, sh.n_kv_heads, s, hkv, 0, 0);
     const uint32_t q_s = smem_u32(smem + C::kQOffset), kt_s = smem_u32(smem + C::kKtOffset), vt_s = smem_u32(smem + C::kVtOffset);
 
-    // codes -> fp16 tiles of the 64 tokens from j0 on, into buffer `buf`: a work item is (8 tokens, one group)
-    // (with fewer items than threads the warps that take them alternate from tile to tile, so that every warp
-    // dequantises every other tile and goes straight on to the MMAs on the tiles between)
+    // codes -> fp16 tiles of the 64 tokens from j0 on, into buffer `buf`, by the 128 producer threads: a work item
+    // is (8 tokens, one group), 8 G items per tile (one per thread for c = 8, two for c = 4)
     auto dequantise_groups = [&](int64_t j0, int buf) {
         for (int item = threadIdx.x - C::kWarps * 32; item < 8 * G; item += C::kProducerWarps * 32) {
             const int g = item % G, oct = item / G;                      // tokens 8 oct .. 8 oct + 7 of the tile
