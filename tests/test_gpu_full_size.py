@@ -168,3 +168,47 @@ def test_config6_llama2_7b_2c8b_decode_full_size():
     ties, total, a, r = check_items(w, 0, st, seeded_items(w, 8, 606))
     assert ties <= total // 500
     print(f"config 6: {total} codes checked, {ties} near-ties, attention max-abs {a:.2e} rel-L2 {r:.2e}")
+
+
+def test_prefill_chunk_full_size():
+    # cq_prefill_attn at the size the benchmark times it (4 sequences x 8192 cached tokens, the newest 2048 as
+    # queries, 32 query heads on 8 KV heads, CQ-8c8b).  Row i of a sequence is Eq. 1 for one query over the first
+    # len - n_q + i + 1 tokens: sampled rows of sampled (sequence, KV head) items are checked against the oracle's
+    # single-query attention over that prefix, with the oracle's own codes in the items' cache slices.
+    w0 = synth.WORKLOADS[2]
+    n_seq, cap, n_q = 4, 8192, 2048
+    w = synth.Workload("prefill_mistral_7b_gqa_8c8b_chunk2048_of_8192", 8, w0.c, w0.b, 1, n_seq, w0.n_q_heads, w0.n_kv_heads, cap)
+    st = bench.DecodeState(w, 0, torch.device(DEV), cq)
+    D, c, b, R = w.head_dim, w.c, w.b, w.n_q_heads // w.n_kv_heads
+    items = seeded_items(w, 3, 808)
+    oracle_codes = {}
+    for (s, h) in items:
+        for is_v, buf, cb in ((False, st.k_codes, st.k_cb), (True, st.v_codes, st.v_cb)):
+            x = item_activations(w, 0, is_v, h, s, cap)
+            res = oracle.encode(x.numpy().reshape(cap, 1, D), cb[h:h + 1].cpu().numpy(), c, b)
+            oracle_codes[(s, h, is_v)] = res[0].reshape(1, cap, 1, w.G)
+            patched = cq.cq_codes_from_rowmajor(torch.from_numpy(res[0].astype(np.uint8).reshape(1, cap, 1, w.G)).to(DEV), D, c, b)
+            buf[item_slice(w, cap, s, h)] = patched
+    g = torch.Generator(device="cpu").manual_seed(88)
+    q = torch.randn(n_seq, n_q, w.n_q_heads, D, generator=g).to(torch.float16)
+    out = cq.cq_prefill_attn(q.to(DEV), st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.seq_lens, st.scale, c, b, cap)
+    torch.cuda.synchronize()
+    out = out.cpu().numpy()
+    rng = np.random.default_rng(809)
+    worst_abs = worst_rel = 0.0
+    for (s, h) in items:
+        n = int(st.lens_cpu[s])
+        # first and last query, the rows around a 64-token tile edge and a 32-query row-tile edge, and random ones
+        rows = sorted({0, 1, 31, 32, 63, 64, n_q - 1} | {int(v) for v in rng.integers(0, n_q, size=9)})
+        for i in rows:
+            prefix = n - n_q + i + 1
+            if prefix < 1:
+                assert (out[s, i, h * R:(h + 1) * R] == 0).all()
+                continue
+            qr = q[s, i, h * R:(h + 1) * R].numpy().reshape(1, R, D)
+            ref = oracle.decode_dense(qr, oracle_codes[(s, h, False)], oracle_codes[(s, h, True)],
+                                      st.k_cb[h:h + 1].cpu().numpy(), st.v_cb[h:h + 1].cpu().numpy(),
+                                      np.array([prefix], np.int32), st.scale, c, b)
+            a, r = H.check_attn(out[s, i, h * R:(h + 1) * R], ref[0], f"prefill item (seq {s}, kv head {h}) row {i}")
+            worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
+    print(f"prefill: {len(items)} items, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
