@@ -212,3 +212,39 @@ def test_prefill_chunk_full_size():
             a, r = H.check_attn(out[s, i, h * R:(h + 1) * R], ref[0], f"prefill item (seq {s}, kv head {h}) row {i}")
             worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
     print(f"prefill: {len(items)} items, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
+
+
+def test_pre_rope_decode_full_size():
+    # cq_decode_attn_rope on config 1's shape (16 x 32 heads x 4096 tokens, CQ-4c8b, the tuned kernel), with the
+    # rotary tables of base 10000 that the benchmark uses: sampled (sequence, head) items against the oracle's
+    # dequantise-rotate-attend form, the oracle's own codes in the items' cache slices.
+    w = synth.WORKLOADS[1]
+    st = bench.DecodeState(w, 0, torch.device(DEV), cq)
+    cap, D, c, b = st.cap, w.head_dim, w.c, w.b
+    R = w.n_q_heads // w.n_kv_heads
+    items = seeded_items(w, 12, 909)
+    oracle_codes = {}
+    for (s, h) in items:
+        for is_v, buf, cb in ((False, st.k_codes, st.k_cb), (True, st.v_codes, st.v_cb)):
+            x = item_activations(w, 0, is_v, h, s, cap)
+            res = oracle.encode(x.numpy().reshape(cap, 1, D), cb[h:h + 1].cpu().numpy(), c, b)
+            oracle_codes[(s, h, is_v)] = res[0].reshape(1, cap, 1, w.G)
+            patched = cq.cq_codes_from_rowmajor(torch.from_numpy(res[0].astype(np.uint8).reshape(1, cap, 1, w.G)).to(DEV), D, c, b)
+            buf[item_slice(w, cap, s, h)] = patched
+    P = D // 2
+    ang = np.arange(cap, dtype=np.float64)[:, None] * (10000.0 ** (-np.arange(P, dtype=np.float64) / P))[None, :]
+    cs, sn = np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+    out = cq.cq_decode_attn_rope(st.q, st.k_codes, st.v_codes, st.k_cb, st.v_cb, st.seq_lens, torch.from_numpy(cs).to(DEV),
+                                 torch.from_numpy(sn).to(DEV), st.scale, c, b, cap, workspace=st.ws, variant=2)
+    torch.cuda.synchronize()
+    out = out.cpu().numpy()
+    worst_abs = worst_rel = 0.0
+    for (s, h) in items:
+        n = int(st.lens_cpu[s])
+        q = st.q[s, h * R:(h + 1) * R].cpu().numpy().reshape(1, R, D)
+        ref = oracle.decode_dense_rope(q, oracle_codes[(s, h, False)], oracle_codes[(s, h, True)],
+                                       st.k_cb[h:h + 1].cpu().numpy(), st.v_cb[h:h + 1].cpu().numpy(),
+                                       np.array([n], np.int32), cs, sn, st.scale, c, b)
+        a, r = H.check_attn(out[s, h * R:(h + 1) * R], ref[0], f"pre-RoPE item (seq {s}, head {h})")
+        worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
+    print(f"pre-RoPE decode: {len(items)} items, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
