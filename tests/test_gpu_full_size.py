@@ -248,3 +248,51 @@ def test_pre_rope_decode_full_size():
         a, r = H.check_attn(out[s, h * R:(h + 1) * R], ref[0], f"pre-RoPE item (seq {s}, head {h})")
         worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
     print(f"pre-RoPE decode: {len(items)} items, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
+
+
+def test_config2_decode_step_full_size():
+    # The call the benchmark times on config 2: cq_decode_step (the new token's K and V are encoded and written
+    # at the last position inside the attention launch, which then attends over all tokens and writes the output).
+    # Sampled (sequence, KV head) items hold the oracle's codes; afterwards the appended codes must be the oracle's
+    # codes of the new vectors (near-tie rule) and the outputs the oracle's attention over the updated cache.
+    w = synth.WORKLOADS[2]
+    st = bench.DecodeState(w, 0, torch.device(DEV), cq)
+    assert st.fused_launches == 1
+    cap, D, c, b = st.cap, w.head_dim, w.c, w.b
+    R = w.n_q_heads // w.n_kv_heads
+    items = seeded_items(w, 4, 212, must=[(w.n_seq - 1, 5)])
+    codes = {}
+    for (s, h) in items:
+        for is_v, buf, cb in ((False, st.k_codes, st.k_cb), (True, st.v_codes, st.v_cb)):
+            x = item_activations(w, 0, is_v, h, s, cap)
+            res = oracle.encode(x.numpy().reshape(cap, 1, D), cb[h:h + 1].cpu().numpy(), c, b)
+            codes[(s, h, is_v)] = res[0].reshape(1, cap, 1, w.G).copy()
+            buf[item_slice(w, cap, s, h)] = cq.cq_codes_from_rowmajor(
+                torch.from_numpy(res[0].astype(np.uint8).reshape(1, cap, 1, w.G)).to(DEV), D, c, b)
+    st.step(cq)
+    torch.cuda.synchronize()
+    out = st.out.cpu().numpy()
+    ties = total = 0
+    worst_abs = worst_rel = 0.0
+    for (s, h) in items:
+        n = int(st.lens_cpu[s])
+        for is_v, buf, cb, new in ((False, st.k_codes, st.k_cb, st.k_new), (True, st.v_codes, st.v_cb, st.v_new)):
+            xn = new[s, h].cpu().numpy().reshape(1, 1, D)
+            cbh = cb[h:h + 1].cpu().numpy()
+            res = oracle.encode(xn, cbh, c, b)
+            got = cq.cq_codes_to_rowmajor(buf[item_slice(w, cap, s, h)].clone(), 1, cap, 1, D, c, b).cpu().numpy()
+            got = got.reshape(cap, w.G)
+            t, tot = H.check_codes(xn, cbh, got[n - 1].reshape(1, 1, w.G), c, b, res)
+            ties += t
+            total += tot
+            # every other position of the item is untouched
+            keep = codes[(s, h, is_v)].reshape(cap, w.G)
+            assert (got[:n - 1] == keep[:n - 1]).all() and (got[n:] == keep[n:]).all()
+            codes[(s, h, is_v)][0, n - 1, 0] = res[0].reshape(w.G)
+        q = st.q[s, h * R:(h + 1) * R].cpu().numpy().reshape(1, R, D)
+        ref = oracle.decode_dense(q, codes[(s, h, False)], codes[(s, h, True)], st.k_cb[h:h + 1].cpu().numpy(),
+                                  st.v_cb[h:h + 1].cpu().numpy(), np.array([n], np.int32), st.scale, c, b)
+        a, r = H.check_attn(out[s, h * R:(h + 1) * R], ref[0], f"step item (seq {s}, kv head {h})")
+        worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
+    assert ties <= 1
+    print(f"config 2 step: {total} appended codes checked, {ties} near-ties, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
