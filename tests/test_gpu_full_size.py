@@ -250,17 +250,20 @@ def test_pre_rope_decode_full_size():
     print(f"pre-RoPE decode: {len(items)} items, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
 
 
-def test_config2_decode_step_full_size():
-    # The call the benchmark times on config 2: cq_decode_step (the new token's K and V are encoded and written
-    # at the last position inside the attention launch, which then attends over all tokens and writes the output).
-    # Sampled (sequence, KV head) items hold the oracle's codes; afterwards the appended codes must be the oracle's
-    # codes of the new vectors (near-tie rule) and the outputs the oracle's attention over the updated cache.
-    w = synth.WORKLOADS[2]
+@pytest.mark.parametrize("wi,n_items,seed", [(2, 4, 212), (4, 4, 414), (1, 8, 111)])
+def test_decode_step_full_size(wi, n_items, seed):
+    # The call the benchmark times: cq_decode_step (the new token's K and V are encoded and written at the last
+    # position inside the attention launch, which then attends over all tokens), on config 2 (the kernel with two
+    # heads per table word, one launch), on config 4's ragged layer and on config 1 (the appending instances of the
+    # one-head-per-word kernel).  Sampled (sequence, KV head) items hold the oracle's codes; afterwards the
+    # appended codes must be the oracle's codes of the new vectors (near-tie rule) and the outputs the oracle's
+    # attention over the updated cache.
+    w = synth.WORKLOADS[wi]
     st = bench.DecodeState(w, 0, torch.device(DEV), cq)
-    assert st.fused_launches == 1
+    assert st.fused_launches <= 2 and (wi != 2 or st.fused_launches == 1)
     cap, D, c, b = st.cap, w.head_dim, w.c, w.b
     R = w.n_q_heads // w.n_kv_heads
-    items = seeded_items(w, 4, 212, must=[(w.n_seq - 1, 5)])
+    items = seeded_items(w, n_items, seed, must=[(w.n_seq - 1, w.n_kv_heads - 3)])
     codes = {}
     for (s, h) in items:
         for is_v, buf, cb in ((False, st.k_codes, st.k_cb), (True, st.v_codes, st.v_cb)):
@@ -295,4 +298,4 @@ def test_config2_decode_step_full_size():
         a, r = H.check_attn(out[s, h * R:(h + 1) * R], ref[0], f"step item (seq {s}, kv head {h})")
         worst_abs, worst_rel = max(worst_abs, a), max(worst_rel, r)
     assert ties <= 1
-    print(f"config 2 step: {total} appended codes checked, {ties} near-ties, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
+    print(f"config {wi} step: {total} appended codes checked, {ties} near-ties, attention max-abs {worst_abs:.2e} rel-L2 {worst_rel:.2e}")
