@@ -47,6 +47,27 @@ def test_kmeanspp_init_is_bit_equal(c, b, n_heads, n_vec, weighted):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("c,b,n_vec,weighted", [(8, 8, 5000, True), (4, 6, 4096, False), (8, 4, 6200, True), (2, 5, 2049, False)])
+def test_kmeanspp_init_is_bit_equal_over_several_tiles(c, b, n_vec, weighted):
+    # more vectors than one tile of the draw's in-order sum (2048): the running sums kept at the tile ends decide
+    # where the walk for the drawn vector starts; uniforms at both ends of [0, 1) and runs of zero contributions
+    # (whole tiles of them in the weighted cases) are part of the input
+    x = calib(340 + c, n_vec, 1, False, c)
+    G = 128 // c
+    w = fisher_like_weights(c + b, n_vec, 1, G) if weighted else None
+    if weighted:
+        w[::5] = 0
+        w[:2100] = 0                                                     # the first tile, and part of the second
+        w[4200:4900] = 0
+    u = torch.rand(1, G, 1 << b, dtype=torch.float64, generator=torch.Generator().manual_seed(40 + b))
+    u[0, :, 1] = 0.0
+    u[0, :, 2] = 1.0 - 2.0 ** -53
+    u[0, ::2, 3] = 2.0 ** -40
+    want, chosen = oracle.kmeanspp_init(x.numpy(), None if w is None else w.numpy(), u.numpy(), c, b)
+    got = cq.cq_kmeanspp_init(x.to(DEV), None if w is None else w.to(DEV), u.to(DEV), c, b).cpu().numpy()
+    assert np.array_equal(got, want)
+
+
 @pytest.mark.parametrize("c,b,n_heads,n_vec,weighted", [(8, 8, 2, 3000, False), (8, 8, 2, 3000, True), (4, 8, 2, 2000, True),
                                                        (2, 8, 1, 2500, False), (8, 4, 2, 500, True)])
 def test_one_iteration_from_common_state(c, b, n_heads, n_vec, weighted):
